@@ -1,0 +1,256 @@
+/*
+ * sbc.h -- C ABI of the B200 Sparse Binary Compression library.
+ *
+ * Sparse Binary Compression (Sattler, Wiedemann, Mueller, Samek,
+ * arXiv 1805.08768) sends, per tensor and per communication round, the
+ * positions of a p-fraction of a client's accumulated weight update plus ONE
+ * fp32 value.  This library is the per-tensor hot path of that scheme on one
+ * NVIDIA B200 (sm_100a): the client-side encode and the server-side
+ * decode-and-sum.  Everything below runs as CUDA kernels on the caller's
+ * stream; there is no CPU fallback.
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA global-memory addresses on the current
+ *     device, "host" pointers are ordinary process memory.
+ *   - The caller owns every buffer.  Except where an entry point says
+ *     otherwise the library allocates nothing and keeps no state between
+ *     calls.
+ *   - Device work is enqueued on `stream` and the call returns without
+ *     waiting for it, unless the entry point says that it synchronises.
+ *   - Return value: SBC_OK or a negative sbc_status code.  Errors the host
+ *     can see (null or misaligned pointer, size out of range, capacity too
+ *     small) are returned at once and nothing is enqueued.  Errors only the
+ *     device can see (non-finite input, corrupt stream) are recorded in the
+ *     stream header's status word / the status word passed to the decoder
+ *     and the kernels stop writing results; they never trap.
+ *   - Positions are flat 0-based element indices, numel < 2^31.
+ */
+#ifndef SBC_H
+#define SBC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Same type as cudaStream_t (an opaque driver handle); 0 is the default stream. */
+typedef struct CUstream_st *sbc_cuda_stream_t;
+
+enum sbc_status {
+    SBC_OK = 0,
+    SBC_EINVAL = -1,     /* bad argument */
+    SBC_ECAPACITY = -2,  /* an output or workspace buffer is too small */
+    SBC_ENONFINITE = -3, /* residual + update holds an Inf or NaN */
+    SBC_ECORRUPT = -4,   /* a stream failed validation while decoding */
+    SBC_ETIMEOUT = -5,   /* a bounded device-side wait gave up (unused so far: no kernel waits) */
+    SBC_ECUDA = -6       /* a CUDA runtime call failed */
+};
+
+/* Bits of the device-side status words (stream header offset 60, decoder status word). */
+#define SBC_STATUS_NONFINITE 0x1u
+#define SBC_STATUS_CORRUPT 0x2u
+#define SBC_STATUS_RANGE 0x4u /* a decoded position fell outside [0, numel) */
+#define SBC_STATUS_INTERNAL 0x8u
+
+/*
+ * Stream container (little-endian).  The paper's message is the Golomb bit
+ * string of the position gaps plus one mean value per tensor (Section 2,
+ * "Optimal Position Encoding"); tensor shapes are known to both sides
+ * (Supplement, "Golomb Position Decoding").  The container keeps that bit
+ * string unchanged as its payload and adds what a parallel decoder needs:
+ *
+ *   bytes 0..63   header
+ *      0 u32 magic "SBC1"      4 u32 version (1)     8 u64 numel
+ *     16 u64 k (positions)    24 u64 nbits (payload bits)
+ *     32 u64 payload_offset   40 u32 b (Golomb parameter b*)
+ *     44 u32 side (0: +mu kept, 1: -mu kept)          48 f32 mu (signed)
+ *     52 u32 chunk_codewords  56 u32 n_chunks         60 u32 status
+ *   bytes 64..    chunk table, n_chunks entries of
+ *                 { u64 bit offset of codeword c*chunk_codewords,
+ *                   i64 position decoded just before it (-1 for c = 0) }
+ *   payload_offset..  payload: codeword i = q ones, a zero, r in b bits
+ *                 (MSB first), where gap-1 = q*2^b + r (Algorithm 3); stream
+ *                 bit j is bit 7-(j%8) of byte j/8; zero padded to 16 bytes.
+ */
+#define SBC_MAGIC 0x31434253u
+#define SBC_VERSION 1u
+#define SBC_HEADER_BYTES 64u
+#define SBC_CHUNK_CODEWORDS 256u
+#define SBC_CHUNK_ENTRY_BYTES 16u
+
+typedef struct sbc_stream_info {
+    uint32_t magic, version;
+    uint64_t numel, k, nbits, payload_offset;
+    uint32_t b, side;
+    float mu;
+    uint32_t chunk_codewords, n_chunks, status;
+    uint64_t total_bytes; /* payload_offset + payload bytes rounded up to 16 */
+} sbc_stream_info;
+
+/* ---- host-side pure functions (no CUDA calls) ------------------------- */
+
+/* Number of positions sent for a tensor of numel elements at sparsity p:
+ * k = max(1, floor(p * numel)), at most numel.  The paper's top_p% (Algorithm
+ * 2) does not say how p*|W| is rounded; this is the convention used here.
+ * Returns 0 if numel <= 0 or p is not in (0, 1). */
+int64_t sbc_kept_count(int64_t numel, double p);
+
+/* Golomb parameter b* = 1 + floor(log2(log(phi-1)/log(1-p))), phi the golden
+ * ratio (Algorithm 3), clamped at 0.  Returns -1 if p is not in (0, 1). */
+int sbc_golomb_b(double p);
+
+/* Mean position bits b + 1/(1-(1-p)^(2^b)) (Section 2, equation for b_pos):
+ * the expected codeword length when gaps are geometric. */
+double sbc_mean_position_bits(double p, int b);
+
+/* Capacity, in bytes, that out_stream must have for sbc_encode(numel, p):
+ * header + chunk table + the largest possible payload,
+ * k(1+b) + floor((numel-k)/2^b) bits, rounded up to 16 bytes.  0 on bad
+ * arguments. */
+size_t sbc_stream_bytes(int64_t numel, double p);
+
+/* Bytes of device scratch sbc_encode(numel, p) needs.  0 on bad arguments. */
+size_t sbc_workspace_bytes(int64_t numel, double p);
+
+/* ---- client side ------------------------------------------------------- */
+
+/*
+ * One client step for one tensor (Algorithm 1, client lines
+ * "dW_i <- R_i + ...", "dW_i* <- compress(dW_i)", "R_i <- dW_i - dW_i*",
+ * "msg_i <- encode(dW_i*)"; Algorithm 2; Algorithm 3):
+ *
+ *   A      = residual + update                 (fp32, elementwise)
+ *   val+   = the k largest entries of A,  val- = the k largest of -A
+ *            (equal values: lower index first; exactly k each)
+ *   mu+    = mean(val+), mu- = mean(val-)      (sums exact, one fp64 divide)
+ *   kept   = positions of val+ if mu+ >= mu-, else of val-
+ *   mu     = (float)mu+  or  (float)(-mu-)
+ *   residual = A, except residual[j] = A[j] - mu for j in kept
+ *   out_stream = container(kept positions in ascending order, mu)
+ *   *out_mu = mu
+ *
+ * update     device, numel floats, read only, 4-byte aligned (16 preferred)
+ * residual   device, numel floats, in: R_old, out: R_new; must not alias update
+ * numel      1 .. 2^31-1
+ * p          sparsity, 0 < p < 1, with sbc_golomb_b(p) <= 30
+ * out_stream device, 16-byte aligned, out_capacity >= sbc_stream_bytes(numel, p)
+ * out_mu     device, one float (may be NULL)
+ * workspace  device, 256-byte aligned, workspace_bytes >= sbc_workspace_bytes
+ *            (numel, p); contents are scratch, nothing carries between calls
+ * stream     CUDA stream the work is enqueued on
+ *
+ * Asynchronous.  If A holds a non-finite value the header's status word gets
+ * SBC_STATUS_NONFINITE, residual holds A and no payload is produced; read the
+ * header with sbc_stream_info to find out.
+ */
+int sbc_encode(const float *update, float *residual, int64_t numel, double p,
+               void *out_stream, size_t out_capacity, float *out_mu,
+               void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream);
+
+/*
+ * sbc_encode with timing marks: the same work, plus, when `marks` is not NULL,
+ * a cudaEventRecord on `stream` at each stage boundary.  marks is a host array
+ * of SBC_MARK_COUNT events the caller created (entries may be NULL).  The
+ * interval BOUNDS->COLLECT holds exactly one kernel, the streaming pass that
+ * reads update and residual and writes the residual (Algorithm 1's accumulate
+ * fused with the candidate gathering for Algorithm 2).
+ */
+typedef struct CUevent_st *sbc_cuda_event_t; /* same type as cudaEvent_t */
+enum sbc_mark {
+    SBC_MARK_BEGIN = 0, /* before anything is enqueued */
+    SBC_MARK_BOUNDS,    /* scratch cleared, threshold bounds estimated from the sample */
+    SBC_MARK_COLLECT,   /* residual = A written, candidate lists gathered */
+    SBC_MARK_EXACT,     /* exact-select route over A done (a no-op unless the bounds failed) */
+    SBC_MARK_SELECT,    /* k-th entries, means, side, mu, residual write-back done */
+    SBC_MARK_END,       /* positions compacted, Golomb payload, chunk table and header written */
+    SBC_MARK_COUNT
+};
+int sbc_encode_ex(const float *update, float *residual, int64_t numel, double p,
+                  void *out_stream, size_t out_capacity, float *out_mu,
+                  void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream,
+                  const sbc_cuda_event_t *marks);
+
+/* Number of kernels one sbc_encode call launches (memsets not counted), and
+ * one sbc_decode_accumulate call for n_clients streams. */
+int sbc_encode_launches(void);
+int sbc_decode_launches(int n_clients);
+
+/* What the last sbc_encode that used `workspace` did; synchronises `stream`. */
+typedef struct sbc_encode_diag {
+    uint32_t status;        /* SBC_STATUS_* bits */
+    uint32_t exact_route;   /* 1 if the bounds from the sample failed and the exact route ran */
+    uint32_t candidates[2]; /* entries gathered per side (>= k) */
+    uint32_t capacity;      /* capacity of each candidate list */
+    float bound_lo, bound_hi; /* candidates were: value >= bound_lo, value <= bound_hi */
+    double mu_pos, mu_neg;  /* the two means of Algorithm 2 */
+} sbc_encode_diag;
+int sbc_encode_diag_get(const void *workspace, sbc_encode_diag *host_out, sbc_cuda_stream_t stream);
+
+/*
+ * Host-buffer form of sbc_encode for callers whose update lives in host
+ * memory: copies update_host to update_dev, encodes, copies the finished
+ * container (its true length, *out_bytes_host) and mu back, and synchronises
+ * `stream`.  The residual is the encoder's persistent state (Algorithm 1) and
+ * stays on the device.  update_dev: device scratch of numel floats;
+ * stream_dev: device scratch of out_capacity bytes.  Pinned host memory makes
+ * the copies asynchronous up to the final synchronise.
+ */
+int sbc_encode_host(const float *update_host, float *update_dev, float *residual_dev,
+                    int64_t numel, double p, void *out_stream_host, void *stream_dev,
+                    size_t out_capacity, size_t *out_bytes_host, float *out_mu_host,
+                    void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream);
+
+/* Copies the header of a device-resident stream to the host and fills
+ * *host_out.  Synchronises `stream`.  Returns SBC_OK, SBC_ECORRUPT if the
+ * magic/version are wrong, SBC_ENONFINITE if the status word says so. */
+int sbc_stream_info_get(const void *stream_dev, sbc_stream_info *host_out,
+                        sbc_cuda_stream_t stream);
+
+/* ---- server side ------------------------------------------------------- */
+
+/*
+ * Decode n_clients streams and add them into a dense tensor (Algorithm 4 for
+ * each stream; Algorithm 1, server line "dW <- 1/|I_t| sum dW_i*", without
+ * the 1/|I_t| factor, which is the caller's):
+ *
+ *   out_dense[j] += mu_c   for every client c and every position j it sent.
+ *
+ * streams    HOST array of n_clients DEVICE pointers to containers written
+ *            by sbc_encode for the same numel (16-byte aligned)
+ * n_clients  >= 0
+ * out_dense  device, numel floats, in/out (zero it first for a plain sum)
+ * numel      must equal the numel in every header
+ * status_dev device, one uint32 the kernels OR error bits into (may be NULL;
+ *            the caller zeroes it).  A stream whose header fails validation
+ *            contributes nothing; a chunk whose codewords run out of the
+ *            payload or past numel stops there; a chunk that does not end
+ *            where the table says the next one starts is reported after its
+ *            (in-range) positions were added.  When the word is non-zero
+ *            out_dense is not to be trusted.
+ * Asynchronous.  The order of the fp32 additions into one element is not
+ * fixed, so sums over several clients agree with a sequential sum to
+ * rounding (<= n_clients ulps of the partial sums), not bit for bit.
+ */
+int sbc_decode_accumulate(const void *const *streams, int n_clients,
+                          float *out_dense, int64_t numel, uint32_t *status_dev,
+                          sbc_cuda_stream_t stream);
+
+/*
+ * Host-buffer form of sbc_decode_accumulate: copies the n_clients containers
+ * (streams_host[c], stream_bytes[c] bytes each) into staging_dev (device
+ * scratch of staging_bytes >= sum of the sizes rounded up to 16 each), zeroes
+ * dense_dev (device, numel floats), decodes and sums into it, copies the
+ * result to out_dense_host and the status word to *status_host, and
+ * synchronises `stream`.  Returns SBC_ECORRUPT if the status word is non-zero.
+ */
+int sbc_decode_accumulate_host(const void *const *streams_host, const size_t *stream_bytes,
+                               int n_clients, float *out_dense_host, float *dense_dev,
+                               int64_t numel, void *staging_dev, size_t staging_bytes,
+                               uint32_t *status_host, sbc_cuda_stream_t stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SBC_H */

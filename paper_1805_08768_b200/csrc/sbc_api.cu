@@ -1,0 +1,412 @@
+// Host side of the SBC C ABI: argument checks, workspace layout, kernel launches.
+// Declared and documented in include/sbc.h.
+#include <cmath>
+#include <cstring>
+
+#include "../../include/sbc.h"
+#include "sbc_common.cuh"
+#include "sbc_decode.cuh"
+#include "sbc_exact.cuh"
+#include "sbc_front.cuh"
+#include "sbc_golomb.cuh"
+#include "sbc_select.cuh"
+
+namespace sbc {
+namespace {
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Host-side plan of one encode problem: scalar parameters and the byte offset
+// of every scratch array inside the workspace.
+struct Plan {
+    long long n, k;
+    int b;
+    uint32_t cap, m, n_xtiles, n_mask_words, n_mask_tiles, n_len_blocks, n_chunks;
+    uint32_t s_target[2];
+    unsigned long long payload_offset;
+    size_t stream_bytes;
+    size_t off_prob, off_mu, off_ctl, off_hists, off_sample, off_cand[2], off_buf[2][2], off_mask,
+        off_mask_tile, off_xtile[2], off_idx, off_blklen, total;
+    size_t zero_begin, zero_end;  // Ctl + Hists, cleared before every call
+};
+
+bool valid_p(double p) { return p > 0.0 && p < 1.0; }
+
+bool make_plan(long long n, double p, Plan* pl) {
+    if (n <= 0 || n >= (1ll << 31) || !valid_p(p)) return false;
+    const int b = sbc_golomb_b(p);
+    if (b < 0 || b > 30) return false;
+    const long long k = sbc_kept_count(n, p);
+    pl->n = n;
+    pl->k = k;
+    pl->b = b;
+    pl->cap = (uint32_t)std::min<long long>(n, 2 * k + 1024);
+    pl->m = n <= (long long)kSampleMax ? (uint32_t)n : kSampleMax;
+    // Rank looked up in the sample.  If the sample is the whole tensor the
+    // rank is k itself; otherwise the expected rank plus six standard
+    // deviations of a binomial count (and a little), so that the bound falls
+    // below the true k-th value except with negligible probability -- and if
+    // it does not, the exact route takes over.
+    uint32_t target;
+    if ((long long)pl->m == n) {
+        target = (uint32_t)k;
+    } else {
+        const double expect = (double)k * (double)pl->m / (double)n;
+        const double t = std::ceil(expect + 6.0 * std::sqrt(expect) + 8.0);
+        target = (uint32_t)std::min<double>(t, (double)pl->m);
+    }
+    pl->s_target[0] = pl->s_target[1] = target;
+    pl->n_xtiles = (uint32_t)((n + kXTile - 1) / kXTile);
+    pl->n_mask_words = (uint32_t)align_up((size_t)((n + 31) / 32), 4);
+    pl->n_mask_tiles = (pl->n_mask_words + kMaskTileWords - 1) / kMaskTileWords;
+    pl->n_len_blocks = (uint32_t)((k + kLenBlock - 1) / kLenBlock);
+    pl->n_chunks = (uint32_t)((k + kChunkCodewords - 1) / kChunkCodewords);
+    pl->payload_offset = SBC_HEADER_BYTES + (unsigned long long)pl->n_chunks * SBC_CHUNK_ENTRY_BYTES;
+    const unsigned long long bits_bound =
+        (unsigned long long)k * (1ull + b) + ((unsigned long long)(n - k) >> b);
+    pl->stream_bytes = (size_t)pl->payload_offset + align_up((size_t)((bits_bound + 7) / 8), 16);
+
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    pl->off_prob = take(sizeof(Prob));
+    pl->off_mu = take(sizeof(float));  // where the host-buffer form parks mu
+    pl->zero_begin = off;
+    pl->off_ctl = take(sizeof(Ctl));
+    pl->off_hists = take(sizeof(Hists));
+    pl->zero_end = off;
+    pl->off_sample = take((size_t)pl->m * 4);
+    for (int s = 0; s < 2; ++s) pl->off_cand[s] = take((size_t)pl->cap * 8);
+    for (int s = 0; s < 2; ++s)
+        for (int j = 0; j < 2; ++j) pl->off_buf[s][j] = take((size_t)pl->cap * 8);
+    pl->off_mask = take((size_t)pl->n_mask_words * 4);
+    pl->off_mask_tile = take((size_t)pl->n_mask_tiles * 4);
+    for (int s = 0; s < 2; ++s) pl->off_xtile[s] = take((size_t)pl->n_xtiles * 4);
+    pl->off_idx = take((size_t)k * 4);
+    pl->off_blklen = take((size_t)pl->n_len_blocks * 8);
+    pl->total = off;
+    return true;
+}
+
+// Writes the problem descriptor where the kernels read it.
+__global__ void k_put_prob(Prob* dst, const Prob src) { *dst = src; }
+
+int sm_count() {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0)
+        return 148;
+    return sms;
+}
+
+inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsigned max_blocks) {
+    unsigned long long g = (work_items + per_block - 1) / per_block;
+    if (g < 1) g = 1;
+    if (g > max_blocks) g = max_blocks;
+    return (unsigned)g;
+}
+
+}  // namespace
+}  // namespace sbc
+
+using namespace sbc;
+
+extern "C" {
+
+int64_t sbc_kept_count(int64_t numel, double p) {
+    if (numel <= 0 || !valid_p(p)) return 0;
+    int64_t k = (int64_t)std::floor(p * (double)numel);
+    if (k < 1) k = 1;
+    if (k > numel) k = numel;
+    return k;
+}
+
+int sbc_golomb_b(double p) {
+    if (!valid_p(p)) return -1;
+    const double golden = (1.0 + std::sqrt(5.0)) * 0.5;
+    const double x = std::log(golden - 1.0) / std::log(1.0 - p);
+    const int b = 1 + (int)std::floor(std::log2(x));
+    return b < 0 ? 0 : b;
+}
+
+double sbc_mean_position_bits(double p, int b) {
+    return (double)b + 1.0 / (1.0 - std::pow(1.0 - p, std::ldexp(1.0, b)));
+}
+
+size_t sbc_stream_bytes(int64_t numel, double p) {
+    Plan pl;
+    return make_plan(numel, p, &pl) ? pl.stream_bytes : 0;
+}
+
+size_t sbc_workspace_bytes(int64_t numel, double p) {
+    Plan pl;
+    return make_plan(numel, p, &pl) ? pl.total : 0;
+}
+
+int sbc_encode(const float* update, float* residual, int64_t numel, double p, void* out_stream,
+               size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
+               sbc_cuda_stream_t stream) {
+    return sbc_encode_ex(update, residual, numel, p, out_stream, out_capacity, out_mu, workspace,
+                         workspace_bytes, stream, nullptr);
+}
+
+int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p, void* out_stream,
+                  size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
+                  sbc_cuda_stream_t stream, const sbc_cuda_event_t* marks) {
+    Plan pl;
+    if (!update || !residual || !out_stream || !workspace) return SBC_EINVAL;
+    if (!make_plan(numel, p, &pl)) return SBC_EINVAL;
+    if (((uintptr_t)update & 3) || ((uintptr_t)residual & 3) || ((uintptr_t)out_stream & 15) ||
+        ((uintptr_t)workspace & 255) || (out_mu && ((uintptr_t)out_mu & 3)))
+        return SBC_EINVAL;
+    {   // update and residual must not overlap
+        const uintptr_t u0 = (uintptr_t)update, r0 = (uintptr_t)residual, len = (uintptr_t)numel * 4;
+        if (u0 < r0 + len && r0 < u0 + len) return SBC_EINVAL;
+    }
+    if (out_capacity < pl.stream_bytes || workspace_bytes < pl.total) return SBC_ECAPACITY;
+
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    Prob P;
+    std::memset(&P, 0, sizeof(P));
+    P.update = update;
+    P.residual = residual;
+    P.n = pl.n;
+    P.k = pl.k;
+    P.b = pl.b;
+    P.vec_ok = (((uintptr_t)update | (uintptr_t)residual) & 15) == 0;
+    P.stream = static_cast<uint8_t*>(out_stream);
+    P.stream_cap = out_capacity;
+    P.out_mu = out_mu;
+    P.ctl = reinterpret_cast<Ctl*>(ws + pl.off_ctl);
+    P.hists = reinterpret_cast<Hists*>(ws + pl.off_hists);
+    P.sample_keys = reinterpret_cast<uint32_t*>(ws + pl.off_sample);
+    for (int s = 0; s < 2; ++s) {
+        P.cand[s] = reinterpret_cast<unsigned long long*>(ws + pl.off_cand[s]);
+        for (int j = 0; j < 2; ++j) P.buf[s][j] = reinterpret_cast<unsigned long long*>(ws + pl.off_buf[s][j]);
+        P.x_tile_cnt[s] = reinterpret_cast<uint32_t*>(ws + pl.off_xtile[s]);
+        P.s_target[s] = pl.s_target[s];
+    }
+    P.mask = reinterpret_cast<uint32_t*>(ws + pl.off_mask);
+    P.mask_tile_cnt = reinterpret_cast<uint32_t*>(ws + pl.off_mask_tile);
+    P.idx = reinterpret_cast<uint32_t*>(ws + pl.off_idx);
+    P.blk_len = reinterpret_cast<unsigned long long*>(ws + pl.off_blklen);
+    P.cap = pl.cap;
+    P.m = pl.m;
+    P.n_xtiles = pl.n_xtiles;
+    P.n_mask_words = pl.n_mask_words;
+    P.n_mask_tiles = pl.n_mask_tiles;
+    P.n_len_blocks = pl.n_len_blocks;
+    P.n_chunks = pl.n_chunks;
+    P.payload_offset = pl.payload_offset;
+
+    cudaStream_t st = stream;
+    auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
+    mark(SBC_MARK_BEGIN);
+    Prob* dP = reinterpret_cast<Prob*>(ws + pl.off_prob);
+    const unsigned sms = (unsigned)sm_count();
+    const dim3 blk(kBlock);
+
+    // scratch that must start at zero: control block + histograms, the kept
+    // mask, and the chunk table + payload area the packer ORs into
+    if (cudaMemsetAsync(ws + pl.zero_begin, 0, pl.zero_end - pl.zero_begin, st) != cudaSuccess ||
+        cudaMemsetAsync(P.mask, 0, (size_t)pl.n_mask_words * 4, st) != cudaSuccess ||
+        cudaMemsetAsync(P.stream + SBC_HEADER_BYTES, 0, pl.stream_bytes - SBC_HEADER_BYTES, st) != cudaSuccess)
+        return SBC_ECUDA;
+    k_put_prob<<<1, 1, 0, st>>>(dP, P);
+
+    // 1. bounds from the sample, then the streaming accumulate + collect pass
+    const unsigned g_sample = grid_for(pl.m, kBlock * 8, sms * 4);
+    k_sample0<<<dim3(g_sample), blk, 0, st>>>(dP);
+    k_sample1<<<dim3(g_sample), blk, 0, st>>>(dP);
+    mark(SBC_MARK_BOUNDS);
+    const unsigned g_main = grid_for((unsigned long long)pl.n, kBlock * kPerThread * 2, sms * 6);
+    if (P.vec_ok) k_add_collect<true><<<dim3(g_main), blk, 0, st>>>(dP);
+    else          k_add_collect<false><<<dim3(g_main), blk, 0, st>>>(dP);
+
+    mark(SBC_MARK_COLLECT);
+
+    // 2. exact route over A (returns immediately unless the bounds failed)
+    const unsigned g_x = grid_for((unsigned long long)pl.n, kBlock * 16, sms * 8);
+    k_exact_hist<0><<<dim3(g_x), blk, 0, st>>>(dP);
+    k_exact_hist<1><<<dim3(g_x), blk, 0, st>>>(dP);
+    k_exact_hist<2><<<dim3(g_x), blk, 0, st>>>(dP);
+    const unsigned g_xt = grid_for(pl.n_xtiles, 1, sms * 8);
+    k_exact_tiecount<<<dim3(g_xt), blk, 0, st>>>(dP);
+    k_exact_tiescan<<<dim3(1), blk, 0, st>>>(dP);
+    k_exact_collect<<<dim3(g_xt), blk, 0, st>>>(dP);
+
+    mark(SBC_MARK_EXACT);
+
+    // 3. exact k-th composite of each candidate list, sums, side, residual
+    const unsigned g_c = grid_for(pl.cap, kBlock * 4, sms * 4);
+    k_select_hist0<<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
+    k_select_filter<0><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
+    k_select_filter<1><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
+    k_select_filter<2><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
+    k_select_filter<3><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
+    k_select_filter<4><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
+    k_sums_decide<<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
+    k_apply<<<dim3(g_c), blk, 0, st>>>(dP);
+
+    mark(SBC_MARK_SELECT);
+
+    // 4. Golomb stage
+    const unsigned g_m = grid_for(pl.n_mask_tiles, 1, sms * 8);
+    k_mask_count<<<dim3(g_m), blk, 0, st>>>(dP);
+    k_mask_scan<<<dim3(1), blk, 0, st>>>(dP);
+    k_mask_compact<<<dim3(g_m), blk, 0, st>>>(dP);
+    const unsigned g_l = grid_for(pl.n_len_blocks, 1, sms * 8);
+    k_len_sum<<<dim3(g_l), blk, 0, st>>>(dP);
+    k_len_scan_header<<<dim3(1), blk, 0, st>>>(dP);
+    k_pack<<<dim3(g_l), blk, 0, st>>>(dP);
+    mark(SBC_MARK_END);
+
+    return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
+}
+
+int sbc_encode_launches(void) { return 24; }  // put_prob, 2 sample, 1 collect, 6 exact, 8 select, 6 Golomb
+
+int sbc_decode_launches(int n_clients) {
+    return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;
+}
+
+int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cuda_stream_t stream) {
+    if (!workspace || !host_out) return SBC_EINVAL;
+    Plan pl;
+    make_plan(1024, 0.5, &pl);  // the control block sits at a fixed offset
+    Prob P;
+    Ctl c;
+    const uint8_t* ws = static_cast<const uint8_t*>(workspace);
+    if (cudaMemcpyAsync(&P, ws + pl.off_prob, sizeof(P), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemcpyAsync(&c, ws + pl.off_ctl, sizeof(c), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return SBC_ECUDA;
+    host_out->status = c.status;
+    host_out->exact_route = c.use_fallback;
+    host_out->candidates[0] = c.cand_cnt[0];
+    host_out->candidates[1] = c.cand_cnt[1];
+    host_out->capacity = P.cap;
+    host_out->bound_lo = c.lo_f;
+    host_out->bound_hi = c.hi_f;
+    host_out->mu_pos = c.mu64[0];
+    host_out->mu_neg = c.mu64[1];
+    return SBC_OK;
+}
+
+int sbc_encode_host(const float* update_host, float* update_dev, float* residual_dev, int64_t numel,
+                    double p, void* out_stream_host, void* stream_dev, size_t out_capacity,
+                    size_t* out_bytes_host, float* out_mu_host, void* workspace, size_t workspace_bytes,
+                    sbc_cuda_stream_t stream) {
+    if (!update_host || !update_dev || !out_stream_host || !stream_dev || !out_bytes_host || numel <= 0)
+        return SBC_EINVAL;
+    if (!workspace) return SBC_EINVAL;
+    if (cudaMemcpyAsync(update_dev, update_host, (size_t)numel * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return SBC_ECUDA;
+    Plan pl;
+    if (!make_plan(numel, p, &pl)) return SBC_EINVAL;
+    if (workspace_bytes < pl.total) return SBC_ECAPACITY;
+    float* mu_dev = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.off_mu);
+    const int rc = sbc_encode(update_dev, residual_dev, numel, p, stream_dev, out_capacity, mu_dev,
+                              workspace, workspace_bytes, stream);
+    if (rc != SBC_OK) return rc;
+    sbc_stream_info info;
+    const int irc = sbc_stream_info_get(stream_dev, &info, stream);  // synchronises
+    if (irc != SBC_OK) return irc;
+    if (info.total_bytes > out_capacity) return SBC_ECAPACITY;
+    float mu = 0.f;
+    if (cudaMemcpyAsync(out_stream_host, stream_dev, info.total_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemcpyAsync(&mu, mu_dev, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return SBC_ECUDA;
+    *out_bytes_host = info.total_bytes;
+    if (out_mu_host) *out_mu_host = mu;
+    return SBC_OK;
+}
+
+int sbc_stream_info_get(const void* stream_dev, sbc_stream_info* host_out, sbc_cuda_stream_t stream) {
+    if (!stream_dev || !host_out) return SBC_EINVAL;
+    uint8_t h[SBC_HEADER_BYTES];
+    if (cudaMemcpyAsync(h, stream_dev, SBC_HEADER_BYTES, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return SBC_ECUDA;
+    sbc_stream_info& o = *host_out;
+    std::memcpy(&o.magic, h + 0, 4);
+    std::memcpy(&o.version, h + 4, 4);
+    std::memcpy(&o.numel, h + 8, 8);
+    std::memcpy(&o.k, h + 16, 8);
+    std::memcpy(&o.nbits, h + 24, 8);
+    std::memcpy(&o.payload_offset, h + 32, 8);
+    std::memcpy(&o.b, h + 40, 4);
+    std::memcpy(&o.side, h + 44, 4);
+    std::memcpy(&o.mu, h + 48, 4);
+    std::memcpy(&o.chunk_codewords, h + 52, 4);
+    std::memcpy(&o.n_chunks, h + 56, 4);
+    std::memcpy(&o.status, h + 60, 4);
+    o.total_bytes = o.payload_offset + align_up((size_t)((o.nbits + 7) / 8), 16);
+    if (o.magic != SBC_MAGIC || o.version != SBC_VERSION) return SBC_ECORRUPT;
+    if (o.status & SBC_STATUS_NONFINITE) return SBC_ENONFINITE;
+    if (o.status) return SBC_ECORRUPT;
+    return SBC_OK;
+}
+
+int sbc_decode_accumulate(const void* const* streams, int n_clients, float* out_dense, int64_t numel,
+                          uint32_t* status_dev, sbc_cuda_stream_t stream) {
+    if (n_clients < 0 || numel <= 0 || numel >= (1ll << 31) || !out_dense) return SBC_EINVAL;
+    if (n_clients > 0 && !streams) return SBC_EINVAL;
+    if (((uintptr_t)out_dense & 3) || ((uintptr_t)status_dev & 3)) return SBC_EINVAL;
+    for (int c = 0; c < n_clients; ++c)
+        if (!streams[c] || ((uintptr_t)streams[c] & 15)) return SBC_EINVAL;
+    const unsigned sms = (unsigned)sm_count();
+    for (int first = 0; first < n_clients; first += kMaxClientsPerLaunch) {
+        DecodeArgs a;
+        std::memset(&a, 0, sizeof(a));
+        a.n_clients = std::min(kMaxClientsPerLaunch, n_clients - first);
+        for (int c = 0; c < a.n_clients; ++c) a.streams[c] = static_cast<const uint8_t*>(streams[first + c]);
+        a.out = out_dense;
+        a.n = numel;
+        a.status = status_dev;
+        // at most ceil(numel / 256) chunks per client
+        const unsigned long long max_items =
+            (unsigned long long)a.n_clients * (unsigned long long)((numel + kChunkCodewords - 1) / kChunkCodewords);
+        const unsigned grid = grid_for(max_items, 128, sms * 16);
+        k_decode_accumulate<<<grid, 128, 0, stream>>>(a);
+    }
+    return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
+}
+
+int sbc_decode_accumulate_host(const void* const* streams_host, const size_t* stream_bytes, int n_clients,
+                               float* out_dense_host, float* dense_dev, int64_t numel, void* staging_dev,
+                               size_t staging_bytes, uint32_t* status_host, sbc_cuda_stream_t stream) {
+    if (n_clients < 0 || n_clients > 4096 || numel <= 0 || !out_dense_host || !dense_dev || !staging_dev)
+        return SBC_EINVAL;
+    if (n_clients > 0 && (!streams_host || !stream_bytes)) return SBC_EINVAL;
+    if ((uintptr_t)staging_dev & 15) return SBC_EINVAL;
+    // staging layout: one status word (16 bytes), then the containers
+    size_t need = 16;
+    for (int c = 0; c < n_clients; ++c) need += align_up(stream_bytes[c], 16);
+    if (staging_bytes < need) return SBC_ECAPACITY;
+    uint8_t* base = static_cast<uint8_t*>(staging_dev);
+    const void* dev_ptrs[4096];
+    size_t off = 16;
+    if (cudaMemsetAsync(base, 0, 16, stream) != cudaSuccess ||
+        cudaMemsetAsync(dense_dev, 0, (size_t)numel * 4, stream) != cudaSuccess)
+        return SBC_ECUDA;
+    for (int c = 0; c < n_clients; ++c) {
+        if (!streams_host[c] || stream_bytes[c] < SBC_HEADER_BYTES) return SBC_EINVAL;
+        if (cudaMemcpyAsync(base + off, streams_host[c], stream_bytes[c], cudaMemcpyHostToDevice, stream) != cudaSuccess)
+            return SBC_ECUDA;
+        dev_ptrs[c] = base + off;
+        off += align_up(stream_bytes[c], 16);
+    }
+    const int rc = sbc_decode_accumulate(dev_ptrs, n_clients, dense_dev, numel,
+                                         reinterpret_cast<uint32_t*>(base), stream);
+    if (rc != SBC_OK) return rc;
+    uint32_t status = 0;
+    if (cudaMemcpyAsync(out_dense_host, dense_dev, (size_t)numel * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemcpyAsync(&status, base, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+        return SBC_ECUDA;
+    if (status_host) *status_host = status;
+    return status ? SBC_ECORRUPT : SBC_OK;
+}
+
+}  // extern "C"

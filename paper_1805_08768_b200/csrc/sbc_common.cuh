@@ -1,0 +1,223 @@
+// Shared definitions for the SBC CUDA kernels (sm_100a).
+//
+// Vocabulary (paper notation): A = R + dW is the accumulated update
+// (Algorithm 1), k the number of kept positions per side (Algorithm 2),
+// b the Golomb parameter b* (Algorithm 3).  "side 0" is the positive side
+// (val+), "side 1" the negative side (val-).
+//
+// Ordering trick used throughout: every fp32 value maps to an unsigned
+// 32-bit key whose integer order is the value order (with -0 folded onto
+// +0); side 1 uses the complemented key, so both sides are always "take the
+// largest".  A candidate is one 64-bit composite, key in the high word and
+// the complemented index in the low word, so that a larger composite means
+// "larger value, or equal value and lower index" -- exactly the tie rule.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace sbc {
+
+constexpr int kBlock = 256;           // threads per block for every kernel here
+constexpr int kHistBins = 2048;       // 11-bit radix digits
+constexpr uint32_t kSampleMax = 1u << 20;  // elements looked at to bound the thresholds
+constexpr int kXTile = 4096;          // elements per tile in the exact-select fallback
+constexpr int kMaskTileWords = 2048;  // 32-bit mask words per compaction tile
+constexpr int kLenBlock = 1024;       // codewords per block in the length scan / packer
+constexpr int kChunkCodewords = 256;  // codewords per chunk-table entry
+constexpr int kSumBins = 254;         // one exact integer bin per fp32 exponent
+
+// Stages that use the "last block to finish does the serial step" pattern.
+enum Stage : int {
+    ST_SAMPLE0 = 0, ST_SAMPLE1, ST_COLLECT, ST_XH0, ST_XH1, ST_XH2,
+    ST_BH0_S0, ST_BH0_S1,
+    ST_BF0_S0, ST_BF0_S1, ST_BF1_S0, ST_BF1_S1, ST_BF2_S0, ST_BF2_S1,
+    ST_BF3_S0, ST_BF3_S1, ST_BF4_S0, ST_BF4_S1,
+    ST_SUM, ST_COUNT
+};
+
+// Device-side control block of one encode call; zeroed before the first kernel.
+struct Ctl {
+    uint32_t status;            // SBC_STATUS_* bits
+    uint32_t use_fallback;      // 1: the candidate pass did not bracket both thresholds
+    uint32_t done[ST_COUNT];    // tickets for the last-block pattern
+    // threshold bounds from the sample
+    uint32_t s_bin0[2], s_rank[2];
+    float lo_f, hi_f;           // candidates: !(a < lo_f) for side 0, !(a > hi_f) for side 1
+    // candidate lists
+    uint32_t cand_cnt[2];
+    // exact select over A (fallback)
+    uint32_t x_prefix[2], x_rank[2], x_thr[2], x_ties_take[2], x_ties_have[2];
+    // select over the candidate lists
+    unsigned long long b_prefix[2];
+    uint32_t b_rank[2];
+    uint32_t list_cnt[2][6];
+    unsigned long long thr[2];  // kept <=> composite >= thr[side]
+    // sums and decision
+    long long bins[2][256];
+    double mu64[2];
+    uint32_t side;
+    float mu32;
+    // Golomb stage
+    unsigned long long nbits;
+    uint32_t kept_total;
+    uint32_t pad_;
+};
+
+// Zeroed scratch that sits right behind Ctl.
+struct Hists {
+    uint32_t s0[kHistBins];
+    uint32_t s1[2][kHistBins];
+    uint32_t x[3][2][kHistBins];
+    uint32_t b[6][2][kHistBins];
+};
+
+// Everything a kernel needs to know about one encode problem.  Lives in
+// device memory (first bytes of the workspace); kernels index it by blockIdx.y.
+struct Prob {
+    const float* update;
+    float* residual;
+    long long n;
+    long long k;
+    int b;
+    int vec_ok;                 // 1: update and residual are 16-byte aligned
+    uint8_t* stream;            // container out
+    unsigned long long stream_cap;
+    float* out_mu;
+    Ctl* ctl;
+    Hists* hists;
+    uint32_t* sample_keys;
+    unsigned long long* cand[2];
+    unsigned long long* buf[2][2];   // ping-pong lists of the candidate select
+    uint32_t* mask;
+    uint32_t* mask_tile_cnt;
+    uint32_t* x_tile_cnt[2];
+    uint32_t* idx;              // sorted kept positions
+    unsigned long long* blk_len;
+    uint32_t cap;               // capacity of each candidate list
+    uint32_t m;                 // sample size
+    uint32_t s_target[2];       // rank looked up in the sample, per side
+    uint32_t n_xtiles, n_mask_words, n_mask_tiles, n_len_blocks, n_chunks;
+    unsigned long long payload_offset;
+};
+
+// ---------------------------------------------------------------- keys
+
+__device__ __forceinline__ uint32_t key_of_bits(uint32_t bits) {
+    if (bits == 0x80000000u) bits = 0u;  // -0 ranks with +0
+    return (bits & 0x80000000u) ? ~bits : (bits | 0x80000000u);
+}
+__device__ __forceinline__ uint32_t bits_of_key(uint32_t key) {
+    return (key & 0x80000000u) ? (key & 0x7fffffffu) : ~key;
+}
+__device__ __forceinline__ uint32_t side_key(int side, uint32_t key) { return side ? ~key : key; }
+__device__ __forceinline__ unsigned long long make_composite(uint32_t skey, uint32_t idx) {
+    return ((unsigned long long)skey << 32) | (unsigned long long)(~idx);
+}
+__device__ __forceinline__ uint32_t composite_index(unsigned long long c) { return ~(uint32_t)c; }
+
+// ---------------------------------------------------------------- scans
+
+__device__ __forceinline__ unsigned lane_id() { return threadIdx.x & 31u; }
+
+template <typename T>
+__device__ __forceinline__ T warp_inclusive_scan(T v) {
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        T o = __shfl_up_sync(0xffffffffu, v, d);
+        if ((int)lane_id() >= d) v += o;
+    }
+    return v;
+}
+
+// Exclusive scan over the kBlock threads of a block; *total gets the block sum.
+// s_warp: shared scratch of kBlock/32 + 1 elements.  All threads must call.
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T v, T* s_warp, T* total) {
+    const int warp = threadIdx.x >> 5;
+    T incl = warp_inclusive_scan(v);
+    __syncthreads();  // s_warp may still be read from a previous call
+    if (lane_id() == 31) s_warp[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        T w = (lane_id() < kBlock / 32) ? s_warp[lane_id()] : T(0);
+        T wi = warp_inclusive_scan(w);
+        if (lane_id() < kBlock / 32) s_warp[lane_id()] = wi - w;
+        if (lane_id() == kBlock / 32 - 1) s_warp[kBlock / 32] = wi;
+    }
+    __syncthreads();
+    if (total) *total = s_warp[kBlock / 32];
+    return s_warp[warp] + incl - v;
+}
+
+// ---------------------------------------------------------------- last-block ticket
+
+// True in exactly one block: the one that finishes last among n_blocks.  Every
+// thread must have issued its global writes before calling; all threads call.
+__device__ __forceinline__ bool last_block_ticket(uint32_t* counter, uint32_t n_blocks) {
+    __shared__ uint32_t s_is_last;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = atomicAdd(counter, 1u);
+        s_is_last = (t == n_blocks - 1u) ? 1u : 0u;
+    }
+    __syncthreads();
+    bool last = s_is_last != 0u;
+    if (last) __threadfence();
+    return last;
+}
+
+// ---------------------------------------------------------------- histogram pick
+
+struct Pick {
+    uint32_t bin;    // bin that holds the rank-th largest entry
+    uint32_t rank;   // rank inside that bin (1 = largest in the bin)
+    uint32_t count;  // entries in that bin
+    uint32_t found;
+};
+
+// Walk a histogram from its top bin down and find where the `rank`-th entry
+// falls.  `mirror` reads bin i of the view as hist[nbins-1-i] (the same counts
+// seen from the complemented key).  All kBlock threads call; result in *out
+// (shared) after the trailing barrier.
+__device__ __forceinline__ void block_pick_desc(const uint32_t* hist, int nbins, bool mirror,
+                                                uint32_t rank, uint32_t* s_scan, Pick* out) {
+    const int per = (nbins + kBlock - 1) / kBlock;  // bins per thread, walked top-down
+    uint32_t h[kHistBins / kBlock];
+    uint32_t sum = 0;
+#pragma unroll
+    for (int j = 0; j < kHistBins / kBlock; ++j) {
+        int view = nbins - 1 - ((int)threadIdx.x * per + j);
+        uint32_t v = 0;
+        if (j < per && view >= 0) v = __ldcg(hist + (mirror ? nbins - 1 - view : view));
+        h[j] = v;
+        sum += v;
+    }
+    if (threadIdx.x == 0) out->found = 0u;
+    uint32_t total;
+    uint32_t cum = block_exclusive_scan<uint32_t>(sum, s_scan, &total);
+#pragma unroll
+    for (int j = 0; j < kHistBins / kBlock; ++j) {
+        if (j < per) {
+            if (cum < rank && rank <= cum + h[j]) {
+                out->bin = (uint32_t)(nbins - 1 - ((int)threadIdx.x * per + j));
+                out->rank = rank - cum;
+                out->count = h[j];
+                out->found = 1u;
+            }
+            cum += h[j];
+        }
+    }
+    __syncthreads();
+}
+
+// Add `v` to a shared-memory histogram with one atomic per distinct bin per warp.
+__device__ __forceinline__ void warp_hist_add(uint32_t* s_hist, uint32_t bin, bool valid) {
+    unsigned active = __ballot_sync(0xffffffffu, valid);
+    if (!valid) return;
+    unsigned peers = __match_any_sync(active, bin);
+    if ((int)lane_id() == __ffs(peers) - 1) atomicAdd(&s_hist[bin], (uint32_t)__popc(peers));
+}
+
+}  // namespace sbc

@@ -1,0 +1,228 @@
+// Exact-select route over the whole accumulated tensor A (Algorithm 2's top_p
+// by radix selection on the fp32 bit patterns).  Runs only when the candidate
+// pass could not bracket both thresholds; every kernel returns at once
+// otherwise.  Result: exactly k composites per side in the candidate lists.
+#pragma once
+#include "sbc_common.cuh"
+#include "../../include/sbc.h"
+
+namespace sbc {
+
+__device__ __forceinline__ bool exact_route_active(const Ctl* ctl) {
+    return ctl->use_fallback != 0u && ctl->status == 0u;
+}
+
+// One radix level (0: key bits 31..21, 1: bits 20..10, 2: bits 9..0) for both
+// sides; the last block extends the two prefixes.
+template <int LEVEL>
+__global__ void __launch_bounds__(kBlock) k_exact_hist(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (!exact_route_active(ctl)) return;
+    constexpr int kBins = (LEVEL == 2) ? 1024 : kHistBins;
+    __shared__ uint32_t s_hist[2][kHistBins];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ Pick s_pick;
+    for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) (&s_hist[0][0])[i] = 0u;
+    __syncthreads();
+    const uint32_t pre[2] = {ctl->x_prefix[0], ctl->x_prefix[1]};
+    const float* __restrict__ A = P.residual;
+    const long long stride = (long long)gridDim.x * kBlock;
+    for (long long base = (long long)blockIdx.x * kBlock; base < P.n; base += stride) {
+        const long long i = base + threadIdx.x;
+        const bool valid = i < P.n;
+        const uint32_t key = valid ? key_of_bits(__float_as_uint(A[i])) : 0u;
+        if (LEVEL == 0) {
+            warp_hist_add(s_hist[0], key >> 21, valid);
+        } else {
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                const uint32_t sk = side_key(s, key);
+                if (LEVEL == 1)
+                    warp_hist_add(s_hist[s], (sk >> 10) & 2047u, valid && (sk >> 21) == pre[s]);
+                else
+                    warp_hist_add(s_hist[s], sk & 1023u, valid && (sk >> 10) == pre[s]);
+            }
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kHistBins; i += kBlock) {
+        if (LEVEL == 0) {
+            const uint32_t v = s_hist[0][i];
+            if (v) {
+                atomicAdd(&P.hists->x[0][0][i], v);
+                atomicAdd(&P.hists->x[0][1][kHistBins - 1 - i], v);  // same counts, complemented key
+            }
+        } else {
+            for (int s = 0; s < 2; ++s) {
+                const uint32_t v = s_hist[s][i];
+                if (v) atomicAdd(&P.hists->x[LEVEL][s][i], v);
+            }
+        }
+    }
+    if (last_block_ticket(&ctl->done[ST_XH0 + LEVEL], gridDim.x)) {
+        for (int s = 0; s < 2; ++s) {
+            const uint32_t rank = (LEVEL == 0) ? (uint32_t)P.k : ctl->x_rank[s];
+            block_pick_desc(P.hists->x[LEVEL][s], kBins, false, rank, s_scan, &s_pick);
+            if (threadIdx.x == 0) {
+                const uint32_t prefix =
+                    (LEVEL == 0) ? s_pick.bin : ((pre[s] << (LEVEL == 1 ? 11 : 10)) | s_pick.bin);
+                ctl->x_prefix[s] = prefix;
+                ctl->x_rank[s] = s_pick.rank;
+                if (LEVEL == 2) {
+                    ctl->x_thr[s] = prefix;             // side key of the k-th entry
+                    ctl->x_ties_take[s] = s_pick.rank;  // equal entries to keep (lowest indices)
+                    ctl->x_ties_have[s] = s_pick.count;
+                    ctl->cand_cnt[s] = 0u;              // the lists are rebuilt from scratch
+                }
+                if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+__device__ __forceinline__ bool tie_ranks_needed(const Ctl* ctl, int s) {
+    return ctl->x_ties_take[s] < ctl->x_ties_have[s];
+}
+
+// Entries equal to the threshold, per tile of kXTile elements.
+__global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (!exact_route_active(ctl)) return;
+    if (!tie_ranks_needed(ctl, 0) && !tie_ranks_needed(ctl, 1)) return;
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    const uint32_t thr[2] = {ctl->x_thr[0], ctl->x_thr[1]};
+    const float* __restrict__ A = P.residual;
+    for (uint32_t tile = blockIdx.x; tile < P.n_xtiles; tile += gridDim.x) {
+        uint32_t c = 0u;  // side 0 in the low half, side 1 in the high half
+        for (int j = 0; j < kXTile / kBlock; ++j) {
+            const long long i = (long long)tile * kXTile + j * kBlock + threadIdx.x;
+            if (i < P.n) {
+                const uint32_t key = key_of_bits(__float_as_uint(A[i]));
+                c += (key == thr[0]) ? 1u : 0u;
+                c += (~key == thr[1]) ? 0x10000u : 0u;
+            }
+        }
+        uint32_t total;
+        block_exclusive_scan<uint32_t>(c, s_scan, &total);
+        if (threadIdx.x == 0) {
+            P.x_tile_cnt[0][tile] = total & 0xffffu;
+            P.x_tile_cnt[1][tile] = total >> 16;
+        }
+    }
+}
+
+// In-place exclusive scan of the per-tile tie counts (one block).
+__global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (!exact_route_active(ctl)) return;
+    if (!tie_ranks_needed(ctl, 0) && !tie_ranks_needed(ctl, 1)) return;
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    const uint32_t per = (P.n_xtiles + kBlock - 1) / kBlock;
+    for (int s = 0; s < 2; ++s) {
+        uint32_t* cnt = P.x_tile_cnt[s];
+        const uint32_t lo = threadIdx.x * per;
+        const uint32_t hi = min(lo + per, P.n_xtiles);
+        uint32_t sum = 0u;
+        for (uint32_t t = lo; t < hi; ++t) sum += cnt[t];
+        uint32_t run = block_exclusive_scan<uint32_t>(sum, s_scan, nullptr);
+        for (uint32_t t = lo; t < hi; ++t) {
+            const uint32_t v = cnt[t];
+            cnt[t] = run;
+            run += v;
+        }
+        __syncthreads();
+    }
+}
+
+// Gather exactly k composites per side: everything strictly beyond the
+// threshold plus the lowest-index ties.  Each warp owns 512 consecutive
+// elements of a tile and walks them 32 at a time, so the rank of a tie is
+// (ties in earlier tiles) + (earlier warps) + (earlier steps) + (lower lanes).
+__global__ void __launch_bounds__(kBlock) k_exact_collect(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (!exact_route_active(ctl)) return;
+    constexpr int kSteps = kXTile / kBlock;  // 16 steps of 32 lanes per warp
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ uint32_t s_warp_ties[2][kBlock / 32];
+    __shared__ uint32_t s_base[2];
+    const int warp = threadIdx.x >> 5, lane = lane_id();
+    const uint32_t thr[2] = {ctl->x_thr[0], ctl->x_thr[1]};
+    const uint32_t take[2] = {ctl->x_ties_take[0], ctl->x_ties_take[1]};
+    const bool ranked[2] = {tie_ranks_needed(ctl, 0), tie_ranks_needed(ctl, 1)};
+    const float* __restrict__ A = P.residual;
+    for (uint32_t tile = blockIdx.x; tile < P.n_xtiles; tile += gridDim.x) {
+        const long long wbase = (long long)tile * kXTile + (long long)warp * (kXTile / (kBlock / 32));
+        uint32_t key[kSteps];
+        unsigned inb = 0u;
+#pragma unroll
+        for (int j = 0; j < kSteps; ++j) {
+            const long long i = wbase + j * 32 + lane;
+            key[j] = 0u;
+            if (i < P.n) {
+                key[j] = key_of_bits(__float_as_uint(A[i]));
+                inb |= 1u << j;
+            }
+        }
+        unsigned emit[2] = {0u, 0u};
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            if (!ranked[s]) {
+#pragma unroll
+                for (int j = 0; j < kSteps; ++j)
+                    emit[s] |= ((inb >> j) & 1u) && (side_key(s, key[j]) >= thr[s]) ? (1u << j) : 0u;
+            } else {
+                uint32_t wt = 0u;
+#pragma unroll
+                for (int j = 0; j < kSteps; ++j)
+                    wt += __popc(__ballot_sync(0xffffffffu,
+                                               ((inb >> j) & 1u) && side_key(s, key[j]) == thr[s]));
+                if (lane == 0) s_warp_ties[s][warp] = wt;
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            if (!ranked[s]) continue;
+            uint32_t run = P.x_tile_cnt[s][tile];
+            for (int w = 0; w < warp; ++w) run += s_warp_ties[s][w];
+#pragma unroll
+            for (int j = 0; j < kSteps; ++j) {
+                const bool in = (inb >> j) & 1u;
+                const uint32_t sk = side_key(s, key[j]);
+                const unsigned tb = __ballot_sync(0xffffffffu, in && sk == thr[s]);
+                const uint32_t my_rank = run + __popc(tb & ((1u << lane) - 1u));
+                const bool keep = in && (sk > thr[s] || (sk == thr[s] && my_rank < take[s]));
+                emit[s] |= keep ? (1u << j) : 0u;
+                run += __popc(tb);
+            }
+        }
+        const uint32_t packed = (uint32_t)__popc(emit[0]) | ((uint32_t)__popc(emit[1]) << 16);
+        uint32_t total;
+        const uint32_t excl = block_exclusive_scan<uint32_t>(packed, s_scan, &total);
+        if (threadIdx.x == 0) {
+            s_base[0] = (total & 0xffffu) ? atomicAdd(&ctl->cand_cnt[0], total & 0xffffu) : 0u;
+            s_base[1] = (total >> 16) ? atomicAdd(&ctl->cand_cnt[1], total >> 16) : 0u;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            uint32_t pos = s_base[s] + (s ? (excl >> 16) : (excl & 0xffffu));
+#pragma unroll
+            for (int j = 0; j < kSteps; ++j) {
+                if ((emit[s] >> j) & 1u) {
+                    const long long i = wbase + j * 32 + lane;
+                    if (pos < P.cap) P.cand[s][pos] = make_composite(side_key(s, key[j]), (uint32_t)i);
+                    ++pos;
+                }
+            }
+        }
+        __syncthreads();  // s_base / s_warp_ties are reused by the next tile
+    }
+}
+
+}  // namespace sbc

@@ -1,0 +1,238 @@
+// Front half of sbc_encode: accumulate A = R + dW (Algorithm 1) and gather,
+// for each side, a candidate list that is guaranteed to contain the k
+// entries Algorithm 2's top_p selects.
+//
+// Fast route: bound both thresholds from a strided sample, then ONE pass over
+// the tensor writes A and appends everything at or beyond the bounds.
+// Exact route (taken when the bounds did not bracket k entries, e.g. heavy
+// ties or a sample that misrepresents the tensor): three radix-histogram
+// passes over A find both k-th keys exactly, a tie-rank pass orders equal
+// values by index, and a last pass gathers exactly k entries per side.
+#pragma once
+#include "sbc_common.cuh"
+#include "../../include/sbc.h"
+
+namespace sbc {
+
+// ---------------------------------------------------------------- sample
+
+__device__ __forceinline__ long long sample_element(const Prob& P, uint32_t i) {
+    if ((long long)P.m == P.n) return (long long)i;
+    const uint32_t seg = i >> 5, lane = i & 31u;
+    const unsigned long long n_lines = (unsigned long long)(P.n >> 5);
+    const unsigned long long n_seg = P.m >> 5;
+    return (long long)(((unsigned long long)seg * n_lines) / n_seg) * 32 + lane;
+}
+
+// Level 0: keys of the sampled A values, histogram of their top 11 bits; the
+// last block locates the bin of the target rank for each side.
+__global__ void __launch_bounds__(kBlock) k_sample0(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    __shared__ uint32_t s_hist[kHistBins];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ Pick s_pick;
+    for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
+    __syncthreads();
+    for (uint32_t base = blockIdx.x * kBlock; base < P.m; base += gridDim.x * kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const bool valid = i < P.m;
+        uint32_t key = 0u;
+        if (valid) {
+            const long long e = sample_element(P, i);
+            const float a = __fadd_rn(P.residual[e], P.update[e]);
+            key = key_of_bits(__float_as_uint(a));
+            P.sample_keys[i] = key;
+        }
+        warp_hist_add(s_hist, key >> 21, valid);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kHistBins; i += kBlock) {
+        const uint32_t v = s_hist[i];
+        if (v) atomicAdd(&P.hists->s0[i], v);
+    }
+    if (last_block_ticket(&ctl->done[ST_SAMPLE0], gridDim.x)) {
+        for (int s = 0; s < 2; ++s) {
+            block_pick_desc(P.hists->s0, kHistBins, s == 1, P.s_target[s], s_scan, &s_pick);
+            if (threadIdx.x == 0) {
+                ctl->s_bin0[s] = s_pick.bin;
+                ctl->s_rank[s] = s_pick.rank;
+                if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// Level 1: next 11 bits inside the located bins; the last block turns the
+// 22-bit prefixes into the two float bounds used by the candidate pass.
+__global__ void __launch_bounds__(kBlock) k_sample1(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    __shared__ uint32_t s_hist[2][kHistBins];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ Pick s_pick;
+    for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) (&s_hist[0][0])[i] = 0u;
+    __syncthreads();
+    const uint32_t bin0[2] = {ctl->s_bin0[0], ctl->s_bin0[1]};
+    for (uint32_t base = blockIdx.x * kBlock; base < P.m; base += gridDim.x * kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const bool valid = i < P.m;
+        const uint32_t key = valid ? P.sample_keys[i] : 0u;
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            const uint32_t sk = side_key(s, key);
+            warp_hist_add(s_hist[s], (sk >> 10) & 2047u, valid && (sk >> 21) == bin0[s]);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) {
+        const uint32_t v = (&s_hist[0][0])[i];
+        if (v) atomicAdd(&P.hists->s1[0][0] + i, v);
+    }
+    if (last_block_ticket(&ctl->done[ST_SAMPLE1], gridDim.x)) {
+        for (int s = 0; s < 2; ++s) {
+            block_pick_desc(P.hists->s1[s], kHistBins, false, ctl->s_rank[s], s_scan, &s_pick);
+            if (threadIdx.x == 0) {
+                const uint32_t lower = (bin0[s] << 21) | (s_pick.bin << 10);  // side key, low bits 0
+                if (s == 0) ctl->lo_f = __uint_as_float(bits_of_key(lower));
+                else        ctl->hi_f = __uint_as_float(bits_of_key(~lower));
+                if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// ---------------------------------------------------------------- accumulate + collect
+
+constexpr int kUnroll = 2;                    // float4 loads per array per thread per step
+constexpr int kPerThread = 4 * kUnroll;       // elements per thread per step
+constexpr int kWarpChunk = 32 * kPerThread;   // elements per warp per step
+constexpr int kStage = kWarpChunk;            // staged candidates per warp per side
+
+// The streaming pass: A = R + dW written over R (12 bytes per element), two
+// float compares per element, and a rare append of (key, index) composites
+// through per-warp shared-memory staging so that the global list counters see
+// one atomic per few hundred candidates.
+template <bool VEC>
+__global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    __shared__ unsigned long long s_stage[kBlock / 32][2][kStage];
+    const int warp = threadIdx.x >> 5, lane = lane_id();
+    const float lo = ctl->lo_f, hi = ctl->hi_f;
+    const long long n = P.n;
+    const float* __restrict__ U = P.update;
+    float* __restrict__ R = P.residual;
+    uint32_t wcnt[2] = {0u, 0u};
+    bool bad = false;
+
+    auto flush = [&](int s) {
+        if (wcnt[s] == 0u) return;  // warp-uniform
+        __syncwarp();
+        uint32_t base = 0u;
+        if (lane == 0) base = atomicAdd(&ctl->cand_cnt[s], wcnt[s]);
+        base = __shfl_sync(0xffffffffu, base, 0);
+        for (uint32_t i = lane; i < wcnt[s]; i += 32)
+            if (base + i < P.cap) P.cand[s][base + i] = s_stage[warp][s][i];
+        __syncwarp();
+        wcnt[s] = 0u;
+    };
+
+    const long long n_chunks = (n + kWarpChunk - 1) / kWarpChunk;
+    const long long total_warps = (long long)gridDim.x * (kBlock / 32);
+    for (long long chunk = (long long)blockIdx.x * (kBlock / 32) + warp; chunk < n_chunks;
+         chunk += total_warps) {
+        const long long base = chunk * kWarpChunk;
+        float a[kPerThread];
+        long long first[kUnroll];  // index of this thread's first element in each group
+        unsigned inb = 0u;
+        if (VEC) {
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) {
+                const long long e0 = base + (long long)(u * 32 + lane) * 4;
+                first[u] = e0;
+                if (e0 + 3 < n) {
+                    const float4 x = __ldcs(reinterpret_cast<const float4*>(U + e0));
+                    const float4 r = __ldcs(reinterpret_cast<const float4*>(R + e0));
+                    float4 y;
+                    y.x = __fadd_rn(r.x, x.x); y.y = __fadd_rn(r.y, x.y);
+                    y.z = __fadd_rn(r.z, x.z); y.w = __fadd_rn(r.w, x.w);
+                    __stcs(reinterpret_cast<float4*>(R + e0), y);
+                    a[4 * u + 0] = y.x; a[4 * u + 1] = y.y; a[4 * u + 2] = y.z; a[4 * u + 3] = y.w;
+                    inb |= 0xfu << (4 * u);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        a[4 * u + j] = 0.f;
+                        if (e0 + j < n) {
+                            a[4 * u + j] = __fadd_rn(R[e0 + j], U[e0 + j]);
+                            R[e0 + j] = a[4 * u + j];
+                            inb |= 1u << (4 * u + j);
+                        }
+                    }
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < kPerThread; ++j) {
+                const long long e = base + j * 32 + lane;
+                a[j] = 0.f;
+                if (e < n) {
+                    a[j] = __fadd_rn(R[e], U[e]);
+                    R[e] = a[j];
+                    inb |= 1u << j;
+                }
+            }
+            first[0] = base + lane;
+        }
+        unsigned pm = 0u, qm = 0u;
+#pragma unroll
+        for (int j = 0; j < kPerThread; ++j) {
+            pm |= (!(a[j] < lo) ? 1u : 0u) << j;   // also true for NaN
+            qm |= (!(a[j] > hi) ? 1u : 0u) << j;
+        }
+        pm &= inb;
+        qm &= inb;
+        if (__any_sync(0xffffffffu, (pm | qm) != 0u)) {
+            const uint32_t packed = (uint32_t)__popc(pm) | ((uint32_t)__popc(qm) << 16);
+            const uint32_t incl = warp_inclusive_scan(packed);
+            const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
+            const uint32_t excl = incl - packed;
+#pragma unroll
+            for (int s = 0; s < 2; ++s) {
+                const uint32_t tot_s = s ? (tot >> 16) : (tot & 0xffffu);
+                if (tot_s == 0u) continue;
+                if (wcnt[s] + tot_s > (uint32_t)kStage) flush(s);
+                uint32_t off = wcnt[s] + (s ? (excl >> 16) : (excl & 0xffffu));
+                const unsigned mask = s ? qm : pm;
+#pragma unroll
+                for (int j = 0; j < kPerThread; ++j) {
+                    if ((mask >> j) & 1u) {
+                        const uint32_t bits = __float_as_uint(a[j]);
+                        if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;
+                        const long long e = VEC ? first[j / 4] + (j % 4) : first[0] + j * 32;
+                        s_stage[warp][s][off++] =
+                            make_composite(side_key(s, key_of_bits(bits)), (uint32_t)e);
+                    }
+                }
+                wcnt[s] += tot_s;
+            }
+            __syncwarp();
+        }
+    }
+    flush(0);
+    flush(1);
+    if (bad) atomicOr(&ctl->status, SBC_STATUS_NONFINITE);
+
+    if (last_block_ticket(&ctl->done[ST_COLLECT], gridDim.x)) {
+        if (threadIdx.x == 0) {
+            const uint32_t c0 = __ldcg(&ctl->cand_cnt[0]), c1 = __ldcg(&ctl->cand_cnt[1]);
+            const bool ok = c0 >= (uint32_t)P.k && c0 <= P.cap && c1 >= (uint32_t)P.k && c1 <= P.cap;
+            ctl->use_fallback = ok ? 0u : 1u;
+        }
+    }
+}
+
+}  // namespace sbc

@@ -1,0 +1,217 @@
+// Golomb position coding (Algorithm 3) and decoding (Algorithm 4).
+//
+// Encode: kept-position bitmask -> ascending position list (popcount scan)
+// -> per-codeword lengths q + 1 + b -> exclusive scan = bit offsets ->
+// every codeword ORs its own bits into the pre-zeroed payload.
+// Decode: one thread per chunk of kChunkCodewords codewords, started from the
+// chunk table (bit offset, previous position), adds mu into the dense tensor.
+#pragma once
+#include "sbc_common.cuh"
+#include "../../include/sbc.h"
+
+namespace sbc {
+
+// ---------------------------------------------------------------- mask -> sorted positions
+
+__global__ void __launch_bounds__(kBlock) k_mask_count(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    if (P.ctl->status) return;
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    constexpr int kPer = kMaskTileWords / kBlock;  // 8 words per thread
+    for (uint32_t tile = blockIdx.x; tile < P.n_mask_tiles; tile += gridDim.x) {
+        uint32_t c = 0u;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t w = tile * kMaskTileWords + threadIdx.x * kPer + j;
+            if (w < P.n_mask_words) c += __popc(P.mask[w]);
+        }
+        uint32_t total;
+        block_exclusive_scan<uint32_t>(c, s_scan, &total);
+        if (threadIdx.x == 0) P.mask_tile_cnt[tile] = total;
+    }
+}
+
+__global__ void __launch_bounds__(kBlock) k_mask_scan(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (ctl->status) return;
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    const uint32_t per = (P.n_mask_tiles + kBlock - 1) / kBlock;
+    const uint32_t lo = threadIdx.x * per, hi = min(lo + per, P.n_mask_tiles);
+    uint32_t sum = 0u;
+    for (uint32_t t = lo; t < hi; ++t) sum += P.mask_tile_cnt[t];
+    uint32_t total;
+    uint32_t run = block_exclusive_scan<uint32_t>(sum, s_scan, &total);
+    for (uint32_t t = lo; t < hi; ++t) {
+        const uint32_t v = P.mask_tile_cnt[t];
+        P.mask_tile_cnt[t] = run;
+        run += v;
+    }
+    if (threadIdx.x == 0) {
+        ctl->kept_total = total;
+        if (total != (uint32_t)P.k) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+    }
+}
+
+__global__ void __launch_bounds__(kBlock) k_mask_compact(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    if (P.ctl->status) return;
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    constexpr int kPer = kMaskTileWords / kBlock;
+    for (uint32_t tile = blockIdx.x; tile < P.n_mask_tiles; tile += gridDim.x) {
+        uint32_t words[kPer];
+        uint32_t c = 0u;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t w = tile * kMaskTileWords + threadIdx.x * kPer + j;
+            words[j] = (w < P.n_mask_words) ? P.mask[w] : 0u;
+            c += __popc(words[j]);
+        }
+        uint32_t pos = P.mask_tile_cnt[tile] + block_exclusive_scan<uint32_t>(c, s_scan, nullptr);
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            uint32_t w = words[j];
+            const uint32_t first = (tile * kMaskTileWords + threadIdx.x * kPer + j) << 5;
+            while (w) {
+                const int bit = __ffs(w) - 1;
+                w &= w - 1u;
+                if (pos < (uint32_t)P.k) P.idx[pos] = first + bit;
+                ++pos;
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------- lengths, offsets, header
+
+__device__ __forceinline__ unsigned long long codeword_len(const Prob& P, uint32_t i, uint32_t* gap) {
+    const long long prev = i ? (long long)P.idx[i - 1] : -1ll;
+    const uint32_t g = (uint32_t)((long long)P.idx[i] - prev - 1);  // gap - 1 of Algorithm 3
+    *gap = g;
+    return (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
+}
+
+__global__ void __launch_bounds__(kBlock) k_len_sum(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    if (P.ctl->status) return;
+    __shared__ unsigned long long s_scan[kBlock / 32 + 1];
+    constexpr int kPer = kLenBlock / kBlock;
+    for (uint32_t blk = blockIdx.x; blk < P.n_len_blocks; blk += gridDim.x) {
+        unsigned long long sum = 0ull;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t i = blk * kLenBlock + threadIdx.x * kPer + j;
+            uint32_t g;
+            if (i < (uint32_t)P.k) sum += codeword_len(P, i, &g);
+        }
+        unsigned long long total;
+        block_exclusive_scan<unsigned long long>(sum, s_scan, &total);
+        if (threadIdx.x == 0) P.blk_len[blk] = total;
+    }
+}
+
+__device__ __forceinline__ void store_u32(uint8_t* p, uint32_t v) { *reinterpret_cast<uint32_t*>(p) = v; }
+__device__ __forceinline__ void store_u64(uint8_t* p, unsigned long long v) {
+    *reinterpret_cast<unsigned long long*>(p) = v;
+}
+
+// Scan of the per-block bit counts; also writes the container header, always,
+// so that a failed encode still leaves a header that says why.
+__global__ void __launch_bounds__(kBlock) k_len_scan_header(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    __shared__ unsigned long long s_scan[kBlock / 32 + 1];
+    const bool ok = ctl->status == 0u;  // uniform: nothing writes status while this kernel runs
+    unsigned long long total = 0ull;
+    if (ok) {
+        const uint32_t per = (P.n_len_blocks + kBlock - 1) / kBlock;
+        const uint32_t lo = threadIdx.x * per, hi = min(lo + per, P.n_len_blocks);
+        unsigned long long sum = 0ull;
+        for (uint32_t t = lo; t < hi; ++t) sum += P.blk_len[t];
+        unsigned long long run = block_exclusive_scan<unsigned long long>(sum, s_scan, &total);
+        for (uint32_t t = lo; t < hi; ++t) {
+            const unsigned long long v = P.blk_len[t];
+            P.blk_len[t] = run;
+            run += v;
+        }
+    }
+    if (threadIdx.x == 0) {
+        ctl->nbits = total;
+        uint8_t* h = P.stream;
+        store_u32(h + 0, SBC_MAGIC);
+        store_u32(h + 4, SBC_VERSION);
+        store_u64(h + 8, (unsigned long long)P.n);
+        store_u64(h + 16, ok ? (unsigned long long)P.k : 0ull);
+        store_u64(h + 24, total);
+        store_u64(h + 32, ok ? P.payload_offset : (unsigned long long)SBC_HEADER_BYTES);
+        store_u32(h + 40, (uint32_t)P.b);
+        store_u32(h + 44, ok ? ctl->side : 0u);
+        store_u32(h + 48, ok ? __float_as_uint(ctl->mu32) : 0u);
+        store_u32(h + 52, SBC_CHUNK_CODEWORDS);
+        store_u32(h + 56, ok ? P.n_chunks : 0u);
+        store_u32(h + 60, ctl->status);
+    }
+}
+
+// ---------------------------------------------------------------- bit packer
+
+// OR `count` (1..32) bits, given right-aligned in `value`, into the payload at
+// stream bit `off`.  Stream bit j lives in byte j/8 at bit 7-(j%8); a 32-bit
+// word assembled MSB-first is therefore stored byte-swapped.
+__device__ __forceinline__ void or_bits(uint32_t* words, unsigned long long off, int count,
+                                        uint32_t value) {
+    const unsigned long long w = off >> 5;
+    const int sh = (int)(off & 31ull);
+    const unsigned long long window = (unsigned long long)value << (64 - count - sh);
+    const uint32_t hi = (uint32_t)(window >> 32), lo = (uint32_t)window;
+    if (hi) atomicOr(words + w, __byte_perm(hi, 0u, 0x0123));
+    if (lo) atomicOr(words + w + 1, __byte_perm(lo, 0u, 0x0123));
+}
+
+__global__ void __launch_bounds__(kBlock) k_pack(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    if (P.ctl->status) return;
+    __shared__ unsigned long long s_scan[kBlock / 32 + 1];
+    constexpr int kPer = kLenBlock / kBlock;
+    uint32_t* words = reinterpret_cast<uint32_t*>(P.stream + P.payload_offset);
+    uint8_t* table = P.stream + SBC_HEADER_BYTES;
+    const int b = P.b;
+    for (uint32_t blk = blockIdx.x; blk < P.n_len_blocks; blk += gridDim.x) {
+        unsigned long long len[kPer];
+        uint32_t gap[kPer];
+        unsigned long long sum = 0ull;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t i = blk * kLenBlock + threadIdx.x * kPer + j;
+            len[j] = 0ull;
+            gap[j] = 0u;
+            if (i < (uint32_t)P.k) len[j] = codeword_len(P, i, &gap[j]);
+            sum += len[j];
+        }
+        unsigned long long off = P.blk_len[blk] + block_exclusive_scan<unsigned long long>(sum, s_scan, nullptr);
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t i = blk * kLenBlock + threadIdx.x * kPer + j;
+            if (i >= (uint32_t)P.k) continue;
+            if (i % kChunkCodewords == 0) {
+                uint8_t* e = table + (size_t)(i / kChunkCodewords) * SBC_CHUNK_ENTRY_BYTES;
+                store_u64(e, off);
+                store_u64(e + 8, (unsigned long long)(i ? (long long)P.idx[i - 1] : -1ll));
+            }
+            unsigned long long pos = off;
+            uint32_t q = gap[j] >> b;
+            // q ones: head up to a word boundary, whole words, then the rest
+            if (q) {
+                const int head = min((uint32_t)(32 - (int)(pos & 31ull)) & 31u, q);
+                if (head) { or_bits(words, pos, head, 0xffffffffu >> (32 - head)); pos += head; q -= head; }
+                while (q >= 32u) { words[pos >> 5] = 0xffffffffu; pos += 32; q -= 32u; }
+                if (q) { or_bits(words, pos, (int)q, 0xffffffffu >> (32 - q)); pos += q; }
+            }
+            // the terminating zero and r in b bits, MSB first: 1 + b <= 31 bits
+            or_bits(words, pos, 1 + b, gap[j] & ((1u << b) - 1u));
+            off += len[j];
+        }
+    }
+}
+
+}  // namespace sbc

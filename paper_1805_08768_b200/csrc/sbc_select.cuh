@@ -1,0 +1,248 @@
+// Exact k-th largest composite of each candidate list (Algorithm 2: exactly k
+// kept entries, equal values ordered by index), by MSB-first radix selection
+// with 11-bit digits over the 64-bit composites.  Each level keeps only the
+// entries that fall in the selected bucket, so the lists shrink quickly.
+// Then the exact sums, the two means, the side choice and mu (Algorithm 2),
+// and the residual write-back at the kept positions (Algorithm 1).
+#pragma once
+#include "sbc_common.cuh"
+#include "../../include/sbc.h"
+
+namespace sbc {
+
+__device__ __forceinline__ int digit_shift(int level) { return level < 5 ? 53 - 11 * level : 0; }
+__device__ __forceinline__ int digit_bits(int level) { return level < 5 ? 11 : 9; }
+__device__ __forceinline__ uint32_t digit_of(unsigned long long c, int level) {
+    return (uint32_t)(c >> digit_shift(level)) & ((1u << digit_bits(level)) - 1u);
+}
+
+// Histogram of the top digit over a whole candidate list.  grid.z = side.
+__global__ void __launch_bounds__(kBlock) k_select_hist0(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (ctl->status) return;
+    const int s = blockIdx.z;
+    __shared__ uint32_t s_hist[kHistBins];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ Pick s_pick;
+    for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
+    __syncthreads();
+    const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
+    const unsigned long long* __restrict__ src = P.cand[s];
+    for (uint32_t base = blockIdx.x * kBlock; base < cnt; base += gridDim.x * kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const bool valid = i < cnt;
+        const unsigned long long c = valid ? src[i] : 0ull;
+        warp_hist_add(s_hist, digit_of(c, 0), valid);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kHistBins; i += kBlock) {
+        const uint32_t v = s_hist[i];
+        if (v) atomicAdd(&P.hists->b[0][s][i], v);
+    }
+    if (last_block_ticket(&ctl->done[ST_BH0_S0 + s], gridDim.x)) {
+        block_pick_desc(P.hists->b[0][s], kHistBins, false, (uint32_t)P.k, s_scan, &s_pick);
+        if (threadIdx.x == 0) {
+            ctl->b_prefix[s] = s_pick.bin;
+            ctl->b_rank[s] = s_pick.rank;
+            if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+        }
+    }
+}
+
+// Keep the entries whose level-L digit is the selected one, histogram their
+// next digit, and let the last block select at level L+1.  grid.z = side.
+template <int LEVEL>
+__global__ void __launch_bounds__(kBlock) k_select_filter(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (ctl->status) return;
+    const int s = blockIdx.z;
+    constexpr int kItems = 4;
+    __shared__ uint32_t s_hist[kHistBins];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ uint32_t s_base;
+    __shared__ Pick s_pick;
+    for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
+    __syncthreads();
+    const uint32_t cnt = (LEVEL == 0) ? min(ctl->cand_cnt[s], P.cap) : ctl->list_cnt[s][LEVEL];
+    const unsigned long long* __restrict__ src = (LEVEL == 0) ? P.cand[s] : P.buf[s][(LEVEL - 1) & 1];
+    unsigned long long* __restrict__ dst = P.buf[s][LEVEL & 1];
+    const uint32_t sel = (uint32_t)ctl->b_prefix[s] & ((1u << digit_bits(LEVEL)) - 1u);
+    for (uint32_t base = blockIdx.x * (kBlock * kItems); base < cnt; base += gridDim.x * (kBlock * kItems)) {
+        unsigned long long c[kItems];
+        unsigned match = 0u;
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const uint32_t i = base + j * kBlock + threadIdx.x;
+            c[j] = (i < cnt) ? src[i] : 0ull;
+            const bool m = (i < cnt) && digit_of(c[j], LEVEL) == sel;
+            match |= m ? (1u << j) : 0u;
+            warp_hist_add(s_hist, digit_of(c[j], LEVEL + 1), m);
+        }
+        uint32_t total;
+        const uint32_t excl = block_exclusive_scan<uint32_t>((uint32_t)__popc(match), s_scan, &total);
+        if (threadIdx.x == 0) s_base = total ? atomicAdd(&ctl->list_cnt[s][LEVEL + 1], total) : 0u;
+        __syncthreads();
+        uint32_t pos = s_base + excl;
+#pragma unroll
+        for (int j = 0; j < kItems; ++j)
+            if ((match >> j) & 1u) { if (pos < P.cap) dst[pos] = c[j]; ++pos; }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < kHistBins; i += kBlock) {
+        const uint32_t v = s_hist[i];
+        if (v) atomicAdd(&P.hists->b[LEVEL + 1][s][i], v);
+    }
+    if (last_block_ticket(&ctl->done[ST_BF0_S0 + 2 * LEVEL + s], gridDim.x)) {
+        block_pick_desc(P.hists->b[LEVEL + 1][s], 1 << digit_bits(LEVEL + 1), false,
+                        ctl->b_rank[s], s_scan, &s_pick);
+        if (threadIdx.x == 0) {
+            const unsigned long long prefix =
+                (ctl->b_prefix[s] << digit_bits(LEVEL + 1)) | (unsigned long long)s_pick.bin;
+            ctl->b_prefix[s] = prefix;
+            ctl->b_rank[s] = s_pick.rank;
+            if (LEVEL + 1 == 5) ctl->thr[s] = prefix;  // the k-th largest composite itself
+            if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+        }
+    }
+}
+
+// ---------------------------------------------------------------- exact sums, means, side
+
+// Round the exact integer sum_s bins[s] * 2^s (units of 2^-149) to fp64,
+// nearest-even.  One thread.
+__device__ double bins_to_double(const long long* bins) {
+    unsigned long long acc[6] = {0, 0, 0, 0, 0, 0};  // 384-bit two's complement
+    for (int s = 0; s < kSumBins; ++s) {
+        const long long v = __ldcg(bins + s);
+        if (v == 0) continue;
+        const int limb = s >> 6, off = s & 63;
+        unsigned long long part[3];
+        part[0] = (unsigned long long)v << off;
+        part[1] = off ? (unsigned long long)(v >> (64 - off)) : (v < 0 ? ~0ull : 0ull);
+        part[2] = v < 0 ? ~0ull : 0ull;
+        unsigned long long carry = 0;
+        for (int l = limb; l < 6; ++l) {
+            const unsigned long long add = part[min(l - limb, 2)];
+            const unsigned long long t = acc[l] + add;
+            const unsigned long long c1 = t < add;
+            const unsigned long long t2 = t + carry;
+            const unsigned long long c2 = t2 < carry;
+            acc[l] = t2;
+            carry = c1 | c2;
+        }
+    }
+    const bool neg = (acc[5] >> 63) != 0;
+    if (neg) {
+        unsigned long long carry = 1;
+        for (int l = 0; l < 6; ++l) {
+            acc[l] = ~acc[l] + carry;
+            carry = (carry && acc[l] == 0) ? 1 : 0;
+        }
+    }
+    int top = -1;
+    for (int l = 5; l >= 0; --l)
+        if (acc[l]) { top = l * 64 + 63 - __clzll((long long)acc[l]); break; }
+    if (top < 0) return 0.0;
+    // shift right so that bit `top` lands on bit 52, tracking round and sticky bits
+    const int drop = top - 52;
+    unsigned long long sig = 0;
+    bool round_bit = false, sticky = false;
+    if (drop <= 0) {
+        sig = acc[0] << (-drop);  // top <= 52: everything sits in limb 0
+    } else {
+        const int limb = drop >> 6, off = drop & 63;
+        const unsigned long long lo = acc[limb];
+        const unsigned long long hi = (limb + 1 < 6) ? acc[limb + 1] : 0ull;
+        sig = off ? ((lo >> off) | (hi << (64 - off))) : lo;
+        sig &= (1ull << 53) - 1ull;
+        const int rpos = drop - 1;
+        round_bit = (acc[rpos >> 6] >> (rpos & 63)) & 1ull;
+        for (int l = 0; l < (rpos >> 6); ++l) sticky |= acc[l] != 0;
+        if (rpos & 63) sticky |= (acc[rpos >> 6] & ((1ull << (rpos & 63)) - 1ull)) != 0;
+    }
+    if (round_bit && (sticky || (sig & 1ull))) sig += 1ull;
+    const double mag = scalbn((double)sig, drop - 149);  // sig <= 2^53: exact
+    return neg ? -mag : mag;
+}
+
+// Sum the kept values of both lists exactly: a value is m * 2^(e-150) with an
+// integer m of at most 24 bits, so one 64-bit integer per exponent holds the
+// sum of up to 2^39 of them and integer addition makes the result independent
+// of the order of the atomics.  grid.z = side.  The last block turns the bins
+// into mu+ and mu- and takes Algorithm 2's side decision.
+__global__ void __launch_bounds__(kBlock) k_sums_decide(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (ctl->status) return;
+    const int s = blockIdx.z;
+    __shared__ unsigned long long s_bins[256];
+    s_bins[threadIdx.x] = 0ull;
+    __syncthreads();
+    const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
+    const unsigned long long thr = ctl->thr[s];
+    const unsigned long long* __restrict__ src = P.cand[s];
+    const int lane = lane_id();
+    for (uint32_t base = blockIdx.x * kBlock; base < cnt; base += gridDim.x * kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const unsigned long long c = (i < cnt) ? src[i] : 0ull;
+        const bool kept = (i < cnt) && c >= thr;
+        const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
+        const uint32_t e = (bits >> 23) & 0xffu;
+        int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
+        if (bits >> 31) m = -m;
+        const int bin = e ? (int)e - 1 : 0;
+        unsigned todo = __ballot_sync(0xffffffffu, kept);
+        while (todo) {
+            const int leader = __ffs(todo) - 1;
+            const int lbin = __shfl_sync(0xffffffffu, bin, leader);
+            const bool same = kept && bin == lbin;
+            const int part = __reduce_add_sync(0xffffffffu, same ? m : 0);
+            if (lane == leader) atomicAdd(&s_bins[lbin], (unsigned long long)(long long)part);
+            todo &= ~__ballot_sync(0xffffffffu, same);
+        }
+    }
+    __syncthreads();
+    {
+        const unsigned long long v = s_bins[threadIdx.x];
+        if (v) atomicAdd(reinterpret_cast<unsigned long long*>(&ctl->bins[s][threadIdx.x]), v);
+    }
+    if (last_block_ticket(&ctl->done[ST_SUM], gridDim.x * gridDim.z)) {
+        if (threadIdx.x == 0) {
+            const double kd = (double)P.k;
+            const double mu_pos = bins_to_double(ctl->bins[0]) / kd;
+            const double mu_neg = -bins_to_double(ctl->bins[1]) / kd;  // val- holds negated entries
+            const uint32_t side = (mu_pos >= mu_neg) ? 0u : 1u;
+            const float mu = side ? (float)(-mu_neg) : (float)mu_pos;
+            ctl->mu64[0] = mu_pos;
+            ctl->mu64[1] = mu_neg;
+            ctl->side = side;
+            ctl->mu32 = mu;
+            if (P.out_mu) *P.out_mu = mu;
+        }
+    }
+}
+
+// R_j = A_j - mu at the kept positions of the chosen side, and one mask bit per
+// kept position for the ordered compaction that follows.
+__global__ void __launch_bounds__(kBlock) k_apply(const Prob* __restrict__ probs) {
+    const Prob& P = probs[blockIdx.y];
+    Ctl* ctl = P.ctl;
+    if (ctl->status) return;
+    const int s = (int)ctl->side;
+    const float mu = ctl->mu32;
+    const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
+    const unsigned long long thr = ctl->thr[s];
+    const unsigned long long* __restrict__ src = P.cand[s];
+    for (uint32_t i = blockIdx.x * kBlock + threadIdx.x; i < cnt; i += gridDim.x * kBlock) {
+        const unsigned long long c = src[i];
+        if (c >= thr) {
+            const uint32_t idx = composite_index(c);
+            P.residual[idx] = __fsub_rn(P.residual[idx], mu);
+            atomicOr(&P.mask[idx >> 5], 1u << (idx & 31u));
+        }
+    }
+}
+
+}  // namespace sbc

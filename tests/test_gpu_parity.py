@@ -1,0 +1,243 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI.
+
+Bar: kept index sets, side, Golomb bit strings and the whole container
+byte-exact; mu bit-identical (both sides round the exact sum once); residual
+bit-identical (same fp32 operations); decoded aggregate within
+1e-6 * sum_c |mu_c| per element (the order of fp32 atomic adds is free).
+"""
+import zlib
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1805_08768_b200 import binding as sbc
+from paper_1805_08768_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():  # pragma: no cover - the CPU box deselects with -m "not gpu"
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+DEV = torch.device("cuda:0")
+
+
+def gpu_encode(upd: np.ndarray, res: np.ndarray, p: float, offset_elems: int = 0):
+    """Run sbc_encode on device copies; returns (stream bytes, mu, new residual, info)."""
+    n = upd.size
+    if offset_elems:  # deliberately misaligned views (4-byte aligned only)
+        ubuf = torch.zeros(n + offset_elems + 4, dtype=torch.float32, device=DEV)
+        rbuf = torch.zeros(n + offset_elems + 4, dtype=torch.float32, device=DEV)
+        u = ubuf[offset_elems:offset_elems + n]
+        r = rbuf[offset_elems:offset_elems + n]
+        u.copy_(torch.from_numpy(upd))
+        r.copy_(torch.from_numpy(res))
+    else:
+        u = torch.from_numpy(upd).to(DEV)
+        r = torch.from_numpy(res).to(DEV)
+    cap = sbc.sbc_stream_bytes(n, p)
+    out = torch.full((cap + 64,), 0xAB, dtype=torch.uint8, device=DEV)   # canary behind the capacity
+    ws_bytes = sbc.sbc_workspace_bytes(n, p)
+    ws = torch.full((ws_bytes + 256,), 0xCD, dtype=torch.uint8, device=DEV)
+    mu = torch.full((1,), float("nan"), dtype=torch.float32, device=DEV)
+    sbc.sbc_encode(u, r, p, out_stream=out[:cap], out_mu=mu, workspace=ws[:ws_bytes])
+    info = sbc.sbc_stream_info_get(out)
+    torch.cuda.synchronize()
+    assert bool((out[cap:] == 0xAB).all()), "write past the stream capacity"
+    assert bool((ws[ws_bytes:] == 0xCD).all()), "write past the workspace"
+    stream = out[: info.total_bytes].cpu().numpy()
+    return stream, np.float32(mu.item()), r.cpu().numpy(), info, out
+
+
+def check_against_oracle(upd, res, p, offset_elems=0):
+    want_res = res.copy()
+    want_stream, want_mu = oracle.encode(upd, want_res, p)
+    stream, mu, got_res, info, _ = gpu_encode(upd, res, p, offset_elems)
+    h = oracle.parse_header(want_stream)
+    assert (info.k, info.b, info.side, info.nbits) == (h.k, h.b, h.side, h.nbits)
+    assert mu.view(np.uint32) == want_mu.view(np.uint32), (mu, want_mu)
+    assert stream.size == want_stream.size
+    assert np.array_equal(stream, want_stream)
+    assert np.array_equal(got_res.view(np.uint32), want_res.view(np.uint32))
+    return stream, mu
+
+
+@pytest.mark.parametrize("name,upd,res,p", workloads.adversarial_cases(),
+                         ids=[c[0] for c in workloads.adversarial_cases()])
+def test_encode_adversarial_cases(name, upd, res, p):
+    check_against_oracle(upd, res, p)
+
+
+def test_config1_round_trip():
+    n, p = 2**20, 0.01
+    upd = workloads.normal_flat(n, 1e-3, workloads.seed_for(1))
+    res = np.zeros(n, dtype=np.float32)
+    stream, mu = check_against_oracle(upd, res, p)
+    # decode into a zeroed dense tensor = the binarised update
+    want = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate([stream], want)
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sbc.sbc_decode_accumulate([torch.from_numpy(stream).to(DEV)], dense, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert np.array_equal(dense.cpu().numpy(), want)      # one client: exact
+    assert np.count_nonzero(want) == oracle.kept_count(n, p)
+
+
+@pytest.mark.parametrize("n", [1, 2, 31, 32, 33, 255, 257, 1023, 4095, 4097, 65537, 300001, 1500007])
+@pytest.mark.parametrize("p", [0.01, 0.001])
+def test_encode_ragged_sizes(n, p):
+    rng = np.random.default_rng(n)
+    upd = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    res = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    check_against_oracle(upd, res, p)
+
+
+@pytest.mark.parametrize("offset", [1, 2, 3])
+def test_encode_misaligned_pointers(offset):
+    rng = np.random.default_rng(offset)
+    n = 70001
+    upd = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    res = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    check_against_oracle(upd, res, 0.01, offset_elems=offset)
+
+
+@pytest.mark.parametrize("dist", ["student_t", "laplace", "uniform", "lognormal_signed"])
+@pytest.mark.parametrize("p", [0.1, 0.01, 1e-3, 1e-4])
+def test_encode_distributions(dist, p):
+    rng = np.random.default_rng(zlib.crc32(f"{dist}:{p}".encode()))
+    n = 1 << 21                      # above the sample size: the bounds come from a strided sample
+    if dist == "student_t":
+        upd = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
+    elif dist == "laplace":
+        upd = rng.laplace(0, 1e-3, n).astype(np.float32)
+    elif dist == "uniform":
+        upd = rng.uniform(-1, 1, n).astype(np.float32)
+    else:
+        upd = (np.exp(rng.standard_normal(n) * 3) * rng.choice([-1.0, 1.0], n)).astype(np.float32)
+    check_against_oracle(upd, np.zeros(n, dtype=np.float32), p)
+
+
+def test_unrepresentative_sample_takes_the_exact_route():
+    # large values only where the strided sample does not look, plus a block of ties
+    n = (1 << 21) + 12345
+    rng = np.random.default_rng(42)
+    upd = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    upd[5::64] = 7.0           # many equal large values: ties at the positive threshold
+    upd[9::128] = -9.0
+    check_against_oracle(upd, np.zeros(n, dtype=np.float32), 0.01)
+    sparse = np.zeros(n, dtype=np.float32)                     # fewer non-zeros than k
+    sparse[rng.choice(n, 1000, replace=False)] = rng.standard_normal(1000).astype(np.float32)
+    check_against_oracle(sparse, np.zeros(n, dtype=np.float32), 0.01)
+
+
+def test_multi_round_residual_carry():
+    n, p = 250000, 0.001
+    res_gpu = np.zeros(n, dtype=np.float32)
+    res_cpu = np.zeros(n, dtype=np.float32)
+    for rnd in range(4):
+        upd = workloads.normal_flat(n, 1e-3, workloads.seed_for(2, rnd))
+        want_stream, want_mu = oracle.encode(upd, res_cpu, p)
+        stream, mu, res_gpu, _, _ = gpu_encode(upd, res_gpu, p)
+        assert np.array_equal(stream, want_stream) and mu == want_mu
+        assert np.array_equal(res_gpu.view(np.uint32), res_cpu.view(np.uint32))
+
+
+def test_encode_is_deterministic():
+    n, p = 1 << 20, 0.01
+    upd = workloads.student_t_flat(n, 77)
+    a = gpu_encode(upd, np.zeros(n, dtype=np.float32), p)
+    b = gpu_encode(upd, np.zeros(n, dtype=np.float32), p)
+    assert np.array_equal(a[0], b[0]) and a[1] == b[1] and np.array_equal(a[2], b[2])
+
+
+def test_decode_aggregate_eight_clients():
+    n, p = 400000, 0.001
+    streams_np, dev_streams, mus = [], [], []
+    for c in range(8):
+        upd = workloads.normal_flat(n, 1e-3, workloads.seed_for(4, 0, c))
+        stream, mu, _, _, _ = gpu_encode(upd, np.zeros(n, dtype=np.float32), p)
+        streams_np.append(stream)
+        dev_streams.append(torch.from_numpy(stream).to(DEV))
+        mus.append(abs(float(mu)))
+    want = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate(streams_np, want)
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sbc.sbc_decode_accumulate(dev_streams, dense, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    got = dense.cpu().numpy()
+    assert np.array_equal(got != 0, want != 0)
+    assert np.max(np.abs(got.astype(np.float64) - want)) <= 1e-6 * sum(mus)
+    # adds onto existing contents, and more than one launch worth of clients
+    dense.fill_(1.0)
+    sbc.sbc_decode_accumulate(dev_streams * 5, dense)
+    torch.cuda.synchronize()
+    want5 = np.ones(n, dtype=np.float64) + 5.0 * want.astype(np.float64)
+    assert np.max(np.abs(dense.cpu().numpy() - want5)) <= 1e-6 * (1 + 5 * sum(mus))
+
+
+def test_non_finite_input_is_reported_not_encoded():
+    n = 100000
+    upd = workloads.normal_flat(n, 1e-3, 5)
+    upd[777] = np.inf
+    u = torch.from_numpy(upd).to(DEV)
+    r = torch.zeros(n, dtype=torch.float32, device=DEV)
+    out, _ = sbc.sbc_encode(u, r, 0.01)
+    info = sbc.sbc_stream_info_get(out, check=False)
+    assert info.status & sbc.STATUS_NONFINITE
+    with pytest.raises(sbc.SbcError):
+        sbc.sbc_stream_info_get(out)
+    assert np.array_equal(r.cpu().numpy().view(np.uint32), upd.view(np.uint32))  # residual holds A
+    # the decoder refuses a stream whose header carries an error
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sbc.sbc_decode_accumulate([out], dense, status=status)
+    torch.cuda.synchronize()
+    assert status.item() & sbc.STATUS_CORRUPT and not bool(dense.any())
+
+
+def test_corrupt_streams_set_status_and_stay_in_bounds():
+    n, p = 200000, 0.01
+    upd = workloads.normal_flat(n, 1e-3, 6)
+    stream, _, _, info, _ = gpu_encode(upd, np.zeros(n, dtype=np.float32), p)
+    guard = 4096
+
+    def run(mutated: np.ndarray):
+        dense = torch.zeros(n + guard, dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        sbc.sbc_decode_accumulate([torch.from_numpy(mutated).to(DEV)], dense[:n], status=status)
+        torch.cuda.synchronize()
+        assert not bool(dense[n:].any()), "decoder wrote outside the tensor"
+        return status.item()
+
+    assert run(stream) == 0
+    bad = stream.copy(); bad[0] ^= 1                 # magic
+    assert run(bad) & sbc.STATUS_CORRUPT
+    bad = stream.copy(); bad[8:16].view("<u8")[0] = n + 1   # numel mismatch
+    assert run(bad) & sbc.STATUS_CORRUPT
+    bad = stream.copy(); bad[info.payload_offset:] = 0xFF    # endless unary runs
+    assert run(bad) != 0
+    bad = stream.copy(); bad[info.payload_offset:info.payload_offset + 64] = 0xFF
+    assert run(bad) != 0                                      # positions run past numel
+    bad = stream.copy(); bad[64:72].view("<u8")[0] = 2**40    # chunk table offset outside the payload
+    assert run(bad) & sbc.STATUS_CORRUPT
+
+
+def test_argument_errors_are_returned_at_once():
+    n = 1000
+    u = torch.zeros(n, dtype=torch.float32, device=DEV)
+    r = torch.zeros(n, dtype=torch.float32, device=DEV)
+    with pytest.raises(sbc.SbcError) as e:
+        sbc.sbc_encode(u, r, 1.5, out_stream=torch.empty(4096, dtype=torch.uint8, device=DEV),
+                       workspace=torch.empty(1 << 20, dtype=torch.uint8, device=DEV))
+    assert e.value.code == sbc.SBC_EINVAL
+    with pytest.raises(sbc.SbcError) as e:
+        sbc.sbc_encode(u, r, 0.01, out_stream=torch.empty(16, dtype=torch.uint8, device=DEV))
+    assert e.value.code == sbc.SBC_ECAPACITY
+    with pytest.raises(sbc.SbcError) as e:
+        sbc.sbc_encode(u, u, 0.01)                      # aliasing
+    assert e.value.code == sbc.SBC_EINVAL

@@ -206,9 +206,9 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     const dim3 blk(kBlock);
 
     // scratch that must start at zero: control block + histograms, the kept
-    // mask, and the chunk table + payload area the packer ORs into
+    // mask and its per-tile counts (adjacent in the workspace), and the chunk table + payload area the packer ORs into
     if (cudaMemsetAsync(ws + pl.zero_begin, 0, pl.zero_end - pl.zero_begin, st) != cudaSuccess ||
-        cudaMemsetAsync(P.mask, 0, (size_t)pl.n_mask_words * 4, st) != cudaSuccess ||
+        cudaMemsetAsync(P.mask, 0, pl.off_mask_tile + (size_t)pl.n_mask_tiles * 4 - pl.off_mask, st) != cudaSuccess ||
         cudaMemsetAsync(P.stream + SBC_HEADER_BYTES, 0, pl.stream_bytes - SBC_HEADER_BYTES, st) != cudaSuccess)
         return SBC_ECUDA;
     k_put_prob<<<1, 1, 0, st>>>(dP, P);
@@ -218,7 +218,7 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     k_sample0<<<dim3(g_sample), blk, 0, st>>>(dP);
     k_sample1<<<dim3(g_sample), blk, 0, st>>>(dP);
     mark(SBC_MARK_BOUNDS);
-    const unsigned g_main = grid_for((unsigned long long)pl.n, kBlock * kPerThread * 2, sms * 6);
+    const unsigned g_main = grid_for((unsigned long long)pl.n, kBlock * kPerThread, sms * kCollectBlocksPerSM);
     if (P.vec_ok) k_add_collect<true><<<dim3(g_main), blk, 0, st>>>(dP);
     else          k_add_collect<false><<<dim3(g_main), blk, 0, st>>>(dP);
 
@@ -245,13 +245,12 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     k_select_filter<3><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
     k_select_filter<4><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
     k_sums_decide<<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_apply<<<dim3(g_c), blk, 0, st>>>(dP);
+    k_mark<<<dim3(g_c), blk, 0, st>>>(dP);
 
     mark(SBC_MARK_SELECT);
 
     // 4. Golomb stage
     const unsigned g_m = grid_for(pl.n_mask_tiles, 1, sms * 8);
-    k_mask_count<<<dim3(g_m), blk, 0, st>>>(dP);
     k_mask_scan<<<dim3(1), blk, 0, st>>>(dP);
     k_mask_compact<<<dim3(g_m), blk, 0, st>>>(dP);
     const unsigned g_l = grid_for(pl.n_len_blocks, 1, sms * 8);
@@ -263,7 +262,7 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
-int sbc_encode_launches(void) { return 24; }  // put_prob, 2 sample, 1 collect, 6 exact, 8 select, 6 Golomb
+int sbc_encode_launches(void) { return 23; }  // put_prob, 2 sample, 1 collect, 6 exact, 8 select, 5 Golomb
 
 int sbc_decode_launches(int n_clients) {
     return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;

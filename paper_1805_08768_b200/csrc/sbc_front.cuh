@@ -106,15 +106,17 @@ __global__ void __launch_bounds__(kBlock) k_sample1(const Prob* __restrict__ pro
 
 // ---------------------------------------------------------------- accumulate + collect
 
-constexpr int kUnroll = 2;                    // float4 loads per array per thread per step
+constexpr int kUnroll = 4;                    // float4 loads per array per thread per step
 constexpr int kPerThread = 4 * kUnroll;       // elements per thread per step
 constexpr int kWarpChunk = 32 * kPerThread;   // elements per warp per step
-constexpr int kStage = kWarpChunk;            // staged candidates per warp per side
+constexpr int kStage = 128;                   // staged candidates per warp per side
+constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 warps, 128 B in flight per thread)
 
 // The streaming pass: A = R + dW written over R (12 bytes per element), two
 // float compares per element, and a rare append of (key, index) composites
 // through per-warp shared-memory staging so that the global list counters see
-// one atomic per few hundred candidates.
+// one atomic per hundred or so candidates.  Each thread has eight 16-byte
+// loads in flight before it touches any of them.
 template <bool VEC>
 __global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__ probs) {
     const Prob& P = probs[blockIdx.y];
@@ -146,35 +148,26 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__
          chunk += total_warps) {
         const long long base = chunk * kWarpChunk;
         float a[kPerThread];
-        long long first[kUnroll];  // index of this thread's first element in each group
         unsigned inb = 0u;
-        if (VEC) {
+        const bool vec_layout = VEC && (base + kWarpChunk <= n);  // warp-uniform
+        if (vec_layout) {
+            // thread owns elements base + (u*32 + lane)*4 + {0..3}, u = 0..kUnroll-1
+            const float4* __restrict__ u4 = reinterpret_cast<const float4*>(U + base) + lane;
+            float4* __restrict__ r4 = reinterpret_cast<float4*>(R + base) + lane;
+            float4 x[kUnroll], r[kUnroll];
+#pragma unroll
+            for (int u = 0; u < kUnroll; ++u) { x[u] = __ldcs(u4 + u * 32); r[u] = __ldcs(r4 + u * 32); }
 #pragma unroll
             for (int u = 0; u < kUnroll; ++u) {
-                const long long e0 = base + (long long)(u * 32 + lane) * 4;
-                first[u] = e0;
-                if (e0 + 3 < n) {
-                    const float4 x = __ldcs(reinterpret_cast<const float4*>(U + e0));
-                    const float4 r = __ldcs(reinterpret_cast<const float4*>(R + e0));
-                    float4 y;
-                    y.x = __fadd_rn(r.x, x.x); y.y = __fadd_rn(r.y, x.y);
-                    y.z = __fadd_rn(r.z, x.z); y.w = __fadd_rn(r.w, x.w);
-                    __stcs(reinterpret_cast<float4*>(R + e0), y);
-                    a[4 * u + 0] = y.x; a[4 * u + 1] = y.y; a[4 * u + 2] = y.z; a[4 * u + 3] = y.w;
-                    inb |= 0xfu << (4 * u);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        a[4 * u + j] = 0.f;
-                        if (e0 + j < n) {
-                            a[4 * u + j] = __fadd_rn(R[e0 + j], U[e0 + j]);
-                            R[e0 + j] = a[4 * u + j];
-                            inb |= 1u << (4 * u + j);
-                        }
-                    }
-                }
+                float4 y;
+                y.x = __fadd_rn(r[u].x, x[u].x); y.y = __fadd_rn(r[u].y, x[u].y);
+                y.z = __fadd_rn(r[u].z, x[u].z); y.w = __fadd_rn(r[u].w, x[u].w);
+                __stcs(r4 + u * 32, y);
+                a[4 * u + 0] = y.x; a[4 * u + 1] = y.y; a[4 * u + 2] = y.z; a[4 * u + 3] = y.w;
             }
+            inb = (1u << kPerThread) - 1u;
         } else {
+            // ragged tail or unaligned pointers: thread owns elements base + j*32 + lane
 #pragma unroll
             for (int j = 0; j < kPerThread; ++j) {
                 const long long e = base + j * 32 + lane;
@@ -185,7 +178,6 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__
                     inb |= 1u << j;
                 }
             }
-            first[0] = base + lane;
         }
         unsigned pm = 0u, qm = 0u;
 #pragma unroll
@@ -205,19 +197,31 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__
                 const uint32_t tot_s = s ? (tot >> 16) : (tot & 0xffffu);
                 if (tot_s == 0u) continue;
                 if (wcnt[s] + tot_s > (uint32_t)kStage) flush(s);
-                uint32_t off = wcnt[s] + (s ? (excl >> 16) : (excl & 0xffffu));
+                // more candidates in one step than the stage holds (dense ties): straight to the list
+                const bool direct = tot_s > (uint32_t)kStage;
+                uint32_t off = s ? (excl >> 16) : (excl & 0xffffu);
+                if (direct) {
+                    uint32_t gbase = 0u;
+                    if (lane == 0) gbase = atomicAdd(&ctl->cand_cnt[s], tot_s);
+                    off += __shfl_sync(0xffffffffu, gbase, 0);
+                } else {
+                    off += wcnt[s];
+                    wcnt[s] += tot_s;
+                }
                 const unsigned mask = s ? qm : pm;
 #pragma unroll
                 for (int j = 0; j < kPerThread; ++j) {
                     if ((mask >> j) & 1u) {
                         const uint32_t bits = __float_as_uint(a[j]);
                         if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;
-                        const long long e = VEC ? first[j / 4] + (j % 4) : first[0] + j * 32;
-                        s_stage[warp][s][off++] =
-                            make_composite(side_key(s, key_of_bits(bits)), (uint32_t)e);
+                        const long long e = vec_layout ? base + (long long)(((j >> 2) * 32 + lane) * 4 + (j & 3))
+                                                       : base + j * 32 + lane;
+                        const unsigned long long c = make_composite(side_key(s, key_of_bits(bits)), (uint32_t)e);
+                        if (direct) { if (off < P.cap) P.cand[s][off] = c; }
+                        else s_stage[warp][s][off] = c;
+                        ++off;
                     }
                 }
-                wcnt[s] += tot_s;
             }
             __syncwarp();
         }

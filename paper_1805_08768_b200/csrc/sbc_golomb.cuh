@@ -13,69 +13,73 @@ namespace sbc {
 
 // ---------------------------------------------------------------- mask -> sorted positions
 
-__global__ void __launch_bounds__(kBlock) k_mask_count(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
-    if (P.ctl->status) return;
-    __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    constexpr int kPer = kMaskTileWords / kBlock;  // 8 words per thread
-    for (uint32_t tile = blockIdx.x; tile < P.n_mask_tiles; tile += gridDim.x) {
-        uint32_t c = 0u;
-#pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            const uint32_t w = tile * kMaskTileWords + threadIdx.x * kPer + j;
-            if (w < P.n_mask_words) c += __popc(P.mask[w]);
-        }
-        uint32_t total;
-        block_exclusive_scan<uint32_t>(c, s_scan, &total);
-        if (threadIdx.x == 0) P.mask_tile_cnt[tile] = total;
-    }
-}
-
+// In-place exclusive scan of the kept-position counts per mask tile (one block).
 __global__ void __launch_bounds__(kBlock) k_mask_scan(const Prob* __restrict__ probs) {
     const Prob& P = probs[blockIdx.y];
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    const uint32_t per = (P.n_mask_tiles + kBlock - 1) / kBlock;
-    const uint32_t lo = threadIdx.x * per, hi = min(lo + per, P.n_mask_tiles);
-    uint32_t sum = 0u;
-    for (uint32_t t = lo; t < hi; ++t) sum += P.mask_tile_cnt[t];
-    uint32_t total;
-    uint32_t run = block_exclusive_scan<uint32_t>(sum, s_scan, &total);
-    for (uint32_t t = lo; t < hi; ++t) {
-        const uint32_t v = P.mask_tile_cnt[t];
-        P.mask_tile_cnt[t] = run;
-        run += v;
+    constexpr int kPer = 8;
+    uint32_t carry = 0u;
+    for (uint32_t base = 0; base < P.n_mask_tiles; base += kBlock * kPer) {
+        uint32_t v[kPer];
+        uint32_t sum = 0u;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t t = base + threadIdx.x * kPer + j;
+            v[j] = (t < P.n_mask_tiles) ? P.mask_tile_cnt[t] : 0u;
+            sum += v[j];
+        }
+        uint32_t total;
+        uint32_t run = carry + block_exclusive_scan<uint32_t>(sum, s_scan, &total);
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t t = base + threadIdx.x * kPer + j;
+            if (t < P.n_mask_tiles) P.mask_tile_cnt[t] = run;
+            run += v[j];
+        }
+        carry += total;
     }
     if (threadIdx.x == 0) {
-        ctl->kept_total = total;
-        if (total != (uint32_t)P.k) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+        ctl->kept_total = carry;
+        if (carry != (uint32_t)P.k) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
     }
 }
 
+// Mask -> ascending position list, and the residual write-back R_j = A_j - mu
+// (Algorithm 1) at those positions, walked in address order.
 __global__ void __launch_bounds__(kBlock) k_mask_compact(const Prob* __restrict__ probs) {
     const Prob& P = probs[blockIdx.y];
     if (P.ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    static_assert(kMaskTileWords / kBlock == 8, "eight words per thread");
     constexpr int kPer = kMaskTileWords / kBlock;
+    const float mu = P.ctl->mu32;
     for (uint32_t tile = blockIdx.x; tile < P.n_mask_tiles; tile += gridDim.x) {
         uint32_t words[kPer];
         uint32_t c = 0u;
+        const uint32_t w0 = tile * kMaskTileWords + threadIdx.x * kPer;
+        if (w0 + kPer <= P.n_mask_words) {
+            const uint4 lo = *reinterpret_cast<const uint4*>(P.mask + w0);
+            const uint4 hi = *reinterpret_cast<const uint4*>(P.mask + w0 + 4);
+            words[0] = lo.x; words[1] = lo.y; words[2] = lo.z; words[3] = lo.w;
+            words[4] = hi.x; words[5] = hi.y; words[6] = hi.z; words[7] = hi.w;
+        } else {
 #pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            const uint32_t w = tile * kMaskTileWords + threadIdx.x * kPer + j;
-            words[j] = (w < P.n_mask_words) ? P.mask[w] : 0u;
-            c += __popc(words[j]);
+            for (int j = 0; j < kPer; ++j) words[j] = (w0 + j < P.n_mask_words) ? P.mask[w0 + j] : 0u;
         }
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) c += __popc(words[j]);
         uint32_t pos = P.mask_tile_cnt[tile] + block_exclusive_scan<uint32_t>(c, s_scan, nullptr);
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             uint32_t w = words[j];
-            const uint32_t first = (tile * kMaskTileWords + threadIdx.x * kPer + j) << 5;
+            const uint32_t first = (w0 + j) << 5;
             while (w) {
-                const int bit = __ffs(w) - 1;
+                const uint32_t idx = first + (__ffs(w) - 1);
                 w &= w - 1u;
-                if (pos < (uint32_t)P.k) P.idx[pos] = first + bit;
+                if (pos < (uint32_t)P.k) P.idx[pos] = idx;
+                P.residual[idx] = __fsub_rn(P.residual[idx], mu);
                 ++pos;
             }
         }
@@ -124,15 +128,25 @@ __global__ void __launch_bounds__(kBlock) k_len_scan_header(const Prob* __restri
     const bool ok = ctl->status == 0u;  // uniform: nothing writes status while this kernel runs
     unsigned long long total = 0ull;
     if (ok) {
-        const uint32_t per = (P.n_len_blocks + kBlock - 1) / kBlock;
-        const uint32_t lo = threadIdx.x * per, hi = min(lo + per, P.n_len_blocks);
-        unsigned long long sum = 0ull;
-        for (uint32_t t = lo; t < hi; ++t) sum += P.blk_len[t];
-        unsigned long long run = block_exclusive_scan<unsigned long long>(sum, s_scan, &total);
-        for (uint32_t t = lo; t < hi; ++t) {
-            const unsigned long long v = P.blk_len[t];
-            P.blk_len[t] = run;
-            run += v;
+        constexpr int kPer = 8;
+        for (uint32_t base = 0; base < P.n_len_blocks; base += kBlock * kPer) {
+            unsigned long long v[kPer];
+            unsigned long long sum = 0ull;
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const uint32_t t = base + threadIdx.x * kPer + j;
+                v[j] = (t < P.n_len_blocks) ? P.blk_len[t] : 0ull;
+                sum += v[j];
+            }
+            unsigned long long part;
+            unsigned long long run = total + block_exclusive_scan<unsigned long long>(sum, s_scan, &part);
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const uint32_t t = base + threadIdx.x * kPer + j;
+                if (t < P.n_len_blocks) P.blk_len[t] = run;
+                run += v[j];
+            }
+            total += part;
         }
     }
     if (threadIdx.x == 0) {

@@ -115,7 +115,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Prob* __restrict
 __device__ double bins_to_double(const long long* bins) {
     unsigned long long acc[6] = {0, 0, 0, 0, 0, 0};  // 384-bit two's complement
     for (int s = 0; s < kSumBins; ++s) {
-        const long long v = __ldcg(bins + s);
+        const long long v = bins[s];
         if (v == 0) continue;
         const int limb = s >> 6, off = s & 63;
         unsigned long long part[3];
@@ -177,46 +177,59 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Prob* __restrict__
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
-    __shared__ unsigned long long s_bins[256];
-    s_bins[threadIdx.x] = 0ull;
+    __shared__ unsigned long long s_bins[2][256];
+    s_bins[0][threadIdx.x] = 0ull;
     __syncthreads();
     const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
     const unsigned long long thr = ctl->thr[s];
     const unsigned long long* __restrict__ src = P.cand[s];
-    const int lane = lane_id();
-    for (uint32_t base = blockIdx.x * kBlock; base < cnt; base += gridDim.x * kBlock) {
-        const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < cnt) ? src[i] : 0ull;
-        const bool kept = (i < cnt) && c >= thr;
+    // Almost every kept value shares the exponent of the threshold value or the
+    // next one up: those two bins are summed in registers, the rest goes
+    // straight to the shared bins.
+    const uint32_t thr_bits = bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
+    const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
+    const int bin_b = bin_a + 1;
+    long long acc_a = 0, acc_b = 0;
+    for (uint32_t i = blockIdx.x * kBlock + threadIdx.x; i < cnt; i += gridDim.x * kBlock) {
+        const unsigned long long c = src[i];
+        if (c < thr) continue;
         const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
         const uint32_t e = (bits >> 23) & 0xffu;
         int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
         if (bits >> 31) m = -m;
         const int bin = e ? (int)e - 1 : 0;
-        unsigned todo = __ballot_sync(0xffffffffu, kept);
-        while (todo) {
-            const int leader = __ffs(todo) - 1;
-            const int lbin = __shfl_sync(0xffffffffu, bin, leader);
-            const bool same = kept && bin == lbin;
-            const int part = __reduce_add_sync(0xffffffffu, same ? m : 0);
-            if (lane == leader) atomicAdd(&s_bins[lbin], (unsigned long long)(long long)part);
-            todo &= ~__ballot_sync(0xffffffffu, same);
-        }
+        if (bin == bin_a) acc_a += m;
+        else if (bin == bin_b) acc_b += m;
+        else atomicAdd(&s_bins[0][bin], (unsigned long long)(long long)m);
+    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) {
+        acc_a += __shfl_down_sync(0xffffffffu, acc_a, d);
+        acc_b += __shfl_down_sync(0xffffffffu, acc_b, d);
+    }
+    if (lane_id() == 0) {
+        if (acc_a) atomicAdd(&s_bins[0][bin_a], (unsigned long long)acc_a);
+        if (acc_b && bin_b < kSumBins) atomicAdd(&s_bins[0][bin_b], (unsigned long long)acc_b);
     }
     __syncthreads();
     {
-        const unsigned long long v = s_bins[threadIdx.x];
+        const unsigned long long v = s_bins[0][threadIdx.x];
         if (v) atomicAdd(reinterpret_cast<unsigned long long*>(&ctl->bins[s][threadIdx.x]), v);
     }
     if (last_block_ticket(&ctl->done[ST_SUM], gridDim.x * gridDim.z)) {
+        s_bins[0][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[0][threadIdx.x]);
+        s_bins[1][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[1][threadIdx.x]);
+        __syncthreads();
+        if (threadIdx.x < 2) {  // one thread per side rounds its exact sum
+            const double sum = bins_to_double(reinterpret_cast<const long long*>(s_bins[threadIdx.x]));
+            ctl->mu64[threadIdx.x] = threadIdx.x ? -sum / (double)P.k : sum / (double)P.k;
+        }
+        __syncthreads();
         if (threadIdx.x == 0) {
-            const double kd = (double)P.k;
-            const double mu_pos = bins_to_double(ctl->bins[0]) / kd;
-            const double mu_neg = -bins_to_double(ctl->bins[1]) / kd;  // val- holds negated entries
+            const double mu_pos = ctl->mu64[0];
+            const double mu_neg = ctl->mu64[1];  // val- holds the negated entries
             const uint32_t side = (mu_pos >= mu_neg) ? 0u : 1u;
             const float mu = side ? (float)(-mu_neg) : (float)mu_pos;
-            ctl->mu64[0] = mu_pos;
-            ctl->mu64[1] = mu_neg;
             ctl->side = side;
             ctl->mu32 = mu;
             if (P.out_mu) *P.out_mu = mu;
@@ -224,23 +237,30 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Prob* __restrict__
     }
 }
 
-// R_j = A_j - mu at the kept positions of the chosen side, and one mask bit per
-// kept position for the ordered compaction that follows.
-__global__ void __launch_bounds__(kBlock) k_apply(const Prob* __restrict__ probs) {
+// One mask bit per kept position of the chosen side (for the ordered
+// compaction that follows) and the number of kept positions per mask tile.
+__global__ void __launch_bounds__(kBlock) k_mark(const Prob* __restrict__ probs) {
     const Prob& P = probs[blockIdx.y];
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = (int)ctl->side;
-    const float mu = ctl->mu32;
     const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
     const unsigned long long thr = ctl->thr[s];
     const unsigned long long* __restrict__ src = P.cand[s];
-    for (uint32_t i = blockIdx.x * kBlock + threadIdx.x; i < cnt; i += gridDim.x * kBlock) {
-        const unsigned long long c = src[i];
-        if (c >= thr) {
-            const uint32_t idx = composite_index(c);
-            P.residual[idx] = __fsub_rn(P.residual[idx], mu);
-            atomicOr(&P.mask[idx >> 5], 1u << (idx & 31u));
+    constexpr int kTileShift = 16;  // kMaskTileWords * 32 = 65536 positions per tile
+    static_assert(kMaskTileWords * 32 == (1 << kTileShift), "tile size");
+    for (uint32_t base = blockIdx.x * kBlock; base < cnt; base += gridDim.x * kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const unsigned long long c = (i < cnt) ? src[i] : 0ull;
+        const bool kept = (i < cnt) && c >= thr;
+        const uint32_t idx = composite_index(c);
+        if (kept) atomicOr(&P.mask[idx >> 5], 1u << (idx & 31u));
+        // neighbours in the list are neighbours in the tensor: one counter update per tile per warp
+        const unsigned active = __ballot_sync(0xffffffffu, kept);
+        if (kept) {
+            const uint32_t tile = idx >> kTileShift;
+            const unsigned peers = __match_any_sync(active, tile);
+            if ((int)lane_id() == __ffs(peers) - 1) atomicAdd(&P.mask_tile_cnt[tile], (uint32_t)__popc(peers));
         }
     }
 }

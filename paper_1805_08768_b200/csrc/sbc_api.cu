@@ -254,7 +254,7 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     k_mask_scan<<<dim3(1), blk, 0, st>>>(dP);
     k_mask_compact<<<dim3(g_m), blk, 0, st>>>(dP);
     const unsigned g_l = grid_for(pl.n_len_blocks, 1, sms * 8);
-    k_len_sum<<<dim3(g_l), blk, 0, st>>>(dP);
+    k_len_sum_residual<<<dim3(g_l), blk, 0, st>>>(dP);
     k_len_scan_header<<<dim3(1), blk, 0, st>>>(dP);
     k_pack<<<dim3(g_l), blk, 0, st>>>(dP);
     mark(SBC_MARK_END);
@@ -363,11 +363,12 @@ int sbc_decode_accumulate(const void* const* streams, int n_clients, float* out_
         a.out = out_dense;
         a.n = numel;
         a.status = status_dev;
-        // at most ceil(numel / 256) chunks per client
-        const unsigned long long max_items =
-            (unsigned long long)a.n_clients * (unsigned long long)((numel + kChunkCodewords - 1) / kChunkCodewords);
-        const unsigned grid = grid_for(max_items, 128, sms * 16);
-        k_decode_accumulate<<<grid, 128, 0, stream>>>(a);
+        // at most ceil(numel / 256) chunks per client, 32 chunks per warp, two warps per block
+        const unsigned long long max_groups =
+            (unsigned long long)a.n_clients *
+            (unsigned long long)((numel + kChunkCodewords * 32 - 1) / (kChunkCodewords * 32));
+        const unsigned grid = grid_for(max_groups, kDecodeThreads / 32, sms * 5);
+        k_decode_accumulate<<<grid, kDecodeThreads, 0, stream>>>(a);
     }
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }

@@ -38,10 +38,60 @@ __device__ __forceinline__ uint32_t peek32(const StreamView& v, unsigned long lo
     return __funnelshift_l(lo, hi, sh);
 }
 
-__global__ void __launch_bounds__(128) k_decode_accumulate(const DecodeArgs args) {
+constexpr int kDecodeThreads = 64;            // two warps per block
+constexpr int kDecodeWarpWords = 5632;        // staged payload words per warp (22 KB)
+
+// Sequential MSB-first bit reader over a warp's staged (byte-swapped) words, or over global memory when the group's payload did not fit the stage.
+// `cur` holds the next 64 - (32 - avail) ... bits left-aligned: bits [63, 64-avail)
+// are valid; one word is always fetched ahead so that its latency is hidden.
+struct BitReader {
+    const uint32_t* sw;
+    const StreamView* v;
+    unsigned long long first_word;  // stream word index of sw[0]
+    uint32_t n_staged;
+    bool staged;
+    unsigned long long cur;   // unread bits, left-aligned
+    int avail;                // valid bits in cur (>= 32 after every refill)
+    unsigned long long next_index;  // stream word index of `ahead`
+    uint32_t ahead;           // word already fetched, not yet in cur
+
+    __device__ __forceinline__ uint32_t fetch(unsigned long long w) const {
+        if (staged) {
+            const unsigned long long r = w - first_word;
+            return (r < n_staged) ? sw[r] : 0u;
+        }
+        return (w < v->n_words) ? __byte_perm(__ldg(v->words + w), 0u, 0x0123) : 0u;
+    }
+    __device__ __forceinline__ void start(unsigned long long pos) {
+        const unsigned long long w = pos >> 5;
+        const int sh = (int)(pos & 31ull);
+        cur = (((unsigned long long)fetch(w) << 32) | (unsigned long long)fetch(w + 1)) << sh;
+        avail = 64 - sh;
+        next_index = w + 2;
+        ahead = fetch(next_index);
+    }
+    __device__ __forceinline__ uint32_t top32() const { return (uint32_t)(cur >> 32); }
+    __device__ __forceinline__ void skip(int count) {  // count <= 32 <= avail
+        cur <<= count;
+        avail -= count;
+        if (avail <= 32) {
+            cur |= (unsigned long long)ahead << (32 - avail);
+            avail += 32;
+            ++next_index;
+            ahead = fetch(next_index);
+        }
+    }
+};
+
+// One warp per group of 32 consecutive chunks: the group's payload is one
+// contiguous bit range, copied once (coalesced) into shared memory; then every
+// lane parses its chunk's kChunkCodewords codewords from there (Algorithm 4)
+// and adds mu at each position (Algorithm 1, server sum).
+__global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate(const DecodeArgs args) {
     __shared__ StreamView s_view[kMaxClientsPerLaunch];
-    __shared__ uint32_t s_first[kMaxClientsPerLaunch + 1];  // first work item of each client
-    const int tid = threadIdx.x;
+    __shared__ uint32_t s_first[kMaxClientsPerLaunch + 1];  // first work item (group) of each client
+    __shared__ uint32_t s_words[kDecodeThreads / 32][kDecodeWarpWords];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid < args.n_clients) {
         const uint8_t* h = args.streams[tid];
         StreamView v;
@@ -71,54 +121,130 @@ __global__ void __launch_bounds__(128) k_decode_accumulate(const DecodeArgs args
     __syncthreads();
     if (tid == 0) {
         uint32_t run = 0u;
-        for (int c = 0; c < args.n_clients; ++c) { s_first[c] = run; run += s_view[c].n_chunks; }
+        for (int c = 0; c < args.n_clients; ++c) { s_first[c] = run; run += (s_view[c].n_chunks + 31u) / 32u; }
         s_first[args.n_clients] = run;
     }
     __syncthreads();
     const uint32_t total = s_first[args.n_clients];
-    for (uint32_t item = blockIdx.x * blockDim.x + tid; item < total; item += gridDim.x * blockDim.x) {
+    const uint32_t warps_total = gridDim.x * (kDecodeThreads / 32);
+    uint32_t* sw = s_words[warp];
+    for (uint32_t item = blockIdx.x * (kDecodeThreads / 32) + warp; item < total; item += warps_total) {
         int c = 0;
         while (item >= s_first[c + 1]) ++c;
         const StreamView& v = s_view[c];
-        const uint32_t chunk = item - s_first[c];
-        const uint8_t* e = v.table + (size_t)chunk * SBC_CHUNK_ENTRY_BYTES;
+        const uint32_t chunk0 = (item - s_first[c]) * 32u;
+        const uint32_t chunk = chunk0 + lane;
+        const bool has = chunk < v.n_chunks;
+        const uint8_t* e = v.table + (size_t)(has ? chunk : chunk0) * SBC_CHUNK_ENTRY_BYTES;
         unsigned long long pos = load_u64(e);
         long long prev = (long long)load_u64(e + 8);
-        const unsigned long long first_cw = (unsigned long long)chunk * kChunkCodewords;
-        const uint32_t count = (uint32_t)min((unsigned long long)kChunkCodewords, v.k - first_cw);
+        // bit range of the whole group: from its first chunk to the next group's first chunk
+        const unsigned long long gbeg = __shfl_sync(0xffffffffu, pos, 0);
+        const uint32_t chunk_end = min(chunk0 + 32u, v.n_chunks);
+        const unsigned long long gend =
+            (chunk_end < v.n_chunks) ? load_u64(v.table + (size_t)chunk_end * SBC_CHUNK_ENTRY_BYTES) : v.nbits;
         uint32_t err = 0u;
-        if (pos >= v.nbits || prev < -1 || prev >= args.n) err = SBC_STATUS_CORRUPT;
-        for (uint32_t i = 0; i < count && !err; ++i) {
-            // unary part: count ones up to the first zero
-            unsigned long long q = 0ull;
-            while (true) {
-                const uint32_t ones = __clz(~peek32(v, pos));  // 32 when the window is all ones
-                q += ones;
-                pos += ones;
-                if (ones < 32u) break;
-                if (pos >= v.nbits) { err = SBC_STATUS_CORRUPT; break; }
-            }
-            if (err) break;
-            pos += 1ull;  // the zero
-            const uint32_t r = v.b ? (peek32(v, pos) >> (32 - v.b)) : 0u;
-            pos += v.b;
-            if (pos > v.nbits) { err = SBC_STATUS_CORRUPT; break; }
-            const unsigned long long step = (q << v.b) + r + 1ull;
-            if (q > (unsigned long long)args.n || (unsigned long long)(args.n - 1 - prev) < step) {
-                err = SBC_STATUS_RANGE;
-                break;
-            }
-            prev += (long long)step;
-            atomicAdd(args.out + prev, v.mu);
+        const bool range_ok = gbeg <= gend && gend <= v.nbits;  // warp-uniform
+        if (!range_ok) err = SBC_STATUS_CORRUPT;
+        const unsigned long long first_word = gbeg >> 5;
+        const unsigned long long n_group_words = range_ok ? ((gend + 31ull) >> 5) - first_word : 0ull;
+        const bool staged = range_ok && n_group_words + 2ull <= (unsigned long long)kDecodeWarpWords;
+        const uint32_t n_staged = staged ? (uint32_t)n_group_words : 0u;
+        __syncwarp();
+        // asynchronous 4-byte copies: all of the group's words are in flight at once
+        for (uint32_t i = lane; i < n_staged; i += 32) {
+            const uint32_t dst = (uint32_t)__cvta_generic_to_shared(sw + i);
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(v.words + first_word + i));
         }
-        if (!err) {
-            // the chunk must end exactly where the table says the next one starts
-            if (chunk + 1u < v.n_chunks) {
-                if (load_u64(e + SBC_CHUNK_ENTRY_BYTES) != pos ||
-                    (long long)load_u64(e + SBC_CHUNK_ENTRY_BYTES + 8) != prev)
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        // MSB-first words for the parser, and two zero words so that a 96-bit read never leaves the stage
+        for (uint32_t i = lane; i < n_staged; i += 32) sw[i] = __byte_perm(sw[i], 0u, 0x0123);
+        if (staged && lane < 2) sw[n_staged + lane] = 0u;
+        __syncwarp();
+        if (has && !err) {
+            const unsigned long long first_cw = (unsigned long long)chunk * kChunkCodewords;
+            const uint32_t count = (uint32_t)min((unsigned long long)kChunkCodewords, v.k - first_cw);
+            if (pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n) err = SBC_STATUS_CORRUPT;
+            const uint32_t b = v.b;
+            const float mu = v.mu;
+            if (staged) {
+                // Fast path: bit positions relative to the stage fit 32 bits; every codeword
+                // is cut out of a 64-bit window rebuilt from three staged words.
+                uint32_t rel = (uint32_t)(pos - (first_word << 5));
+                const uint32_t rel_end = (uint32_t)(gend - (first_word << 5));
+                for (uint32_t i = 0; i < count; ++i) {
+                    if (rel >= rel_end) { err = SBC_STATUS_CORRUPT; break; }
+                    uint32_t w = rel >> 5;
+                    int sh = (int)(rel & 31u);
+                    uint32_t hi = __funnelshift_l(sw[w + 1], sw[w], sh);
+                    uint32_t lo = __funnelshift_l(sw[w + 2], sw[w + 1], sh);
+                    uint32_t ones = __clz(~hi);
+                    unsigned long long q = ones;
+                    while (ones == 32u) {  // rare: a run of 32 or more ones
+                        rel += 32u;
+                        if (rel >= rel_end) break;
+                        w = rel >> 5;
+                        hi = __funnelshift_l(sw[w + 1], sw[w], sh);
+                        lo = __funnelshift_l(sw[w + 2], sw[w + 1], sh);
+                        ones = __clz(~hi);
+                        q += ones;
+                    }
+                    if (rel >= rel_end) { err = SBC_STATUS_CORRUPT; break; }
+                    const unsigned long long win = ((unsigned long long)hi << 32) | (unsigned long long)lo;
+                    const uint32_t r = b ? (uint32_t)((win << (ones + 1u)) >> (64u - b)) : 0u;
+                    rel += ones + 1u + b;
+                    const unsigned long long step = (q << b) + r + 1ull;
+                    if (q > (unsigned long long)args.n || (unsigned long long)(args.n - 1 - prev) < step) {
+                        err = SBC_STATUS_RANGE;
+                        break;
+                    }
+                    prev += (long long)step;
+                    atomicAdd(args.out + prev, mu);
+                }
+                pos = (first_word << 5) + rel;
+            } else {
+                // Long unary runs made the group larger than the stage: read global memory.
+                BitReader br;
+                br.sw = sw; br.v = &v; br.first_word = first_word; br.n_staged = 0u; br.staged = false;
+                br.start(pos);
+                const unsigned long long room = v.nbits - pos;  // no codeword of this chunk may reach past it
+                unsigned long long used = 0ull;
+                for (uint32_t i = 0; i < count; ++i) {
+                    uint32_t ones = __clz(~br.top32());
+                    unsigned long long q = ones;
+                    while (ones == 32u) {
+                        br.skip(32);
+                        used += 32ull;
+                        if (used > room) break;
+                        ones = __clz(~br.top32());
+                        q += ones;
+                    }
+                    if (used > room) { err = SBC_STATUS_CORRUPT; break; }
+                    br.skip((int)ones + 1);  // the rest of the ones and the zero
+                    const uint32_t r = b ? (br.top32() >> (32 - b)) : 0u;
+                    br.skip((int)b);
+                    used += ones + 1u + b;
+                    const unsigned long long step = (q << b) + r + 1ull;
+                    if (q > (unsigned long long)args.n || (unsigned long long)(args.n - 1 - prev) < step) {
+                        err = SBC_STATUS_RANGE;
+                        break;
+                    }
+                    prev += (long long)step;
+                    atomicAdd(args.out + prev, mu);
+                }
+                if (!err && used > room) err = SBC_STATUS_CORRUPT;
+                pos += used;
+            }
+            if (!err) {
+                // the chunk must end exactly where the table says the next one starts
+                if (chunk + 1u < v.n_chunks) {
+                    if (load_u64(e + SBC_CHUNK_ENTRY_BYTES) != pos ||
+                        (long long)load_u64(e + SBC_CHUNK_ENTRY_BYTES + 8) != prev)
+                        err = SBC_STATUS_CORRUPT;
+                } else if (pos != v.nbits) {
                     err = SBC_STATUS_CORRUPT;
-            } else if (pos != v.nbits) {
-                err = SBC_STATUS_CORRUPT;
+                }
             }
         }
         if (err && args.status) atomicOr(args.status, err);

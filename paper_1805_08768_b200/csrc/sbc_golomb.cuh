@@ -46,15 +46,13 @@ __global__ void __launch_bounds__(kBlock) k_mask_scan(const Prob* __restrict__ p
     }
 }
 
-// Mask -> ascending position list, and the residual write-back R_j = A_j - mu
-// (Algorithm 1) at those positions, walked in address order.
+// Mask -> ascending position list.
 __global__ void __launch_bounds__(kBlock) k_mask_compact(const Prob* __restrict__ probs) {
     const Prob& P = probs[blockIdx.y];
     if (P.ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     static_assert(kMaskTileWords / kBlock == 8, "eight words per thread");
     constexpr int kPer = kMaskTileWords / kBlock;
-    const float mu = P.ctl->mu32;
     for (uint32_t tile = blockIdx.x; tile < P.n_mask_tiles; tile += gridDim.x) {
         uint32_t words[kPer];
         uint32_t c = 0u;
@@ -79,7 +77,6 @@ __global__ void __launch_bounds__(kBlock) k_mask_compact(const Prob* __restrict_
                 const uint32_t idx = first + (__ffs(w) - 1);
                 w &= w - 1u;
                 if (pos < (uint32_t)P.k) P.idx[pos] = idx;
-                P.residual[idx] = __fsub_rn(P.residual[idx], mu);
                 ++pos;
             }
         }
@@ -95,18 +92,34 @@ __device__ __forceinline__ unsigned long long codeword_len(const Prob& P, uint32
     return (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
 }
 
-__global__ void __launch_bounds__(kBlock) k_len_sum(const Prob* __restrict__ probs) {
+// Bits of each block of kLenBlock codewords, and -- since this is the first
+// walk over the ordered position list -- the residual write-back
+// R_j = A_j - mu at the kept positions (Algorithm 1), in address order.
+__global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Prob* __restrict__ probs) {
     const Prob& P = probs[blockIdx.y];
     if (P.ctl->status) return;
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     constexpr int kPer = kLenBlock / kBlock;
+    const float mu = P.ctl->mu32;
+    const uint32_t k = (uint32_t)P.k;
     for (uint32_t blk = blockIdx.x; blk < P.n_len_blocks; blk += gridDim.x) {
+        const uint32_t i0 = blk * kLenBlock + threadIdx.x * kPer;
+        uint32_t pos[kPer];
+        float r[kPer];
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) pos[j] = (i0 + j < k) ? P.idx[i0 + j] : 0u;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) r[j] = (i0 + j < k) ? P.residual[pos[j]] : 0.f;
+        long long prev = (i0 && i0 < k) ? (long long)P.idx[i0 - 1] : -1ll;
         unsigned long long sum = 0ull;
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
-            const uint32_t i = blk * kLenBlock + threadIdx.x * kPer + j;
-            uint32_t g;
-            if (i < (uint32_t)P.k) sum += codeword_len(P, i, &g);
+            if (i0 + j < k) {
+                P.residual[pos[j]] = __fsub_rn(r[j], mu);
+                const uint32_t g = (uint32_t)((long long)pos[j] - prev - 1);
+                sum += (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
+                prev = pos[j];
+            }
         }
         unsigned long long total;
         block_exclusive_scan<unsigned long long>(sum, s_scan, &total);

@@ -150,6 +150,36 @@ def run_reference(args):
 
 # ------------------------------------------------------------------ our arm
 
+# DRAM traffic of one k_add_collect launch from the ncu capture summarised in
+# profiles/k_add_collect_2p26_ncu_full.md: (536.93 + 225.39) MB at 2^26 elements, p = 1e-2.
+# Traffic is proportional to the element count, so it is scaled by numel / 2^26.  Valid only for
+# the kernel source it was taken from: a different hash of the file reports null.
+NCU_TRAFFIC_BYTES_AT_2P26 = 762.32e6
+NCU_TRAFFIC_SOURCE_SHA256 = "4353e0316d569b6791d5f74546ddfe74a17da3dc4f9339e8d8586bf04367a59d"
+
+
+def measured_traffic(numel: int):
+    import hashlib
+    path = os.path.join(ROOT, "paper_1805_08768_b200", "csrc", "sbc_front.cuh")
+    try:
+        with open(path, "rb") as fh:
+            if hashlib.sha256(fh.read()).hexdigest() != NCU_TRAFFIC_SOURCE_SHA256:
+                return None
+    except OSError:
+        return None
+    return NCU_TRAFFIC_BYTES_AT_2P26 * numel / float(1 << 26)
+
+
+def reduce_max_over_ranks(value: float, dist, device) -> float:
+    """Max of a per-rank scalar over all ranks (the slowest rank sets the job's time)."""
+    if dist is None:
+        return value
+    import torch
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
 def load_peak():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -241,10 +271,7 @@ def run_ours(args):
             stage_ms[i][s] += marks[s].elapsed_time(marks[s + 1])
         collect_ms_all.append(marks[sbc.MARK_BOUNDS].elapsed_time(marks[sbc.MARK_COLLECT]))
     timed_ms = sum(enc_ms) + sum(dec_ms)
-    if dist is not None:
-        t = torch.tensor([timed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        timed_ms = float(t.item())
+    timed_ms = reduce_max_over_ranks(timed_ms, dist, dev)
     if int(status.item()) != 0:
         raise RuntimeError(f"decoder reported status {int(status.item())}")
 
@@ -264,7 +291,7 @@ def run_ours(args):
     collect_ms = sum(collect_ms_all) / len(collect_ms_all)
     achieved = ALGO_BYTES_PER_ELEM * n / (collect_ms * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": None, "kernel": "k_add_collect", "launches_timed": len(collect_ms_all),
+                "traffic": measured_traffic(n), "kernel": "k_add_collect", "launches_timed": len(collect_ms_all),
                 "avg_ms": collect_ms, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": ALGO_BYTES_PER_ELEM * n}
 

@@ -38,6 +38,22 @@ __device__ __forceinline__ uint32_t peek32(const StreamView& v, unsigned long lo
     return __funnelshift_l(lo, hi, sh);
 }
 
+// out[j] += mu.  The hardware fp32 atomic add treats subnormal inputs and results as zero, which
+// is harmless (far below the stated tolerance) unless the transmitted value itself is tiny; then
+// an IEEE add is done with a compare-and-swap retry instead.  The retry count is bounded: every
+// failed attempt means another thread's add succeeded.
+__device__ __forceinline__ uint32_t add_at(float* p, float mu, bool ieee_path) {
+    if (!ieee_path) { atomicAdd(p, mu); return 0u; }
+    unsigned int* u = reinterpret_cast<unsigned int*>(p);
+    unsigned int old = *u;
+    for (int tries = 0; tries < (1 << 20); ++tries) {
+        const unsigned int assumed = old;
+        old = atomicCAS(u, assumed, __float_as_uint(__fadd_rn(__uint_as_float(assumed), mu)));
+        if (old == assumed) return 0u;
+    }
+    return SBC_STATUS_INTERNAL;
+}
+
 constexpr int kDecodeThreads = 64;            // two warps per block
 constexpr int kDecodeWarpWords = 5632;        // staged payload words per warp (22 KB)
 
@@ -168,6 +184,7 @@ __global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate(const Deco
             if (pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n) err = SBC_STATUS_CORRUPT;
             const uint32_t b = v.b;
             const float mu = v.mu;
+            const bool tiny = fabsf(mu) < 7.888609052e-31f;  // 2^-100
             if (staged) {
                 // Fast path: bit positions relative to the stage fit 32 bits; every codeword
                 // is cut out of a 64-bit window rebuilt from three staged words.
@@ -200,7 +217,7 @@ __global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate(const Deco
                         break;
                     }
                     prev += (long long)step;
-                    atomicAdd(args.out + prev, mu);
+                    err |= add_at(args.out + prev, mu, tiny);
                 }
                 pos = (first_word << 5) + rel;
             } else {
@@ -231,7 +248,7 @@ __global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate(const Deco
                         break;
                     }
                     prev += (long long)step;
-                    atomicAdd(args.out + prev, mu);
+                    err |= add_at(args.out + prev, mu, tiny);
                 }
                 if (!err && used > room) err = SBC_STATUS_CORRUPT;
                 pos += used;

@@ -1,0 +1,54 @@
+"""Host-side logic of bench.py: the max-over-ranks reduction (2 gloo ranks on CPU), the
+reference arm under a 2-rank launch, and the traffic figure's source check."""
+import json
+import os
+import subprocess
+import sys
+
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+import bench  # noqa: E402
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    mine = 10.0 + 5.0 * rank                     # rank 1 is the slow one
+    got = bench.reduce_max_over_ranks(mine, dist, torch.device("cpu"))
+    with open(os.path.join(out_dir, f"r{rank}.txt"), "w") as fh:
+        fh.write(repr(got))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_max_over_ranks_with_two_gloo_ranks(tmp_path):
+    mp.spawn(_worker, args=(2, 29611, str(tmp_path)), nprocs=2, join=True)
+    assert [float(open(tmp_path / f"r{r}.txt").read()) for r in range(2)] == [15.0, 15.0]
+    assert bench.reduce_max_over_ranks(3.5, None, None) == 3.5
+
+
+def test_reference_arm_prints_one_line_from_rank_zero_only():
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+           "--master-addr", "127.0.0.1", "--master-port", "29613", os.path.join(ROOT, "bench.py"),
+           "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "1", "--cpu-sample", "4096"]
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [l for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    rec = json.loads(lines[0])
+    assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["unit"] == "Gelem/s"
+    assert rec["cpu_baseline"]["kind"] == "oracle" and rec["e2e"]["h2d_bytes_per_step"] == 0
+    assert rec["value"] > 0
+
+
+def test_traffic_figure_is_tied_to_the_kernel_source(monkeypatch):
+    full = bench.measured_traffic(1 << 30)
+    if full is not None:                          # counters still match the kernel source
+        assert abs(full - 16 * bench.NCU_TRAFFIC_BYTES_AT_2P26) < 1.0
+    monkeypatch.setattr(bench, "NCU_TRAFFIC_SOURCE_SHA256", "0" * 64)
+    assert bench.measured_traffic(1 << 30) is None

@@ -241,3 +241,19 @@ def test_argument_errors_are_returned_at_once():
     with pytest.raises(sbc.SbcError) as e:
         sbc.sbc_encode(u, u, 0.01)                      # aliasing
     assert e.value.code == sbc.SBC_EINVAL
+
+
+def test_decode_of_a_subnormal_mu_is_exact():
+    # the transmitted value itself is subnormal: the sum must not be flushed to zero
+    n = 5000
+    rng = np.random.default_rng(3)
+    upd = (rng.standard_normal(n) * 1e-41).astype(np.float32)
+    stream, mu, _, _, _ = gpu_encode(upd, np.zeros(n, dtype=np.float32), 0.02)
+    assert mu != 0 and abs(float(mu)) < 1.2e-38
+    want = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate([stream, stream, stream], want)
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    s = torch.from_numpy(stream).to(DEV)
+    sbc.sbc_decode_accumulate([s, s, s], dense)
+    torch.cuda.synchronize()
+    assert np.array_equal(dense.cpu().numpy().view(np.uint32), want.view(np.uint32))

@@ -202,6 +202,40 @@ int sbc_encode_host(const float *update_host, float *update_dev, float *residual
                     size_t out_capacity, size_t *out_bytes_host, float *out_mu_host,
                     void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream);
 
+/*
+ * sbc_encode without a workspace argument, for callers that must not allocate.
+ * (The paper has no counterpart; this is a packaging variant of sbc_encode.)
+ *
+ * Who needs it: code that is handed a stream and its tensors but no allocator
+ * -- a compression hook called from inside a training framework's
+ * communication step, a plug-in in a serving process, a control loop that is
+ * forbidden to allocate once it is running.  For them cudaMalloc is either
+ * unavailable or harmful (it can synchronise the whole device and stall
+ * streams that belong to someone else), and they have no pool to carve the
+ * scratch of sbc_encode from.
+ *
+ * The scratch of this variant is a fixed array of SBC_STATIC_WORKSPACE_BYTES
+ * that is part of the library image: every GPU that loads the library holds
+ * those bytes until the process exits.  Consequences the caller must know:
+ *   - Only problems with sbc_workspace_bytes(numel, p) <=
+ *     SBC_STATIC_WORKSPACE_BYTES fit (up to about 3.5 M elements at p = 0.01,
+ *     17 M at p = 0.001);
+ *     larger ones are refused with SBC_ECAPACITY and nothing is enqueued.
+ *   - There is ONE array per GPU, shared by every call in the process.  Two
+ *     calls whose device work can overlap (different streams, different
+ *     threads) race on it and corrupt each other; issue them on one stream or
+ *     order them with events.  The array keeps whatever the previous call
+ *     left; each call clears the parts that must start at zero itself.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and remembers it; make that first call outside any
+ *     stream capture.  No call allocates or frees memory.
+ * Everything else (arguments, results, errors, asynchrony) is as sbc_encode.
+ */
+#define SBC_STATIC_WORKSPACE_BYTES (8u << 20)
+int sbc_encode_static(const float *update, float *residual, int64_t numel, double p,
+                      void *out_stream, size_t out_capacity, float *out_mu,
+                      sbc_cuda_stream_t stream);
+
 /* Copies the header of a device-resident stream to the host and fills
  * *host_out.  Synchronises `stream`.  Returns SBC_OK, SBC_ECORRUPT if the
  * magic/version are wrong, SBC_ENONFINITE if the status word says so. */

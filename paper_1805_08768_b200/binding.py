@@ -25,8 +25,9 @@ EXPORTS = [
     "sbc_kept_count", "sbc_golomb_b", "sbc_mean_position_bits", "sbc_stream_bytes",
     "sbc_workspace_bytes", "sbc_encode", "sbc_encode_ex", "sbc_encode_launches", "sbc_decode_launches",
     "sbc_encode_diag_get", "sbc_encode_host", "sbc_stream_info_get", "sbc_decode_accumulate",
-    "sbc_decode_accumulate_host",
+    "sbc_decode_accumulate_host", "sbc_encode_static",
 ]
+STATIC_WORKSPACE_BYTES = 8 << 20
 MARK_BEGIN, MARK_BOUNDS, MARK_COLLECT, MARK_EXACT, MARK_SELECT, MARK_END, MARK_COUNT = range(7)
 MARK_NAMES = ["bounds", "collect", "exact", "select", "golomb"]  # interval i = mark i -> mark i+1
 
@@ -96,6 +97,9 @@ def lib() -> C.CDLL:
         L.sbc_decode_accumulate_host.argtypes = [C.POINTER(C.c_void_p), C.POINTER(C.c_size_t), C.c_int,
                                                  C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_size_t,
                                                  C.POINTER(C.c_uint32), C.c_void_p]
+        L.sbc_encode_static.restype = C.c_int
+        L.sbc_encode_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_double, C.c_void_p, C.c_size_t,
+                                        C.c_void_p, C.c_void_p]
         L.sbc_stream_info_get.restype = C.c_int
         L.sbc_stream_info_get.argtypes = [C.c_void_p, C.POINTER(StreamInfo), C.c_void_p]
         L.sbc_decode_accumulate.restype = C.c_int
@@ -169,6 +173,19 @@ def sbc_encode(update: torch.Tensor, residual: torch.Tensor, p: float,
                             workspace.data_ptr(), workspace.numel(), _cuda_stream(stream))
     _check(code, "sbc_encode")
     return out_stream, out_mu
+
+
+def sbc_encode_static(update: torch.Tensor, residual: torch.Tensor, p: float, out_stream: torch.Tensor,
+                      out_mu: torch.Tensor, stream=None) -> None:
+    """sbc_encode for callers that may not allocate: the scratch is a fixed array inside the
+    library (one per GPU, shared by all calls -- do not overlap calls).  The caller passes every
+    input and output; problems whose scratch exceeds STATIC_WORKSPACE_BYTES raise SBC_ECAPACITY."""
+    _dev_f32(update, "update")
+    _dev_f32(residual, "residual")
+    code = lib().sbc_encode_static(update.data_ptr(), residual.data_ptr(), update.numel(), float(p),
+                                   out_stream.data_ptr(), out_stream.numel(), out_mu.data_ptr(),
+                                   _cuda_stream(stream))
+    _check(code, "sbc_encode_static")
 
 
 def sbc_encode_ex(update: torch.Tensor, residual: torch.Tensor, p: float, out_stream: torch.Tensor,

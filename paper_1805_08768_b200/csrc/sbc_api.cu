@@ -2,6 +2,7 @@
 // Declared and documented in include/sbc.h.
 #include <cmath>
 #include <cstring>
+#include <mutex>
 
 #include "../../include/sbc.h"
 #include "sbc_common.cuh"
@@ -260,6 +261,47 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     mark(SBC_MARK_END);
 
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
+}
+
+// ---- sbc_encode_static: scratch that lives in the library image --------------------------
+//
+// File-scope device array used as the workspace of sbc_encode_static.  In host code this name is
+// only a handle for the runtime, not a device address: the address is looked up per device with
+// cudaGetSymbolAddress below and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_workspace[SBC_STATIC_WORKSPACE_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mutex;
+void* g_static_ptr[kMaxDevices] = {};  // device address of g_static_workspace, per device ordinal
+
+// Device address of the static workspace on the current device; looked up on first use.
+int static_workspace_ptr(void** out) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return SBC_ECUDA;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_workspace) != cudaSuccess || !ptr) return SBC_ECUDA;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return SBC_OK;
+}
+}  // namespace
+
+int sbc_encode_static(const float* update, float* residual, int64_t numel, double p, void* out_stream,
+                      size_t out_capacity, float* out_mu, sbc_cuda_stream_t stream) {
+    const size_t need = sbc_workspace_bytes(numel, p);
+    if (need == 0) return SBC_EINVAL;
+    if (need > (size_t)SBC_STATIC_WORKSPACE_BYTES) return SBC_ECAPACITY;  // problem too large for the fixed scratch
+    void* ws = nullptr;
+    const int rc = static_workspace_ptr(&ws);
+    if (rc != SBC_OK) return rc;
+    // Same launches as sbc_encode; they clear the control block, histograms, mask and payload area
+    // themselves, so stale contents of the shared array from an earlier call do not matter.
+    return sbc_encode(update, residual, numel, p, out_stream, out_capacity, out_mu, ws,
+                      (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
 }
 
 int sbc_encode_launches(void) { return 23; }  // put_prob, 2 sample, 1 collect, 6 exact, 8 select, 5 Golomb

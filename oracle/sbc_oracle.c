@@ -190,6 +190,18 @@ static int cmp_i64(const void *x, const void *y) {
     return (a > b) - (a < b);
 }
 
+void sbc_oracle_side_and_mu(double sum_top, double sum_bottom, int64_t k, int *side,
+                            float *mu32, double *mu_pos, double *mu_neg) {
+    /* Algorithm 2: mu+ = mean(val+), mu- = mean(val-) with val- the negated k smallest;
+     * "if mu+ >= mu-" keeps the positive side; the value sent is mu+ or -mu-. */
+    double mp = sum_top / (double)k;
+    double mn = -sum_bottom / (double)k;
+    if (mp >= mn) { *side = 0; *mu32 = (float)mp; }
+    else          { *side = 1; *mu32 = (float)(-mn); }
+    if (mu_pos) *mu_pos = mp;
+    if (mu_neg) *mu_neg = mn;
+}
+
 int sbc_oracle_compress(float *a, int64_t n, int64_t k, int64_t *kept_sorted,
                         int *side, float *mu32, double *mu_pos,
                         double *mu_neg) {
@@ -203,13 +215,11 @@ int sbc_oracle_compress(float *a, int64_t n, int64_t k, int64_t *kept_sorted,
     sbc_oracle_topk(a, n, k, 1, neg_idx);
 
     /* mu+ = mean(val+), mu- = mean(val-); val- holds the negated entries */
-    double mp = sbc_oracle_exact_sum(a, pos_idx, k) / (double)k;
-    double mn = -sbc_oracle_exact_sum(a, neg_idx, k) / (double)k;
-
-    const int64_t *kept;
+    double mp, mn;
     float mu;
-    if (mp >= mn) { *side = 0; kept = pos_idx; mu = (float)mp; }
-    else          { *side = 1; kept = neg_idx; mu = (float)(-mn); }
+    sbc_oracle_side_and_mu(sbc_oracle_exact_sum(a, pos_idx, k), sbc_oracle_exact_sum(a, neg_idx, k),
+                           k, side, &mu, &mp, &mn);
+    const int64_t *kept = *side ? neg_idx : pos_idx;
 
     /* R = dW - dW*: dW* is mu on the kept positions and 0 elsewhere */
     for (int64_t j = 0; j < k; ++j) {
@@ -354,34 +364,16 @@ size_t sbc_oracle_stream_bytes(int64_t n, double p) {
     return sbc_oracle_container_bytes(k, sbc_oracle_payload_bits_bound(n, k, b));
 }
 
-int sbc_oracle_encode(const float *update, float *residual, int64_t n, double p,
-                      uint8_t *out, size_t cap, size_t *out_len, float *out_mu) {
-    if (!update || !residual || !out || n <= 0 || n >= ((int64_t)1 << 31) ||
-        !(p > 0.0 && p < 1.0))
-        return -2;
-    int64_t k = sbc_oracle_kept_count(n, p);
-    int b = sbc_oracle_golomb_b(p);
-    if (b > 30) return -2;
-
-    /* Algorithm 1: dW_i = R_i + (SGD_n(W_i) - W_i) */
-    if (sbc_oracle_accumulate(update, residual, n) != 0) return -1;
-
-    /* Algorithm 2 and R_i = dW_i - dW_i* */
-    int64_t *I = (int64_t *)malloc((size_t)k * sizeof(int64_t));
-    if (!I) return -2;
-    int side;
-    float mu;
-    sbc_oracle_compress(residual, n, k, I, &side, &mu, NULL, NULL);
-
+int sbc_oracle_container(const int64_t *I, int64_t k, int64_t n, int b, int side, float mu,
+                         uint8_t *out, size_t cap, size_t *out_len) {
     /* Algorithm 3 into the payload area */
     uint64_t nchunks = n_chunks_for(k);
     size_t payload_offset = SBC_ORACLE_HEADER_BYTES + SBC_ORACLE_CHUNK_ENTRY_BYTES * (size_t)nchunks;
-    if (cap < payload_offset) { free(I); return -3; }
-    uint64_t nbits = sbc_oracle_golomb_encode(I, k, b, out + payload_offset,
-                                              cap - payload_offset);
-    if (nbits == UINT64_MAX) { free(I); return -3; }
+    if (cap < payload_offset) return -3;
+    uint64_t nbits = sbc_oracle_golomb_encode(I, k, b, out + payload_offset, cap - payload_offset);
+    if (nbits == UINT64_MAX) return -3;
     size_t total = sbc_oracle_container_bytes(k, nbits);
-    if (cap < total) { free(I); return -3; }
+    if (cap < total) return -3;
     for (size_t z = payload_offset + (size_t)((nbits + 7) / 8); z < total; ++z) out[z] = 0;
 
     /* chunk table: bit offset of codeword c*C and the position before it */
@@ -413,11 +405,33 @@ int sbc_oracle_encode(const float *update, float *residual, int64_t n, double p,
     put_u32(out + 52, SBC_ORACLE_CHUNK_CODEWORDS);
     put_u32(out + 56, (uint32_t)nchunks);
     put_u32(out + 60, 0u);
-
     if (out_len) *out_len = total;
-    if (out_mu) *out_mu = mu;
-    free(I);
     return 0;
+}
+
+int sbc_oracle_encode(const float *update, float *residual, int64_t n, double p,
+                      uint8_t *out, size_t cap, size_t *out_len, float *out_mu) {
+    if (!update || !residual || !out || n <= 0 || n >= ((int64_t)1 << 31) ||
+        !(p > 0.0 && p < 1.0))
+        return -2;
+    int64_t k = sbc_oracle_kept_count(n, p);
+    int b = sbc_oracle_golomb_b(p);
+    if (b > 30) return -2;
+
+    /* Algorithm 1: dW_i = R_i + (SGD_n(W_i) - W_i) */
+    if (sbc_oracle_accumulate(update, residual, n) != 0) return -1;
+
+    /* Algorithm 2 and R_i = dW_i - dW_i* */
+    int64_t *I = (int64_t *)malloc((size_t)k * sizeof(int64_t));
+    if (!I) return -2;
+    int side;
+    float mu;
+    sbc_oracle_compress(residual, n, k, I, &side, &mu, NULL, NULL);
+
+    int rc = sbc_oracle_container(I, k, n, b, side, mu, out, cap, out_len);
+    if (rc == 0 && out_mu) *out_mu = mu;
+    free(I);
+    return rc;
 }
 
 int sbc_oracle_decode_accumulate(const uint8_t *const *streams, int n_clients,

@@ -80,6 +80,12 @@ int sbc_oracle_compress(float *a_inout, int64_t n, int64_t k,
                         int64_t *kept_sorted, int *side, float *mu32,
                         double *mu_pos, double *mu_neg);
 
+/* Algorithm 2's decision from the two (exactly rounded) sums: sum_top over the
+ * k largest entries, sum_bottom over the k smallest.  mu+ = sum_top/k,
+ * mu- = -sum_bottom/k; side 0 iff mu+ >= mu-; mu32 = (float)mu+ or (float)(-mu-). */
+void sbc_oracle_side_and_mu(double sum_top, double sum_bottom, int64_t k, int *side,
+                            float *mu32, double *mu_pos, double *mu_neg);
+
 /* Upper bound on payload bits: k(1+b) + floor((n-k)/2^b). */
 uint64_t sbc_oracle_payload_bits_bound(int64_t n, int64_t k, int b);
 
@@ -99,6 +105,11 @@ int64_t sbc_oracle_golomb_decode(const uint8_t *payload, uint64_t nbits, int b,
 size_t sbc_oracle_container_bytes(int64_t k, uint64_t nbits);
 /* Capacity bound for (n, p): container_bytes(k, payload_bits_bound). */
 size_t sbc_oracle_stream_bytes(int64_t n, double p);
+
+/* Container (header, chunk table, Algorithm 3 payload) for an ascending
+ * position list.  Returns 0, or -3 if cap is too small. */
+int sbc_oracle_container(const int64_t *sorted_idx, int64_t k, int64_t n, int b, int side,
+                         float mu, uint8_t *out, size_t cap, size_t *out_len);
 
 /* Whole client step: accumulate, compress, residual write-back, encode into a
  * container (header, chunk table, payload).  Returns 0 on success, -1 for

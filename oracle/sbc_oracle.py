@@ -14,7 +14,7 @@ __all__ = [
     "kept_count", "golomb_b", "mean_position_bits", "accumulate", "topk",
     "exact_sum", "compress", "payload_bits_bound", "golomb_encode",
     "golomb_decode", "container_bytes", "stream_bytes", "encode",
-    "decode_accumulate", "parse_header", "StreamHeader",
+    "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container",
     "HEADER_BYTES", "CHUNK_CODEWORDS", "CHUNK_ENTRY_BYTES", "MAGIC",
 ]
 
@@ -54,6 +54,10 @@ _container_bytes = _sig("sbc_oracle_container_bytes", C.c_size_t, C.c_int64, C.c
 _stream_bytes = _sig("sbc_oracle_stream_bytes", C.c_size_t, C.c_int64, C.c_double)
 _encode = _sig("sbc_oracle_encode", C.c_int, _f32p, _f32p, C.c_int64, C.c_double, _u8p,
                C.c_size_t, C.POINTER(C.c_size_t), C.POINTER(C.c_float))
+_side_mu = _sig("sbc_oracle_side_and_mu", None, C.c_double, C.c_double, C.c_int64, C.POINTER(C.c_int),
+                C.POINTER(C.c_float), C.POINTER(C.c_double), C.POINTER(C.c_double))
+_container = _sig("sbc_oracle_container", C.c_int, _i64p, C.c_int64, C.c_int64, C.c_int, C.c_int,
+                  C.c_float, _u8p, C.c_size_t, C.POINTER(C.c_size_t))
 _decode_acc = _sig("sbc_oracle_decode_accumulate", C.c_int, C.POINTER(C.c_void_p), C.c_int,
                    _f32p, C.c_int64)
 
@@ -148,6 +152,26 @@ def encode(update: np.ndarray, residual: np.ndarray, p: float, cap: int = None):
     if rc != 0:
         raise ValueError(f"sbc_oracle_encode failed: {rc}")
     return out[: out_len.value].copy(), np.float32(mu.value)
+
+
+def side_and_mu(sum_top: float, sum_bottom: float, k: int):
+    """Algorithm 2's decision from the two exact sums.  Returns (side, mu32, mu_pos, mu_neg)."""
+    side, mu = C.c_int(), C.c_float()
+    mp, mn = C.c_double(), C.c_double()
+    _side_mu(sum_top, sum_bottom, k, C.byref(side), C.byref(mu), C.byref(mp), C.byref(mn))
+    return side.value, np.float32(mu.value), mp.value, mn.value
+
+
+def container(sorted_idx, n: int, p: float, side: int, mu) -> np.ndarray:
+    """Header + chunk table + Algorithm 3 payload for an ascending position list."""
+    idx = np.ascontiguousarray(sorted_idx, dtype=np.int64)
+    cap = stream_bytes(n, p)
+    out = np.zeros(cap, dtype=np.uint8)
+    out_len = C.c_size_t()
+    rc = _container(idx, idx.size, n, golomb_b(p), int(side), float(mu), out, cap, C.byref(out_len))
+    if rc != 0:
+        raise ValueError(f"sbc_oracle_container failed: {rc}")
+    return out[: out_len.value].copy()
 
 
 def decode_accumulate(streams, out_dense: np.ndarray) -> None:

@@ -1,0 +1,172 @@
+"""GPU parity on the five workload configurations (shapes of the paper's networks, synthetic values).
+
+Configs 1-4 run the oracle on the full tensors (one thread per tensor: the C oracle releases the
+GIL).  Config 5 (2^30 elements) is too large for the oracle's full sort, so its expected result is
+assembled from independent pieces: torch's own sort for the two thresholds, the oracle's exact
+sum / decision / container builder for everything after the selection.
+"""
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_1805_08768_b200 import binding as sbc
+from paper_1805_08768_b200 import workloads
+
+pytestmark = pytest.mark.gpu
+
+if not torch.cuda.is_available():  # pragma: no cover
+    pytest.skip("needs a CUDA device", allow_module_level=True)
+
+DEV = torch.device("cuda:0")
+POOL = ThreadPoolExecutor(max_workers=16)
+
+
+class Client:
+    """Device-side state of one client: residuals, streams, scratch (allocated once, reused per round)."""
+
+    def __init__(self, sizes, p):
+        self.p = p
+        self.res = [torch.zeros(n, dtype=torch.float32, device=DEV) for n in sizes]
+        self.out = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=DEV) for n in sizes]
+        self.mu = [torch.empty(1, dtype=torch.float32, device=DEV) for _ in sizes]
+        self.ws = torch.empty(max(sbc.sbc_workspace_bytes(n, p) for n in sizes), dtype=torch.uint8, device=DEV)
+
+    def encode_round(self, tensors):
+        for t, upd in enumerate(tensors):
+            sbc.sbc_encode(torch.from_numpy(upd).to(DEV), self.res[t], self.p, self.out[t], self.mu[t], self.ws)
+        torch.cuda.synchronize()
+        got = []
+        for t in range(len(tensors)):
+            info = sbc.sbc_stream_info_get(self.out[t])
+            got.append((self.out[t][: info.total_bytes].cpu().numpy(), np.float32(self.mu[t].item())))
+        return got
+
+
+def oracle_round(tensors, residuals, p):
+    return list(POOL.map(lambda ur: oracle.encode(ur[0], ur[1], p), zip(tensors, residuals)))
+
+
+def assert_round_equal(got, want, client, residuals_cpu, label):
+    for t, ((gs, gm), (ws_, wm)) in enumerate(zip(got, want)):
+        assert np.array_equal(gs, ws_), f"{label}: container of tensor {t} differs"
+        assert gm.view(np.uint32) == wm.view(np.uint32), f"{label}: mu of tensor {t} differs"
+        assert np.array_equal(client.res[t].cpu().numpy().view(np.uint32), residuals_cpu[t].view(np.uint32)), \
+            f"{label}: residual of tensor {t} differs"
+
+
+def test_config2_resnet50_shapes_ten_rounds():
+    shapes = workloads.resnet50_shapes()
+    sizes = [int(np.prod(s)) for _, s, _ in shapes]
+    assert len(sizes) == 161 and sum(sizes) == 25557032 and sum(1 for n in sizes if n < 1000) == 84
+    p = 0.001
+    client = Client(sizes, p)
+    res_cpu = [np.zeros(n, dtype=np.float32) for n in sizes]
+    for rnd in range(10):
+        tensors = workloads.resnet50_update(workloads.seed_for(2, rnd))
+        want = oracle_round(tensors, res_cpu, p)
+        got = client.encode_round(tensors)
+        assert_round_equal(got, want, client, res_cpu, f"round {rnd}")
+
+
+@pytest.mark.parametrize("p", [0.01, 0.001])
+def test_config3_word_lstm_shapes_four_rounds(p):
+    sizes = [int(np.prod(s)) for _, s in workloads.word_lstm_shapes()]
+    assert sum(sizes) == 19765200
+    client = Client(sizes, p)
+    res_cpu = [np.zeros(n, dtype=np.float32) for n in sizes]
+    for rnd in range(4):
+        tensors = workloads.word_lstm_update(workloads.seed_for(3, rnd))
+        want = oracle_round(tensors, res_cpu, p)
+        got = client.encode_round(tensors)
+        assert_round_equal(got, want, client, res_cpu, f"p={p} round {rnd}")
+
+
+def test_config4_eight_clients_decode_aggregate():
+    shapes = workloads.resnet50_shapes()
+    sizes = [int(np.prod(s)) for _, s, _ in shapes]
+    p = 0.001
+    per_client = []
+    for c in range(8):
+        tensors = workloads.resnet50_update(workloads.seed_for(4, 0, c))
+        client = Client(sizes, p)
+        res_cpu = [np.zeros(n, dtype=np.float32) for n in sizes]
+        want = oracle_round(tensors, res_cpu, p)
+        got = client.encode_round(tensors)
+        assert_round_equal(got, want, client, res_cpu, f"client {c}")
+        per_client.append((client, want))
+    # one dense aggregate per tensor, the 8 streams decoded and summed on the device
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dense = [torch.zeros(n, dtype=torch.float32, device=DEV) for n in sizes]
+    for t in range(len(sizes)):
+        sbc.sbc_decode_accumulate([cl.out[t] for cl, _ in per_client], dense[t], status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+
+    def expected(t):
+        want = np.zeros(sizes[t], dtype=np.float32)
+        oracle.decode_accumulate([w[t][0] for _, w in per_client], want)
+        return want
+
+    for t, want in enumerate(POOL.map(expected, range(len(sizes)))):
+        got = dense[t].cpu().numpy()
+        tol = 1e-6 * sum(abs(float(w[t][1])) for _, w in per_client)
+        assert np.array_equal(got != 0, want != 0) or tol > 0
+        assert np.max(np.abs(got.astype(np.float64) - want)) <= tol, f"aggregate of tensor {t}"
+
+
+def test_config5_flat_2p30_sweep_against_independent_selection():
+    n = 1 << 30
+    update = workloads.student_t_flat_torch(n, workloads.seed_for(5), DEV)
+    # independent selection: torch's sort gives both order statistics for every p at once
+    sorted_vals = torch.sort(update).values
+    for p in (1e-2, 1e-3, 1e-4):
+        k, b = oracle.kept_count(n, p), oracle.golomb_b(p)
+        t_top = sorted_vals[n - k]          # k-th largest
+        t_bot = sorted_vals[k - 1]          # k-th smallest
+        top = torch.nonzero(update >= t_top).flatten()
+        bot = torch.nonzero(update <= t_bot).flatten()
+        # continuous data: no ties expected at the thresholds; if there are, keep the lowest indices
+        if top.numel() > k:
+            ties = torch.nonzero(update[top] == t_top).flatten()
+            keep = torch.ones(top.numel(), dtype=torch.bool, device=DEV)
+            keep[ties[k - (top.numel() - ties.numel()):]] = False
+            top = top[keep]
+        if bot.numel() > k:
+            ties = torch.nonzero(update[bot] == t_bot).flatten()
+            keep = torch.ones(bot.numel(), dtype=torch.bool, device=DEV)
+            keep[ties[k - (bot.numel() - ties.numel()):]] = False
+            bot = bot[keep]
+        assert top.numel() == k and bot.numel() == k
+        top_vals = update[top].cpu().numpy()
+        bot_vals = update[bot].cpu().numpy()
+        ar = np.arange(k, dtype=np.int64)
+        side, mu, _, _ = oracle.side_and_mu(oracle.exact_sum(top_vals, ar), oracle.exact_sum(bot_vals, ar), k)
+        kept = (bot if side else top)
+        want_stream = oracle.container(kept.cpu().numpy(), n, p, side, mu)
+        del top, bot
+
+        residual = torch.zeros(n, dtype=torch.float32, device=DEV)
+        out, mu_dev = sbc.sbc_encode(update, residual, p)
+        info = sbc.sbc_stream_info_get(out)
+        got_stream = out[: info.total_bytes].cpu().numpy()
+        assert (info.k, info.b, info.side) == (k, b, side)
+        assert np.float32(mu_dev.item()).view(np.uint32) == mu.view(np.uint32)
+        assert np.array_equal(got_stream, want_stream), f"p={p}: container differs"
+        # residual: A everywhere (zero residual in: A = update), A - mu on the kept positions
+        expect_res = update.clone()
+        expect_res[kept] = update[kept] - float(mu)
+        assert torch.equal(residual.view(torch.int32), expect_res.view(torch.int32)), f"p={p}: residual differs"
+        del expect_res
+        # decode into a zeroed tensor: mu on the kept positions, zero elsewhere
+        dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        sbc.sbc_decode_accumulate([out], dense, status=status)
+        expect = torch.zeros(n, dtype=torch.float32, device=DEV)
+        expect[kept] = float(mu)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        assert torch.equal(dense.view(torch.int32), expect.view(torch.int32)), f"p={p}: decoded tensor differs"
+        del dense, expect, residual, kept

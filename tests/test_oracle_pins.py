@@ -375,3 +375,19 @@ def test_rejects_bad_arguments_and_non_finite_input():
     bad[0] ^= 0xFF
     with pytest.raises(ValueError):
         oracle.decode_accumulate([bad], np.zeros(3, dtype=np.float32))
+
+
+def test_side_and_mu_and_container_entry_points():
+    # Algorithm 2's decision from the two sums (worked example: sums 3.5 and -5.5 over k = 2)
+    assert oracle.side_and_mu(3.5, -5.5, 2) == (1, np.float32(-2.75), 1.75, 2.75)
+    assert oracle.side_and_mu(2.0, -2.0, 2)[:2] == (0, np.float32(1.0))          # tie keeps the positive side
+    assert oracle.side_and_mu(-1.0, -9.0, 3)[:2] == (1, np.float32(-3.0))
+    # the container built from a position list is the one encode() emits
+    rng = np.random.default_rng(21)
+    n, p = 40000, 0.01
+    upd = rng.standard_normal(n).astype(np.float32)
+    res = np.zeros(n, dtype=np.float32)
+    stream, mu = oracle.encode(upd, res, p)
+    h = oracle.parse_header(stream)
+    kept = np.sort(_brute_topk(upd, h.k, bool(h.side)))
+    assert np.array_equal(oracle.container(kept, n, p, h.side, mu), stream)

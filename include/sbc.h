@@ -150,6 +150,33 @@ int sbc_encode(const float *update, float *residual, int64_t numel, double p,
                void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream);
 
 /*
+ * sbc_encode for many tensors at once (a model's parameter tensors in one
+ * communication round; the paper applies the method per tensor, with one mean
+ * per tensor -- Section 2, "Optimal Position Encoding").  Exactly the results
+ * of n_tensors separate sbc_encode calls, but every kernel is launched once
+ * for the whole batch, so small tensors do not pay a launch sequence each.
+ *
+ * descs      HOST array of n_tensors descriptors (fields as the sbc_encode
+ *            arguments of the same name; p may differ per tensor).  Read
+ *            before the call returns.
+ * workspace  device, 256-byte aligned, >= sbc_workspace_bytes_batch(...)
+ * If any tensor has a host-visible argument error nothing is enqueued.
+ * Device-side errors are reported per tensor in its stream header.
+ */
+typedef struct sbc_tensor_desc {
+    const float *update;
+    float *residual;
+    int64_t numel;
+    double p;
+    void *out_stream;
+    size_t out_capacity;
+    float *out_mu;
+} sbc_tensor_desc;
+size_t sbc_workspace_bytes_batch(int n_tensors, const sbc_tensor_desc *descs);
+int sbc_encode_batch(int n_tensors, const sbc_tensor_desc *descs, void *workspace,
+                     size_t workspace_bytes, sbc_cuda_stream_t stream);
+
+/*
  * sbc_encode with timing marks: the same work, plus, when `marks` is not NULL,
  * a cudaEventRecord on `stream` at each stage boundary.  marks is a host array
  * of SBC_MARK_COUNT events the caller created (entries may be NULL).  The
@@ -270,6 +297,27 @@ int sbc_stream_info_get(const void *stream_dev, sbc_stream_info *host_out,
 int sbc_decode_accumulate(const void *const *streams, int n_clients,
                           float *out_dense, int64_t numel, uint32_t *status_dev,
                           sbc_cuda_stream_t stream);
+
+/*
+ * sbc_decode_accumulate for many tensors at once: for every tensor t,
+ * out_dense[t][j] += mu_{c,t} over the n_clients streams of that tensor
+ * (Algorithm 1, server sum line, per tensor).  One launch for the batch.
+ *
+ * descs      HOST array of n_tensors descriptors; descs[t].streams is a HOST
+ *            array of n_clients DEVICE pointers.  Read before the call returns.
+ * n_clients  1 .. 32 (the same for every tensor)
+ * workspace  device, 256-byte aligned, >= sbc_decode_workspace_bytes_batch(n_tensors)
+ * status_dev as in sbc_decode_accumulate (one word for the whole batch)
+ */
+typedef struct sbc_decode_desc {
+    const void *const *streams;
+    float *out_dense;
+    int64_t numel;
+} sbc_decode_desc;
+size_t sbc_decode_workspace_bytes_batch(int n_tensors);
+int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_desc *descs,
+                                uint32_t *status_dev, void *workspace, size_t workspace_bytes,
+                                sbc_cuda_stream_t stream);
 
 /*
  * Host-buffer form of sbc_decode_accumulate: copies the n_clients containers

@@ -25,7 +25,8 @@ EXPORTS = [
     "sbc_kept_count", "sbc_golomb_b", "sbc_mean_position_bits", "sbc_stream_bytes",
     "sbc_workspace_bytes", "sbc_encode", "sbc_encode_ex", "sbc_encode_launches", "sbc_decode_launches",
     "sbc_encode_diag_get", "sbc_encode_host", "sbc_stream_info_get", "sbc_decode_accumulate",
-    "sbc_decode_accumulate_host", "sbc_encode_static",
+    "sbc_decode_accumulate_host", "sbc_encode_static", "sbc_workspace_bytes_batch", "sbc_encode_batch",
+    "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch",
 ]
 STATIC_WORKSPACE_BYTES = 8 << 20
 MARK_BEGIN, MARK_BOUNDS, MARK_COLLECT, MARK_EXACT, MARK_SELECT, MARK_END, MARK_COUNT = range(7)
@@ -54,6 +55,15 @@ class EncodeDiag(C.Structure):
         ("capacity", C.c_uint32), ("bound_lo", C.c_float), ("bound_hi", C.c_float),
         ("mu_pos", C.c_double), ("mu_neg", C.c_double),
     ]
+
+
+class TensorDesc(C.Structure):
+    _fields_ = [("update", C.c_void_p), ("residual", C.c_void_p), ("numel", C.c_int64), ("p", C.c_double),
+                ("out_stream", C.c_void_p), ("out_capacity", C.c_size_t), ("out_mu", C.c_void_p)]
+
+
+class DecodeDesc(C.Structure):
+    _fields_ = [("streams", C.POINTER(C.c_void_p)), ("out_dense", C.c_void_p), ("numel", C.c_int64)]
 
 
 _lib = None
@@ -100,6 +110,15 @@ def lib() -> C.CDLL:
         L.sbc_encode_static.restype = C.c_int
         L.sbc_encode_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_double, C.c_void_p, C.c_size_t,
                                         C.c_void_p, C.c_void_p]
+        L.sbc_workspace_bytes_batch.restype = C.c_size_t
+        L.sbc_workspace_bytes_batch.argtypes = [C.c_int, C.POINTER(TensorDesc)]
+        L.sbc_encode_batch.restype = C.c_int
+        L.sbc_encode_batch.argtypes = [C.c_int, C.POINTER(TensorDesc), C.c_void_p, C.c_size_t, C.c_void_p]
+        L.sbc_decode_workspace_bytes_batch.restype = C.c_size_t
+        L.sbc_decode_workspace_bytes_batch.argtypes = [C.c_int]
+        L.sbc_decode_accumulate_batch.restype = C.c_int
+        L.sbc_decode_accumulate_batch.argtypes = [C.c_int, C.c_int, C.POINTER(DecodeDesc), C.c_void_p, C.c_void_p,
+                                                  C.c_size_t, C.c_void_p]
         L.sbc_stream_info_get.restype = C.c_int
         L.sbc_stream_info_get.argtypes = [C.c_void_p, C.POINTER(StreamInfo), C.c_void_p]
         L.sbc_decode_accumulate.restype = C.c_int
@@ -173,6 +192,62 @@ def sbc_encode(update: torch.Tensor, residual: torch.Tensor, p: float,
                             workspace.data_ptr(), workspace.numel(), _cuda_stream(stream))
     _check(code, "sbc_encode")
     return out_stream, out_mu
+
+
+def sbc_workspace_bytes_batch(numels: Sequence[int], ps: Sequence[float]) -> int:
+    n = len(numels)
+    descs = (TensorDesc * n)()
+    for t in range(n):
+        descs[t].numel = int(numels[t])
+        descs[t].p = float(ps[t])
+    return int(lib().sbc_workspace_bytes_batch(n, descs))
+
+
+def sbc_encode_batch(updates: Sequence[torch.Tensor], residuals: Sequence[torch.Tensor], ps: Sequence[float],
+                     out_streams: Sequence[torch.Tensor], out_mus: Sequence[torch.Tensor],
+                     workspace: torch.Tensor, stream=None) -> None:
+    """sbc_encode of every tensor of a round with one launch sequence for the whole batch."""
+    n = len(updates)
+    descs = (TensorDesc * n)()
+    for t in range(n):
+        _dev_f32(updates[t], "update")
+        _dev_f32(residuals[t], "residual")
+        descs[t].update = updates[t].data_ptr()
+        descs[t].residual = residuals[t].data_ptr()
+        descs[t].numel = updates[t].numel()
+        descs[t].p = float(ps[t])
+        descs[t].out_stream = out_streams[t].data_ptr()
+        descs[t].out_capacity = out_streams[t].numel()
+        descs[t].out_mu = out_mus[t].data_ptr()
+    code = lib().sbc_encode_batch(n, descs, workspace.data_ptr(), workspace.numel(), _cuda_stream(stream))
+    _check(code, "sbc_encode_batch")
+
+
+def sbc_decode_workspace_bytes_batch(n_tensors: int) -> int:
+    return int(lib().sbc_decode_workspace_bytes_batch(n_tensors))
+
+
+def sbc_decode_accumulate_batch(streams_per_tensor: Sequence[Sequence[torch.Tensor]],
+                                out_denses: Sequence[torch.Tensor], workspace: torch.Tensor,
+                                status: Optional[torch.Tensor] = None, stream=None) -> None:
+    """out_denses[t][j] += mu for every client stream of every tensor t; one launch for the batch."""
+    n = len(out_denses)
+    n_clients = len(streams_per_tensor[0])
+    descs = (DecodeDesc * n)()
+    keep = []
+    for t in range(n):
+        if len(streams_per_tensor[t]) != n_clients:
+            raise ValueError("every tensor needs the same number of client streams")
+        _dev_f32(out_denses[t], "out_dense")
+        ptrs = (C.c_void_p * n_clients)(*[s.data_ptr() for s in streams_per_tensor[t]])
+        keep.append(ptrs)
+        descs[t].streams = ptrs
+        descs[t].out_dense = out_denses[t].data_ptr()
+        descs[t].numel = out_denses[t].numel()
+    code = lib().sbc_decode_accumulate_batch(n, n_clients, descs,
+                                             status.data_ptr() if status is not None else None,
+                                             workspace.data_ptr(), workspace.numel(), _cuda_stream(stream))
+    _check(code, "sbc_decode_accumulate_batch")
 
 
 def sbc_encode_static(update: torch.Tensor, residual: torch.Tensor, p: float, out_stream: torch.Tensor,

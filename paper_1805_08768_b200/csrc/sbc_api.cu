@@ -3,6 +3,7 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
+#include <vector>
 
 #include "../../include/sbc.h"
 #include "sbc_common.cuh"
@@ -17,8 +18,14 @@ namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-// Host-side plan of one encode problem: scalar parameters and the byte offset
-// of every scratch array inside the workspace.
+constexpr size_t kProbSlotBytes = 256;  // one problem descriptor, padded
+static_assert(sizeof(Prob) <= kProbSlotBytes, "descriptor must fit its slot");
+
+// Host-side plan of one encode problem: scalar parameters and the layout of its scratch, which
+// comes in three parts so that a batch can keep each part contiguous across problems:
+//   zero part  control block + radix histograms (cleared before every call)
+//   mask part  kept-position bitmask + per-tile counts (cleared before every call)
+//   rest       everything that needs no clearing
 struct Plan {
     long long n, k;
     int b;
@@ -26,9 +33,11 @@ struct Plan {
     uint32_t s_target[2];
     unsigned long long payload_offset;
     size_t stream_bytes;
-    size_t off_prob, off_mu, off_ctl, off_hists, off_sample, off_cand[2], off_buf[2][2], off_mask,
-        off_mask_tile, off_xtile[2], off_idx, off_blklen, total;
-    size_t zero_begin, zero_end;  // Ctl + Hists, cleared before every call
+    size_t zero_bytes, off_ctl, off_hists;                 // offsets inside the zero part
+    size_t mask_bytes, off_mask, off_mask_tile;            // inside the mask part
+    size_t rest_bytes, off_mu, off_sample, off_cand[2], off_buf[2][2], off_xtile[2], off_idx,
+        off_blklen;                                        // inside the rest
+    size_t total;                                          // single problem: slot + zero + mask + rest
 };
 
 bool valid_p(double p) { return p > 0.0 && p < 1.0; }
@@ -69,27 +78,83 @@ bool make_plan(long long n, double p, Plan* pl) {
 
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
-    pl->off_prob = take(sizeof(Prob));
-    pl->off_mu = take(sizeof(float));  // where the host-buffer form parks mu
-    pl->zero_begin = off;
     pl->off_ctl = take(sizeof(Ctl));
     pl->off_hists = take(sizeof(Hists));
-    pl->zero_end = off;
+    pl->zero_bytes = off;
+    off = 0;
+    pl->off_mask = take((size_t)pl->n_mask_words * 4);
+    pl->off_mask_tile = take((size_t)pl->n_mask_tiles * 4);
+    pl->mask_bytes = off;
+    off = 0;
+    pl->off_mu = take(sizeof(float));  // where the host-buffer form parks mu
     pl->off_sample = take((size_t)pl->m * 4);
     for (int s = 0; s < 2; ++s) pl->off_cand[s] = take((size_t)pl->cap * 8);
     for (int s = 0; s < 2; ++s)
         for (int j = 0; j < 2; ++j) pl->off_buf[s][j] = take((size_t)pl->cap * 8);
-    pl->off_mask = take((size_t)pl->n_mask_words * 4);
-    pl->off_mask_tile = take((size_t)pl->n_mask_tiles * 4);
     for (int s = 0; s < 2; ++s) pl->off_xtile[s] = take((size_t)pl->n_xtiles * 4);
     pl->off_idx = take((size_t)k * 4);
     pl->off_blklen = take((size_t)pl->n_len_blocks * 8);
-    pl->total = off;
+    pl->rest_bytes = off;
+    pl->total = kProbSlotBytes + pl->zero_bytes + pl->mask_bytes + pl->rest_bytes;
     return true;
 }
 
-// Writes the problem descriptor where the kernels read it.
-__global__ void k_put_prob(Prob* dst, const Prob src) { *dst = src; }
+struct TensorArgs {
+    const float* update;
+    float* residual;
+    void* out_stream;
+    size_t out_capacity;
+    float* out_mu;
+};
+
+// Host-visible argument errors of one tensor (nothing is enqueued if any tensor fails).
+int check_tensor(const TensorArgs& a, const Plan& pl) {
+    if (!a.update || !a.residual || !a.out_stream) return SBC_EINVAL;
+    if (((uintptr_t)a.update & 3) || ((uintptr_t)a.residual & 3) || ((uintptr_t)a.out_stream & 15) ||
+        (a.out_mu && ((uintptr_t)a.out_mu & 3)))
+        return SBC_EINVAL;
+    const uintptr_t u0 = (uintptr_t)a.update, r0 = (uintptr_t)a.residual, len = (uintptr_t)pl.n * 4;
+    if (u0 < r0 + len && r0 < u0 + len) return SBC_EINVAL;  // update and residual must not overlap
+    if (a.out_capacity < pl.stream_bytes) return SBC_ECAPACITY;
+    return SBC_OK;
+}
+
+Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* mask, uint8_t* rest) {
+    Prob P;
+    std::memset(&P, 0, sizeof(P));
+    P.update = a.update;
+    P.residual = a.residual;
+    P.n = pl.n;
+    P.k = pl.k;
+    P.b = pl.b;
+    P.vec_ok = (((uintptr_t)a.update | (uintptr_t)a.residual) & 15) == 0;
+    P.stream = static_cast<uint8_t*>(a.out_stream);
+    P.stream_cap = a.out_capacity;
+    P.stream_bytes = pl.stream_bytes;
+    P.out_mu = a.out_mu;
+    P.ctl = reinterpret_cast<Ctl*>(zero + pl.off_ctl);
+    P.hists = reinterpret_cast<Hists*>(zero + pl.off_hists);
+    P.mask = reinterpret_cast<uint32_t*>(mask + pl.off_mask);
+    P.mask_tile_cnt = reinterpret_cast<uint32_t*>(mask + pl.off_mask_tile);
+    P.sample_keys = reinterpret_cast<uint32_t*>(rest + pl.off_sample);
+    for (int s = 0; s < 2; ++s) {
+        P.cand[s] = reinterpret_cast<unsigned long long*>(rest + pl.off_cand[s]);
+        for (int j = 0; j < 2; ++j) P.buf[s][j] = reinterpret_cast<unsigned long long*>(rest + pl.off_buf[s][j]);
+        P.x_tile_cnt[s] = reinterpret_cast<uint32_t*>(rest + pl.off_xtile[s]);
+        P.s_target[s] = pl.s_target[s];
+    }
+    P.idx = reinterpret_cast<uint32_t*>(rest + pl.off_idx);
+    P.blk_len = reinterpret_cast<unsigned long long*>(rest + pl.off_blklen);
+    P.cap = pl.cap;
+    P.m = pl.m;
+    P.n_xtiles = pl.n_xtiles;
+    P.n_mask_words = pl.n_mask_words;
+    P.n_mask_tiles = pl.n_mask_tiles;
+    P.n_len_blocks = pl.n_len_blocks;
+    P.n_chunks = pl.n_chunks;
+    P.payload_offset = pl.payload_offset;
+    return P;
+}
 
 int sm_count() {
     int dev = 0, sms = 0;
@@ -104,6 +169,92 @@ inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsi
     if (g < 1) g = 1;
     if (g > max_blocks) g = max_blocks;
     return (unsigned)g;
+}
+
+// Blocks one problem gets for each kind of work.
+void block_counts(const Plan& pl, unsigned sms, unsigned nb[WK_COUNT]) {
+    nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8, sms * 4);
+    nb[WK_MAIN] = grid_for((unsigned long long)pl.n, kBlock * kPerThread, sms * kCollectBlocksPerSM);
+    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16, sms * 8);
+    nb[WK_XTILE] = grid_for(pl.n_xtiles, 1, sms * 8);
+    nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
+    nb[WK_MASK] = grid_for(pl.n_mask_tiles, 1, sms * 8);
+    nb[WK_LEN] = grid_for(pl.n_len_blocks, 1, sms * 8);
+    nb[WK_ONE] = 1;
+    nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
+}
+
+// Problem descriptors and prefix tables reach the device as kernel arguments, a few per launch:
+// no host staging buffer whose lifetime the caller would have to care about.
+constexpr int kProbsPerPut = 14;
+struct ProbChunk { Prob p[kProbsPerPut]; };
+static_assert(sizeof(ProbChunk) <= 3600, "kernel argument limit");
+static_assert(sizeof(DecodeArgs) % 4 == 0, "copied as words");
+__global__ void k_put_probs(Prob* dst, const ProbChunk src, int count) {
+    if ((int)threadIdx.x < count) dst[threadIdx.x] = src.p[threadIdx.x];
+}
+constexpr int kWordsPerPut = 896;
+struct WordChunk { uint32_t v[kWordsPerPut]; };
+__global__ void k_put_words(uint32_t* dst, const WordChunk src, int count) {
+    for (int i = threadIdx.x; i < count; i += blockDim.x) dst[i] = src.v[i];
+}
+
+// Zero the chunk table and payload area of every problem's output stream (batch form; a single
+// encode uses one memset instead).
+__global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
+    uint4* dst = reinterpret_cast<uint4*>(P.stream + SBC_HEADER_BYTES);
+    const unsigned long long count = (P.stream_bytes - SBC_HEADER_BYTES) / 16ull;
+    for (unsigned long long i = (unsigned long long)S.bx * kBlock + threadIdx.x; i < count;
+         i += (unsigned long long)S.nb * kBlock)
+        dst[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
+// a single problem) say how each kind of work is spread over the problems.
+void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK_COUNT],
+                   const uint32_t* const* prefix, cudaStream_t st, const sbc_cuda_event_t* marks) {
+    auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
+    auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs}; };
+    const dim3 blk(kBlock);
+    auto g1 = [&](int kind) { return dim3(grid[kind]); };
+    auto g2 = [&](int kind) { return dim3(grid[kind], 1, 2); };  // z = side
+
+    // 1. bounds from the sample, then the streaming accumulate + collect pass
+    k_sample0<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
+    k_sample1<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
+    mark(SBC_MARK_BOUNDS);
+    k_add_collect<<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
+    mark(SBC_MARK_COLLECT);
+
+    // 2. exact route over A (returns immediately unless the bounds failed)
+    k_exact_hist<0><<<g1(WK_EXACT), blk, 0, st>>>(B(WK_EXACT));
+    k_exact_hist<1><<<g1(WK_EXACT), blk, 0, st>>>(B(WK_EXACT));
+    k_exact_hist<2><<<g1(WK_EXACT), blk, 0, st>>>(B(WK_EXACT));
+    k_exact_tiecount<<<g1(WK_XTILE), blk, 0, st>>>(B(WK_XTILE));
+    k_exact_tiescan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
+    k_exact_collect<<<g1(WK_XTILE), blk, 0, st>>>(B(WK_XTILE));
+    mark(SBC_MARK_EXACT);
+
+    // 3. exact k-th composite of each candidate list, sums, side, mask of the kept positions
+    k_select_hist0<<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    k_select_filter<0><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    k_select_filter<1><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    k_select_filter<2><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    k_select_filter<3><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    k_select_filter<4><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    k_sums_decide<<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    k_mark<<<g1(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    mark(SBC_MARK_SELECT);
+
+    // 4. ordered positions, residual write-back, Golomb payload, chunk table, header
+    k_mask_scan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
+    k_mask_compact<<<g1(WK_MASK), blk, 0, st>>>(B(WK_MASK));
+    k_len_sum_residual<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));
+    k_len_scan_header<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
+    k_pack<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));
+    mark(SBC_MARK_END);
 }
 
 }  // namespace
@@ -154,112 +305,124 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
                   size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
                   sbc_cuda_stream_t stream, const sbc_cuda_event_t* marks) {
     Plan pl;
-    if (!update || !residual || !out_stream || !workspace) return SBC_EINVAL;
+    if (!workspace || ((uintptr_t)workspace & 255)) return SBC_EINVAL;
     if (!make_plan(numel, p, &pl)) return SBC_EINVAL;
-    if (((uintptr_t)update & 3) || ((uintptr_t)residual & 3) || ((uintptr_t)out_stream & 15) ||
-        ((uintptr_t)workspace & 255) || (out_mu && ((uintptr_t)out_mu & 3)))
-        return SBC_EINVAL;
-    {   // update and residual must not overlap
-        const uintptr_t u0 = (uintptr_t)update, r0 = (uintptr_t)residual, len = (uintptr_t)numel * 4;
-        if (u0 < r0 + len && r0 < u0 + len) return SBC_EINVAL;
-    }
-    if (out_capacity < pl.stream_bytes || workspace_bytes < pl.total) return SBC_ECAPACITY;
+    const TensorArgs a = {update, residual, out_stream, out_capacity, out_mu};
+    const int rc = check_tensor(a, pl);
+    if (rc != SBC_OK) return rc;
+    if (workspace_bytes < pl.total) return SBC_ECAPACITY;
 
+    // workspace: [descriptor][zero part][mask part][rest]
     uint8_t* ws = static_cast<uint8_t*>(workspace);
-    Prob P;
-    std::memset(&P, 0, sizeof(P));
-    P.update = update;
-    P.residual = residual;
-    P.n = pl.n;
-    P.k = pl.k;
-    P.b = pl.b;
-    P.vec_ok = (((uintptr_t)update | (uintptr_t)residual) & 15) == 0;
-    P.stream = static_cast<uint8_t*>(out_stream);
-    P.stream_cap = out_capacity;
-    P.out_mu = out_mu;
-    P.ctl = reinterpret_cast<Ctl*>(ws + pl.off_ctl);
-    P.hists = reinterpret_cast<Hists*>(ws + pl.off_hists);
-    P.sample_keys = reinterpret_cast<uint32_t*>(ws + pl.off_sample);
-    for (int s = 0; s < 2; ++s) {
-        P.cand[s] = reinterpret_cast<unsigned long long*>(ws + pl.off_cand[s]);
-        for (int j = 0; j < 2; ++j) P.buf[s][j] = reinterpret_cast<unsigned long long*>(ws + pl.off_buf[s][j]);
-        P.x_tile_cnt[s] = reinterpret_cast<uint32_t*>(ws + pl.off_xtile[s]);
-        P.s_target[s] = pl.s_target[s];
-    }
-    P.mask = reinterpret_cast<uint32_t*>(ws + pl.off_mask);
-    P.mask_tile_cnt = reinterpret_cast<uint32_t*>(ws + pl.off_mask_tile);
-    P.idx = reinterpret_cast<uint32_t*>(ws + pl.off_idx);
-    P.blk_len = reinterpret_cast<unsigned long long*>(ws + pl.off_blklen);
-    P.cap = pl.cap;
-    P.m = pl.m;
-    P.n_xtiles = pl.n_xtiles;
-    P.n_mask_words = pl.n_mask_words;
-    P.n_mask_tiles = pl.n_mask_tiles;
-    P.n_len_blocks = pl.n_len_blocks;
-    P.n_chunks = pl.n_chunks;
-    P.payload_offset = pl.payload_offset;
+    uint8_t* zero = ws + kProbSlotBytes;
+    uint8_t* mask = zero + pl.zero_bytes;
+    uint8_t* rest = mask + pl.mask_bytes;
+    const Prob P = make_prob(a, pl, zero, mask, rest);
+    Prob* d_prob = reinterpret_cast<Prob*>(ws);
 
     cudaStream_t st = stream;
-    auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
-    mark(SBC_MARK_BEGIN);
-    Prob* dP = reinterpret_cast<Prob*>(ws + pl.off_prob);
-    const unsigned sms = (unsigned)sm_count();
-    const dim3 blk(kBlock);
-
-    // scratch that must start at zero: control block + histograms, the kept
-    // mask and its per-tile counts (adjacent in the workspace), and the chunk table + payload area the packer ORs into
-    if (cudaMemsetAsync(ws + pl.zero_begin, 0, pl.zero_end - pl.zero_begin, st) != cudaSuccess ||
-        cudaMemsetAsync(P.mask, 0, pl.off_mask_tile + (size_t)pl.n_mask_tiles * 4 - pl.off_mask, st) != cudaSuccess ||
+    if (marks && marks[SBC_MARK_BEGIN]) cudaEventRecord(marks[SBC_MARK_BEGIN], st);
+    // scratch that must start at zero: control block + histograms, mask + tile counts (adjacent),
+    // and the chunk table + payload area the packer ORs into
+    if (cudaMemsetAsync(zero, 0, pl.zero_bytes + pl.mask_bytes, st) != cudaSuccess ||
         cudaMemsetAsync(P.stream + SBC_HEADER_BYTES, 0, pl.stream_bytes - SBC_HEADER_BYTES, st) != cudaSuccess)
         return SBC_ECUDA;
-    k_put_prob<<<1, 1, 0, st>>>(dP, P);
+    ProbChunk chunk;
+    chunk.p[0] = P;
+    k_put_probs<<<1, 32, 0, st>>>(d_prob, chunk, 1);
 
-    // 1. bounds from the sample, then the streaming accumulate + collect pass
-    const unsigned g_sample = grid_for(pl.m, kBlock * 8, sms * 4);
-    k_sample0<<<dim3(g_sample), blk, 0, st>>>(dP);
-    k_sample1<<<dim3(g_sample), blk, 0, st>>>(dP);
-    mark(SBC_MARK_BOUNDS);
-    const unsigned g_main = grid_for((unsigned long long)pl.n, kBlock * kPerThread, sms * kCollectBlocksPerSM);
-    if (P.vec_ok) k_add_collect<true><<<dim3(g_main), blk, 0, st>>>(dP);
-    else          k_add_collect<false><<<dim3(g_main), blk, 0, st>>>(dP);
+    unsigned grid[WK_COUNT];
+    block_counts(pl, (unsigned)sm_count(), grid);
+    launch_encode(d_prob, 1u, grid, nullptr, st, marks);
+    return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
+}
 
-    mark(SBC_MARK_COLLECT);
+size_t sbc_workspace_bytes_batch(int n_tensors, const sbc_tensor_desc* descs) {
+    if (n_tensors <= 0 || !descs) return 0;
+    size_t total = align_up((size_t)n_tensors * sizeof(Prob), 256) +
+                   align_up((size_t)WK_COUNT * (size_t)(n_tensors + 1) * 4, 256);
+    for (int t = 0; t < n_tensors; ++t) {
+        Plan pl;
+        if (!make_plan(descs[t].numel, descs[t].p, &pl)) return 0;
+        total += pl.zero_bytes + pl.mask_bytes + pl.rest_bytes;
+    }
+    return total;
+}
 
-    // 2. exact route over A (returns immediately unless the bounds failed)
-    const unsigned g_x = grid_for((unsigned long long)pl.n, kBlock * 16, sms * 8);
-    k_exact_hist<0><<<dim3(g_x), blk, 0, st>>>(dP);
-    k_exact_hist<1><<<dim3(g_x), blk, 0, st>>>(dP);
-    k_exact_hist<2><<<dim3(g_x), blk, 0, st>>>(dP);
-    const unsigned g_xt = grid_for(pl.n_xtiles, 1, sms * 8);
-    k_exact_tiecount<<<dim3(g_xt), blk, 0, st>>>(dP);
-    k_exact_tiescan<<<dim3(1), blk, 0, st>>>(dP);
-    k_exact_collect<<<dim3(g_xt), blk, 0, st>>>(dP);
+int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspace, size_t workspace_bytes,
+                     sbc_cuda_stream_t stream) {
+    if (n_tensors <= 0 || !descs || !workspace || ((uintptr_t)workspace & 255)) return SBC_EINVAL;
+    if (n_tensors > (1 << 20)) return SBC_EINVAL;
+    std::vector<Plan> plans((size_t)n_tensors);
+    size_t zero_total = 0, mask_total = 0, rest_total = 0;
+    for (int t = 0; t < n_tensors; ++t) {
+        if (!make_plan(descs[t].numel, descs[t].p, &plans[t])) return SBC_EINVAL;
+        const TensorArgs a = {descs[t].update, descs[t].residual, descs[t].out_stream, descs[t].out_capacity,
+                              descs[t].out_mu};
+        const int rc = check_tensor(a, plans[t]);
+        if (rc != SBC_OK) return rc;
+        zero_total += plans[t].zero_bytes;
+        mask_total += plans[t].mask_bytes;
+        rest_total += plans[t].rest_bytes;
+    }
+    const size_t probs_bytes = align_up((size_t)n_tensors * sizeof(Prob), 256);
+    const size_t prefix_bytes = align_up((size_t)WK_COUNT * (size_t)(n_tensors + 1) * 4, 256);
+    if (workspace_bytes < probs_bytes + prefix_bytes + zero_total + mask_total + rest_total) return SBC_ECAPACITY;
 
-    mark(SBC_MARK_EXACT);
+    // workspace: [descriptors][prefix tables][zero parts][mask parts][rests]
+    uint8_t* ws = static_cast<uint8_t*>(workspace);
+    Prob* d_probs = reinterpret_cast<Prob*>(ws);
+    uint32_t* d_prefix = reinterpret_cast<uint32_t*>(ws + probs_bytes);
+    uint8_t* zero = ws + probs_bytes + prefix_bytes;
+    uint8_t* mask = zero + zero_total;
+    uint8_t* rest = mask + mask_total;
 
-    // 3. exact k-th composite of each candidate list, sums, side, residual
-    const unsigned g_c = grid_for(pl.cap, kBlock * 4, sms * 4);
-    k_select_hist0<<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_select_filter<0><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_select_filter<1><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_select_filter<2><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_select_filter<3><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_select_filter<4><<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_sums_decide<<<dim3(g_c, 1, 2), blk, 0, st>>>(dP);
-    k_mark<<<dim3(g_c), blk, 0, st>>>(dP);
+    const unsigned sms = (unsigned)sm_count();
+    const size_t row_len = (size_t)n_tensors + 1;
+    std::vector<Prob> probs((size_t)n_tensors);
+    std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
+    {
+        uint8_t *z = zero, *m = mask, *r = rest;
+        for (int t = 0; t < n_tensors; ++t) {
+            const TensorArgs a = {descs[t].update, descs[t].residual, descs[t].out_stream,
+                                  descs[t].out_capacity, descs[t].out_mu};
+            probs[t] = make_prob(a, plans[t], z, m, r);
+            z += plans[t].zero_bytes;
+            m += plans[t].mask_bytes;
+            r += plans[t].rest_bytes;
+            unsigned nb[WK_COUNT];
+            block_counts(plans[t], sms, nb);
+            for (int kind = 0; kind < WK_COUNT; ++kind) {
+                uint32_t* row = prefix.data() + (size_t)kind * row_len;
+                const unsigned long long next = (unsigned long long)row[t] + nb[kind];
+                if (next > 0x7fffffffull) return SBC_EINVAL;  // more blocks than one grid can hold
+                row[t + 1] = (uint32_t)next;
+            }
+        }
+    }
 
-    mark(SBC_MARK_SELECT);
-
-    // 4. Golomb stage
-    const unsigned g_m = grid_for(pl.n_mask_tiles, 1, sms * 8);
-    k_mask_scan<<<dim3(1), blk, 0, st>>>(dP);
-    k_mask_compact<<<dim3(g_m), blk, 0, st>>>(dP);
-    const unsigned g_l = grid_for(pl.n_len_blocks, 1, sms * 8);
-    k_len_sum_residual<<<dim3(g_l), blk, 0, st>>>(dP);
-    k_len_scan_header<<<dim3(1), blk, 0, st>>>(dP);
-    k_pack<<<dim3(g_l), blk, 0, st>>>(dP);
-    mark(SBC_MARK_END);
-
+    cudaStream_t st = stream;
+    if (cudaMemsetAsync(zero, 0, zero_total + mask_total, st) != cudaSuccess) return SBC_ECUDA;
+    for (int first = 0; first < n_tensors; first += kProbsPerPut) {
+        ProbChunk chunk;
+        const int count = std::min(kProbsPerPut, n_tensors - first);
+        for (int i = 0; i < count; ++i) chunk.p[i] = probs[first + i];
+        k_put_probs<<<1, 32, 0, st>>>(d_probs + first, chunk, count);
+    }
+    for (size_t first = 0; first < prefix.size(); first += kWordsPerPut) {
+        WordChunk chunk;
+        const int count = (int)std::min<size_t>(kWordsPerPut, prefix.size() - first);
+        std::memcpy(chunk.v, prefix.data() + first, (size_t)count * 4);
+        k_put_words<<<1, 256, 0, st>>>(d_prefix + first, chunk, count);
+    }
+    unsigned grid[WK_COUNT];
+    const uint32_t* d_rows[WK_COUNT];
+    for (int kind = 0; kind < WK_COUNT; ++kind) {
+        d_rows[kind] = d_prefix + (size_t)kind * row_len;
+        grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
+    }
+    k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors});
+    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -317,8 +480,8 @@ int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cu
     Prob P;
     Ctl c;
     const uint8_t* ws = static_cast<const uint8_t*>(workspace);
-    if (cudaMemcpyAsync(&P, ws + pl.off_prob, sizeof(P), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-        cudaMemcpyAsync(&c, ws + pl.off_ctl, sizeof(c), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+    if (cudaMemcpyAsync(&P, ws, sizeof(P), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        cudaMemcpyAsync(&c, ws + kProbSlotBytes + pl.off_ctl, sizeof(c), cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return SBC_ECUDA;
     host_out->status = c.status;
@@ -345,7 +508,8 @@ int sbc_encode_host(const float* update_host, float* update_dev, float* residual
     Plan pl;
     if (!make_plan(numel, p, &pl)) return SBC_EINVAL;
     if (workspace_bytes < pl.total) return SBC_ECAPACITY;
-    float* mu_dev = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + pl.off_mu);
+    float* mu_dev = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kProbSlotBytes + pl.zero_bytes +
+                                             pl.mask_bytes + pl.off_mu);
     const int rc = sbc_encode(update_dev, residual_dev, numel, p, stream_dev, out_capacity, mu_dev,
                               workspace, workspace_bytes, stream);
     if (rc != SBC_OK) return rc;
@@ -412,6 +576,54 @@ int sbc_decode_accumulate(const void* const* streams, int n_clients, float* out_
         const unsigned grid = grid_for(max_groups, kDecodeThreads / 32, sms * 5);
         k_decode_accumulate<<<grid, kDecodeThreads, 0, stream>>>(a);
     }
+    return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
+}
+
+size_t sbc_decode_workspace_bytes_batch(int n_tensors) {
+    return n_tensors > 0 ? align_up((size_t)n_tensors * sizeof(DecodeArgs), 256) : 0;
+}
+
+int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_desc* descs, uint32_t* status_dev,
+                                void* workspace, size_t workspace_bytes, sbc_cuda_stream_t stream) {
+    if (n_tensors <= 0 || n_tensors > 65535 || n_clients <= 0 || n_clients > kMaxClientsPerLaunch || !descs ||
+        !workspace || ((uintptr_t)workspace & 255) || ((uintptr_t)status_dev & 3))
+        return SBC_EINVAL;
+    if (workspace_bytes < sbc_decode_workspace_bytes_batch(n_tensors)) return SBC_ECAPACITY;
+    long long max_numel = 0;
+    for (int t = 0; t < n_tensors; ++t) {
+        const sbc_decode_desc& d = descs[t];
+        if (!d.streams || !d.out_dense || ((uintptr_t)d.out_dense & 3) || d.numel <= 0 || d.numel >= (1ll << 31))
+            return SBC_EINVAL;
+        for (int c = 0; c < n_clients; ++c)
+            if (!d.streams[c] || ((uintptr_t)d.streams[c] & 15)) return SBC_EINVAL;
+        max_numel = std::max<long long>(max_numel, d.numel);
+    }
+    // argument blocks reach the device as kernel arguments, a few per launch
+    constexpr int kArgsPerPut = 3584 / (int)sizeof(DecodeArgs);
+    static_assert(kArgsPerPut >= 1, "argument block too large");
+    DecodeArgs* d_args = static_cast<DecodeArgs*>(workspace);
+    for (int first = 0; first < n_tensors; first += kArgsPerPut) {
+        WordChunk chunk;
+        const int count = std::min(kArgsPerPut, n_tensors - first);
+        for (int i = 0; i < count; ++i) {
+            DecodeArgs a;
+            std::memset(&a, 0, sizeof(a));
+            a.n_clients = n_clients;
+            for (int c = 0; c < n_clients; ++c) a.streams[c] = static_cast<const uint8_t*>(descs[first + i].streams[c]);
+            a.out = descs[first + i].out_dense;
+            a.n = descs[first + i].numel;
+            a.status = status_dev;
+            std::memcpy(reinterpret_cast<uint8_t*>(chunk.v) + (size_t)i * sizeof(DecodeArgs), &a, sizeof(a));
+        }
+        const int words = count * (int)(sizeof(DecodeArgs) / 4);
+        k_put_words<<<1, 256, 0, stream>>>(reinterpret_cast<uint32_t*>(d_args + first), chunk, words);
+    }
+    const unsigned long long max_groups =
+        (unsigned long long)n_clients *
+        (unsigned long long)((max_numel + kChunkCodewords * 32 - 1) / (kChunkCodewords * 32));
+    const unsigned gx = grid_for(max_groups, kDecodeThreads / 32,
+                                 std::max(16u, (unsigned)sm_count() * 5u / (unsigned)n_tensors));
+    k_decode_accumulate_batch<<<dim3(gx, (unsigned)n_tensors), kDecodeThreads, 0, stream>>>(d_args);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

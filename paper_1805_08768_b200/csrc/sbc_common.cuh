@@ -73,7 +73,7 @@ struct Hists {
 };
 
 // Everything a kernel needs to know about one encode problem.  Lives in
-// device memory (first bytes of the workspace); kernels index it by blockIdx.y.
+// device memory (first bytes of the workspace).
 struct Prob {
     const float* update;
     float* residual;
@@ -83,6 +83,7 @@ struct Prob {
     int vec_ok;                 // 1: update and residual are 16-byte aligned
     uint8_t* stream;            // container out
     unsigned long long stream_cap;
+    unsigned long long stream_bytes;  // bytes sbc_stream_bytes(n, p) promises to stay within
     float* out_mu;
     Ctl* ctl;
     Hists* hists;
@@ -99,6 +100,39 @@ struct Prob {
     uint32_t s_target[2];       // rank looked up in the sample, per side
     uint32_t n_xtiles, n_mask_words, n_mask_tiles, n_len_blocks, n_chunks;
     unsigned long long payload_offset;
+};
+
+// A launch serves one problem (prefix == nullptr: the grid is that problem's) or a batch: then
+// prefix[i] .. prefix[i+1] are the blocks of problem i for this kernel's kind of work, and a block
+// finds its problem by binary search.
+struct Batch {
+    const Prob* probs;
+    const uint32_t* prefix;  // n_probs + 1 entries, or nullptr
+    uint32_t n_probs;
+};
+struct Slot {
+    const Prob* P;
+    uint32_t bx;  // block index within the problem
+    uint32_t nb;  // blocks working on the problem
+};
+__device__ __forceinline__ Slot resolve(const Batch& B) {
+    Slot s;
+    if (B.prefix == nullptr) {
+        s.P = B.probs; s.bx = blockIdx.x; s.nb = gridDim.x;
+        return s;
+    }
+    uint32_t lo = 0u, hi = B.n_probs;  // invariant: prefix[lo] <= blockIdx.x < prefix[hi]
+    while (hi - lo > 1u) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (B.prefix[mid] <= blockIdx.x) lo = mid; else hi = mid;
+    }
+    s.P = B.probs + lo; s.bx = blockIdx.x - B.prefix[lo]; s.nb = B.prefix[lo + 1] - B.prefix[lo];
+    return s;
+}
+
+// Kinds of work a kernel's grid is sized by (one prefix table per kind in a batch).
+enum WorkKind : int {
+    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_MASK, WK_LEN, WK_ONE, WK_STREAM, WK_COUNT
 };
 
 // ---------------------------------------------------------------- keys

@@ -103,7 +103,7 @@ struct BitReader {
 // contiguous bit range, copied once (coalesced) into shared memory; then every
 // lane parses its chunk's kChunkCodewords codewords from there (Algorithm 4)
 // and adds mu at each position (Algorithm 1, server sum).
-__global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate(const DecodeArgs args) {
+__device__ __forceinline__ void decode_body(const DecodeArgs& args) {
     __shared__ StreamView s_view[kMaxClientsPerLaunch];
     __shared__ uint32_t s_first[kMaxClientsPerLaunch + 1];  // first work item (group) of each client
     __shared__ uint32_t s_words[kDecodeThreads / 32][kDecodeWarpWords];
@@ -266,6 +266,13 @@ __global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate(const Deco
         }
         if (err && args.status) atomicOr(args.status, err);
     }
+}
+
+__global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate(const DecodeArgs args) { decode_body(args); }
+
+// Batch form: blockIdx.y selects the tensor; its arguments sit in device memory.
+__global__ void __launch_bounds__(kDecodeThreads) k_decode_accumulate_batch(const DecodeArgs* __restrict__ all) {
+    decode_body(all[blockIdx.y]);
 }
 
 }  // namespace sbc

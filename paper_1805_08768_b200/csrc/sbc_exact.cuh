@@ -15,8 +15,9 @@ __device__ __forceinline__ bool exact_route_active(const Ctl* ctl) {
 // One radix level (0: key bits 31..21, 1: bits 20..10, 2: bits 9..0) for both
 // sides; the last block extends the two prefixes.
 template <int LEVEL>
-__global__ void __launch_bounds__(kBlock) k_exact_hist(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_exact_hist(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     constexpr int kBins = (LEVEL == 2) ? 1024 : kHistBins;
@@ -27,8 +28,8 @@ __global__ void __launch_bounds__(kBlock) k_exact_hist(const Prob* __restrict__ 
     __syncthreads();
     const uint32_t pre[2] = {ctl->x_prefix[0], ctl->x_prefix[1]};
     const float* __restrict__ A = P.residual;
-    const long long stride = (long long)gridDim.x * kBlock;
-    for (long long base = (long long)blockIdx.x * kBlock; base < P.n; base += stride) {
+    const long long stride = (long long)S.nb * kBlock;
+    for (long long base = (long long)S.bx * kBlock; base < P.n; base += stride) {
         const long long i = base + threadIdx.x;
         const bool valid = i < P.n;
         const uint32_t key = valid ? key_of_bits(__float_as_uint(A[i])) : 0u;
@@ -60,7 +61,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_hist(const Prob* __restrict__ 
             }
         }
     }
-    if (last_block_ticket(&ctl->done[ST_XH0 + LEVEL], gridDim.x)) {
+    if (last_block_ticket(&ctl->done[ST_XH0 + LEVEL], S.nb)) {
         for (int s = 0; s < 2; ++s) {
             const uint32_t rank = (LEVEL == 0) ? (uint32_t)P.k : ctl->x_rank[s];
             block_pick_desc(P.hists->x[LEVEL][s], kBins, false, rank, s_scan, &s_pick);
@@ -87,15 +88,16 @@ __device__ __forceinline__ bool tie_ranks_needed(const Ctl* ctl, int s) {
 }
 
 // Entries equal to the threshold, per tile of kXTile elements.
-__global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     if (!tie_ranks_needed(ctl, 0) && !tie_ranks_needed(ctl, 1)) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     const uint32_t thr[2] = {ctl->x_thr[0], ctl->x_thr[1]};
     const float* __restrict__ A = P.residual;
-    for (uint32_t tile = blockIdx.x; tile < P.n_xtiles; tile += gridDim.x) {
+    for (uint32_t tile = S.bx; tile < P.n_xtiles; tile += S.nb) {
         uint32_t c = 0u;  // side 0 in the low half, side 1 in the high half
         for (int j = 0; j < kXTile / kBlock; ++j) {
             const long long i = (long long)tile * kXTile + j * kBlock + threadIdx.x;
@@ -115,8 +117,9 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Prob* __restric
 }
 
 // In-place exclusive scan of the per-tile tie counts (one block).
-__global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     if (!tie_ranks_needed(ctl, 0) && !tie_ranks_needed(ctl, 1)) return;
@@ -142,8 +145,9 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Prob* __restrict
 // threshold plus the lowest-index ties.  Each warp owns 512 consecutive
 // elements of a tile and walks them 32 at a time, so the rank of a tie is
 // (ties in earlier tiles) + (earlier warps) + (earlier steps) + (lower lanes).
-__global__ void __launch_bounds__(kBlock) k_exact_collect(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     constexpr int kSteps = kXTile / kBlock;  // 16 steps of 32 lanes per warp
@@ -155,7 +159,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_collect(const Prob* __restrict
     const uint32_t take[2] = {ctl->x_ties_take[0], ctl->x_ties_take[1]};
     const bool ranked[2] = {tie_ranks_needed(ctl, 0), tie_ranks_needed(ctl, 1)};
     const float* __restrict__ A = P.residual;
-    for (uint32_t tile = blockIdx.x; tile < P.n_xtiles; tile += gridDim.x) {
+    for (uint32_t tile = S.bx; tile < P.n_xtiles; tile += S.nb) {
         const long long wbase = (long long)tile * kXTile + (long long)warp * (kXTile / (kBlock / 32));
         uint32_t key[kSteps];
         unsigned inb = 0u;

@@ -26,15 +26,16 @@ __device__ __forceinline__ long long sample_element(const Prob& P, uint32_t i) {
 
 // Level 0: keys of the sampled A values, histogram of their top 11 bits; the
 // last block locates the bin of the target rank for each side.
-__global__ void __launch_bounds__(kBlock) k_sample0(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     __shared__ uint32_t s_hist[kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     __shared__ Pick s_pick;
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
-    for (uint32_t base = blockIdx.x * kBlock; base < P.m; base += gridDim.x * kBlock) {
+    for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
         const uint32_t i = base + threadIdx.x;
         const bool valid = i < P.m;
         uint32_t key = 0u;
@@ -51,7 +52,7 @@ __global__ void __launch_bounds__(kBlock) k_sample0(const Prob* __restrict__ pro
         const uint32_t v = s_hist[i];
         if (v) atomicAdd(&P.hists->s0[i], v);
     }
-    if (last_block_ticket(&ctl->done[ST_SAMPLE0], gridDim.x)) {
+    if (last_block_ticket(&ctl->done[ST_SAMPLE0], S.nb)) {
         for (int s = 0; s < 2; ++s) {
             block_pick_desc(P.hists->s0, kHistBins, s == 1, P.s_target[s], s_scan, &s_pick);
             if (threadIdx.x == 0) {
@@ -66,8 +67,9 @@ __global__ void __launch_bounds__(kBlock) k_sample0(const Prob* __restrict__ pro
 
 // Level 1: next 11 bits inside the located bins; the last block turns the
 // 22-bit prefixes into the two float bounds used by the candidate pass.
-__global__ void __launch_bounds__(kBlock) k_sample1(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_sample1(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     __shared__ uint32_t s_hist[2][kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -75,7 +77,7 @@ __global__ void __launch_bounds__(kBlock) k_sample1(const Prob* __restrict__ pro
     for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) (&s_hist[0][0])[i] = 0u;
     __syncthreads();
     const uint32_t bin0[2] = {ctl->s_bin0[0], ctl->s_bin0[1]};
-    for (uint32_t base = blockIdx.x * kBlock; base < P.m; base += gridDim.x * kBlock) {
+    for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
         const uint32_t i = base + threadIdx.x;
         const bool valid = i < P.m;
         const uint32_t key = valid ? P.sample_keys[i] : 0u;
@@ -90,7 +92,7 @@ __global__ void __launch_bounds__(kBlock) k_sample1(const Prob* __restrict__ pro
         const uint32_t v = (&s_hist[0][0])[i];
         if (v) atomicAdd(&P.hists->s1[0][0] + i, v);
     }
-    if (last_block_ticket(&ctl->done[ST_SAMPLE1], gridDim.x)) {
+    if (last_block_ticket(&ctl->done[ST_SAMPLE1], S.nb)) {
         for (int s = 0; s < 2; ++s) {
             block_pick_desc(P.hists->s1[s], kHistBins, false, ctl->s_rank[s], s_scan, &s_pick);
             if (threadIdx.x == 0) {
@@ -117,9 +119,9 @@ constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 wa
 // through per-warp shared-memory staging so that the global list counters see
 // one atomic per hundred or so candidates.  Each thread has eight 16-byte
 // loads in flight before it touches any of them.
-template <bool VEC>
-__global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     __shared__ unsigned long long s_stage[kBlock / 32][2][kStage];
     const int warp = threadIdx.x >> 5, lane = lane_id();
@@ -143,13 +145,13 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__
     };
 
     const long long n_chunks = (n + kWarpChunk - 1) / kWarpChunk;
-    const long long total_warps = (long long)gridDim.x * (kBlock / 32);
-    for (long long chunk = (long long)blockIdx.x * (kBlock / 32) + warp; chunk < n_chunks;
+    const long long total_warps = (long long)S.nb * (kBlock / 32);
+    for (long long chunk = (long long)S.bx * (kBlock / 32) + warp; chunk < n_chunks;
          chunk += total_warps) {
         const long long base = chunk * kWarpChunk;
         float a[kPerThread];
         unsigned inb = 0u;
-        const bool vec_layout = VEC && (base + kWarpChunk <= n);  // warp-uniform
+        const bool vec_layout = P.vec_ok && (base + kWarpChunk <= n);  // warp-uniform
         if (vec_layout) {
             // thread owns elements base + (u*32 + lane)*4 + {0..3}, u = 0..kUnroll-1
             const float4* __restrict__ u4 = reinterpret_cast<const float4*>(U + base) + lane;
@@ -230,7 +232,7 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Prob* __restrict__
     flush(1);
     if (bad) atomicOr(&ctl->status, SBC_STATUS_NONFINITE);
 
-    if (last_block_ticket(&ctl->done[ST_COLLECT], gridDim.x)) {
+    if (last_block_ticket(&ctl->done[ST_COLLECT], S.nb)) {
         if (threadIdx.x == 0) {
             const uint32_t c0 = __ldcg(&ctl->cand_cnt[0]), c1 = __ldcg(&ctl->cand_cnt[1]);
             const bool ok = c0 >= (uint32_t)P.k && c0 <= P.cap && c1 >= (uint32_t)P.k && c1 <= P.cap;

@@ -14,8 +14,9 @@ namespace sbc {
 // ---------------------------------------------------------------- mask -> sorted positions
 
 // In-place exclusive scan of the kept-position counts per mask tile (one block).
-__global__ void __launch_bounds__(kBlock) k_mask_scan(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_mask_scan(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -47,13 +48,14 @@ __global__ void __launch_bounds__(kBlock) k_mask_scan(const Prob* __restrict__ p
 }
 
 // Mask -> ascending position list.
-__global__ void __launch_bounds__(kBlock) k_mask_compact(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_mask_compact(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     if (P.ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     static_assert(kMaskTileWords / kBlock == 8, "eight words per thread");
     constexpr int kPer = kMaskTileWords / kBlock;
-    for (uint32_t tile = blockIdx.x; tile < P.n_mask_tiles; tile += gridDim.x) {
+    for (uint32_t tile = S.bx; tile < P.n_mask_tiles; tile += S.nb) {
         uint32_t words[kPer];
         uint32_t c = 0u;
         const uint32_t w0 = tile * kMaskTileWords + threadIdx.x * kPer;
@@ -95,14 +97,15 @@ __device__ __forceinline__ unsigned long long codeword_len(const Prob& P, uint32
 // Bits of each block of kLenBlock codewords, and -- since this is the first
 // walk over the ordered position list -- the residual write-back
 // R_j = A_j - mu at the kept positions (Algorithm 1), in address order.
-__global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     if (P.ctl->status) return;
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     constexpr int kPer = kLenBlock / kBlock;
     const float mu = P.ctl->mu32;
     const uint32_t k = (uint32_t)P.k;
-    for (uint32_t blk = blockIdx.x; blk < P.n_len_blocks; blk += gridDim.x) {
+    for (uint32_t blk = S.bx; blk < P.n_len_blocks; blk += S.nb) {
         const uint32_t i0 = blk * kLenBlock + threadIdx.x * kPer;
         uint32_t pos[kPer];
         float r[kPer];
@@ -134,8 +137,9 @@ __device__ __forceinline__ void store_u64(uint8_t* p, unsigned long long v) {
 
 // Scan of the per-block bit counts; also writes the container header, always,
 // so that a failed encode still leaves a header that says why.
-__global__ void __launch_bounds__(kBlock) k_len_scan_header(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_len_scan_header(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     const bool ok = ctl->status == 0u;  // uniform: nothing writes status while this kernel runs
@@ -195,15 +199,16 @@ __device__ __forceinline__ void or_bits(uint32_t* words, unsigned long long off,
     if (lo) atomicOr(words + w + 1, __byte_perm(lo, 0u, 0x0123));
 }
 
-__global__ void __launch_bounds__(kBlock) k_pack(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_pack(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     if (P.ctl->status) return;
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     constexpr int kPer = kLenBlock / kBlock;
     uint32_t* words = reinterpret_cast<uint32_t*>(P.stream + P.payload_offset);
     uint8_t* table = P.stream + SBC_HEADER_BYTES;
     const int b = P.b;
-    for (uint32_t blk = blockIdx.x; blk < P.n_len_blocks; blk += gridDim.x) {
+    for (uint32_t blk = S.bx; blk < P.n_len_blocks; blk += S.nb) {
         unsigned long long len[kPer];
         uint32_t gap[kPer];
         unsigned long long sum = 0ull;

@@ -17,8 +17,9 @@ __device__ __forceinline__ uint32_t digit_of(unsigned long long c, int level) {
 }
 
 // Histogram of the top digit over a whole candidate list.  grid.z = side.
-__global__ void __launch_bounds__(kBlock) k_select_hist0(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
@@ -29,7 +30,7 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Prob* __restrict_
     __syncthreads();
     const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
     const unsigned long long* __restrict__ src = P.cand[s];
-    for (uint32_t base = blockIdx.x * kBlock; base < cnt; base += gridDim.x * kBlock) {
+    for (uint32_t base = S.bx * kBlock; base < cnt; base += S.nb * kBlock) {
         const uint32_t i = base + threadIdx.x;
         const bool valid = i < cnt;
         const unsigned long long c = valid ? src[i] : 0ull;
@@ -40,7 +41,7 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Prob* __restrict_
         const uint32_t v = s_hist[i];
         if (v) atomicAdd(&P.hists->b[0][s][i], v);
     }
-    if (last_block_ticket(&ctl->done[ST_BH0_S0 + s], gridDim.x)) {
+    if (last_block_ticket(&ctl->done[ST_BH0_S0 + s], S.nb)) {
         block_pick_desc(P.hists->b[0][s], kHistBins, false, (uint32_t)P.k, s_scan, &s_pick);
         if (threadIdx.x == 0) {
             ctl->b_prefix[s] = s_pick.bin;
@@ -53,8 +54,9 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Prob* __restrict_
 // Keep the entries whose level-L digit is the selected one, histogram their
 // next digit, and let the last block select at level L+1.  grid.z = side.
 template <int LEVEL>
-__global__ void __launch_bounds__(kBlock) k_select_filter(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
@@ -69,7 +71,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Prob* __restrict
     const unsigned long long* __restrict__ src = (LEVEL == 0) ? P.cand[s] : P.buf[s][(LEVEL - 1) & 1];
     unsigned long long* __restrict__ dst = P.buf[s][LEVEL & 1];
     const uint32_t sel = (uint32_t)ctl->b_prefix[s] & ((1u << digit_bits(LEVEL)) - 1u);
-    for (uint32_t base = blockIdx.x * (kBlock * kItems); base < cnt; base += gridDim.x * (kBlock * kItems)) {
+    for (uint32_t base = S.bx * (kBlock * kItems); base < cnt; base += S.nb * (kBlock * kItems)) {
         unsigned long long c[kItems];
         unsigned match = 0u;
 #pragma unroll
@@ -94,7 +96,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Prob* __restrict
         const uint32_t v = s_hist[i];
         if (v) atomicAdd(&P.hists->b[LEVEL + 1][s][i], v);
     }
-    if (last_block_ticket(&ctl->done[ST_BF0_S0 + 2 * LEVEL + s], gridDim.x)) {
+    if (last_block_ticket(&ctl->done[ST_BF0_S0 + 2 * LEVEL + s], S.nb)) {
         block_pick_desc(P.hists->b[LEVEL + 1][s], 1 << digit_bits(LEVEL + 1), false,
                         ctl->b_rank[s], s_scan, &s_pick);
         if (threadIdx.x == 0) {
@@ -172,8 +174,9 @@ __device__ double bins_to_double(const long long* bins) {
 // sum of up to 2^39 of them and integer addition makes the result independent
 // of the order of the atomics.  grid.z = side.  The last block turns the bins
 // into mu+ and mu- and takes Algorithm 2's side decision.
-__global__ void __launch_bounds__(kBlock) k_sums_decide(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
@@ -190,7 +193,7 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Prob* __restrict__
     const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
     const int bin_b = bin_a + 1;
     long long acc_a = 0, acc_b = 0;
-    for (uint32_t i = blockIdx.x * kBlock + threadIdx.x; i < cnt; i += gridDim.x * kBlock) {
+    for (uint32_t i = S.bx * kBlock + threadIdx.x; i < cnt; i += S.nb * kBlock) {
         const unsigned long long c = src[i];
         if (c < thr) continue;
         const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
@@ -216,7 +219,7 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Prob* __restrict__
         const unsigned long long v = s_bins[0][threadIdx.x];
         if (v) atomicAdd(reinterpret_cast<unsigned long long*>(&ctl->bins[s][threadIdx.x]), v);
     }
-    if (last_block_ticket(&ctl->done[ST_SUM], gridDim.x * gridDim.z)) {
+    if (last_block_ticket(&ctl->done[ST_SUM], S.nb * gridDim.z)) {
         s_bins[0][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[0][threadIdx.x]);
         s_bins[1][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[1][threadIdx.x]);
         __syncthreads();
@@ -239,8 +242,9 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Prob* __restrict__
 
 // One mask bit per kept position of the chosen side (for the ordered
 // compaction that follows) and the number of kept positions per mask tile.
-__global__ void __launch_bounds__(kBlock) k_mark(const Prob* __restrict__ probs) {
-    const Prob& P = probs[blockIdx.y];
+__global__ void __launch_bounds__(kBlock) k_mark(const Batch B) {
+    const Slot S = resolve(B);
+    const Prob& P = *S.P;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = (int)ctl->side;
@@ -249,7 +253,7 @@ __global__ void __launch_bounds__(kBlock) k_mark(const Prob* __restrict__ probs)
     const unsigned long long* __restrict__ src = P.cand[s];
     constexpr int kTileShift = 16;  // kMaskTileWords * 32 = 65536 positions per tile
     static_assert(kMaskTileWords * 32 == (1 << kTileShift), "tile size");
-    for (uint32_t base = blockIdx.x * kBlock; base < cnt; base += gridDim.x * kBlock) {
+    for (uint32_t base = S.bx * kBlock; base < cnt; base += S.nb * kBlock) {
         const uint32_t i = base + threadIdx.x;
         const unsigned long long c = (i < cnt) ? src[i] : 0ull;
         const bool kept = (i < cnt) && c >= thr;

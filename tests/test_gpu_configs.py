@@ -27,17 +27,27 @@ POOL = ThreadPoolExecutor(max_workers=16)
 class Client:
     """Device-side state of one client: residuals, streams, scratch (allocated once, reused per round)."""
 
-    def __init__(self, sizes, p):
-        self.p = p
+    def __init__(self, sizes, p, batched=True):
+        self.p, self.batched = p, batched
         self.res = [torch.zeros(n, dtype=torch.float32, device=DEV) for n in sizes]
         self.out = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=DEV) for n in sizes]
         self.mu = [torch.empty(1, dtype=torch.float32, device=DEV) for _ in sizes]
-        self.ws = torch.empty(max(sbc.sbc_workspace_bytes(n, p) for n in sizes), dtype=torch.uint8, device=DEV)
+        if batched:
+            ws_bytes = sbc.sbc_workspace_bytes_batch(sizes, [p] * len(sizes))
+        else:
+            ws_bytes = max(sbc.sbc_workspace_bytes(n, p) for n in sizes)
+        self.ws = torch.full((ws_bytes + 256,), 0xCD, dtype=torch.uint8, device=DEV)
+        self.ws_bytes = ws_bytes
 
     def encode_round(self, tensors):
-        for t, upd in enumerate(tensors):
-            sbc.sbc_encode(torch.from_numpy(upd).to(DEV), self.res[t], self.p, self.out[t], self.mu[t], self.ws)
+        ups = [torch.from_numpy(u).to(DEV) for u in tensors]
+        if self.batched:
+            sbc.sbc_encode_batch(ups, self.res, [self.p] * len(ups), self.out, self.mu, self.ws[: self.ws_bytes])
+        else:
+            for t, u in enumerate(ups):
+                sbc.sbc_encode(u, self.res[t], self.p, self.out[t], self.mu[t], self.ws[: self.ws_bytes])
         torch.cuda.synchronize()
+        assert bool((self.ws[self.ws_bytes:] == 0xCD).all()), "write past the workspace"
         got = []
         for t in range(len(tensors)):
             info = sbc.sbc_stream_info_get(self.out[t])
@@ -100,10 +110,19 @@ def test_config4_eight_clients_decode_aggregate():
     # one dense aggregate per tensor, the 8 streams decoded and summed on the device
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
     dense = [torch.zeros(n, dtype=torch.float32, device=DEV) for n in sizes]
-    for t in range(len(sizes)):
-        sbc.sbc_decode_accumulate([cl.out[t] for cl, _ in per_client], dense[t], status=status)
+    dws = torch.empty(sbc.sbc_decode_workspace_bytes_batch(len(sizes)), dtype=torch.uint8, device=DEV)
+    sbc.sbc_decode_accumulate_batch([[cl.out[t] for cl, _ in per_client] for t in range(len(sizes))],
+                                    dense, dws, status=status)
     torch.cuda.synchronize()
     assert status.item() == 0
+    # the one-tensor-per-call form gives the same sums (to the stated tolerance)
+    dense1 = [torch.zeros(n, dtype=torch.float32, device=DEV) for n in sizes]
+    for t in range(0, len(sizes), 7):
+        sbc.sbc_decode_accumulate([cl.out[t] for cl, _ in per_client], dense1[t], status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    for t in range(0, len(sizes), 7):
+        assert torch.allclose(dense[t], dense1[t], rtol=0, atol=1e-6)
 
     def expected(t):
         want = np.zeros(sizes[t], dtype=np.float32)
@@ -170,3 +189,30 @@ def test_config5_flat_2p30_sweep_against_independent_selection():
         assert status.item() == 0
         assert torch.equal(dense.view(torch.int32), expect.view(torch.int32)), f"p={p}: decoded tensor differs"
         del dense, expect, residual, kept
+
+
+def test_batch_and_single_tensor_calls_agree_with_mixed_sparsities():
+    rng = np.random.default_rng(77)
+    sizes = [1, 64, 1000, 4097, 70001, 300000, 2_000_003, 5, 131072]
+    ps = [0.5, 0.001, 0.01, 0.1, 0.001, 0.01, 0.001, 0.2, 0.0001]
+    ups = [(rng.standard_normal(n) * 1e-3).astype(np.float32) for n in sizes]
+    ups[3][:] = 0.0                                  # an all-zero tensor in the middle of the batch (exact route)
+    res0 = [(rng.standard_normal(n) * 1e-3).astype(np.float32) for n in sizes]
+    res0[3][:] = 0.0
+    want_res = [r.copy() for r in res0]
+    want = [oracle.encode(u, r, p) for u, r, p in zip(ups, want_res, ps)]
+    d_up = [torch.from_numpy(u).to(DEV) for u in ups]
+    d_res = [torch.from_numpy(r).to(DEV) for r in res0]
+    outs = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=DEV) for n, p in zip(sizes, ps)]
+    mus = [torch.empty(1, dtype=torch.float32, device=DEV) for _ in sizes]
+    ws = torch.empty(sbc.sbc_workspace_bytes_batch(sizes, ps), dtype=torch.uint8, device=DEV)
+    sbc.sbc_encode_batch(d_up, d_res, ps, outs, mus, ws)
+    torch.cuda.synchronize()
+    for t, (ws_, wm) in enumerate(want):
+        info = sbc.sbc_stream_info_get(outs[t])
+        assert np.array_equal(outs[t][: info.total_bytes].cpu().numpy(), ws_), f"tensor {t}"
+        assert np.float32(mus[t].item()).view(np.uint32) == wm.view(np.uint32)
+        assert np.array_equal(d_res[t].cpu().numpy().view(np.uint32), want_res[t].view(np.uint32))
+    # a bad descriptor anywhere in the batch: nothing runs
+    with pytest.raises(sbc.SbcError):
+        sbc.sbc_encode_batch(d_up, d_res, ps[:-1] + [1.5], outs, mus, ws)

@@ -223,6 +223,52 @@ def sbc_encode_batch(updates: Sequence[torch.Tensor], residuals: Sequence[torch.
     _check(code, "sbc_encode_batch")
 
 
+class EncodeBatch:
+    """The marshalled descriptors of a batch, built once and reused every round (same tensors)."""
+
+    def __init__(self, updates, residuals, ps, out_streams, out_mus, workspace):
+        self.n = len(updates)
+        self.descs = (TensorDesc * self.n)()
+        self.keep = (list(updates), list(residuals), list(out_streams), list(out_mus), workspace)
+        for t in range(self.n):
+            _dev_f32(updates[t], "update")
+            _dev_f32(residuals[t], "residual")
+            d = self.descs[t]
+            d.update, d.residual, d.numel, d.p = updates[t].data_ptr(), residuals[t].data_ptr(), updates[t].numel(), float(ps[t])
+            d.out_stream, d.out_capacity, d.out_mu = out_streams[t].data_ptr(), out_streams[t].numel(), out_mus[t].data_ptr()
+        self.ws_ptr, self.ws_bytes = workspace.data_ptr(), workspace.numel()
+
+    def run(self, stream=None) -> None:
+        _check(lib().sbc_encode_batch(self.n, self.descs, self.ws_ptr, self.ws_bytes, _cuda_stream(stream)),
+               "sbc_encode_batch")
+
+
+class DecodeBatch:
+    """The marshalled descriptors of a batched decode, built once and reused."""
+
+    def __init__(self, streams_per_tensor, out_denses, workspace, status=None):
+        self.n = len(out_denses)
+        self.n_clients = len(streams_per_tensor[0])
+        self.descs = (DecodeDesc * self.n)()
+        self.keep = [streams_per_tensor, out_denses, workspace, status]
+        for t in range(self.n):
+            if len(streams_per_tensor[t]) != self.n_clients:
+                raise ValueError("every tensor needs the same number of client streams")
+            _dev_f32(out_denses[t], "out_dense")
+            ptrs = (C.c_void_p * self.n_clients)(*[s.data_ptr() for s in streams_per_tensor[t]])
+            self.keep.append(ptrs)
+            self.descs[t].streams = ptrs
+            self.descs[t].out_dense = out_denses[t].data_ptr()
+            self.descs[t].numel = out_denses[t].numel()
+        self.status_ptr = status.data_ptr() if status is not None else None
+        self.ws_ptr, self.ws_bytes = workspace.data_ptr(), workspace.numel()
+
+    def run(self, stream=None) -> None:
+        _check(lib().sbc_decode_accumulate_batch(self.n, self.n_clients, self.descs, self.status_ptr,
+                                                 self.ws_ptr, self.ws_bytes, _cuda_stream(stream)),
+               "sbc_decode_accumulate_batch")
+
+
 def sbc_decode_workspace_bytes_batch(n_tensors: int) -> int:
     return int(lib().sbc_decode_workspace_bytes_batch(n_tensors))
 

@@ -51,7 +51,16 @@ bool make_plan(long long n, double p, Plan* pl) {
     pl->k = k;
     pl->b = b;
     pl->cap = (uint32_t)std::min<long long>(n, 2 * k + 1024);
-    pl->m = n <= (long long)kSampleMax ? (uint32_t)n : kSampleMax;
+    // Sample size: a sixteenth of the tensor, but at least 128/p elements (so that the rank looked
+    // up below is >= 128 and its relative margin stays small) and at most 2^20; whole 32-element
+    // segments unless the sample is the whole tensor.
+    {
+        const long long want = std::max<long long>(n / 16, (long long)std::ceil(128.0 / p));
+        long long m = std::min<long long>(std::min<long long>(want, (long long)kSampleMax), n);
+        if (m < n) m = std::max<long long>(32, m / 32 * 32);
+        if (m >= n || (n >> 5) < (m >> 5)) m = n;
+        pl->m = (uint32_t)m;
+    }
     // Rank looked up in the sample.  If the sample is the whole tensor the
     // rank is k itself; otherwise the expected rank plus six standard
     // deviations of a binomial count (and a little), so that the bound falls
@@ -171,12 +180,15 @@ inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsi
     return (unsigned)g;
 }
 
-// Blocks one problem gets for each kind of work.
-void block_counts(const Plan& pl, unsigned sms, unsigned nb[WK_COUNT]) {
-    nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8, sms * 4);
+// Blocks one problem gets for each kind of work.  `coarsen` (1 for a single problem) makes the
+// blocks of the sample and exact-route kernels that many times larger: every block of those
+// kernels pays for clearing and flushing a shared-memory histogram, and a batch of hundreds of
+// problems has parallelism to spare.
+void block_counts(const Plan& pl, unsigned sms, unsigned coarsen, unsigned nb[WK_COUNT]) {
+    nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8 * coarsen, sms * 4);
     nb[WK_MAIN] = grid_for((unsigned long long)pl.n, kBlock * kPerThread, sms * kCollectBlocksPerSM);
-    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16, sms * 8);
-    nb[WK_XTILE] = grid_for(pl.n_xtiles, 1, sms * 8);
+    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarsen, sms * 8);
+    nb[WK_XTILE] = grid_for(pl.n_xtiles, coarsen, sms * 8);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
     nb[WK_MASK] = grid_for(pl.n_mask_tiles, 1, sms * 8);
     nb[WK_LEN] = grid_for(pl.n_len_blocks, 1, sms * 8);
@@ -184,26 +196,15 @@ void block_counts(const Plan& pl, unsigned sms, unsigned nb[WK_COUNT]) {
     nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
 }
 
-// Problem descriptors and prefix tables reach the device as kernel arguments, a few per launch:
-// no host staging buffer whose lifetime the caller would have to care about.
-constexpr int kProbsPerPut = 14;
-struct ProbChunk { Prob p[kProbsPerPut]; };
-static_assert(sizeof(ProbChunk) <= 3600, "kernel argument limit");
-static_assert(sizeof(DecodeArgs) % 4 == 0, "copied as words");
-__global__ void k_put_probs(Prob* dst, const ProbChunk src, int count) {
-    if ((int)threadIdx.x < count) dst[threadIdx.x] = src.p[threadIdx.x];
-}
-constexpr int kWordsPerPut = 896;
-struct WordChunk { uint32_t v[kWordsPerPut]; };
-__global__ void k_put_words(uint32_t* dst, const WordChunk src, int count) {
-    for (int i = threadIdx.x; i < count; i += blockDim.x) dst[i] = src.v[i];
-}
+// A single problem's descriptor reaches the device as a kernel argument.
+__global__ void k_put_prob(Prob* dst, const Prob src) { *dst = src; }
 
 // Zero the chunk table and payload area of every problem's output stream (batch form; a single
 // encode uses one memset instead).
 __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     uint4* dst = reinterpret_cast<uint4*>(P.stream + SBC_HEADER_BYTES);
     const unsigned long long count = (P.stream_bytes - SBC_HEADER_BYTES) / 16ull;
     for (unsigned long long i = (unsigned long long)S.bx * kBlock + threadIdx.x; i < count;
@@ -327,12 +328,10 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     if (cudaMemsetAsync(zero, 0, pl.zero_bytes + pl.mask_bytes, st) != cudaSuccess ||
         cudaMemsetAsync(P.stream + SBC_HEADER_BYTES, 0, pl.stream_bytes - SBC_HEADER_BYTES, st) != cudaSuccess)
         return SBC_ECUDA;
-    ProbChunk chunk;
-    chunk.p[0] = P;
-    k_put_probs<<<1, 32, 0, st>>>(d_prob, chunk, 1);
+    k_put_prob<<<1, 1, 0, st>>>(d_prob, P);
 
     unsigned grid[WK_COUNT];
-    block_counts(pl, (unsigned)sm_count(), grid);
+    block_counts(pl, (unsigned)sm_count(), 1u, grid);
     launch_encode(d_prob, 1u, grid, nullptr, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
@@ -378,6 +377,10 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     uint8_t* rest = mask + mask_total;
 
     const unsigned sms = (unsigned)sm_count();
+    // aim at about eight blocks per SM over the whole batch for the histogram-carrying kernels
+    unsigned long long fine_blocks = 0;
+    for (int t = 0; t < n_tensors; ++t) fine_blocks += (plans[t].m + kBlock * 8 - 1) / (kBlock * 8);
+    const unsigned coarsen = (unsigned)std::min<unsigned long long>(64, std::max<unsigned long long>(1, fine_blocks / (sms * 8ull)));
     const size_t row_len = (size_t)n_tensors + 1;
     std::vector<Prob> probs((size_t)n_tensors);
     std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
@@ -391,7 +394,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
             m += plans[t].mask_bytes;
             r += plans[t].rest_bytes;
             unsigned nb[WK_COUNT];
-            block_counts(plans[t], sms, nb);
+            block_counts(plans[t], sms, coarsen, nb);
             for (int kind = 0; kind < WK_COUNT; ++kind) {
                 uint32_t* row = prefix.data() + (size_t)kind * row_len;
                 const unsigned long long next = (unsigned long long)row[t] + nb[kind];
@@ -403,17 +406,15 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
 
     cudaStream_t st = stream;
     if (cudaMemsetAsync(zero, 0, zero_total + mask_total, st) != cudaSuccess) return SBC_ECUDA;
-    for (int first = 0; first < n_tensors; first += kProbsPerPut) {
-        ProbChunk chunk;
-        const int count = std::min(kProbsPerPut, n_tensors - first);
-        for (int i = 0; i < count; ++i) chunk.p[i] = probs[first + i];
-        k_put_probs<<<1, 32, 0, st>>>(d_probs + first, chunk, count);
-    }
-    for (size_t first = 0; first < prefix.size(); first += kWordsPerPut) {
-        WordChunk chunk;
-        const int count = (int)std::min<size_t>(kWordsPerPut, prefix.size() - first);
-        std::memcpy(chunk.v, prefix.data() + first, (size_t)count * 4);
-        k_put_words<<<1, 256, 0, st>>>(d_prefix + first, chunk, count);
+    // Descriptors and tables are adjacent in the workspace: one copy from a host buffer laid out
+    // the same way.  The source is ordinary (pageable) memory, which the runtime reads out before
+    // cudaMemcpyAsync returns, so the buffer may die with this call.
+    {
+        std::vector<uint8_t> image(probs_bytes + prefix.size() * 4, 0);
+        std::memcpy(image.data(), probs.data(), probs.size() * sizeof(Prob));
+        std::memcpy(image.data() + probs_bytes, prefix.data(), prefix.size() * 4);
+        if (cudaMemcpyAsync(ws, image.data(), image.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return SBC_ECUDA;
     }
     unsigned grid[WK_COUNT];
     const uint32_t* d_rows[WK_COUNT];
@@ -598,25 +599,21 @@ int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_d
             if (!d.streams[c] || ((uintptr_t)d.streams[c] & 15)) return SBC_EINVAL;
         max_numel = std::max<long long>(max_numel, d.numel);
     }
-    // argument blocks reach the device as kernel arguments, a few per launch
-    constexpr int kArgsPerPut = 3584 / (int)sizeof(DecodeArgs);
-    static_assert(kArgsPerPut >= 1, "argument block too large");
+    // one copy of all argument blocks from an ordinary host buffer (read out before the call returns)
     DecodeArgs* d_args = static_cast<DecodeArgs*>(workspace);
-    for (int first = 0; first < n_tensors; first += kArgsPerPut) {
-        WordChunk chunk;
-        const int count = std::min(kArgsPerPut, n_tensors - first);
-        for (int i = 0; i < count; ++i) {
-            DecodeArgs a;
-            std::memset(&a, 0, sizeof(a));
-            a.n_clients = n_clients;
-            for (int c = 0; c < n_clients; ++c) a.streams[c] = static_cast<const uint8_t*>(descs[first + i].streams[c]);
-            a.out = descs[first + i].out_dense;
-            a.n = descs[first + i].numel;
-            a.status = status_dev;
-            std::memcpy(reinterpret_cast<uint8_t*>(chunk.v) + (size_t)i * sizeof(DecodeArgs), &a, sizeof(a));
+    {
+        std::vector<DecodeArgs> args((size_t)n_tensors);
+        std::memset(static_cast<void*>(args.data()), 0, args.size() * sizeof(DecodeArgs));
+        for (int t = 0; t < n_tensors; ++t) {
+            args[t].n_clients = n_clients;
+            for (int c = 0; c < n_clients; ++c) args[t].streams[c] = static_cast<const uint8_t*>(descs[t].streams[c]);
+            args[t].out = descs[t].out_dense;
+            args[t].n = descs[t].numel;
+            args[t].status = status_dev;
         }
-        const int words = count * (int)(sizeof(DecodeArgs) / 4);
-        k_put_words<<<1, 256, 0, stream>>>(reinterpret_cast<uint32_t*>(d_args + first), chunk, words);
+        if (cudaMemcpyAsync(d_args, args.data(), args.size() * sizeof(DecodeArgs), cudaMemcpyHostToDevice,
+                            stream) != cudaSuccess)
+            return SBC_ECUDA;
     }
     const unsigned long long max_groups =
         (unsigned long long)n_clients *

@@ -115,18 +115,27 @@ struct Slot {
     uint32_t bx;  // block index within the problem
     uint32_t nb;  // blocks working on the problem
 };
-__device__ __forceinline__ Slot resolve(const Batch& B) {
+// Finds the block's problem and copies its descriptor into shared memory (all threads call):
+// kernels then read the descriptor at shared-memory cost and the compiler knows that their global
+// stores cannot change it.
+__device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
     Slot s;
+    const Prob* src;
     if (B.prefix == nullptr) {
-        s.P = B.probs; s.bx = blockIdx.x; s.nb = gridDim.x;
-        return s;
+        src = B.probs; s.bx = blockIdx.x; s.nb = gridDim.x;
+    } else {
+        uint32_t lo = 0u, hi = B.n_probs;  // invariant: prefix[lo] <= blockIdx.x < prefix[hi]
+        while (hi - lo > 1u) {
+            const uint32_t mid = (lo + hi) >> 1;
+            if (B.prefix[mid] <= blockIdx.x) lo = mid; else hi = mid;
+        }
+        src = B.probs + lo; s.bx = blockIdx.x - B.prefix[lo]; s.nb = B.prefix[lo + 1] - B.prefix[lo];
     }
-    uint32_t lo = 0u, hi = B.n_probs;  // invariant: prefix[lo] <= blockIdx.x < prefix[hi]
-    while (hi - lo > 1u) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (B.prefix[mid] <= blockIdx.x) lo = mid; else hi = mid;
-    }
-    s.P = B.probs + lo; s.bx = blockIdx.x - B.prefix[lo]; s.nb = B.prefix[lo + 1] - B.prefix[lo];
+    static_assert(sizeof(Prob) % 8 == 0, "copied as 8-byte words");
+    for (int i = threadIdx.x; i < (int)(sizeof(Prob) / 8); i += blockDim.x)
+        reinterpret_cast<unsigned long long*>(s_prob)[i] = reinterpret_cast<const unsigned long long*>(src)[i];
+    __syncthreads();
+    s.P = s_prob;
     return s;
 }
 

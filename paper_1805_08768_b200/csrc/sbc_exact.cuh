@@ -16,8 +16,9 @@ __device__ __forceinline__ bool exact_route_active(const Ctl* ctl) {
 // sides; the last block extends the two prefixes.
 template <int LEVEL>
 __global__ void __launch_bounds__(kBlock) k_exact_hist(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     constexpr int kBins = (LEVEL == 2) ? 1024 : kHistBins;
@@ -89,8 +90,9 @@ __device__ __forceinline__ bool tie_ranks_needed(const Ctl* ctl, int s) {
 
 // Entries equal to the threshold, per tile of kXTile elements.
 __global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     if (!tie_ranks_needed(ctl, 0) && !tie_ranks_needed(ctl, 1)) return;
@@ -118,8 +120,9 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Batch B) {
 
 // In-place exclusive scan of the per-tile tie counts (one block).
 __global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     if (!tie_ranks_needed(ctl, 0) && !tie_ranks_needed(ctl, 1)) return;
@@ -146,8 +149,9 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Batch B) {
 // elements of a tile and walks them 32 at a time, so the rank of a tie is
 // (ties in earlier tiles) + (earlier warps) + (earlier steps) + (lower lanes).
 __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     constexpr int kSteps = kXTile / kBlock;  // 16 steps of 32 lanes per warp

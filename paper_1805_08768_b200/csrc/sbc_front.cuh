@@ -27,8 +27,9 @@ __device__ __forceinline__ long long sample_element(const Prob& P, uint32_t i) {
 // Level 0: keys of the sampled A values, histogram of their top 11 bits; the
 // last block locates the bin of the target rank for each side.
 __global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     __shared__ uint32_t s_hist[kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -68,8 +69,9 @@ __global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
 // Level 1: next 11 bits inside the located bins; the last block turns the
 // 22-bit prefixes into the two float bounds used by the candidate pass.
 __global__ void __launch_bounds__(kBlock) k_sample1(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     __shared__ uint32_t s_hist[2][kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -120,8 +122,9 @@ constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 wa
 // one atomic per hundred or so candidates.  Each thread has eight 16-byte
 // loads in flight before it touches any of them.
 __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     __shared__ unsigned long long s_stage[kBlock / 32][2][kStage];
     const int warp = threadIdx.x >> 5, lane = lane_id();
@@ -131,6 +134,10 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
     float* __restrict__ R = P.residual;
     uint32_t wcnt[2] = {0u, 0u};
     bool bad = false;
+    const uint32_t cap = P.cap;
+    unsigned long long* const cand0 = P.cand[0];
+    unsigned long long* const cand1 = P.cand[1];
+    const bool vec_ok = P.vec_ok != 0;
 
     auto flush = [&](int s) {
         if (wcnt[s] == 0u) return;  // warp-uniform
@@ -139,7 +146,7 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
         if (lane == 0) base = atomicAdd(&ctl->cand_cnt[s], wcnt[s]);
         base = __shfl_sync(0xffffffffu, base, 0);
         for (uint32_t i = lane; i < wcnt[s]; i += 32)
-            if (base + i < P.cap) P.cand[s][base + i] = s_stage[warp][s][i];
+            if (base + i < cap) (s ? cand1 : cand0)[base + i] = s_stage[warp][s][i];
         __syncwarp();
         wcnt[s] = 0u;
     };
@@ -151,7 +158,7 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
         const long long base = chunk * kWarpChunk;
         float a[kPerThread];
         unsigned inb = 0u;
-        const bool vec_layout = P.vec_ok && (base + kWarpChunk <= n);  // warp-uniform
+        const bool vec_layout = vec_ok && (base + kWarpChunk <= n);  // warp-uniform
         if (vec_layout) {
             // thread owns elements base + (u*32 + lane)*4 + {0..3}, u = 0..kUnroll-1
             const float4* __restrict__ u4 = reinterpret_cast<const float4*>(U + base) + lane;
@@ -219,7 +226,7 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
                         const long long e = vec_layout ? base + (long long)(((j >> 2) * 32 + lane) * 4 + (j & 3))
                                                        : base + j * 32 + lane;
                         const unsigned long long c = make_composite(side_key(s, key_of_bits(bits)), (uint32_t)e);
-                        if (direct) { if (off < P.cap) P.cand[s][off] = c; }
+                        if (direct) { if (off < cap) (s ? cand1 : cand0)[off] = c; }
                         else s_stage[warp][s][off] = c;
                         ++off;
                     }

@@ -15,8 +15,9 @@ namespace sbc {
 
 // In-place exclusive scan of the kept-position counts per mask tile (one block).
 __global__ void __launch_bounds__(kBlock) k_mask_scan(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -49,8 +50,9 @@ __global__ void __launch_bounds__(kBlock) k_mask_scan(const Batch B) {
 
 // Mask -> ascending position list.
 __global__ void __launch_bounds__(kBlock) k_mask_compact(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     if (P.ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     static_assert(kMaskTileWords / kBlock == 8, "eight words per thread");
@@ -98,8 +100,9 @@ __device__ __forceinline__ unsigned long long codeword_len(const Prob& P, uint32
 // walk over the ordered position list -- the residual write-back
 // R_j = A_j - mu at the kept positions (Algorithm 1), in address order.
 __global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     if (P.ctl->status) return;
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     constexpr int kPer = kLenBlock / kBlock;
@@ -138,8 +141,9 @@ __device__ __forceinline__ void store_u64(uint8_t* p, unsigned long long v) {
 // Scan of the per-block bit counts; also writes the container header, always,
 // so that a failed encode still leaves a header that says why.
 __global__ void __launch_bounds__(kBlock) k_len_scan_header(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     const bool ok = ctl->status == 0u;  // uniform: nothing writes status while this kernel runs
@@ -200,8 +204,9 @@ __device__ __forceinline__ void or_bits(uint32_t* words, unsigned long long off,
 }
 
 __global__ void __launch_bounds__(kBlock) k_pack(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     if (P.ctl->status) return;
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     constexpr int kPer = kLenBlock / kBlock;

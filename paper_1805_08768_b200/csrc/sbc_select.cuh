@@ -18,8 +18,9 @@ __device__ __forceinline__ uint32_t digit_of(unsigned long long c, int level) {
 
 // Histogram of the top digit over a whole candidate list.  grid.z = side.
 __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
@@ -55,8 +56,9 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
 // next digit, and let the last block select at level L+1.  grid.z = side.
 template <int LEVEL>
 __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
@@ -175,8 +177,9 @@ __device__ double bins_to_double(const long long* bins) {
 // of the order of the atomics.  grid.z = side.  The last block turns the bins
 // into mu+ and mu- and takes Algorithm 2's side decision.
 __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
@@ -243,8 +246,9 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
 // One mask bit per kept position of the chosen side (for the ordered
 // compaction that follows) and the number of kept positions per mask tile.
 __global__ void __launch_bounds__(kBlock) k_mark(const Batch B) {
-    const Slot S = resolve(B);
-    const Prob& P = *S.P;
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = (int)ctl->side;

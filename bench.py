@@ -151,11 +151,11 @@ def run_reference(args):
 # ------------------------------------------------------------------ our arm
 
 # DRAM traffic of one k_add_collect launch from the ncu capture summarised in
-# profiles/k_add_collect_2p26_ncu_full.md: (536.93 + 225.39) MB at 2^26 elements, p = 1e-2.
+# profiles/k_add_collect_2p26_ncu_full.md: (536.91 + 227.77) MB at 2^26 elements, p = 1e-2.
 # Traffic is proportional to the element count, so it is scaled by numel / 2^26.  Valid only for
 # the kernel source it was taken from: a different hash of the file reports null.
-NCU_TRAFFIC_BYTES_AT_2P26 = 762.32e6
-NCU_TRAFFIC_SOURCE_SHA256 = "4353e0316d569b6791d5f74546ddfe74a17da3dc4f9339e8d8586bf04367a59d"
+NCU_TRAFFIC_BYTES_AT_2P26 = 764.68e6
+NCU_TRAFFIC_SOURCE_SHA256 = "ae35c48d5bdd0eeca1577e1cdbbb1ab9ed720b9b80b92356b35afcdc9d69beb6"
 
 
 def measured_traffic(numel: int):

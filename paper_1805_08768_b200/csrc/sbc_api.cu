@@ -24,20 +24,20 @@ static_assert(sizeof(Prob) <= kProbSlotBytes, "descriptor must fit its slot");
 // Host-side plan of one encode problem: scalar parameters and the layout of its scratch, which
 // comes in three parts so that a batch can keep each part contiguous across problems:
 //   zero part  control block + radix histograms (cleared before every call)
-//   mask part  kept-position bitmask + per-tile counts (cleared before every call)
+//   tile part  per-tile counts of kept positions, both sides, and bucket fill counters (cleared)
 //   rest       everything that needs no clearing
 struct Plan {
     long long n, k;
     int b;
-    uint32_t cap, m, n_xtiles, n_mask_words, n_mask_tiles, n_len_blocks, n_chunks;
+    uint32_t cap, m, n_xtiles, n_tiles, n_len_blocks, n_chunks;
     uint32_t s_target[2];
     unsigned long long payload_offset;
     size_t stream_bytes;
     size_t zero_bytes, off_ctl, off_hists;                 // offsets inside the zero part
-    size_t mask_bytes, off_mask, off_mask_tile;            // inside the mask part
+    size_t tile_bytes, off_tile_cnt[2], off_tile_fill;     // inside the tile part
     size_t rest_bytes, off_mu, off_sample, off_cand[2], off_buf[2][2], off_xtile[2], off_idx,
         off_blklen;                                        // inside the rest
-    size_t total;                                          // single problem: slot + zero + mask + rest
+    size_t total;                                          // single problem: slot + zero + tile + rest
 };
 
 bool valid_p(double p) { return p > 0.0 && p < 1.0; }
@@ -76,8 +76,7 @@ bool make_plan(long long n, double p, Plan* pl) {
     }
     pl->s_target[0] = pl->s_target[1] = target;
     pl->n_xtiles = (uint32_t)((n + kXTile - 1) / kXTile);
-    pl->n_mask_words = (uint32_t)align_up((size_t)((n + 31) / 32), 4);
-    pl->n_mask_tiles = (pl->n_mask_words + kMaskTileWords - 1) / kMaskTileWords;
+    pl->n_tiles = (uint32_t)((n + (1ll << kTileShift) - 1) >> kTileShift);
     pl->n_len_blocks = (uint32_t)((k + kLenBlock - 1) / kLenBlock);
     pl->n_chunks = (uint32_t)((k + kChunkCodewords - 1) / kChunkCodewords);
     pl->payload_offset = SBC_HEADER_BYTES + (unsigned long long)pl->n_chunks * SBC_CHUNK_ENTRY_BYTES;
@@ -91,9 +90,9 @@ bool make_plan(long long n, double p, Plan* pl) {
     pl->off_hists = take(sizeof(Hists));
     pl->zero_bytes = off;
     off = 0;
-    pl->off_mask = take((size_t)pl->n_mask_words * 4);
-    pl->off_mask_tile = take((size_t)pl->n_mask_tiles * 4);
-    pl->mask_bytes = off;
+    for (int s = 0; s < 2; ++s) pl->off_tile_cnt[s] = take((size_t)(pl->n_tiles + 1) * 4);
+    pl->off_tile_fill = take((size_t)pl->n_tiles * 4);
+    pl->tile_bytes = off;
     off = 0;
     pl->off_mu = take(sizeof(float));  // where the host-buffer form parks mu
     pl->off_sample = take((size_t)pl->m * 4);
@@ -104,7 +103,7 @@ bool make_plan(long long n, double p, Plan* pl) {
     pl->off_idx = take((size_t)k * 4);
     pl->off_blklen = take((size_t)pl->n_len_blocks * 8);
     pl->rest_bytes = off;
-    pl->total = kProbSlotBytes + pl->zero_bytes + pl->mask_bytes + pl->rest_bytes;
+    pl->total = kProbSlotBytes + pl->zero_bytes + pl->tile_bytes + pl->rest_bytes;
     return true;
 }
 
@@ -128,7 +127,7 @@ int check_tensor(const TensorArgs& a, const Plan& pl) {
     return SBC_OK;
 }
 
-Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* mask, uint8_t* rest) {
+Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile, uint8_t* rest) {
     Prob P;
     std::memset(&P, 0, sizeof(P));
     P.update = a.update;
@@ -143,8 +142,8 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* mask
     P.out_mu = a.out_mu;
     P.ctl = reinterpret_cast<Ctl*>(zero + pl.off_ctl);
     P.hists = reinterpret_cast<Hists*>(zero + pl.off_hists);
-    P.mask = reinterpret_cast<uint32_t*>(mask + pl.off_mask);
-    P.mask_tile_cnt = reinterpret_cast<uint32_t*>(mask + pl.off_mask_tile);
+    for (int s = 0; s < 2; ++s) P.tile_cnt[s] = reinterpret_cast<uint32_t*>(tile + pl.off_tile_cnt[s]);
+    P.tile_fill = reinterpret_cast<uint32_t*>(tile + pl.off_tile_fill);
     P.sample_keys = reinterpret_cast<uint32_t*>(rest + pl.off_sample);
     for (int s = 0; s < 2; ++s) {
         P.cand[s] = reinterpret_cast<unsigned long long*>(rest + pl.off_cand[s]);
@@ -157,8 +156,7 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* mask
     P.cap = pl.cap;
     P.m = pl.m;
     P.n_xtiles = pl.n_xtiles;
-    P.n_mask_words = pl.n_mask_words;
-    P.n_mask_tiles = pl.n_mask_tiles;
+    P.n_tiles = pl.n_tiles;
     P.n_len_blocks = pl.n_len_blocks;
     P.n_chunks = pl.n_chunks;
     P.payload_offset = pl.payload_offset;
@@ -190,7 +188,8 @@ void block_counts(const Plan& pl, unsigned sms, unsigned coarsen, unsigned nb[WK
     nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarsen, sms * 8);
     nb[WK_XTILE] = grid_for(pl.n_xtiles, coarsen, sms * 8);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
-    nb[WK_MASK] = grid_for(pl.n_mask_tiles, 1, sms * 8);
+    nb[WK_SCATTER] = grid_for(pl.cap, kBlock * 4, sms * 8);
+    nb[WK_MASK] = grid_for(pl.n_tiles, 1, sms * 8);
     nb[WK_LEN] = grid_for(pl.n_len_blocks, 1, sms * 8);
     nb[WK_ONE] = 1;
     nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
@@ -238,7 +237,7 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     k_exact_collect<<<g1(WK_XTILE), blk, 0, st>>>(B(WK_XTILE));
     mark(SBC_MARK_EXACT);
 
-    // 3. exact k-th composite of each candidate list, sums, side, mask of the kept positions
+    // 3. exact k-th composite of each candidate list, sums, side
     k_select_hist0<<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
     k_select_filter<0><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
     k_select_filter<1><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
@@ -246,12 +245,12 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     k_select_filter<3><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
     k_select_filter<4><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
     k_sums_decide<<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
-    k_mark<<<g1(WK_CAND), blk, 0, st>>>(B(WK_CAND));
     mark(SBC_MARK_SELECT);
 
     // 4. ordered positions, residual write-back, Golomb payload, chunk table, header
-    k_mask_scan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
-    k_mask_compact<<<g1(WK_MASK), blk, 0, st>>>(B(WK_MASK));
+    k_tile_scan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
+    k_scatter<<<g1(WK_SCATTER), blk, 0, st>>>(B(WK_SCATTER));
+    k_tile_sort<<<g1(WK_MASK), blk, 0, st>>>(B(WK_MASK));
     k_len_sum_residual<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));
     k_len_scan_header<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
     k_pack<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));
@@ -313,19 +312,19 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     if (rc != SBC_OK) return rc;
     if (workspace_bytes < pl.total) return SBC_ECAPACITY;
 
-    // workspace: [descriptor][zero part][mask part][rest]
+    // workspace: [descriptor][zero part][tile part][rest]
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     uint8_t* zero = ws + kProbSlotBytes;
-    uint8_t* mask = zero + pl.zero_bytes;
-    uint8_t* rest = mask + pl.mask_bytes;
-    const Prob P = make_prob(a, pl, zero, mask, rest);
+    uint8_t* tile = zero + pl.zero_bytes;
+    uint8_t* rest = tile + pl.tile_bytes;
+    const Prob P = make_prob(a, pl, zero, tile, rest);
     Prob* d_prob = reinterpret_cast<Prob*>(ws);
 
     cudaStream_t st = stream;
     if (marks && marks[SBC_MARK_BEGIN]) cudaEventRecord(marks[SBC_MARK_BEGIN], st);
-    // scratch that must start at zero: control block + histograms, mask + tile counts (adjacent),
+    // scratch that must start at zero: control block + histograms, tile counters (adjacent),
     // and the chunk table + payload area the packer ORs into
-    if (cudaMemsetAsync(zero, 0, pl.zero_bytes + pl.mask_bytes, st) != cudaSuccess ||
+    if (cudaMemsetAsync(zero, 0, pl.zero_bytes + pl.tile_bytes, st) != cudaSuccess ||
         cudaMemsetAsync(P.stream + SBC_HEADER_BYTES, 0, pl.stream_bytes - SBC_HEADER_BYTES, st) != cudaSuccess)
         return SBC_ECUDA;
     k_put_prob<<<1, 1, 0, st>>>(d_prob, P);
@@ -343,7 +342,7 @@ size_t sbc_workspace_bytes_batch(int n_tensors, const sbc_tensor_desc* descs) {
     for (int t = 0; t < n_tensors; ++t) {
         Plan pl;
         if (!make_plan(descs[t].numel, descs[t].p, &pl)) return 0;
-        total += pl.zero_bytes + pl.mask_bytes + pl.rest_bytes;
+        total += pl.zero_bytes + pl.tile_bytes + pl.rest_bytes;
     }
     return total;
 }
@@ -353,7 +352,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     if (n_tensors <= 0 || !descs || !workspace || ((uintptr_t)workspace & 255)) return SBC_EINVAL;
     if (n_tensors > (1 << 20)) return SBC_EINVAL;
     std::vector<Plan> plans((size_t)n_tensors);
-    size_t zero_total = 0, mask_total = 0, rest_total = 0;
+    size_t zero_total = 0, tile_total = 0, rest_total = 0;
     for (int t = 0; t < n_tensors; ++t) {
         if (!make_plan(descs[t].numel, descs[t].p, &plans[t])) return SBC_EINVAL;
         const TensorArgs a = {descs[t].update, descs[t].residual, descs[t].out_stream, descs[t].out_capacity,
@@ -361,20 +360,20 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         const int rc = check_tensor(a, plans[t]);
         if (rc != SBC_OK) return rc;
         zero_total += plans[t].zero_bytes;
-        mask_total += plans[t].mask_bytes;
+        tile_total += plans[t].tile_bytes;
         rest_total += plans[t].rest_bytes;
     }
     const size_t probs_bytes = align_up((size_t)n_tensors * sizeof(Prob), 256);
     const size_t prefix_bytes = align_up((size_t)WK_COUNT * (size_t)(n_tensors + 1) * 4, 256);
-    if (workspace_bytes < probs_bytes + prefix_bytes + zero_total + mask_total + rest_total) return SBC_ECAPACITY;
+    if (workspace_bytes < probs_bytes + prefix_bytes + zero_total + tile_total + rest_total) return SBC_ECAPACITY;
 
-    // workspace: [descriptors][prefix tables][zero parts][mask parts][rests]
+    // workspace: [descriptors][prefix tables][zero parts][tile parts][rests]
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     Prob* d_probs = reinterpret_cast<Prob*>(ws);
     uint32_t* d_prefix = reinterpret_cast<uint32_t*>(ws + probs_bytes);
     uint8_t* zero = ws + probs_bytes + prefix_bytes;
-    uint8_t* mask = zero + zero_total;
-    uint8_t* rest = mask + mask_total;
+    uint8_t* tile = zero + zero_total;
+    uint8_t* rest = tile + tile_total;
 
     const unsigned sms = (unsigned)sm_count();
     // aim at about eight blocks per SM over the whole batch for the histogram-carrying kernels
@@ -385,13 +384,13 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     std::vector<Prob> probs((size_t)n_tensors);
     std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
     {
-        uint8_t *z = zero, *m = mask, *r = rest;
+        uint8_t *z = zero, *m = tile, *r = rest;
         for (int t = 0; t < n_tensors; ++t) {
             const TensorArgs a = {descs[t].update, descs[t].residual, descs[t].out_stream,
                                   descs[t].out_capacity, descs[t].out_mu};
             probs[t] = make_prob(a, plans[t], z, m, r);
             z += plans[t].zero_bytes;
-            m += plans[t].mask_bytes;
+            m += plans[t].tile_bytes;
             r += plans[t].rest_bytes;
             unsigned nb[WK_COUNT];
             block_counts(plans[t], sms, coarsen, nb);
@@ -405,7 +404,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     }
 
     cudaStream_t st = stream;
-    if (cudaMemsetAsync(zero, 0, zero_total + mask_total, st) != cudaSuccess) return SBC_ECUDA;
+    if (cudaMemsetAsync(zero, 0, zero_total + tile_total, st) != cudaSuccess) return SBC_ECUDA;
     // Descriptors and tables are adjacent in the workspace: one copy from a host buffer laid out
     // the same way.  The source is ordinary (pageable) memory, which the runtime reads out before
     // cudaMemcpyAsync returns, so the buffer may die with this call.
@@ -462,7 +461,7 @@ int sbc_encode_static(const float* update, float* residual, int64_t numel, doubl
     void* ws = nullptr;
     const int rc = static_workspace_ptr(&ws);
     if (rc != SBC_OK) return rc;
-    // Same launches as sbc_encode; they clear the control block, histograms, mask and payload area
+    // Same launches as sbc_encode; they clear the control block, histograms, tile counters and payload area
     // themselves, so stale contents of the shared array from an earlier call do not matter.
     return sbc_encode(update, residual, numel, p, out_stream, out_capacity, out_mu, ws,
                       (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
@@ -510,7 +509,7 @@ int sbc_encode_host(const float* update_host, float* update_dev, float* residual
     if (!make_plan(numel, p, &pl)) return SBC_EINVAL;
     if (workspace_bytes < pl.total) return SBC_ECAPACITY;
     float* mu_dev = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kProbSlotBytes + pl.zero_bytes +
-                                             pl.mask_bytes + pl.off_mu);
+                                             pl.tile_bytes + pl.off_mu);
     const int rc = sbc_encode(update_dev, residual_dev, numel, p, stream_dev, out_capacity, mu_dev,
                               workspace, workspace_bytes, stream);
     if (rc != SBC_OK) return rc;

@@ -22,7 +22,8 @@ constexpr int kBlock = 256;           // threads per block for every kernel here
 constexpr int kHistBins = 2048;       // 11-bit radix digits
 constexpr uint32_t kSampleMax = 1u << 20;  // elements looked at to bound the thresholds
 constexpr int kXTile = 4096;          // elements per tile in the exact-select fallback
-constexpr int kMaskTileWords = 2048;  // 32-bit mask words per compaction tile
+constexpr int kTileShift = 18;         // positions per ordering tile = 262144
+constexpr int kTileWords = (1 << kTileShift) / 32;  // bitmask words covering one tile
 constexpr int kLenBlock = 1024;       // codewords per block in the length scan / packer
 constexpr int kChunkCodewords = 256;  // codewords per chunk-table entry
 constexpr int kSumBins = 254;         // one exact integer bin per fp32 exponent
@@ -90,15 +91,15 @@ struct Prob {
     uint32_t* sample_keys;
     unsigned long long* cand[2];
     unsigned long long* buf[2][2];   // ping-pong lists of the candidate select
-    uint32_t* mask;
-    uint32_t* mask_tile_cnt;
+    uint32_t* tile_cnt[2];      // kept positions per tile and side (n_tiles + 1 entries; scanned in place)
+    uint32_t* tile_fill;        // entries already placed in each tile's bucket
     uint32_t* x_tile_cnt[2];
     uint32_t* idx;              // sorted kept positions
     unsigned long long* blk_len;
     uint32_t cap;               // capacity of each candidate list
     uint32_t m;                 // sample size
     uint32_t s_target[2];       // rank looked up in the sample, per side
-    uint32_t n_xtiles, n_mask_words, n_mask_tiles, n_len_blocks, n_chunks;
+    uint32_t n_xtiles, n_tiles, n_len_blocks, n_chunks;
     unsigned long long payload_offset;
 };
 
@@ -141,7 +142,7 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
 
 // Kinds of work a kernel's grid is sized by (one prefix table per kind in a batch).
 enum WorkKind : int {
-    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_MASK, WK_LEN, WK_ONE, WK_STREAM, WK_COUNT
+    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_SCATTER, WK_MASK, WK_LEN, WK_ONE, WK_STREAM, WK_COUNT
 };
 
 // ---------------------------------------------------------------- keys
@@ -209,6 +210,50 @@ __device__ __forceinline__ bool last_block_ticket(uint32_t* counter, uint32_t n_
     bool last = s_is_last != 0u;
     if (last) __threadfence();
     return last;
+}
+
+// Shared-memory window of per-tile counters used by blocks that walk a contiguous span of a
+// nearly position-ordered list: tiles [base, base + kTileWindow), base a little before the tile
+// of the span's first entry.
+constexpr int kTileWindow = 128;
+__device__ __forceinline__ uint32_t tile_window_base(uint32_t first_tile) {
+    return first_tile > 16u ? first_tile - 16u : 0u;
+}
+
+// One counter update per distinct `key` among the warp's `valid` lanes; returns each valid lane's
+// rank within its key group and, through *first, the counter value before the group's update (only
+// meaningful when WANT_OLD).  Fast path: every valid lane has the same key (the common case when
+// neighbouring list entries are neighbours in the tensor).  All 32 lanes must call.
+template <bool WANT_OLD>
+__device__ __forceinline__ uint32_t warp_group_add(uint32_t* counters, uint32_t key, bool valid, uint32_t* first) {
+    const unsigned active = __ballot_sync(0xffffffffu, valid);
+    if (active == 0u) return 0u;
+    const int lead = __ffs(active) - 1;
+    const uint32_t lead_key = __shfl_sync(0xffffffffu, key, lead);
+    const bool uniform = __all_sync(0xffffffffu, !valid || key == lead_key);
+    const unsigned lt = (1u << lane_id()) - 1u;
+    if (uniform) {
+        uint32_t old = 0u;
+        if ((int)lane_id() == lead) {
+            if (WANT_OLD) old = atomicAdd(&counters[key], (uint32_t)__popc(active));
+            else atomicAdd(&counters[key], (uint32_t)__popc(active));
+        }
+        if (WANT_OLD) *first = __shfl_sync(0xffffffffu, old, lead);
+        return (uint32_t)__popc(active & lt);
+    }
+    uint32_t rank = 0u, old = 0u;
+    if (valid) {
+        const unsigned peers = __match_any_sync(active, key);
+        const int leader = __ffs(peers) - 1;
+        if ((int)lane_id() == leader) {
+            if (WANT_OLD) old = atomicAdd(&counters[key], (uint32_t)__popc(peers));
+            else atomicAdd(&counters[key], (uint32_t)__popc(peers));
+        }
+        if (WANT_OLD) old = __shfl_sync(peers, old, leader);
+        rank = (uint32_t)__popc(peers & lt);
+    }
+    if (WANT_OLD) *first = old;
+    return rank;
 }
 
 // ---------------------------------------------------------------- histogram pick

@@ -1,6 +1,6 @@
 // Golomb position coding (Algorithm 3) and decoding (Algorithm 4).
 //
-// Encode: kept-position bitmask -> ascending position list (popcount scan)
+// Encode: kept positions bucketed by tile and ordered inside each tile -> ascending position list
 // -> per-codeword lengths q + 1 + b -> exclusive scan = bit offsets ->
 // every codeword ORs its own bits into the pre-zeroed payload.
 // Decode: one thread per chunk of kChunkCodewords codewords, started from the
@@ -13,23 +13,26 @@ namespace sbc {
 
 // ---------------------------------------------------------------- mask -> sorted positions
 
-// In-place exclusive scan of the kept-position counts per mask tile (one block).
-__global__ void __launch_bounds__(kBlock) k_mask_scan(const Batch B) {
+// In-place exclusive scan of the chosen side's kept-position counts per tile (one block); entry
+// n_tiles receives the total.
+__global__ void __launch_bounds__(kBlock) k_tile_scan(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    uint32_t* __restrict__ cnt = P.tile_cnt[ctl->side];
+    const uint32_t n_tiles = P.n_tiles;
     constexpr int kPer = 8;
     uint32_t carry = 0u;
-    for (uint32_t base = 0; base < P.n_mask_tiles; base += kBlock * kPer) {
+    for (uint32_t base = 0; base < n_tiles; base += kBlock * kPer) {
         uint32_t v[kPer];
         uint32_t sum = 0u;
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             const uint32_t t = base + threadIdx.x * kPer + j;
-            v[j] = (t < P.n_mask_tiles) ? P.mask_tile_cnt[t] : 0u;
+            v[j] = (t < n_tiles) ? cnt[t] : 0u;
             sum += v[j];
         }
         uint32_t total;
@@ -37,53 +40,91 @@ __global__ void __launch_bounds__(kBlock) k_mask_scan(const Batch B) {
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             const uint32_t t = base + threadIdx.x * kPer + j;
-            if (t < P.n_mask_tiles) P.mask_tile_cnt[t] = run;
+            if (t < n_tiles) cnt[t] = run;
             run += v[j];
         }
         carry += total;
     }
     if (threadIdx.x == 0) {
+        cnt[n_tiles] = carry;
         ctl->kept_total = carry;
         if (carry != (uint32_t)P.k) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
     }
 }
 
-// Mask -> ascending position list.
-__global__ void __launch_bounds__(kBlock) k_mask_compact(const Batch B) {
+// Put every tile's bucket of the position list in ascending order.  Small buckets: each thread
+// ranks its entry against the others in shared memory.  Large buckets: the entries set bits in a
+// shared-memory bitmask of the tile, which is then read out in order (popcount scan).
+__global__ void __launch_bounds__(kBlock) k_tile_sort(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     if (P.ctl->status) return;
-    __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    static_assert(kMaskTileWords / kBlock == 8, "eight words per thread");
-    constexpr int kPer = kMaskTileWords / kBlock;
-    for (uint32_t tile = S.bx; tile < P.n_mask_tiles; tile += S.nb) {
-        uint32_t words[kPer];
-        uint32_t c = 0u;
-        const uint32_t w0 = tile * kMaskTileWords + threadIdx.x * kPer;
-        if (w0 + kPer <= P.n_mask_words) {
-            const uint4 lo = *reinterpret_cast<const uint4*>(P.mask + w0);
-            const uint4 hi = *reinterpret_cast<const uint4*>(P.mask + w0 + 4);
-            words[0] = lo.x; words[1] = lo.y; words[2] = lo.z; words[3] = lo.w;
-            words[4] = hi.x; words[5] = hi.y; words[6] = hi.z; words[7] = hi.w;
-        } else {
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) words[j] = (w0 + j < P.n_mask_words) ? P.mask[w0 + j] : 0u;
+    __shared__ uint32_t s_mask[kTileWords];
+    __shared__ uint32_t s_small[kBlock];
+    const uint32_t* __restrict__ tile_base = P.tile_cnt[P.ctl->side];
+    uint32_t* __restrict__ list = P.idx;
+    const uint32_t n_tiles = P.n_tiles;
+    for (uint32_t tile = S.bx; tile < n_tiles; tile += S.nb) {
+        const uint32_t beg = tile_base[tile], end = tile_base[tile + 1];
+        const uint32_t count = end - beg;
+        if (count <= 1u) continue;  // block-uniform
+        if (count <= (uint32_t)kBlock) {
+            const uint32_t x = (threadIdx.x < count) ? list[beg + threadIdx.x] : 0xffffffffu;
+            s_small[threadIdx.x] = x;
+            __syncthreads();
+            uint32_t rank = 0u;
+            for (uint32_t j = 0; j < count; ++j) rank += (s_small[j] < x) ? 1u : 0u;
+            if (threadIdx.x < count) list[beg + rank] = x;
+            __syncthreads();
+            continue;
         }
+        for (int w = threadIdx.x; w < kTileWords; w += kBlock) s_mask[w] = 0u;
+        __syncthreads();
+        for (uint32_t base = beg; base < end; base += 4 * kBlock) {  // four loads in flight per thread
+            uint32_t v[4];
 #pragma unroll
-        for (int j = 0; j < kPer; ++j) c += __popc(words[j]);
-        uint32_t pos = P.mask_tile_cnt[tile] + block_exclusive_scan<uint32_t>(c, s_scan, nullptr);
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t i = base + j * kBlock + threadIdx.x;
+                v[j] = (i < end) ? list[i] : 0xffffffffu;
+            }
 #pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            uint32_t w = words[j];
-            const uint32_t first = (w0 + j) << 5;
+            for (int j = 0; j < 4; ++j) {
+                if (v[j] != 0xffffffffu) {
+                    const uint32_t r = v[j] & ((1u << kTileShift) - 1u);
+                    atomicOr(&s_mask[r >> 5], 1u << (r & 31u));
+                }
+            }
+        }
+        __syncthreads();
+        // read-out: warp w owns words [w*kPerWarp, (w+1)*kPerWarp), lane l takes word it*32 + l of
+        // them in step `it` (conflict-free); order of the output = (warp, step, lane, bit)
+        constexpr int kPerWarp = kTileWords / (kBlock / 32);
+        const int warp = threadIdx.x >> 5, lane = lane_id();
+        uint32_t mine = 0u;
+        for (int it = 0; it < kPerWarp / 32; ++it) mine += __popc(s_mask[warp * kPerWarp + it * 32 + lane]);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, d);
+        if (lane == 0) s_small[warp] = mine;
+        __syncthreads();
+        uint32_t pos = beg;
+        for (int w = 0; w < warp; ++w) pos += s_small[w];
+        for (int it = 0; it < kPerWarp / 32; ++it) {
+            const int word = warp * kPerWarp + it * 32 + lane;
+            uint32_t w = s_mask[word];
+            const uint32_t c = (uint32_t)__popc(w);
+            const uint32_t incl = warp_inclusive_scan(c);
+            uint32_t at = pos + incl - c;
+            const uint32_t first = (tile << kTileShift) + ((uint32_t)word << 5);
             while (w) {
                 const uint32_t idx = first + (__ffs(w) - 1);
                 w &= w - 1u;
-                if (pos < (uint32_t)P.k) P.idx[pos] = idx;
-                ++pos;
+                if (at < end) list[at] = idx;
+                ++at;
             }
+            pos += __shfl_sync(0xffffffffu, incl, 31);
         }
+        __syncthreads();  // s_mask is cleared again for the next tile
     }
 }
 

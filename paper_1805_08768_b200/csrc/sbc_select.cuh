@@ -196,18 +196,38 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
     const int bin_b = bin_a + 1;
     long long acc_a = 0, acc_b = 0;
-    for (uint32_t i = S.bx * kBlock + threadIdx.x; i < cnt; i += S.nb * kBlock) {
-        const unsigned long long c = src[i];
-        if (c < thr) continue;
-        const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
-        const uint32_t e = (bits >> 23) & 0xffu;
-        int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
-        if (bits >> 31) m = -m;
-        const int bin = e ? (int)e - 1 : 0;
-        if (bin == bin_a) acc_a += m;
-        else if (bin == bin_b) acc_b += m;
-        else atomicAdd(&s_bins[0][bin], (unsigned long long)(long long)m);
+    // Each block walks one contiguous span of the list.  The list is nearly in position order, so
+    // a span touches few ordering tiles: their counts are kept in a shared-memory window and
+    // added to the global per-tile counts once per block (entries outside the window go straight
+    // to the global counters).
+    uint32_t* __restrict__ tile_cnt = P.tile_cnt[s];
+    __shared__ uint32_t s_win[kTileWindow];
+    if (threadIdx.x < kTileWindow) s_win[threadIdx.x] = 0u;
+    const uint32_t span = ((cnt + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
+    const uint32_t lo = min(cnt, S.bx * span), hi = min(cnt, lo + span);
+    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(src[lo]) >> kTileShift : 0u);
+    __syncthreads();
+    for (uint32_t base = lo; base < hi; base += kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const unsigned long long c = (i < hi) ? src[i] : 0ull;
+        const bool kept = (i < hi) && c >= thr;
+        if (kept) {
+            const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
+            const uint32_t e = (bits >> 23) & 0xffu;
+            int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
+            if (bits >> 31) m = -m;
+            const int bin = e ? (int)e - 1 : 0;
+            if (bin == bin_a) acc_a += m;
+            else if (bin == bin_b) acc_b += m;
+            else atomicAdd(&s_bins[0][bin], (unsigned long long)(long long)m);
+        }
+        const uint32_t tile = composite_index(c) >> kTileShift;
+        const uint32_t rel = tile - win0;
+        warp_group_add<false>(s_win, rel, kept && rel < (uint32_t)kTileWindow, nullptr);
+        warp_group_add<false>(tile_cnt, tile, kept && rel >= (uint32_t)kTileWindow, nullptr);
     }
+    __syncthreads();
+    if (threadIdx.x < kTileWindow && s_win[threadIdx.x]) atomicAdd(&tile_cnt[win0 + threadIdx.x], s_win[threadIdx.x]);
 #pragma unroll
     for (int d = 16; d > 0; d >>= 1) {
         acc_a += __shfl_down_sync(0xffffffffu, acc_a, d);
@@ -243,9 +263,10 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     }
 }
 
-// One mask bit per kept position of the chosen side (for the ordered
-// compaction that follows) and the number of kept positions per mask tile.
-__global__ void __launch_bounds__(kBlock) k_mark(const Batch B) {
+// Kept positions of the chosen side into per-tile buckets of the position list (tile = 65536
+// consecutive positions; bucket starts come from the scanned tile counts).  Inside a bucket the
+// order is whatever the atomics give; k_tile_sort puts each bucket in order afterwards.
+__global__ void __launch_bounds__(kBlock) k_scatter(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -255,20 +276,47 @@ __global__ void __launch_bounds__(kBlock) k_mark(const Batch B) {
     const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
     const unsigned long long thr = ctl->thr[s];
     const unsigned long long* __restrict__ src = P.cand[s];
-    constexpr int kTileShift = 16;  // kMaskTileWords * 32 = 65536 positions per tile
-    static_assert(kMaskTileWords * 32 == (1 << kTileShift), "tile size");
-    for (uint32_t base = S.bx * kBlock; base < cnt; base += S.nb * kBlock) {
+    const uint32_t* __restrict__ tile_base = P.tile_cnt[s];
+    uint32_t* __restrict__ tile_fill = P.tile_fill;
+    uint32_t* __restrict__ out = P.idx;
+    const uint32_t k = (uint32_t)P.k;
+    // Same span / window scheme as the counting in k_sums_decide: count the span's kept entries
+    // per tile in shared memory, reserve each tile's range of its bucket with ONE global atomic,
+    // then walk the span again and hand out slots from shared-memory counters.
+    __shared__ uint32_t s_win[kTileWindow];
+    __shared__ uint32_t s_first[kTileWindow];
+    if (threadIdx.x < kTileWindow) s_win[threadIdx.x] = 0u;
+    const uint32_t span = ((cnt + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
+    const uint32_t lo = min(cnt, S.bx * span), hi = min(cnt, lo + span);
+    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(src[lo]) >> kTileShift : 0u);
+    __syncthreads();
+    for (uint32_t base = lo; base < hi; base += kBlock) {
         const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < cnt) ? src[i] : 0ull;
-        const bool kept = (i < cnt) && c >= thr;
+        const unsigned long long c = (i < hi) ? src[i] : 0ull;
+        const uint32_t rel = (composite_index(c) >> kTileShift) - win0;
+        warp_group_add<false>(s_win, rel, (i < hi) && c >= thr && rel < (uint32_t)kTileWindow, nullptr);
+    }
+    __syncthreads();
+    if (threadIdx.x < kTileWindow) {
+        const uint32_t c = s_win[threadIdx.x];
+        s_first[threadIdx.x] = c ? atomicAdd(&tile_fill[win0 + threadIdx.x], c) : 0u;
+        s_win[threadIdx.x] = 0u;
+    }
+    __syncthreads();
+    for (uint32_t base = lo; base < hi; base += kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const unsigned long long c = (i < hi) ? src[i] : 0ull;
+        const bool kept = (i < hi) && c >= thr;
         const uint32_t idx = composite_index(c);
-        if (kept) atomicOr(&P.mask[idx >> 5], 1u << (idx & 31u));
-        // neighbours in the list are neighbours in the tensor: one counter update per tile per warp
-        const unsigned active = __ballot_sync(0xffffffffu, kept);
+        const uint32_t tile = idx >> kTileShift;
+        const uint32_t rel = tile - win0;
+        const bool in_win = rel < (uint32_t)kTileWindow;
+        uint32_t first_w = 0u, first_g = 0u;
+        const uint32_t rank_w = warp_group_add<true>(s_win, rel, kept && in_win, &first_w);
+        const uint32_t rank_g = warp_group_add<true>(tile_fill, tile, kept && !in_win, &first_g);
         if (kept) {
-            const uint32_t tile = idx >> kTileShift;
-            const unsigned peers = __match_any_sync(active, tile);
-            if ((int)lane_id() == __ffs(peers) - 1) atomicAdd(&P.mask_tile_cnt[tile], (uint32_t)__popc(peers));
+            const uint32_t slot = tile_base[tile] + (in_win ? s_first[rel] + first_w + rank_w : first_g + rank_g);
+            if (slot < k) out[slot] = idx;
         }
     }
 }

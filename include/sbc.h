@@ -299,6 +299,27 @@ int sbc_decode_accumulate(const void *const *streams, int n_clients,
                           sbc_cuda_stream_t stream);
 
 /*
+ * Decode, scale and apply in one pass (Algorithm 1: server lines
+ * "dW <- 1/|I_t| sum dW_i*" and "W <- W + dW", equally the client line
+ * "W_i <- W_i + dW"; momentum masking, Supplement "Momentum Correction, Warm-up
+ * Training and Momentum Masking": the momentum of every updated weight is set
+ * to zero):
+ *
+ *   weights[j]  += scale * mu_c   for every client c and every position j it sent
+ *   momentum[j]  = 0              at those positions (if momentum != NULL)
+ *
+ * scale is 1/|I_t| for the paper's average, 1 for a plain sum.  Each client's
+ * contribution fl32(scale * mu_c) is added with an fp32 atomic, so the result
+ * agrees with "sum, then scale, then add" to rounding (a few ulps of
+ * |weights[j]| + scale * sum_c |mu_c|), not bit for bit.  Other arguments,
+ * validation and status reporting as sbc_decode_accumulate, which is this call
+ * with scale = 1 and momentum = NULL.
+ */
+int sbc_decode_apply(const void *const *streams, int n_clients, float scale, float *weights,
+                     float *momentum, int64_t numel, uint32_t *status_dev,
+                     sbc_cuda_stream_t stream);
+
+/*
  * sbc_decode_accumulate for many tensors at once: for every tensor t,
  * out_dense[t][j] += mu_{c,t} over the n_clients streams of that tensor
  * (Algorithm 1, server sum line, per tensor).  One launch for the batch.

@@ -453,3 +453,33 @@ int sbc_oracle_decode_accumulate(const uint8_t *const *streams, int n_clients,
     }
     return 0;
 }
+
+/* ------------------------------------------------------------------ */
+/* Algorithm 1, server lines: dW = 1/|I_t| * sum dW_i*,  W = W + dW    */
+/* and momentum masking (Supplement): zero the momentum where a weight */
+/* was updated by a transmitted entry                                  */
+/* ------------------------------------------------------------------ */
+
+int sbc_oracle_decode_apply(const uint8_t *const *streams, int n_clients, float scale,
+                            float *weights, float *momentum, int64_t n) {
+    if (!streams || !weights || n_clients < 0 || n <= 0) return -2;
+    float *sum = (float *)calloc((size_t)n, sizeof(float));
+    float *hit = (float *)calloc((size_t)n, sizeof(float));
+    if (!sum || !hit) { free(sum); free(hit); return -2; }
+    int rc = sbc_oracle_decode_accumulate(streams, n_clients, sum, n); /* sum over i in I_t */
+    for (int c = 0; rc == 0 && c < n_clients; ++c) { /* positions any client transmitted */
+        const uint8_t *s = streams[c];
+        int64_t got = sbc_oracle_golomb_decode(s + get_u64(s + 32), get_u64(s + 24),
+                                               (int)get_u32(s + 40), 1.0f, hit, n);
+        if (got < 0) rc = -4;
+    }
+    for (int64_t j = 0; rc == 0 && j < n; ++j) {
+        volatile float d = scale * sum[j];      /* dW_j = 1/|I_t| * sum */
+        volatile float w = weights[j] + d;      /* W_j = W_j + dW_j */
+        weights[j] = w;
+        if (momentum && hit[j] != 0.0f) momentum[j] = 0.0f;
+    }
+    free(sum);
+    free(hit);
+    return rc;
+}

@@ -126,6 +126,14 @@ int sbc_oracle_encode(const float *update, float *residual, int64_t n, double p,
 int sbc_oracle_decode_accumulate(const uint8_t *const *streams, int n_clients,
                                  float *out_dense, int64_t n);
 
+/* Server / client apply step (Algorithm 1: "dW <- 1/|I_t| sum dW_i*", "W <- W + dW") with
+ * momentum masking (Supplement): weights[j] = fl32(weights[j] + fl32(scale * sum_j)) for every
+ * j, sum_j the fp32 sum of the decoded client tensors in client order; momentum[j] = 0 at every
+ * position some client transmitted (momentum may be NULL).  scale is 1/|I_t| for the paper's
+ * average.  Returns 0 or a negative error. */
+int sbc_oracle_decode_apply(const uint8_t *const *streams, int n_clients, float scale,
+                            float *weights, float *momentum, int64_t n);
+
 #ifdef __cplusplus
 }
 #endif

@@ -14,7 +14,7 @@ __all__ = [
     "kept_count", "golomb_b", "mean_position_bits", "accumulate", "topk",
     "exact_sum", "compress", "payload_bits_bound", "golomb_encode",
     "golomb_decode", "container_bytes", "stream_bytes", "encode",
-    "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container",
+    "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container", "decode_apply",
     "HEADER_BYTES", "CHUNK_CODEWORDS", "CHUNK_ENTRY_BYTES", "MAGIC",
 ]
 
@@ -181,6 +181,20 @@ def decode_accumulate(streams, out_dense: np.ndarray) -> None:
     rc = _decode_acc(ptrs, len(arrs), out_dense, out_dense.size)
     if rc != 0:
         raise ValueError(f"sbc_oracle_decode_accumulate failed: {rc}")
+
+
+_decode_apply = _sig("sbc_oracle_decode_apply", C.c_int, C.POINTER(C.c_void_p), C.c_int, C.c_float,
+                     _f32p, C.c_void_p, C.c_int64)
+
+
+def decode_apply(streams, scale: float, weights: np.ndarray, momentum: np.ndarray = None) -> None:
+    """weights += scale * sum of the decoded streams; momentum zeroed at transmitted positions."""
+    arrs = [np.ascontiguousarray(s, dtype=np.uint8) for s in streams]
+    ptrs = (C.c_void_p * max(len(arrs), 1))(*[a.ctypes.data for a in arrs])
+    mom = momentum.ctypes.data if momentum is not None else None
+    rc = _decode_apply(ptrs, len(arrs), float(scale), weights, mom, weights.size)
+    if rc != 0:
+        raise ValueError(f"sbc_oracle_decode_apply failed: {rc}")
 
 
 @dataclass

@@ -26,7 +26,7 @@ EXPORTS = [
     "sbc_workspace_bytes", "sbc_encode", "sbc_encode_ex", "sbc_encode_launches", "sbc_decode_launches",
     "sbc_encode_diag_get", "sbc_encode_host", "sbc_stream_info_get", "sbc_decode_accumulate",
     "sbc_decode_accumulate_host", "sbc_encode_static", "sbc_workspace_bytes_batch", "sbc_encode_batch",
-    "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch",
+    "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch", "sbc_decode_apply",
 ]
 STATIC_WORKSPACE_BYTES = 8 << 20
 MARK_BEGIN, MARK_BOUNDS, MARK_COLLECT, MARK_EXACT, MARK_SELECT, MARK_END, MARK_COUNT = range(7)
@@ -119,6 +119,9 @@ def lib() -> C.CDLL:
         L.sbc_decode_accumulate_batch.restype = C.c_int
         L.sbc_decode_accumulate_batch.argtypes = [C.c_int, C.c_int, C.POINTER(DecodeDesc), C.c_void_p, C.c_void_p,
                                                   C.c_size_t, C.c_void_p]
+        L.sbc_decode_apply.restype = C.c_int
+        L.sbc_decode_apply.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_int64,
+                                       C.c_void_p, C.c_void_p]
         L.sbc_stream_info_get.restype = C.c_int
         L.sbc_stream_info_get.argtypes = [C.c_void_p, C.POINTER(StreamInfo), C.c_void_p]
         L.sbc_decode_accumulate.restype = C.c_int
@@ -386,3 +389,17 @@ def sbc_decode_accumulate(streams: Sequence[torch.Tensor], out_dense: torch.Tens
                                        status.data_ptr() if status is not None else None,
                                        _cuda_stream(stream))
     _check(code, "sbc_decode_accumulate")
+
+
+def sbc_decode_apply(streams: Sequence[torch.Tensor], scale: float, weights: torch.Tensor,
+                     momentum: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
+                     stream=None) -> None:
+    """Enqueue weights[j] += scale * mu_c at every decoded position; momentum[j] = 0 there."""
+    _dev_f32(weights, "weights")
+    if momentum is not None:
+        _dev_f32(momentum, "momentum")
+    ptrs = (C.c_void_p * max(len(streams), 1))(*[s.data_ptr() for s in streams])
+    code = lib().sbc_decode_apply(ptrs, len(streams), float(scale), weights.data_ptr(),
+                                  momentum.data_ptr() if momentum is not None else None, weights.numel(),
+                                  status.data_ptr() if status is not None else None, _cuda_stream(stream))
+    _check(code, "sbc_decode_apply")

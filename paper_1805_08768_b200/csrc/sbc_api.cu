@@ -555,6 +555,12 @@ int sbc_stream_info_get(const void* stream_dev, sbc_stream_info* host_out, sbc_c
 
 int sbc_decode_accumulate(const void* const* streams, int n_clients, float* out_dense, int64_t numel,
                           uint32_t* status_dev, sbc_cuda_stream_t stream) {
+    return sbc_decode_apply(streams, n_clients, 1.0f, out_dense, nullptr, numel, status_dev, stream);
+}
+
+int sbc_decode_apply(const void* const* streams, int n_clients, float scale, float* out_dense, float* momentum,
+                     int64_t numel, uint32_t* status_dev, sbc_cuda_stream_t stream) {
+    if (!(scale == scale) || std::isinf(scale) || ((uintptr_t)momentum & 3)) return SBC_EINVAL;
     if (n_clients < 0 || numel <= 0 || numel >= (1ll << 31) || !out_dense) return SBC_EINVAL;
     if (n_clients > 0 && !streams) return SBC_EINVAL;
     if (((uintptr_t)out_dense & 3) || ((uintptr_t)status_dev & 3)) return SBC_EINVAL;
@@ -569,6 +575,8 @@ int sbc_decode_accumulate(const void* const* streams, int n_clients, float* out_
         a.out = out_dense;
         a.n = numel;
         a.status = status_dev;
+        a.scale = scale;
+        a.momentum = momentum;
         // at most ceil(numel / 256) chunks per client, 32 chunks per warp, two warps per block
         const unsigned long long max_groups =
             (unsigned long long)a.n_clients *
@@ -609,6 +617,7 @@ int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_d
             args[t].out = descs[t].out_dense;
             args[t].n = descs[t].numel;
             args[t].status = status_dev;
+            args[t].scale = 1.0f;
         }
         if (cudaMemcpyAsync(d_args, args.data(), args.size() * sizeof(DecodeArgs), cudaMemcpyHostToDevice,
                             stream) != cudaSuccess)

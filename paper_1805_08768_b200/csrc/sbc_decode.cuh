@@ -1,5 +1,6 @@
 // Golomb position decoding and server-side sum (Algorithm 4; Algorithm 1,
-// server line "dW <- sum of the decoded client updates").
+// server lines "dW <- 1/|I_t| sum of the decoded client updates", "W <- W + dW";
+// momentum masking of the Supplement as an optional second target).
 #pragma once
 #include "sbc_common.cuh"
 #include "../../include/sbc.h"
@@ -14,6 +15,8 @@ struct DecodeArgs {
     float* out;
     long long n;
     uint32_t* status;  // may be null
+    float scale;       // every transmitted value is multiplied by this before it is added
+    float* momentum;   // may be null: zeroed at every decoded position (momentum masking)
 };
 
 __device__ __forceinline__ uint32_t load_u32(const uint8_t* p) { return *reinterpret_cast<const uint32_t*>(p); }
@@ -183,7 +186,8 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
             const uint32_t count = (uint32_t)min((unsigned long long)kChunkCodewords, v.k - first_cw);
             if (pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n) err = SBC_STATUS_CORRUPT;
             const uint32_t b = v.b;
-            const float mu = v.mu;
+            const float mu = __fmul_rn(v.mu, args.scale);
+            float* __restrict__ momentum = args.momentum;
             const bool tiny = fabsf(mu) < 7.888609052e-31f;  // 2^-100
             if (staged) {
                 // Fast path: bit positions relative to the stage fit 32 bits; every codeword
@@ -218,6 +222,7 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                     }
                     prev += (long long)step;
                     err |= add_at(args.out + prev, mu, tiny);
+                    if (momentum) momentum[prev] = 0.f;
                 }
                 pos = (first_word << 5) + rel;
             } else {
@@ -249,6 +254,7 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                     }
                     prev += (long long)step;
                     err |= add_at(args.out + prev, mu, tiny);
+                    if (momentum) momentum[prev] = 0.f;
                 }
                 if (!err && used > room) err = SBC_STATUS_CORRUPT;
                 pos += used;

@@ -257,3 +257,39 @@ def test_decode_of_a_subnormal_mu_is_exact():
     sbc.sbc_decode_accumulate([s, s, s], dense)
     torch.cuda.synchronize()
     assert np.array_equal(dense.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
+def test_decode_apply_scales_adds_and_masks_momentum():
+    n, p, n_clients = 300000, 0.01, 4
+    rng = np.random.default_rng(12)
+    streams_np, dev_streams, mus = [], [], []
+    for c in range(n_clients):
+        upd = workloads.normal_flat(n, 1e-3, 500 + c)
+        stream, mu, _, _, _ = gpu_encode(upd, np.zeros(n, dtype=np.float32), p)
+        streams_np.append(stream)
+        dev_streams.append(torch.from_numpy(stream).to(DEV))
+        mus.append(abs(float(mu)))
+    w0 = (rng.standard_normal(n) * 0.05).astype(np.float32)
+    m0 = rng.standard_normal(n).astype(np.float32)
+    want_w, want_m = w0.copy(), m0.copy()
+    scale = 1.0 / n_clients
+    oracle.decode_apply(streams_np, scale, want_w, want_m)
+    w = torch.from_numpy(w0).to(DEV)
+    m = torch.from_numpy(m0).to(DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sbc.sbc_decode_apply(dev_streams, scale, w, m, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    got_w, got_m = w.cpu().numpy(), m.cpu().numpy()
+    tol = 1e-6 * (np.abs(w0).astype(np.float64) + scale * sum(mus))
+    assert np.all(np.abs(got_w.astype(np.float64) - want_w) <= tol)
+    untouched = want_m == m0
+    assert np.array_equal(got_w[untouched & (want_w == w0)], w0[untouched & (want_w == w0)])
+    assert np.array_equal(got_m.view(np.uint32), want_m.view(np.uint32))     # momentum mask is exact
+    # one client, scale 1: identical to the oracle bit for bit
+    w1 = torch.from_numpy(w0).to(DEV)
+    sbc.sbc_decode_apply(dev_streams[:1], 1.0, w1)
+    torch.cuda.synchronize()
+    want1 = w0.copy()
+    oracle.decode_apply(streams_np[:1], 1.0, want1)
+    assert np.array_equal(w1.cpu().numpy().view(np.uint32), want1.view(np.uint32))

@@ -391,3 +391,31 @@ def test_side_and_mu_and_container_entry_points():
     h = oracle.parse_header(stream)
     kept = np.sort(_brute_topk(upd, h.k, bool(h.side)))
     assert np.array_equal(oracle.container(kept, n, p, h.side, mu), stream)
+
+
+def test_decode_apply_against_dense_fp64():
+    # Algorithm 1's server lines, checked against a dense fp64 computation from the kept sets
+    rng = np.random.default_rng(31)
+    n, p, n_clients = 30000, 0.01, 4
+    streams, dense64, hit = [], np.zeros(n), np.zeros(n, dtype=bool)
+    for c in range(n_clients):
+        upd = rng.standard_normal(n).astype(np.float32)
+        s, mu = oracle.encode(upd, np.zeros(n, dtype=np.float32), p)
+        streams.append(s)
+        kept = np.sort(_brute_topk(upd, oracle.kept_count(n, p), bool(oracle.parse_header(s).side)))
+        dense64[kept] += float(mu)
+        hit[kept] = True
+    w0 = rng.standard_normal(n).astype(np.float32)
+    m0 = rng.standard_normal(n).astype(np.float32)
+    w, m = w0.copy(), m0.copy()
+    oracle.decode_apply(streams, 1.0 / n_clients, w, m)
+    want = w0.astype(np.float64) + dense64 / n_clients
+    assert np.max(np.abs(w - want)) <= 1e-6 * (np.max(np.abs(w0)) + np.max(np.abs(dense64)))
+    assert np.array_equal(w[~hit], w0[~hit])                 # untouched where nothing was sent
+    assert np.all(m[hit] == 0) and np.array_equal(m[~hit], m0[~hit])
+    # scale 1, zero weights, no momentum: the plain server sum
+    z = np.zeros(n, dtype=np.float32)
+    oracle.decode_apply(streams, 1.0, z)
+    d = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate(streams, d)
+    assert np.array_equal(z, d)

@@ -31,7 +31,7 @@ ALGO_BYTES_PER_ELEM = 12  # read update, read residual, write residual
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--numel", type=int, default=FULL_N, help="elements per update (default 2^30)")
@@ -150,8 +150,8 @@ def run_reference(args):
 
 # ------------------------------------------------------------------ our arm
 
-# DRAM traffic of one k_add_collect launch from the ncu capture summarised in
-# profiles/k_add_collect_2p26_ncu_full.md: (536.91 + 227.77) MB at 2^26 elements, p = 1e-2.
+# DRAM traffic of one k_add_collect launch from an ncu capture at 2^26 elements (its summary
+# is kept with the other profile summaries): (536.91 + 227.77) MB at 2^26 elements, p = 1e-2.
 # Traffic is proportional to the element count, so it is scaled by numel / 2^26.  Valid only for
 # the kernel source it was taken from: a different hash of the file reports null.
 NCU_TRAFFIC_BYTES_AT_2P26 = 764.68e6

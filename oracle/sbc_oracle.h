@@ -15,7 +15,7 @@
  *   Algorithm 4 (Golomb position decoding, supplement)
  *   Eq. for the mean position bits  b_pos = b* + 1 / (1 - (1-p)^(2^b*)).
  *
- * Readings taken where the paper is silent (all listed in the design notes):
+ * Readings taken where the paper is silent:
  *   k = max(1, floor(p*n)) (fp64 product), exactly k entries kept per side,
  *   equal values ordered by lower flat index first, -0 == +0, signed top-k as
  *   Algorithm 2 writes it, the two sums exact (rounded once to fp64), mean =

@@ -326,6 +326,11 @@ def run_ours(args):
         cpu = {"value": g, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc,
                "seconds": dt, "host_cores_available": len(os.sched_getaffinity(0))}
 
+    try:
+        network_shapes = run_network_shapes(torch, sbc, workloads, dev)
+    except Exception as exc:  # context numbers only: never fail the headline for them
+        network_shapes = {"error": repr(exc)}
+
     launches = steps * sum(sbc.sbc_encode_launches() + sbc.sbc_decode_launches(1) for _ in P_SWEEP)
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
@@ -337,11 +342,52 @@ def run_ours(args):
                             "zero fill of the dense tensor is outside the intervals",
                    "parallelism": f"{world} independent client replica(s), no collective"},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-        "clocks": clocks, "per_p": per_p, "wall_s": wall,
+        "clocks": clocks, "per_p": per_p, "network_shapes": network_shapes, "wall_s": wall,
     }
     print(json.dumps(line), flush=True)
     if dist is not None:
         dist.destroy_process_group()
+
+
+def run_network_shapes(torch, sbc, workloads, dev):
+    """Batched encode (one round) and 8-client batched decode on the network-shaped workloads:
+    context numbers next to the headline, timed with CUDA events over 10 repetitions."""
+    import numpy as np
+    out = {}
+    for name, sizes, p, gen in (
+            ("resnet50_shapes_p1e-3", [int(np.prod(s)) for _, s, _ in workloads.resnet50_shapes()], 1e-3,
+             workloads.resnet50_update),
+            ("word_lstm_shapes_p1e-2", [int(np.prod(s)) for _, s in workloads.word_lstm_shapes()], 1e-2,
+             workloads.word_lstm_update)):
+        ups = [torch.from_numpy(u).to(dev) for u in gen(1)]
+        res = [torch.zeros(n, dtype=torch.float32, device=dev) for n in sizes]
+        outs = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=dev) for n in sizes]
+        mus = [torch.empty(1, dtype=torch.float32, device=dev) for _ in sizes]
+        ws = torch.empty(sbc.sbc_workspace_bytes_batch(sizes, [p] * len(sizes)), dtype=torch.uint8, device=dev)
+        enc = sbc.EncodeBatch(ups, res, [p] * len(sizes), outs, mus, ws)
+        dense = [torch.zeros(n, dtype=torch.float32, device=dev) for n in sizes]
+        dws = torch.empty(sbc.sbc_decode_workspace_bytes_batch(len(sizes)), dtype=torch.uint8, device=dev)
+        dec = sbc.DecodeBatch([[o] * 8 for o in outs], dense, dws)
+
+        def timed(fn, reps=10):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(reps):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / reps
+
+        enc_ms, dec_ms = timed(enc.run), timed(dec.run)
+        total = sum(sizes)
+        out[name] = {"tensors": len(sizes), "elements": total, "encode_batch_us": 1e3 * enc_ms,
+                     "encode_gelem_s": total / enc_ms / 1e6,
+                     "encode_algorithmic_gbs": ALGO_BYTES_PER_ELEM * total / enc_ms / 1e6,
+                     "decode_batch_8_clients_us": 1e3 * dec_ms}
+    return out
 
 
 def run_e2e(args, torch, sbc, dev, update, ws, n, world):

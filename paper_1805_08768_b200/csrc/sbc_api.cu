@@ -178,15 +178,17 @@ inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsi
     return (unsigned)g;
 }
 
-// Blocks one problem gets for each kind of work.  `coarsen` (1 for a single problem) makes the
-// blocks of the sample and exact-route kernels that many times larger: every block of those
-// kernels pays for clearing and flushing a shared-memory histogram, and a batch of hundreds of
-// problems has parallelism to spare.
-void block_counts(const Plan& pl, unsigned sms, unsigned coarsen, unsigned nb[WK_COUNT]) {
-    nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8 * coarsen, sms * 4);
+// Blocks one problem gets for each kind of work.  The two coarsening factors (1 for a single
+// problem) make the blocks of the sample kernels and of the exact-route kernels that many times
+// larger: every block of those kernels pays for clearing and flushing a shared-memory histogram
+// (or, for the exact route, usually just for finding out that it is not needed), and a batch of
+// hundreds of problems has parallelism to spare.
+void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned coarse_exact,
+                  unsigned nb[WK_COUNT]) {
+    nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8 * coarse_sample, sms * 4);
     nb[WK_MAIN] = grid_for((unsigned long long)pl.n, kBlock * kPerThread, sms * kCollectBlocksPerSM);
-    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarsen, sms * 8);
-    nb[WK_XTILE] = grid_for(pl.n_xtiles, coarsen, sms * 8);
+    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 8);
+    nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 8);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
     nb[WK_SCATTER] = grid_for(pl.cap, kBlock * 4, sms * 8);
     nb[WK_MASK] = grid_for(pl.n_tiles, 1, sms * 8);
@@ -330,7 +332,7 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
     k_put_prob<<<1, 1, 0, st>>>(d_prob, P);
 
     unsigned grid[WK_COUNT];
-    block_counts(pl, (unsigned)sm_count(), 1u, grid);
+    block_counts(pl, (unsigned)sm_count(), 1u, 1u, grid);
     launch_encode(d_prob, 1u, grid, nullptr, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
@@ -376,10 +378,16 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     uint8_t* rest = tile + tile_total;
 
     const unsigned sms = (unsigned)sm_count();
-    // aim at about eight blocks per SM over the whole batch for the histogram-carrying kernels
-    unsigned long long fine_blocks = 0;
-    for (int t = 0; t < n_tensors; ++t) fine_blocks += (plans[t].m + kBlock * 8 - 1) / (kBlock * 8);
-    const unsigned coarsen = (unsigned)std::min<unsigned long long>(64, std::max<unsigned long long>(1, fine_blocks / (sms * 8ull)));
+    // aim at about six (sample) and two (exact route) blocks per SM over the whole batch
+    unsigned long long fine_sample = 0, fine_exact = 0;
+    for (int t = 0; t < n_tensors; ++t) {
+        fine_sample += (plans[t].m + kBlock * 8 - 1) / (kBlock * 8);
+        fine_exact += (unsigned long long)(plans[t].n + kBlock * 16 - 1) / (kBlock * 16);
+    }
+    auto factor = [&](unsigned long long fine, unsigned per_sm) {
+        return (unsigned)std::min<unsigned long long>(256, std::max<unsigned long long>(1, fine / (sms * per_sm)));
+    };
+    const unsigned coarse_sample = factor(fine_sample, 6), coarse_exact = factor(fine_exact, 2);
     const size_t row_len = (size_t)n_tensors + 1;
     std::vector<Prob> probs((size_t)n_tensors);
     std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
@@ -393,7 +401,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
             m += plans[t].tile_bytes;
             r += plans[t].rest_bytes;
             unsigned nb[WK_COUNT];
-            block_counts(plans[t], sms, coarsen, nb);
+            block_counts(plans[t], sms, coarse_sample, coarse_exact, nb);
             for (int kind = 0; kind < WK_COUNT; ++kind) {
                 uint32_t* row = prefix.data() + (size_t)kind * row_len;
                 const unsigned long long next = (unsigned long long)row[t] + nb[kind];

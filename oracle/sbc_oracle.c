@@ -434,6 +434,121 @@ int sbc_oracle_encode(const float *update, float *residual, int64_t n, double p,
     return rc;
 }
 
+/* ------------------------------------------------------------------ */
+/* Gradient Dropping (the paper's sparsification baseline, Section 1   */
+/* and Table 1): top-p by magnitude, the values themselves are sent    */
+/* ------------------------------------------------------------------ */
+
+static int ranked_abs_desc(const void *x, const void *y) {
+    return ranked_desc(x, y); /* v already holds |a| */
+}
+
+int sbc_oracle_topk_abs(const float *a, int64_t n, int64_t k, int64_t *out_idx) {
+    if (n <= 0 || k < 0 || k > n) return -2;
+    ranked_t *r = (ranked_t *)malloc((size_t)n * sizeof(ranked_t));
+    if (!r) return -2;
+    for (int64_t i = 0; i < n; ++i) { r[i].v = fabsf(a[i]); r[i].i = i; }
+    qsort(r, (size_t)n, sizeof(ranked_t), ranked_abs_desc);
+    for (int64_t j = 0; j < k; ++j) out_idx[j] = r[j].i;
+    free(r);
+    return 0;
+}
+
+/* Algorithm 4 with one value per position instead of one mean: dense[j] += values[i] at the
+ * i-th decoded position.  values: k little-endian fp32. */
+int64_t sbc_oracle_golomb_decode_values(const uint8_t *msg, uint64_t nbits, int b,
+                                        const uint8_t *values, int64_t k, float *dense, int64_t n) {
+    uint64_t i = 0, q = 0;
+    int64_t j = 0, count = 0;
+    while (i < nbits) {
+        if (msg_bit(msg, i) == 0) {
+            if (i + (uint64_t)b >= nbits) return -1;
+            uint64_t r = 0;
+            for (int t = 1; t <= b; ++t) r = (r << 1) | (uint64_t)msg_bit(msg, i + t);
+            j = j + (int64_t)(q << b) + (int64_t)r + 1;
+            if (j < 1 || j > n || count >= k) return -1;
+            uint32_t bits = get_u32(values + 4 * (size_t)count);
+            float v;
+            memcpy(&v, &bits, 4);
+            dense[j - 1] += v;
+            q = 0;
+            i = i + (uint64_t)b + 1;
+            ++count;
+        } else {
+            q = q + 1;
+            i = i + 1;
+        }
+    }
+    if (q != 0) return -1;
+    return count;
+}
+
+size_t sbc_oracle_stream_bytes_values(int64_t n, double p) {
+    int64_t k = sbc_oracle_kept_count(n, p);
+    return sbc_oracle_stream_bytes(n, p) + round_up16((size_t)k * 4);
+}
+
+int sbc_oracle_encode_values(const float *update, float *residual, int64_t n, double p,
+                             uint8_t *out, size_t cap, size_t *out_len) {
+    if (!update || !residual || !out || n <= 0 || n >= ((int64_t)1 << 31) || !(p > 0.0 && p < 1.0))
+        return -2;
+    int64_t k = sbc_oracle_kept_count(n, p);
+    int b = sbc_oracle_golomb_b(p);
+    if (b > 30) return -2;
+    if (sbc_oracle_accumulate(update, residual, n) != 0) return -1; /* dW = R + update */
+    int64_t *I = (int64_t *)malloc((size_t)k * sizeof(int64_t));
+    if (!I) return -2;
+    sbc_oracle_topk_abs(residual, n, k, I);                /* the fraction p with the biggest magnitude */
+    qsort(I, (size_t)k, sizeof(int64_t), cmp_i64);
+
+    uint64_t nchunks = n_chunks_for(k);
+    size_t values_offset = SBC_ORACLE_HEADER_BYTES + SBC_ORACLE_CHUNK_ENTRY_BYTES * (size_t)nchunks;
+    size_t payload_offset = values_offset + round_up16((size_t)k * 4);
+    if (cap < payload_offset) { free(I); return -3; }
+    memset(out + values_offset, 0, payload_offset - values_offset);
+    for (int64_t i = 0; i < k; ++i) {
+        uint32_t bits;
+        float v = residual[I[i]];                          /* dW*_j = dW_j on the kept positions */
+        memcpy(&bits, &v, 4);
+        put_u32(out + values_offset + 4 * (size_t)i, bits);
+        volatile float r = v - v;                          /* R = dW - dW* */
+        residual[I[i]] = r;
+    }
+    uint64_t nbits = sbc_oracle_golomb_encode(I, k, b, out + payload_offset, cap - payload_offset);
+    if (nbits == UINT64_MAX) { free(I); return -3; }
+    size_t total = payload_offset + round_up16((size_t)((nbits + 7) / 8));
+    if (cap < total) { free(I); return -3; }
+    for (size_t z = payload_offset + (size_t)((nbits + 7) / 8); z < total; ++z) out[z] = 0;
+    uint64_t bit_off = 0;
+    int64_t prev = -1;
+    for (int64_t i = 0; i < k; ++i) {
+        if (i % SBC_ORACLE_CHUNK_CODEWORDS == 0) {
+            uint8_t *e = out + SBC_ORACLE_HEADER_BYTES +
+                         SBC_ORACLE_CHUNK_ENTRY_BYTES * (size_t)(i / SBC_ORACLE_CHUNK_CODEWORDS);
+            put_u64(e, bit_off);
+            put_u64(e + 8, (uint64_t)prev);
+        }
+        uint64_t g = (uint64_t)(I[i] - prev - 1);
+        bit_off += (g >> b) + 1 + (uint64_t)b;
+        prev = I[i];
+    }
+    put_u32(out + 0, SBC_ORACLE_MAGIC);
+    put_u32(out + 4, SBC_ORACLE_VERSION);
+    put_u64(out + 8, (uint64_t)n);
+    put_u64(out + 16, (uint64_t)k);
+    put_u64(out + 24, nbits);
+    put_u64(out + 32, (uint64_t)payload_offset);
+    put_u32(out + 40, (uint32_t)b);
+    put_u32(out + 44, SBC_ORACLE_SIDE_VALUES);
+    put_u32(out + 48, 0u);
+    put_u32(out + 52, SBC_ORACLE_CHUNK_CODEWORDS);
+    put_u32(out + 56, (uint32_t)nchunks);
+    put_u32(out + 60, 0u);
+    if (out_len) *out_len = total;
+    free(I);
+    return 0;
+}
+
 int sbc_oracle_decode_accumulate(const uint8_t *const *streams, int n_clients,
                                  float *out_dense, int64_t n) {
     if (!streams || !out_dense || n_clients < 0 || n <= 0) return -2;
@@ -448,7 +563,13 @@ int sbc_oracle_decode_accumulate(const uint8_t *const *streams, int n_clients,
         if (b > 30 || k > (uint64_t)n) return -4;
         float mu;
         memcpy(&mu, &mu_bits, 4);
-        int64_t got = sbc_oracle_golomb_decode(s + off, nbits, (int)b, mu, out_dense, n);
+        int64_t got;
+        if (get_u32(s + 44) == SBC_ORACLE_SIDE_VALUES) /* one fp32 value per position, before the payload */
+            got = sbc_oracle_golomb_decode_values(s + off, nbits, (int)b,
+                                                  s + SBC_ORACLE_HEADER_BYTES + SBC_ORACLE_CHUNK_ENTRY_BYTES * n_chunks_for((int64_t)k),
+                                                  (int64_t)k, out_dense, n);
+        else
+            got = sbc_oracle_golomb_decode(s + off, nbits, (int)b, mu, out_dense, n);
         if (got < 0 || (uint64_t)got != k) return -4;
     }
     return 0;

@@ -49,6 +49,7 @@ extern "C" {
 #define SBC_ORACLE_HEADER_BYTES 64u
 #define SBC_ORACLE_CHUNK_CODEWORDS 256u
 #define SBC_ORACLE_CHUNK_ENTRY_BYTES 16u
+#define SBC_ORACLE_SIDE_VALUES 2u /* header 'side' of a stream that carries one value per position */
 
 /* k = max(1, floor(p*n)), at most n.  (Algorithm 2, "top p%"; reading S1.) */
 int64_t sbc_oracle_kept_count(int64_t n, double p);
@@ -125,6 +126,20 @@ int sbc_oracle_encode(const float *update, float *residual, int64_t n, double p,
  * error (-4 corrupt container). */
 int sbc_oracle_decode_accumulate(const uint8_t *const *streams, int n_clients,
                                  float *out_dense, int64_t n);
+
+/* Gradient Dropping, the sparsification baseline the paper compares with (Section 1: "only
+ * communicate the fraction p entries of the gradient with the biggest magnitude, while also
+ * collecting all other gradients in a residual"; Table 1: 32 value bits + position bits):
+ * A = R + update; kept = the k entries of largest |A| (equal magnitudes: lower index first);
+ * the kept values themselves are sent; R_new = A off the kept set and A - A on it.
+ * Container: header (side = 2, mu = 0) | chunk table | k fp32 values in position order, padded
+ * to 16 bytes | Algorithm 3 payload.  Decoding such a stream adds values[i] at the i-th position. */
+int sbc_oracle_topk_abs(const float *a, int64_t n, int64_t k, int64_t *out_idx);
+size_t sbc_oracle_stream_bytes_values(int64_t n, double p);
+int sbc_oracle_encode_values(const float *update, float *residual, int64_t n, double p,
+                             uint8_t *out, size_t cap, size_t *out_len);
+int64_t sbc_oracle_golomb_decode_values(const uint8_t *payload, uint64_t nbits, int b,
+                                        const uint8_t *values, int64_t k, float *dense, int64_t n);
 
 /* Server / client apply step (Algorithm 1: "dW <- 1/|I_t| sum dW_i*", "W <- W + dW") with
  * momentum masking (Supplement): weights[j] = fl32(weights[j] + fl32(scale * sum_j)) for every

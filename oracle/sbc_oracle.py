@@ -14,7 +14,7 @@ __all__ = [
     "kept_count", "golomb_b", "mean_position_bits", "accumulate", "topk",
     "exact_sum", "compress", "payload_bits_bound", "golomb_encode",
     "golomb_decode", "container_bytes", "stream_bytes", "encode",
-    "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container", "decode_apply",
+    "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container", "decode_apply", "topk_abs", "stream_bytes_values", "encode_values",
     "HEADER_BYTES", "CHUNK_CODEWORDS", "CHUNK_ENTRY_BYTES", "MAGIC",
 ]
 
@@ -195,6 +195,35 @@ def decode_apply(streams, scale: float, weights: np.ndarray, momentum: np.ndarra
     rc = _decode_apply(ptrs, len(arrs), float(scale), weights, mom, weights.size)
     if rc != 0:
         raise ValueError(f"sbc_oracle_decode_apply failed: {rc}")
+
+
+_topk_abs = _sig("sbc_oracle_topk_abs", C.c_int, _f32p, C.c_int64, C.c_int64, _i64p)
+_stream_bytes_values = _sig("sbc_oracle_stream_bytes_values", C.c_size_t, C.c_int64, C.c_double)
+_encode_values = _sig("sbc_oracle_encode_values", C.c_int, _f32p, _f32p, C.c_int64, C.c_double, _u8p,
+                      C.c_size_t, C.POINTER(C.c_size_t))
+
+
+def topk_abs(a: np.ndarray, k: int) -> np.ndarray:
+    out = np.empty(k, dtype=np.int64)
+    if _topk_abs(a, a.size, k, out) != 0:
+        raise ValueError("sbc_oracle_topk_abs failed")
+    return out
+
+
+def stream_bytes_values(n: int, p: float) -> int:
+    return int(_stream_bytes_values(n, p))
+
+
+def encode_values(update: np.ndarray, residual: np.ndarray, p: float) -> np.ndarray:
+    """Gradient Dropping client step: ``residual`` updated in place; returns the stream bytes."""
+    n = update.size
+    cap = stream_bytes_values(n, p)
+    out = np.zeros(cap, dtype=np.uint8)
+    out_len = C.c_size_t()
+    rc = _encode_values(update, residual, n, p, out, cap, C.byref(out_len))
+    if rc != 0:
+        raise ValueError(f"sbc_oracle_encode_values failed: {rc}")
+    return out[: out_len.value].copy()
 
 
 @dataclass

@@ -419,3 +419,59 @@ def test_decode_apply_against_dense_fp64():
     d = np.zeros(n, dtype=np.float32)
     oracle.decode_accumulate(streams, d)
     assert np.array_equal(z, d)
+
+
+# ---------------------------------------------------------------- Gradient Dropping baseline
+
+@pytest.mark.parametrize("seed,n,p", [(1, 10, 0.2), (2, 5000, 0.01), (3, 40000, 0.001), (4, 777, 0.3)])
+def test_gradient_dropping_against_brute_force(seed, n, p):
+    rng = np.random.default_rng(seed)
+    upd = np.round(rng.standard_normal(n) * 4).astype(np.float32) / 4     # ties in magnitude
+    res0 = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    A = (res0 + upd).astype(np.float32)
+    k, b = oracle.kept_count(n, p), oracle.golomb_b(p)
+    res = res0.copy()
+    stream = oracle.encode_values(upd, res, p)
+    h = oracle.parse_header(stream)
+    assert (h.k, h.b, h.side, h.numel) == (k, b, 2, n)
+    # kept set: k largest magnitudes, equal magnitudes by lower index (stable argsort of -|A|)
+    kept = np.sort(np.argsort(-np.abs(A).astype(np.float64), kind="stable")[:k])
+    assert np.array_equal(np.sort(oracle.topk_abs(A, k)), kept)
+    # values travel as they are, in position order, between the chunk table and the payload
+    values = stream[64 + 16 * h.n_chunks: 64 + 16 * h.n_chunks + 4 * k].view("<f4")
+    assert np.array_equal(values.view(np.uint32), A[kept].view(np.uint32))
+    assert h.payload_offset == 64 + 16 * h.n_chunks + ((4 * k + 15) // 16) * 16
+    # residual: everything that was not sent; exactly zero where it was
+    want_res = A.copy()
+    want_res[kept] = 0.0
+    assert np.array_equal(res, want_res)
+    # the position payload is Algorithm 3's, identical to what SBC would emit for the same set
+    payload, nbits = oracle.golomb_encode(kept, b)
+    assert h.nbits == nbits
+    assert bytes(stream[h.payload_offset: h.payload_offset + len(payload)]) == bytes(payload)
+    # decoding gives dW* = A on the kept set
+    dense = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate([stream], dense)
+    want = np.zeros(n, dtype=np.float32)
+    want[kept] = A[kept]
+    assert np.array_equal(dense, want)
+    assert len(stream) <= oracle.stream_bytes_values(n, p)
+
+
+def test_bit_accounting_of_binarisation_and_golomb_coding():
+    # Fig. 2 caption of the paper: binarisation gains about x3 over sparse 32-bit values with
+    # naive 16-bit positions; Golomb coding gains up to another x2 over 16-bit positions
+    n, p = 2**20, 0.01
+    upd = workloads.normal_flat(n, 1e-3, workloads.seed_for(1))
+    sbc_stream, _ = oracle.encode(upd, np.zeros(n, dtype=np.float32), p)
+    gd_stream = oracle.encode_values(upd, np.zeros(n, dtype=np.float32), p)
+    hs, hg = oracle.parse_header(sbc_stream), oracle.parse_header(gd_stream)
+    k = hs.k
+    naive_gd_bits = k * (32 + 16)
+    golomb_gd_bits = k * 32 + hg.nbits
+    sbc_naive_bits = k * 16 + 32
+    sbc_bits = hs.nbits + 32
+    assert 2.8 < naive_gd_bits / sbc_naive_bits < 3.1          # 32 -> 0 value bits
+    assert 1.8 < sbc_naive_bits / sbc_bits < 2.1               # 16 -> ~8.1 position bits
+    assert abs(hg.nbits / k - oracle.mean_position_bits(p, hg.b)) < 0.1
+    assert golomb_gd_bits < naive_gd_bits

@@ -65,7 +65,7 @@ enum sbc_status {
  *      0 u32 magic "SBC1"      4 u32 version (1)     8 u64 numel
  *     16 u64 k (positions)    24 u64 nbits (payload bits)
  *     32 u64 payload_offset   40 u32 b (Golomb parameter b*)
- *     44 u32 side (0: +mu kept, 1: -mu kept)          48 f32 mu (signed)
+ *     44 u32 side (0: +mu kept, 1: -mu kept, 2: values follow the table)  48 f32 mu (signed)
  *     52 u32 chunk_codewords  56 u32 n_chunks         60 u32 status
  *   bytes 64..    chunk table, n_chunks entries of
  *                 { u64 bit offset of codeword c*chunk_codewords,
@@ -79,6 +79,7 @@ enum sbc_status {
 #define SBC_HEADER_BYTES 64u
 #define SBC_CHUNK_CODEWORDS 256u
 #define SBC_CHUNK_ENTRY_BYTES 16u
+#define SBC_SIDE_VALUES 2u /* header 'side' of a stream written by sbc_encode_values */
 
 typedef struct sbc_stream_info {
     uint32_t magic, version;
@@ -148,6 +149,30 @@ size_t sbc_workspace_bytes(int64_t numel, double p);
 int sbc_encode(const float *update, float *residual, int64_t numel, double p,
                void *out_stream, size_t out_capacity, float *out_mu,
                void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream);
+
+/*
+ * Gradient Dropping, the sparsification baseline the paper measures SBC against
+ * (Section 1: send the fraction p of entries with the biggest magnitude, collect
+ * the rest in a residual; Table 1: 32 value bits per entry), with the same
+ * Golomb position code (Algorithm 3):
+ *
+ *   A        = residual + update
+ *   kept     = the k entries of largest |A| (equal magnitudes: lower index first)
+ *   residual = A, except residual[j] = 0 for j in kept
+ *   out_stream = header (side = SBC_SIDE_VALUES, mu = 0) | chunk table |
+ *                k fp32 values A[j] in position order, zero padded to 16 bytes |
+ *                Golomb payload of the kept positions
+ *
+ * out_capacity >= sbc_stream_bytes_values(numel, p); workspace as sbc_encode
+ * (sbc_workspace_bytes).  sbc_decode_accumulate / sbc_decode_apply accept such
+ * streams and add values[i] (times scale) at the i-th position.  Lets the
+ * paper's accounting -- about x3 from binarisation, up to x2 from Golomb coding
+ * (Figure 2) -- be measured on the same tensors.
+ */
+size_t sbc_stream_bytes_values(int64_t numel, double p);
+int sbc_encode_values(const float *update, float *residual, int64_t numel, double p,
+                      void *out_stream, size_t out_capacity, void *workspace,
+                      size_t workspace_bytes, sbc_cuda_stream_t stream);
 
 /*
  * sbc_encode for many tensors at once (a model's parameter tensors in one

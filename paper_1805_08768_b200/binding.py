@@ -26,8 +26,9 @@ EXPORTS = [
     "sbc_workspace_bytes", "sbc_encode", "sbc_encode_ex", "sbc_encode_launches", "sbc_decode_launches",
     "sbc_encode_diag_get", "sbc_encode_host", "sbc_stream_info_get", "sbc_decode_accumulate",
     "sbc_decode_accumulate_host", "sbc_encode_static", "sbc_workspace_bytes_batch", "sbc_encode_batch",
-    "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch", "sbc_decode_apply",
+    "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch", "sbc_decode_apply", "sbc_stream_bytes_values", "sbc_encode_values",
 ]
+SIDE_VALUES = 2
 STATIC_WORKSPACE_BYTES = 8 << 20
 MARK_BEGIN, MARK_BOUNDS, MARK_COLLECT, MARK_EXACT, MARK_SELECT, MARK_END, MARK_COUNT = range(7)
 MARK_NAMES = ["bounds", "collect", "exact", "select", "golomb"]  # interval i = mark i -> mark i+1
@@ -122,6 +123,11 @@ def lib() -> C.CDLL:
         L.sbc_decode_apply.restype = C.c_int
         L.sbc_decode_apply.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_float, C.c_void_p, C.c_void_p, C.c_int64,
                                        C.c_void_p, C.c_void_p]
+        L.sbc_stream_bytes_values.restype = C.c_size_t
+        L.sbc_stream_bytes_values.argtypes = [C.c_int64, C.c_double]
+        L.sbc_encode_values.restype = C.c_int
+        L.sbc_encode_values.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_double, C.c_void_p, C.c_size_t,
+                                        C.c_void_p, C.c_size_t, C.c_void_p]
         L.sbc_stream_info_get.restype = C.c_int
         L.sbc_stream_info_get.argtypes = [C.c_void_p, C.POINTER(StreamInfo), C.c_void_p]
         L.sbc_decode_accumulate.restype = C.c_int
@@ -403,3 +409,25 @@ def sbc_decode_apply(streams: Sequence[torch.Tensor], scale: float, weights: tor
                                   momentum.data_ptr() if momentum is not None else None, weights.numel(),
                                   status.data_ptr() if status is not None else None, _cuda_stream(stream))
     _check(code, "sbc_decode_apply")
+
+
+def sbc_stream_bytes_values(numel: int, p: float) -> int:
+    return int(lib().sbc_stream_bytes_values(numel, p))
+
+
+def sbc_encode_values(update: torch.Tensor, residual: torch.Tensor, p: float,
+                      out_stream: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                      stream=None) -> torch.Tensor:
+    """Gradient Dropping client step (top-p by magnitude, values sent); residual updated in place."""
+    _dev_f32(update, "update")
+    _dev_f32(residual, "residual")
+    n = update.numel()
+    if out_stream is None:
+        out_stream = torch.empty(sbc_stream_bytes_values(n, p), dtype=torch.uint8, device=update.device)
+    if workspace is None:
+        workspace = torch.empty(sbc_workspace_bytes(n, p), dtype=torch.uint8, device=update.device)
+    code = lib().sbc_encode_values(update.data_ptr(), residual.data_ptr(), n, float(p), out_stream.data_ptr(),
+                                   out_stream.numel(), workspace.data_ptr(), workspace.numel(),
+                                   _cuda_stream(stream))
+    _check(code, "sbc_encode_values")
+    return out_stream

@@ -28,7 +28,7 @@ static_assert(sizeof(Prob) <= kProbSlotBytes, "descriptor must fit its slot");
 //   rest       everything that needs no clearing
 struct Plan {
     long long n, k;
-    int b;
+    int b, mode;
     uint32_t cap, m, n_xtiles, n_tiles, n_len_blocks, n_chunks;
     uint32_t s_target[2];
     unsigned long long payload_offset;
@@ -42,7 +42,7 @@ struct Plan {
 
 bool valid_p(double p) { return p > 0.0 && p < 1.0; }
 
-bool make_plan(long long n, double p, Plan* pl) {
+bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary) {
     if (n <= 0 || n >= (1ll << 31) || !valid_p(p)) return false;
     const int b = sbc_golomb_b(p);
     if (b < 0 || b > 30) return false;
@@ -80,6 +80,8 @@ bool make_plan(long long n, double p, Plan* pl) {
     pl->n_len_blocks = (uint32_t)((k + kLenBlock - 1) / kLenBlock);
     pl->n_chunks = (uint32_t)((k + kChunkCodewords - 1) / kChunkCodewords);
     pl->payload_offset = SBC_HEADER_BYTES + (unsigned long long)pl->n_chunks * SBC_CHUNK_ENTRY_BYTES;
+    if (mode == kModeValues) pl->payload_offset += align_up((size_t)k * 4, 16);  // the values sit before the payload
+    pl->mode = mode;
     const unsigned long long bits_bound =
         (unsigned long long)k * (1ull + b) + ((unsigned long long)(n - k) >> b);
     pl->stream_bytes = (size_t)pl->payload_offset + align_up((size_t)((bits_bound + 7) / 8), 16);
@@ -136,6 +138,7 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile
     P.k = pl.k;
     P.b = pl.b;
     P.vec_ok = (((uintptr_t)a.update | (uintptr_t)a.residual) & 15) == 0;
+    P.mode = pl.mode;
     P.stream = static_cast<uint8_t*>(a.out_stream);
     P.stream_cap = a.out_capacity;
     P.stream_bytes = pl.stream_bytes;
@@ -216,7 +219,7 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
 // a single problem) say how each kind of work is spread over the problems.
 void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK_COUNT],
-                   const uint32_t* const* prefix, cudaStream_t st, const sbc_cuda_event_t* marks) {
+                   const uint32_t* const* prefix, int mode, cudaStream_t st, const sbc_cuda_event_t* marks) {
     auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
     auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs}; };
     const dim3 blk(kBlock);
@@ -227,7 +230,8 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     k_sample0<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
     k_sample1<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
     mark(SBC_MARK_BOUNDS);
-    k_add_collect<<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
+    if (mode == kModeValues) k_add_collect<kModeValues><<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
+    else                     k_add_collect<kModeBinary><<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
     mark(SBC_MARK_COLLECT);
 
     // 2. exact route over A (returns immediately unless the bounds failed)
@@ -303,12 +307,12 @@ int sbc_encode(const float* update, float* residual, int64_t numel, double p, vo
                          workspace_bytes, stream, nullptr);
 }
 
-int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p, void* out_stream,
-                  size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
-                  sbc_cuda_stream_t stream, const sbc_cuda_event_t* marks) {
+static int encode_impl(int mode, const float* update, float* residual, int64_t numel, double p, void* out_stream,
+                       size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
+                       sbc_cuda_stream_t stream, const sbc_cuda_event_t* marks) {
     Plan pl;
     if (!workspace || ((uintptr_t)workspace & 255)) return SBC_EINVAL;
-    if (!make_plan(numel, p, &pl)) return SBC_EINVAL;
+    if (!make_plan(numel, p, &pl, mode)) return SBC_EINVAL;
     const TensorArgs a = {update, residual, out_stream, out_capacity, out_mu};
     const int rc = check_tensor(a, pl);
     if (rc != SBC_OK) return rc;
@@ -333,8 +337,26 @@ int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p,
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, 1u, grid);
-    launch_encode(d_prob, 1u, grid, nullptr, st, marks);
+    launch_encode(d_prob, 1u, grid, nullptr, mode, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
+}
+
+int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p, void* out_stream,
+                  size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
+                  sbc_cuda_stream_t stream, const sbc_cuda_event_t* marks) {
+    return encode_impl(kModeBinary, update, residual, numel, p, out_stream, out_capacity, out_mu, workspace,
+                       workspace_bytes, stream, marks);
+}
+
+size_t sbc_stream_bytes_values(int64_t numel, double p) {
+    Plan pl;
+    return make_plan(numel, p, &pl, kModeValues) ? pl.stream_bytes : 0;
+}
+
+int sbc_encode_values(const float* update, float* residual, int64_t numel, double p, void* out_stream,
+                      size_t out_capacity, void* workspace, size_t workspace_bytes, sbc_cuda_stream_t stream) {
+    return encode_impl(kModeValues, update, residual, numel, p, out_stream, out_capacity, nullptr, workspace,
+                       workspace_bytes, stream, nullptr);
 }
 
 size_t sbc_workspace_bytes_batch(int n_tensors, const sbc_tensor_desc* descs) {
@@ -430,7 +452,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
     k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors});
-    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, st, nullptr);
+    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

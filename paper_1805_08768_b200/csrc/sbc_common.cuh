@@ -82,6 +82,7 @@ struct Prob {
     long long k;
     int b;
     int vec_ok;                 // 1: update and residual are 16-byte aligned
+    int mode;                   // kModeBinary (SBC) or kModeValues (top-p by magnitude, values sent)
     uint8_t* stream;            // container out
     unsigned long long stream_cap;
     unsigned long long stream_bytes;  // bytes sbc_stream_bytes(n, p) promises to stay within
@@ -155,6 +156,15 @@ __device__ __forceinline__ uint32_t bits_of_key(uint32_t key) {
     return (key & 0x80000000u) ? (key & 0x7fffffffu) : ~key;
 }
 __device__ __forceinline__ uint32_t side_key(int side, uint32_t key) { return side ? ~key : key; }
+
+// What the selection ranks by.  kModeBinary: the signed value (Algorithm 2 takes the k largest of
+// dW and of -dW).  kModeValues: the magnitude (Gradient Dropping keeps the k entries of largest
+// |dW|); only side 0 exists then.
+constexpr int kModeBinary = 0;
+constexpr int kModeValues = 1;
+__device__ __forceinline__ uint32_t select_key(int mode, uint32_t bits) {
+    return mode == kModeValues ? (bits & 0x7fffffffu) : key_of_bits(bits);
+}
 __device__ __forceinline__ unsigned long long make_composite(uint32_t skey, uint32_t idx) {
     return ((unsigned long long)skey << 32) | (unsigned long long)(~idx);
 }

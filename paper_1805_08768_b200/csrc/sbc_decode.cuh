@@ -30,6 +30,7 @@ struct StreamView {
     unsigned long long k, nbits, n_words;
     uint32_t b, n_chunks;
     float mu;
+    const float* values;  // one value per position (values stream), else null
 };
 
 // 32 stream bits starting at bit `pos`, MSB first; bits past the payload read as 0.
@@ -123,12 +124,18 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
         v.n_words = (v.nbits + 31ull) >> 5;
         v.words = reinterpret_cast<const uint32_t*>(h + payload_offset);
         v.table = h + SBC_HEADER_BYTES;
+        const uint32_t side = load_u32(h + 44);
+        const unsigned long long values_bytes = (side == SBC_SIDE_VALUES) ? ((v.k * 4ull + 15ull) & ~15ull) : 0ull;
+        v.values = (side == SBC_SIDE_VALUES)
+            ? reinterpret_cast<const float*>(h + SBC_HEADER_BYTES + (unsigned long long)v.n_chunks * SBC_CHUNK_ENTRY_BYTES)
+            : nullptr;
         const bool good =
             load_u32(h + 0) == SBC_MAGIC && load_u32(h + 4) == SBC_VERSION &&
             load_u64(h + 8) == (unsigned long long)args.n && load_u32(h + 60) == 0u &&
             load_u32(h + 52) == SBC_CHUNK_CODEWORDS && v.b <= 30u && v.k <= (unsigned long long)args.n &&
             v.n_chunks == (uint32_t)((v.k + kChunkCodewords - 1) / kChunkCodewords) &&
-            payload_offset == SBC_HEADER_BYTES + (unsigned long long)v.n_chunks * SBC_CHUNK_ENTRY_BYTES &&
+            side <= SBC_SIDE_VALUES &&
+            payload_offset == SBC_HEADER_BYTES + (unsigned long long)v.n_chunks * SBC_CHUNK_ENTRY_BYTES + values_bytes &&
             v.nbits >= v.k * (1ull + v.b) &&
             v.nbits <= v.k * (1ull + v.b) + ((unsigned long long)args.n >> v.b);
         if (!good) {
@@ -188,6 +195,7 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
             const uint32_t b = v.b;
             const float mu = __fmul_rn(v.mu, args.scale);
             float* __restrict__ momentum = args.momentum;
+            const float* __restrict__ vals = v.values ? v.values + (size_t)chunk * kChunkCodewords : nullptr;
             const bool tiny = fabsf(mu) < 7.888609052e-31f;  // 2^-100
             if (staged) {
                 // Fast path: bit positions relative to the stage fit 32 bits; every codeword
@@ -221,7 +229,12 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                         break;
                     }
                     prev += (long long)step;
-                    err |= add_at(args.out + prev, mu, tiny);
+                    if (vals) {
+                        const float x = __fmul_rn(vals[i], args.scale);
+                        err |= add_at(args.out + prev, x, fabsf(x) < 7.888609052e-31f);
+                    } else {
+                        err |= add_at(args.out + prev, mu, tiny);
+                    }
                     if (momentum) momentum[prev] = 0.f;
                 }
                 pos = (first_word << 5) + rel;
@@ -253,7 +266,12 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                         break;
                     }
                     prev += (long long)step;
-                    err |= add_at(args.out + prev, mu, tiny);
+                    if (vals) {
+                        const float x = __fmul_rn(vals[i], args.scale);
+                        err |= add_at(args.out + prev, x, fabsf(x) < 7.888609052e-31f);
+                    } else {
+                        err |= add_at(args.out + prev, mu, tiny);
+                    }
                     if (momentum) momentum[prev] = 0.f;
                 }
                 if (!err && used > room) err = SBC_STATUS_CORRUPT;

@@ -33,7 +33,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_hist(const Batch B) {
     for (long long base = (long long)S.bx * kBlock; base < P.n; base += stride) {
         const long long i = base + threadIdx.x;
         const bool valid = i < P.n;
-        const uint32_t key = valid ? key_of_bits(__float_as_uint(A[i])) : 0u;
+        const uint32_t key = valid ? select_key(P.mode, __float_as_uint(A[i])) : 0u;
         if (LEVEL == 0) {
             warp_hist_add(s_hist[0], key >> 21, valid);
         } else {
@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Batch B) {
         for (int j = 0; j < kXTile / kBlock; ++j) {
             const long long i = (long long)tile * kXTile + j * kBlock + threadIdx.x;
             if (i < P.n) {
-                const uint32_t key = key_of_bits(__float_as_uint(A[i]));
+                const uint32_t key = select_key(P.mode, __float_as_uint(A[i]));
                 c += (key == thr[0]) ? 1u : 0u;
                 c += (~key == thr[1]) ? 0x10000u : 0u;
             }
@@ -162,6 +162,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
     const uint32_t thr[2] = {ctl->x_thr[0], ctl->x_thr[1]};
     const uint32_t take[2] = {ctl->x_ties_take[0], ctl->x_ties_take[1]};
     const bool ranked[2] = {tie_ranks_needed(ctl, 0), tie_ranks_needed(ctl, 1)};
+    const bool one_sided = P.mode == kModeValues;  // magnitude selection has no second side
     const float* __restrict__ A = P.residual;
     for (uint32_t tile = S.bx; tile < P.n_xtiles; tile += S.nb) {
         const long long wbase = (long long)tile * kXTile + (long long)warp * (kXTile / (kBlock / 32));
@@ -172,13 +173,14 @@ __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
             const long long i = wbase + j * 32 + lane;
             key[j] = 0u;
             if (i < P.n) {
-                key[j] = key_of_bits(__float_as_uint(A[i]));
+                key[j] = select_key(P.mode, __float_as_uint(A[i]));
                 inb |= 1u << j;
             }
         }
         unsigned emit[2] = {0u, 0u};
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
+            if (s == 1 && one_sided) continue;
             if (!ranked[s]) {
 #pragma unroll
                 for (int j = 0; j < kSteps; ++j)
@@ -195,7 +197,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
         __syncthreads();
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
-            if (!ranked[s]) continue;
+            if (!ranked[s] || (s == 1 && one_sided)) continue;
             uint32_t run = P.x_tile_cnt[s][tile];
             for (int w = 0; w < warp; ++w) run += s_warp_ties[s][w];
 #pragma unroll

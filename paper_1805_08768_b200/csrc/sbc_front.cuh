@@ -43,7 +43,7 @@ __global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
         if (valid) {
             const long long e = sample_element(P, i);
             const float a = __fadd_rn(P.residual[e], P.update[e]);
-            key = key_of_bits(__float_as_uint(a));
+            key = select_key(P.mode, __float_as_uint(a));
             P.sample_keys[i] = key;
         }
         warp_hist_add(s_hist, key >> 21, valid);
@@ -99,8 +99,14 @@ __global__ void __launch_bounds__(kBlock) k_sample1(const Batch B) {
             block_pick_desc(P.hists->s1[s], kHistBins, false, ctl->s_rank[s], s_scan, &s_pick);
             if (threadIdx.x == 0) {
                 const uint32_t lower = (bin0[s] << 21) | (s_pick.bin << 10);  // side key, low bits 0
-                if (s == 0) ctl->lo_f = __uint_as_float(bits_of_key(lower));
-                else        ctl->hi_f = __uint_as_float(bits_of_key(~lower));
+                if (P.mode == kModeValues) {  // the key is the magnitude's bit pattern; no second side
+                    if (s == 0) ctl->lo_f = __uint_as_float(lower);
+                    else        ctl->hi_f = -INFINITY;
+                } else if (s == 0) {
+                    ctl->lo_f = __uint_as_float(bits_of_key(lower));
+                } else {
+                    ctl->hi_f = __uint_as_float(bits_of_key(~lower));
+                }
                 if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
             }
             __syncthreads();
@@ -121,6 +127,7 @@ constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 wa
 // through per-warp shared-memory staging so that the global list counters see
 // one atomic per hundred or so candidates.  Each thread has eight 16-byte
 // loads in flight before it touches any of them.
+template <int MODE>
 __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
@@ -191,8 +198,12 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
         unsigned pm = 0u, qm = 0u;
 #pragma unroll
         for (int j = 0; j < kPerThread; ++j) {
-            pm |= (!(a[j] < lo) ? 1u : 0u) << j;   // also true for NaN
-            qm |= (!(a[j] > hi) ? 1u : 0u) << j;
+            if (MODE == kModeValues) {
+                pm |= (!(fabsf(a[j]) < lo) ? 1u : 0u) << j;   // also true for NaN
+            } else {
+                pm |= (!(a[j] < lo) ? 1u : 0u) << j;          // also true for NaN
+                qm |= (!(a[j] > hi) ? 1u : 0u) << j;
+            }
         }
         pm &= inb;
         qm &= inb;
@@ -225,7 +236,7 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
                         if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;
                         const long long e = vec_layout ? base + (long long)(((j >> 2) * 32 + lane) * 4 + (j & 3))
                                                        : base + j * 32 + lane;
-                        const unsigned long long c = make_composite(side_key(s, key_of_bits(bits)), (uint32_t)e);
+                        const unsigned long long c = make_composite(side_key(s, select_key(MODE, bits)), (uint32_t)e);
                         if (direct) { if (off < cap) (s ? cand1 : cand0)[off] = c; }
                         else s_stage[warp][s][off] = c;
                         ++off;
@@ -242,7 +253,8 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
     if (last_block_ticket(&ctl->done[ST_COLLECT], S.nb)) {
         if (threadIdx.x == 0) {
             const uint32_t c0 = __ldcg(&ctl->cand_cnt[0]), c1 = __ldcg(&ctl->cand_cnt[1]);
-            const bool ok = c0 >= (uint32_t)P.k && c0 <= P.cap && c1 >= (uint32_t)P.k && c1 <= P.cap;
+            const bool ok = c0 >= (uint32_t)P.k && c0 <= P.cap &&
+                            (MODE == kModeValues || (c1 >= (uint32_t)P.k && c1 <= P.cap));
             ctl->use_fallback = ok ? 0u : 1u;
         }
     }

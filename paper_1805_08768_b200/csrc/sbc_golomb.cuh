@@ -149,6 +149,11 @@ __global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
     constexpr int kPer = kLenBlock / kBlock;
     const float mu = P.ctl->mu32;
     const uint32_t k = (uint32_t)P.k;
+    // values mode: the kept values themselves are sent (they sit between the chunk table and the
+    // payload, in position order) and nothing of them stays in the residual
+    float* values = (P.mode == kModeValues)
+        ? reinterpret_cast<float*>(P.stream + SBC_HEADER_BYTES + (size_t)P.n_chunks * SBC_CHUNK_ENTRY_BYTES)
+        : nullptr;
     for (uint32_t blk = S.bx; blk < P.n_len_blocks; blk += S.nb) {
         const uint32_t i0 = blk * kLenBlock + threadIdx.x * kPer;
         uint32_t pos[kPer];
@@ -162,7 +167,8 @@ __global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             if (i0 + j < k) {
-                P.residual[pos[j]] = __fsub_rn(r[j], mu);
+                if (values) values[i0 + j] = r[j];
+                P.residual[pos[j]] = __fsub_rn(r[j], values ? r[j] : mu);
                 const uint32_t g = (uint32_t)((long long)pos[j] - prev - 1);
                 sum += (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
                 prev = pos[j];
@@ -221,7 +227,7 @@ __global__ void __launch_bounds__(kBlock) k_len_scan_header(const Batch B) {
         store_u64(h + 24, total);
         store_u64(h + 32, ok ? P.payload_offset : (unsigned long long)SBC_HEADER_BYTES);
         store_u32(h + 40, (uint32_t)P.b);
-        store_u32(h + 44, ok ? ctl->side : 0u);
+        store_u32(h + 44, ok ? (P.mode == kModeValues ? SBC_SIDE_VALUES : ctl->side) : 0u);
         store_u32(h + 48, ok ? __float_as_uint(ctl->mu32) : 0u);
         store_u32(h + 52, SBC_CHUNK_CODEWORDS);
         store_u32(h + 56, ok ? P.n_chunks : 0u);

@@ -24,6 +24,7 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
+    if (s == 1 && P.mode == kModeValues) return;  // magnitude selection has one side only
     __shared__ uint32_t s_hist[kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     __shared__ Pick s_pick;
@@ -62,6 +63,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
+    if (s == 1 && P.mode == kModeValues) return;
     constexpr int kItems = 4;
     __shared__ uint32_t s_hist[kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -183,6 +185,8 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = blockIdx.z;
+    const bool values_mode = P.mode == kModeValues;
+    if (s == 1 && values_mode) return;
     __shared__ unsigned long long s_bins[2][256];
     s_bins[0][threadIdx.x] = 0ull;
     __syncthreads();
@@ -192,7 +196,7 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     // Almost every kept value shares the exponent of the threshold value or the
     // next one up: those two bins are summed in registers, the rest goes
     // straight to the shared bins.
-    const uint32_t thr_bits = bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
+    const uint32_t thr_bits = values_mode ? (uint32_t)(thr >> 32) : bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
     const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
     const int bin_b = bin_a + 1;
     long long acc_a = 0, acc_b = 0;
@@ -211,7 +215,7 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
         const uint32_t i = base + threadIdx.x;
         const unsigned long long c = (i < hi) ? src[i] : 0ull;
         const bool kept = (i < hi) && c >= thr;
-        if (kept) {
+        if (kept && !values_mode) {  // the means exist only for the binarised form
             const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
             const uint32_t e = (bits >> 23) & 0xffu;
             int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
@@ -242,7 +246,7 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
         const unsigned long long v = s_bins[0][threadIdx.x];
         if (v) atomicAdd(reinterpret_cast<unsigned long long*>(&ctl->bins[s][threadIdx.x]), v);
     }
-    if (last_block_ticket(&ctl->done[ST_SUM], S.nb * gridDim.z)) {
+    if (last_block_ticket(&ctl->done[ST_SUM], values_mode ? S.nb : S.nb * gridDim.z)) {
         s_bins[0][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[0][threadIdx.x]);
         s_bins[1][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[1][threadIdx.x]);
         __syncthreads();
@@ -254,8 +258,8 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
         if (threadIdx.x == 0) {
             const double mu_pos = ctl->mu64[0];
             const double mu_neg = ctl->mu64[1];  // val- holds the negated entries
-            const uint32_t side = (mu_pos >= mu_neg) ? 0u : 1u;
-            const float mu = side ? (float)(-mu_neg) : (float)mu_pos;
+            const uint32_t side = values_mode ? 0u : ((mu_pos >= mu_neg) ? 0u : 1u);
+            const float mu = values_mode ? 0.f : (side ? (float)(-mu_neg) : (float)mu_pos);
             ctl->side = side;
             ctl->mu32 = mu;
             if (P.out_mu) *P.out_mu = mu;

@@ -293,3 +293,70 @@ def test_decode_apply_scales_adds_and_masks_momentum():
     want1 = w0.copy()
     oracle.decode_apply(streams_np[:1], 1.0, want1)
     assert np.array_equal(w1.cpu().numpy().view(np.uint32), want1.view(np.uint32))
+
+
+# ---------------------------------------------------------------- Gradient Dropping baseline
+
+def check_values_mode(upd, res, p):
+    n = upd.size
+    want_res = res.copy()
+    want = oracle.encode_values(upd, want_res, p)
+    u = torch.from_numpy(upd).to(DEV)
+    r = torch.from_numpy(res).to(DEV)
+    cap = sbc.sbc_stream_bytes_values(n, p)
+    assert cap == oracle.stream_bytes_values(n, p)
+    out = torch.full((cap + 64,), 0xAB, dtype=torch.uint8, device=DEV)
+    sbc.sbc_encode_values(u, r, p, out_stream=out[:cap])
+    info = sbc.sbc_stream_info_get(out)
+    torch.cuda.synchronize()
+    assert bool((out[cap:] == 0xAB).all())
+    assert info.side == sbc.SIDE_VALUES and info.mu == 0.0
+    got = out[: info.total_bytes].cpu().numpy()
+    assert got.size == want.size and np.array_equal(got, want)
+    assert np.array_equal(r.cpu().numpy().view(np.uint32), want_res.view(np.uint32))
+    return out, want
+
+
+@pytest.mark.parametrize("name,upd,res,p", workloads.adversarial_cases(),
+                         ids=[c[0] for c in workloads.adversarial_cases()])
+def test_values_mode_adversarial_cases(name, upd, res, p):
+    check_values_mode(upd, res, p)
+
+
+@pytest.mark.parametrize("n,p", [(1 << 21, 0.01), (3_000_001, 0.001), (1 << 22, 1e-4), (70001, 0.1)])
+def test_values_mode_large_and_decode(n, p):
+    rng = np.random.default_rng(n)
+    upd = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
+    res = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    out, want = check_values_mode(upd, res, p)
+    # decode: dW* = A on the kept set; a values stream and a binary stream can be summed together
+    upd2 = workloads.normal_flat(n, 1e-3, 5)
+    s2, _, _, _, out2 = gpu_encode(upd2, np.zeros(n, dtype=np.float32), p)
+    want_dense = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate([want, s2], want_dense)
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sbc.sbc_decode_accumulate([out, out2], dense, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    got = dense.cpu().numpy()
+    assert np.max(np.abs(got.astype(np.float64) - want_dense)) <= 1e-6 * float(np.abs(want_dense).max())
+    one = torch.zeros(n, dtype=torch.float32, device=DEV)
+    sbc.sbc_decode_accumulate([out], one)
+    want_one = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate([want], want_one)
+    torch.cuda.synchronize()
+    assert np.array_equal(one.cpu().numpy().view(np.uint32), want_one.view(np.uint32))
+
+
+def test_values_mode_three_rounds_with_carried_residual():
+    n, p = 500000, 0.001
+    res_cpu = np.zeros(n, dtype=np.float32)
+    r = torch.zeros(n, dtype=torch.float32, device=DEV)
+    for rnd in range(3):
+        upd = workloads.normal_flat(n, 1e-3, 900 + rnd)
+        want = oracle.encode_values(upd, res_cpu, p)
+        out = sbc.sbc_encode_values(torch.from_numpy(upd).to(DEV), r, p)
+        info = sbc.sbc_stream_info_get(out)
+        assert np.array_equal(out[: info.total_bytes].cpu().numpy(), want)
+        assert np.array_equal(r.cpu().numpy().view(np.uint32), res_cpu.view(np.uint32))

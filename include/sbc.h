@@ -175,6 +175,36 @@ int sbc_encode_values(const float *update, float *residual, int64_t numel, doubl
                       size_t workspace_bytes, sbc_cuda_stream_t stream);
 
 /*
+ * sbc_encode with thresholds estimated from a random subsample (Section 2,
+ * "Sparse Binarization": the cost of the selection can be reduced "by randomly
+ * subsampling from W", at the price of noise in the amount of sparsity).  The
+ * caller draws the sample positions; everything else is deterministic:
+ *
+ *   j  = max(1, floor(p * sample_count))
+ *   t+ = j-th largest, t- = j-th smallest of A[sample_idx[0..sample_count)]
+ *   val+ = ALL entries A_i >= t+,  val- = ALL entries A_i <= t-   (about k each)
+ *   means over those sets, side choice, binarisation, residual, stream: as
+ *   sbc_encode, with the header's k = the size of the kept set.
+ *
+ * The estimate is accepted if both sets hold between 1 and min(numel, 2k+1024)
+ * entries (k = sbc_kept_count); otherwise the call produces exactly what
+ * sbc_encode produces.  The selection stage of sbc_encode is skipped, so the
+ * call is cheaper by that stage.
+ *
+ * sample_idx   device, sample_count positions in [0, numel), 4-byte aligned;
+ *              a position >= numel sets SBC_STATUS_RANGE in the header
+ * sample_count 1 .. 2^20
+ * out_capacity >= sbc_stream_bytes_sampled(numel, p)
+ * workspace    >= sbc_workspace_bytes_sampled(numel, p, sample_count)
+ */
+size_t sbc_stream_bytes_sampled(int64_t numel, double p);
+size_t sbc_workspace_bytes_sampled(int64_t numel, double p, int64_t sample_count);
+int sbc_encode_sampled(const float *update, float *residual, int64_t numel, double p,
+                       const uint32_t *sample_idx, int64_t sample_count, void *out_stream,
+                       size_t out_capacity, float *out_mu, void *workspace,
+                       size_t workspace_bytes, sbc_cuda_stream_t stream);
+
+/*
  * sbc_encode for many tensors at once (a model's parameter tensors in one
  * communication round; the paper applies the method per tensor, with one mean
  * per tensor -- Section 2, "Optimal Position Encoding").  Exactly the results

@@ -549,6 +549,80 @@ int sbc_oracle_encode_values(const float *update, float *residual, int64_t n, do
     return 0;
 }
 
+/* ------------------------------------------------------------------ */
+/* Sparse binarisation with thresholds from a random subsample         */
+/* (Section 2, "Sparse Binarization": subsampling reduces the cost of  */
+/* the selection and adds noise to the amount of sparsity)             */
+/* ------------------------------------------------------------------ */
+
+static int cmp_float_desc(const void *x, const void *y) {
+    float a = *(const float *)x, b = *(const float *)y;
+    return (a < b) - (a > b);
+}
+
+int sbc_oracle_encode_sampled(const float *update, float *residual, int64_t n, double p,
+                              const uint32_t *sample_idx, int64_t m, uint8_t *out, size_t cap,
+                              size_t *out_len, float *out_mu) {
+    if (!update || !residual || !out || !sample_idx || m <= 0 || n <= 0 || n >= ((int64_t)1 << 31) ||
+        !(p > 0.0 && p < 1.0))
+        return -2;
+    int64_t k = sbc_oracle_kept_count(n, p);
+    int b = sbc_oracle_golomb_b(p);
+    if (b > 30) return -2;
+    if (sbc_oracle_accumulate(update, residual, n) != 0) return -1;
+    float *a = residual;
+
+    /* thresholds: the floor(p*m)-th largest and smallest of the sampled entries */
+    float *sv = (float *)malloc((size_t)m * sizeof(float));
+    if (!sv) return -2;
+    for (int64_t i = 0; i < m; ++i) {
+        if (sample_idx[i] >= (uint64_t)n) { free(sv); return -2; }
+        sv[i] = a[sample_idx[i]];
+    }
+    qsort(sv, (size_t)m, sizeof(float), cmp_float_desc);
+    int64_t j = (int64_t)floor(p * (double)m);
+    if (j < 1) j = 1;
+    float t_pos = sv[j - 1], t_neg = sv[m - j];
+    free(sv);
+
+    /* val+ = everything at or above t+, val- = everything at or below t- */
+    int64_t limit = 2 * k + 1024;
+    if (limit > n) limit = n;
+    int64_t n_pos = 0, n_neg = 0;
+    for (int64_t i = 0; i < n; ++i) { n_pos += a[i] >= t_pos; n_neg += a[i] <= t_neg; }
+    int64_t *I;
+    int side;
+    float mu;
+    int64_t kept_count;
+    if (n_pos >= 1 && n_pos <= limit && n_neg >= 1 && n_neg <= limit) {
+        int64_t *P = (int64_t *)malloc((size_t)n_pos * sizeof(int64_t));
+        int64_t *N = (int64_t *)malloc((size_t)n_neg * sizeof(int64_t));
+        if (!P || !N) { free(P); free(N); return -2; }
+        int64_t ip = 0, in = 0;
+        for (int64_t i = 0; i < n; ++i) {
+            if (a[i] >= t_pos) P[ip++] = i;
+            if (a[i] <= t_neg) N[in++] = i;
+        }
+        double mp = sbc_oracle_exact_sum(a, P, n_pos) / (double)n_pos;   /* mean(val+) */
+        double mn = -sbc_oracle_exact_sum(a, N, n_neg) / (double)n_neg;  /* mean(val-) */
+        if (mp >= mn) { side = 0; mu = (float)mp; I = P; kept_count = n_pos; free(N); }
+        else          { side = 1; mu = (float)(-mn); I = N; kept_count = n_neg; free(P); }
+        for (int64_t q = 0; q < kept_count; ++q) {
+            volatile float r = a[I[q]] - mu;
+            a[I[q]] = r;
+        }
+    } else { /* estimate rejected: Algorithm 2 with exactly k entries per side */
+        I = (int64_t *)malloc((size_t)k * sizeof(int64_t));
+        if (!I) return -2;
+        sbc_oracle_compress(a, n, k, I, &side, &mu, NULL, NULL);
+        kept_count = k;
+    }
+    int rc = sbc_oracle_container(I, kept_count, n, b, side, mu, out, cap, out_len);
+    if (rc == 0 && out_mu) *out_mu = mu;
+    free(I);
+    return rc;
+}
+
 int sbc_oracle_decode_accumulate(const uint8_t *const *streams, int n_clients,
                                  float *out_dense, int64_t n) {
     if (!streams || !out_dense || n_clients < 0 || n <= 0) return -2;

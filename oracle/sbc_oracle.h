@@ -141,6 +141,18 @@ int sbc_oracle_encode_values(const float *update, float *residual, int64_t n, do
 int64_t sbc_oracle_golomb_decode_values(const uint8_t *payload, uint64_t nbits, int b,
                                         const uint8_t *values, int64_t k, float *dense, int64_t n);
 
+/* Sparse binarisation with thresholds from a subsample (Section 2, "Sparse Binarization": the
+ * selection can be made cheaper "by randomly subsampling from W", which adds noise to the amount
+ * of sparsity).  The caller supplies the m sample positions.  j = max(1, floor(p*m)); t+ / t- =
+ * the j-th largest / smallest sampled entry of A = R + update; val+ = ALL entries >= t+, val- =
+ * ALL entries <= t-; means over those sets, side choice, binarisation, residual and container as
+ * in the exact method, with k = size of the kept set.  If either set is empty or larger than
+ * min(n, 2*kept_count(n,p) + 1024) the estimate is rejected and the exact method is used.
+ * cap: at least sbc_oracle_container_bytes(limit, limit*(1+b) + 2*(n >> b)). */
+int sbc_oracle_encode_sampled(const float *update, float *residual, int64_t n, double p,
+                              const uint32_t *sample_idx, int64_t m, uint8_t *out, size_t cap,
+                              size_t *out_len, float *out_mu);
+
 /* Server / client apply step (Algorithm 1: "dW <- 1/|I_t| sum dW_i*", "W <- W + dW") with
  * momentum masking (Supplement): weights[j] = fl32(weights[j] + fl32(scale * sum_j)) for every
  * j, sum_j the fp32 sum of the decoded client tensors in client order; momentum[j] = 0 at every

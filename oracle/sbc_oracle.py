@@ -14,7 +14,7 @@ __all__ = [
     "kept_count", "golomb_b", "mean_position_bits", "accumulate", "topk",
     "exact_sum", "compress", "payload_bits_bound", "golomb_encode",
     "golomb_decode", "container_bytes", "stream_bytes", "encode",
-    "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container", "decode_apply", "topk_abs", "stream_bytes_values", "encode_values",
+    "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container", "decode_apply", "topk_abs", "stream_bytes_values", "encode_values", "encode_sampled",
     "HEADER_BYTES", "CHUNK_CODEWORDS", "CHUNK_ENTRY_BYTES", "MAGIC",
 ]
 
@@ -224,6 +224,26 @@ def encode_values(update: np.ndarray, residual: np.ndarray, p: float) -> np.ndar
     if rc != 0:
         raise ValueError(f"sbc_oracle_encode_values failed: {rc}")
     return out[: out_len.value].copy()
+
+
+_u32p = np.ctypeslib.ndpointer(dtype=np.uint32, flags="C_CONTIGUOUS")
+_encode_sampled = _sig("sbc_oracle_encode_sampled", C.c_int, _f32p, _f32p, C.c_int64, C.c_double, _u32p,
+                       C.c_int64, _u8p, C.c_size_t, C.POINTER(C.c_size_t), C.POINTER(C.c_float))
+
+
+def encode_sampled(update: np.ndarray, residual: np.ndarray, p: float, sample_idx: np.ndarray):
+    """Client step with thresholds taken from the given subsample.  Returns (stream bytes, mu32)."""
+    n = update.size
+    k, b = kept_count(n, p), golomb_b(p)
+    limit = min(n, 2 * k + 1024)
+    cap = container_bytes(limit, limit * (1 + b) + 2 * (n >> b))
+    out = np.zeros(cap, dtype=np.uint8)
+    out_len, mu = C.c_size_t(), C.c_float()
+    idx = np.ascontiguousarray(sample_idx, dtype=np.uint32)
+    rc = _encode_sampled(update, residual, n, p, idx, idx.size, out, cap, C.byref(out_len), C.byref(mu))
+    if rc != 0:
+        raise ValueError(f"sbc_oracle_encode_sampled failed: {rc}")
+    return out[: out_len.value].copy(), np.float32(mu.value)
 
 
 @dataclass

@@ -26,7 +26,8 @@ EXPORTS = [
     "sbc_workspace_bytes", "sbc_encode", "sbc_encode_ex", "sbc_encode_launches", "sbc_decode_launches",
     "sbc_encode_diag_get", "sbc_encode_host", "sbc_stream_info_get", "sbc_decode_accumulate",
     "sbc_decode_accumulate_host", "sbc_encode_static", "sbc_workspace_bytes_batch", "sbc_encode_batch",
-    "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch", "sbc_decode_apply", "sbc_stream_bytes_values", "sbc_encode_values",
+    "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch", "sbc_decode_apply", "sbc_stream_bytes_values", "sbc_encode_values", "sbc_stream_bytes_sampled",
+    "sbc_workspace_bytes_sampled", "sbc_encode_sampled",
 ]
 SIDE_VALUES = 2
 STATIC_WORKSPACE_BYTES = 8 << 20
@@ -128,6 +129,13 @@ def lib() -> C.CDLL:
         L.sbc_encode_values.restype = C.c_int
         L.sbc_encode_values.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_double, C.c_void_p, C.c_size_t,
                                         C.c_void_p, C.c_size_t, C.c_void_p]
+        L.sbc_stream_bytes_sampled.restype = C.c_size_t
+        L.sbc_stream_bytes_sampled.argtypes = [C.c_int64, C.c_double]
+        L.sbc_workspace_bytes_sampled.restype = C.c_size_t
+        L.sbc_workspace_bytes_sampled.argtypes = [C.c_int64, C.c_double, C.c_int64]
+        L.sbc_encode_sampled.restype = C.c_int
+        L.sbc_encode_sampled.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_double, C.c_void_p, C.c_int64,
+                                         C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.sbc_stream_info_get.restype = C.c_int
         L.sbc_stream_info_get.argtypes = [C.c_void_p, C.POINTER(StreamInfo), C.c_void_p]
         L.sbc_decode_accumulate.restype = C.c_int
@@ -431,3 +439,34 @@ def sbc_encode_values(update: torch.Tensor, residual: torch.Tensor, p: float,
                                    _cuda_stream(stream))
     _check(code, "sbc_encode_values")
     return out_stream
+
+
+def sbc_stream_bytes_sampled(numel: int, p: float) -> int:
+    return int(lib().sbc_stream_bytes_sampled(numel, p))
+
+
+def sbc_workspace_bytes_sampled(numel: int, p: float, sample_count: int) -> int:
+    return int(lib().sbc_workspace_bytes_sampled(numel, p, sample_count))
+
+
+def sbc_encode_sampled(update: torch.Tensor, residual: torch.Tensor, p: float, sample_idx: torch.Tensor,
+                       out_stream: Optional[torch.Tensor] = None, out_mu: Optional[torch.Tensor] = None,
+                       workspace: Optional[torch.Tensor] = None, stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """sbc_encode with the two thresholds taken from the caller's subsample (int32 CUDA positions)."""
+    _dev_f32(update, "update")
+    _dev_f32(residual, "residual")
+    if not (sample_idx.is_cuda and sample_idx.dtype == torch.int32 and sample_idx.is_contiguous()):
+        raise TypeError("sample_idx must be a contiguous int32 CUDA tensor")
+    n, m = update.numel(), sample_idx.numel()
+    dev = update.device
+    if out_stream is None:
+        out_stream = torch.empty(sbc_stream_bytes_sampled(n, p), dtype=torch.uint8, device=dev)
+    if out_mu is None:
+        out_mu = torch.empty(1, dtype=torch.float32, device=dev)
+    if workspace is None:
+        workspace = torch.empty(sbc_workspace_bytes_sampled(n, p, m), dtype=torch.uint8, device=dev)
+    code = lib().sbc_encode_sampled(update.data_ptr(), residual.data_ptr(), n, float(p), sample_idx.data_ptr(), m,
+                                    out_stream.data_ptr(), out_stream.numel(), out_mu.data_ptr(),
+                                    workspace.data_ptr(), workspace.numel(), _cuda_stream(stream))
+    _check(code, "sbc_encode_sampled")
+    return out_stream, out_mu

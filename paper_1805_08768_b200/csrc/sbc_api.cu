@@ -28,7 +28,7 @@ static_assert(sizeof(Prob) <= kProbSlotBytes, "descriptor must fit its slot");
 //   rest       everything that needs no clearing
 struct Plan {
     long long n, k;
-    int b, mode;
+    int b, mode, sampled;
     uint32_t cap, m, n_xtiles, n_tiles, n_len_blocks, n_chunks;
     uint32_t s_target[2];
     unsigned long long payload_offset;
@@ -42,7 +42,7 @@ struct Plan {
 
 bool valid_p(double p) { return p > 0.0 && p < 1.0; }
 
-bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary) {
+bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long long sampled_m = 0) {
     if (n <= 0 || n >= (1ll << 31) || !valid_p(p)) return false;
     const int b = sbc_golomb_b(p);
     if (b < 0 || b > 30) return false;
@@ -74,16 +74,24 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary) {
         const double t = std::ceil(expect + 6.0 * std::sqrt(expect) + 8.0);
         target = (uint32_t)std::min<double>(t, (double)pl->m);
     }
+    pl->sampled = sampled_m > 0;
+    if (pl->sampled) {  // the caller's subsample; its floor(p*m)-th order statistics ARE the thresholds
+        if (sampled_m > (long long)kSampleMax) return false;
+        pl->m = (uint32_t)sampled_m;
+        target = (uint32_t)std::max<long long>(1, (long long)std::floor(p * (double)sampled_m));
+    }
     pl->s_target[0] = pl->s_target[1] = target;
     pl->n_xtiles = (uint32_t)((n + kXTile - 1) / kXTile);
     pl->n_tiles = (uint32_t)((n + (1ll << kTileShift) - 1) >> kTileShift);
-    pl->n_len_blocks = (uint32_t)((k + kLenBlock - 1) / kLenBlock);
-    pl->n_chunks = (uint32_t)((k + kChunkCodewords - 1) / kChunkCodewords);
+    const long long k_max = pl->sampled ? (long long)pl->cap : k;  // most positions a stream can carry
+    pl->n_len_blocks = (uint32_t)((k_max + kLenBlock - 1) / kLenBlock);
+    pl->n_chunks = (uint32_t)((k_max + kChunkCodewords - 1) / kChunkCodewords);
     pl->payload_offset = SBC_HEADER_BYTES + (unsigned long long)pl->n_chunks * SBC_CHUNK_ENTRY_BYTES;
     if (mode == kModeValues) pl->payload_offset += align_up((size_t)k * 4, 16);  // the values sit before the payload
     pl->mode = mode;
     const unsigned long long bits_bound =
-        (unsigned long long)k * (1ull + b) + ((unsigned long long)(n - k) >> b);
+        (unsigned long long)k_max * (1ull + b) + ((unsigned long long)(n - std::min<long long>(n, k_max)) >> b) +
+        (pl->sampled ? ((unsigned long long)n >> b) : 0ull);
     pl->stream_bytes = (size_t)pl->payload_offset + align_up((size_t)((bits_bound + 7) / 8), 16);
 
     size_t off = 0;
@@ -102,7 +110,7 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary) {
     for (int s = 0; s < 2; ++s)
         for (int j = 0; j < 2; ++j) pl->off_buf[s][j] = take((size_t)pl->cap * 8);
     for (int s = 0; s < 2; ++s) pl->off_xtile[s] = take((size_t)pl->n_xtiles * 4);
-    pl->off_idx = take((size_t)k * 4);
+    pl->off_idx = take((size_t)k_max * 4);
     pl->off_blklen = take((size_t)pl->n_len_blocks * 8);
     pl->rest_bytes = off;
     pl->total = kProbSlotBytes + pl->zero_bytes + pl->tile_bytes + pl->rest_bytes;
@@ -139,6 +147,7 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile
     P.b = pl.b;
     P.vec_ok = (((uintptr_t)a.update | (uintptr_t)a.residual) & 15) == 0;
     P.mode = pl.mode;
+    P.sampled = pl.sampled;
     P.stream = static_cast<uint8_t*>(a.out_stream);
     P.stream_cap = a.out_capacity;
     P.stream_bytes = pl.stream_bytes;
@@ -219,7 +228,8 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
 // a single problem) say how each kind of work is spread over the problems.
 void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK_COUNT],
-                   const uint32_t* const* prefix, int mode, cudaStream_t st, const sbc_cuda_event_t* marks) {
+                   const uint32_t* const* prefix, int mode, bool sampled, cudaStream_t st,
+                   const sbc_cuda_event_t* marks) {
     auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
     auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs}; };
     const dim3 blk(kBlock);
@@ -229,6 +239,7 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     // 1. bounds from the sample, then the streaming accumulate + collect pass
     k_sample0<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
     k_sample1<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
+    if (sampled) k_sample2<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
     mark(SBC_MARK_BOUNDS);
     if (mode == kModeValues) k_add_collect<kModeValues><<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
     else                     k_add_collect<kModeBinary><<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
@@ -307,12 +318,14 @@ int sbc_encode(const float* update, float* residual, int64_t numel, double p, vo
                          workspace_bytes, stream, nullptr);
 }
 
-static int encode_impl(int mode, const float* update, float* residual, int64_t numel, double p, void* out_stream,
-                       size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
-                       sbc_cuda_stream_t stream, const sbc_cuda_event_t* marks) {
+static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, const float* update,
+                       float* residual, int64_t numel, double p, void* out_stream, size_t out_capacity,
+                       float* out_mu, void* workspace, size_t workspace_bytes, sbc_cuda_stream_t stream,
+                       const sbc_cuda_event_t* marks) {
     Plan pl;
     if (!workspace || ((uintptr_t)workspace & 255)) return SBC_EINVAL;
-    if (!make_plan(numel, p, &pl, mode)) return SBC_EINVAL;
+    if (sample_idx && (sample_m <= 0 || ((uintptr_t)sample_idx & 3))) return SBC_EINVAL;
+    if (!make_plan(numel, p, &pl, mode, sample_idx ? sample_m : 0)) return SBC_EINVAL;
     const TensorArgs a = {update, residual, out_stream, out_capacity, out_mu};
     const int rc = check_tensor(a, pl);
     if (rc != SBC_OK) return rc;
@@ -323,7 +336,8 @@ static int encode_impl(int mode, const float* update, float* residual, int64_t n
     uint8_t* zero = ws + kProbSlotBytes;
     uint8_t* tile = zero + pl.zero_bytes;
     uint8_t* rest = tile + pl.tile_bytes;
-    const Prob P = make_prob(a, pl, zero, tile, rest);
+    Prob P = make_prob(a, pl, zero, tile, rest);
+    P.sample_idx = sample_idx;
     Prob* d_prob = reinterpret_cast<Prob*>(ws);
 
     cudaStream_t st = stream;
@@ -337,15 +351,33 @@ static int encode_impl(int mode, const float* update, float* residual, int64_t n
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, 1u, grid);
-    launch_encode(d_prob, 1u, grid, nullptr, mode, st, marks);
+    launch_encode(d_prob, 1u, grid, nullptr, mode, pl.sampled != 0, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
 int sbc_encode_ex(const float* update, float* residual, int64_t numel, double p, void* out_stream,
                   size_t out_capacity, float* out_mu, void* workspace, size_t workspace_bytes,
                   sbc_cuda_stream_t stream, const sbc_cuda_event_t* marks) {
-    return encode_impl(kModeBinary, update, residual, numel, p, out_stream, out_capacity, out_mu, workspace,
+    return encode_impl(kModeBinary, nullptr, 0, update, residual, numel, p, out_stream, out_capacity, out_mu, workspace,
                        workspace_bytes, stream, marks);
+}
+
+size_t sbc_stream_bytes_sampled(int64_t numel, double p) {
+    Plan pl;
+    return make_plan(numel, p, &pl, kModeBinary, 32) ? pl.stream_bytes : 0;  // the bound does not depend on m
+}
+
+size_t sbc_workspace_bytes_sampled(int64_t numel, double p, int64_t sample_count) {
+    Plan pl;
+    return (sample_count > 0 && make_plan(numel, p, &pl, kModeBinary, sample_count)) ? pl.total : 0;
+}
+
+int sbc_encode_sampled(const float* update, float* residual, int64_t numel, double p, const uint32_t* sample_idx,
+                       int64_t sample_count, void* out_stream, size_t out_capacity, float* out_mu, void* workspace,
+                       size_t workspace_bytes, sbc_cuda_stream_t stream) {
+    if (!sample_idx) return SBC_EINVAL;
+    return encode_impl(kModeBinary, sample_idx, sample_count, update, residual, numel, p, out_stream, out_capacity,
+                       out_mu, workspace, workspace_bytes, stream, nullptr);
 }
 
 size_t sbc_stream_bytes_values(int64_t numel, double p) {
@@ -355,7 +387,7 @@ size_t sbc_stream_bytes_values(int64_t numel, double p) {
 
 int sbc_encode_values(const float* update, float* residual, int64_t numel, double p, void* out_stream,
                       size_t out_capacity, void* workspace, size_t workspace_bytes, sbc_cuda_stream_t stream) {
-    return encode_impl(kModeValues, update, residual, numel, p, out_stream, out_capacity, nullptr, workspace,
+    return encode_impl(kModeValues, nullptr, 0, update, residual, numel, p, out_stream, out_capacity, nullptr, workspace,
                        workspace_bytes, stream, nullptr);
 }
 
@@ -452,7 +484,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
     k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors});
-    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, st, nullptr);
+    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, false, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

@@ -30,7 +30,7 @@ constexpr int kSumBins = 254;         // one exact integer bin per fp32 exponent
 
 // Stages that use the "last block to finish does the serial step" pattern.
 enum Stage : int {
-    ST_SAMPLE0 = 0, ST_SAMPLE1, ST_COLLECT, ST_XH0, ST_XH1, ST_XH2,
+    ST_SAMPLE0 = 0, ST_SAMPLE1, ST_SAMPLE2, ST_COLLECT, ST_XH0, ST_XH1, ST_XH2,
     ST_BH0_S0, ST_BH0_S1,
     ST_BF0_S0, ST_BF0_S1, ST_BF1_S0, ST_BF1_S1, ST_BF2_S0, ST_BF2_S1,
     ST_BF3_S0, ST_BF3_S1, ST_BF4_S0, ST_BF4_S1,
@@ -44,6 +44,9 @@ struct Ctl {
     uint32_t done[ST_COUNT];    // tickets for the last-block pattern
     // threshold bounds from the sample
     uint32_t s_bin0[2], s_rank[2];
+    uint32_t s_prefix22[2];     // sampled mode: 22-bit prefix of the sample's order statistic
+    uint32_t sampled_ok;        // sampled mode: the estimated thresholds were accepted
+    uint32_t k_final;           // positions actually sent (k, or the count the sampled thresholds gave)
     float lo_f, hi_f;           // candidates: !(a < lo_f) for side 0, !(a > hi_f) for side 1
     // candidate lists
     uint32_t cand_cnt[2];
@@ -69,6 +72,7 @@ struct Ctl {
 struct Hists {
     uint32_t s0[kHistBins];
     uint32_t s1[2][kHistBins];
+    uint32_t s2[2][1024];
     uint32_t x[3][2][kHistBins];
     uint32_t b[6][2][kHistBins];
 };
@@ -83,6 +87,8 @@ struct Prob {
     int b;
     int vec_ok;                 // 1: update and residual are 16-byte aligned
     int mode;                   // kModeBinary (SBC) or kModeValues (top-p by magnitude, values sent)
+    int sampled;                // 1: thresholds are the order statistics of a caller-given subsample
+    const uint32_t* sample_idx; // sampled mode: m positions (device)
     uint8_t* stream;            // container out
     unsigned long long stream_cap;
     unsigned long long stream_bytes;  // bytes sbc_stream_bytes(n, p) promises to stay within
@@ -114,6 +120,7 @@ struct Batch {
 };
 struct Slot {
     const Prob* P;
+    Prob* G;      // the descriptor in global memory (patched when the sent count is only known on the device)
     uint32_t bx;  // block index within the problem
     uint32_t nb;  // blocks working on the problem
 };
@@ -138,6 +145,7 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
         reinterpret_cast<unsigned long long*>(s_prob)[i] = reinterpret_cast<const unsigned long long*>(src)[i];
     __syncthreads();
     s.P = s_prob;
+    s.G = const_cast<Prob*>(src);
     return s;
 }
 

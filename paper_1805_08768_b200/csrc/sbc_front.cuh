@@ -41,7 +41,8 @@ __global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
         const bool valid = i < P.m;
         uint32_t key = 0u;
         if (valid) {
-            const long long e = sample_element(P, i);
+            long long e = P.sampled ? (long long)P.sample_idx[i] : sample_element(P, i);
+            if (e >= P.n) { e = P.n - 1; atomicOr(&ctl->status, SBC_STATUS_RANGE); }  // bad caller-given position
             const float a = __fadd_rn(P.residual[e], P.update[e]);
             key = select_key(P.mode, __float_as_uint(a));
             P.sample_keys[i] = key;
@@ -99,7 +100,10 @@ __global__ void __launch_bounds__(kBlock) k_sample1(const Batch B) {
             block_pick_desc(P.hists->s1[s], kHistBins, false, ctl->s_rank[s], s_scan, &s_pick);
             if (threadIdx.x == 0) {
                 const uint32_t lower = (bin0[s] << 21) | (s_pick.bin << 10);  // side key, low bits 0
-                if (P.mode == kModeValues) {  // the key is the magnitude's bit pattern; no second side
+                if (P.sampled) {  // one more level follows: the exact order statistic is wanted
+                    ctl->s_prefix22[s] = lower >> 10;
+                    ctl->s_rank[s] = s_pick.rank;
+                } else if (P.mode == kModeValues) {  // the key is the magnitude's bit pattern; no second side
                     if (s == 0) ctl->lo_f = __uint_as_float(lower);
                     else        ctl->hi_f = -INFINITY;
                 } else if (s == 0) {
@@ -107,6 +111,48 @@ __global__ void __launch_bounds__(kBlock) k_sample1(const Batch B) {
                 } else {
                     ctl->hi_f = __uint_as_float(bits_of_key(~lower));
                 }
+                if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            }
+            __syncthreads();
+        }
+    }
+}
+
+// Level 2 (sampled mode only): the last 10 key bits, which pins the sample's order statistic
+// exactly; the two thresholds are then that value itself.
+__global__ void __launch_bounds__(kBlock) k_sample2(const Batch B) {
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
+    Ctl* ctl = P.ctl;
+    __shared__ uint32_t s_hist[2][1024];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ Pick s_pick;
+    for (int i = threadIdx.x; i < 2 * 1024; i += kBlock) (&s_hist[0][0])[i] = 0u;
+    __syncthreads();
+    const uint32_t pre[2] = {ctl->s_prefix22[0], ctl->s_prefix22[1]};
+    for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
+        const uint32_t i = base + threadIdx.x;
+        const bool valid = i < P.m;
+        const uint32_t key = valid ? P.sample_keys[i] : 0u;
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            const uint32_t sk = side_key(s, key);
+            warp_hist_add(s_hist[s], sk & 1023u, valid && (sk >> 10) == pre[s]);
+        }
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 2 * 1024; i += kBlock) {
+        const uint32_t v = (&s_hist[0][0])[i];
+        if (v) atomicAdd(&P.hists->s2[0][0] + i, v);
+    }
+    if (last_block_ticket(&ctl->done[ST_SAMPLE2], S.nb)) {
+        for (int s = 0; s < 2; ++s) {
+            block_pick_desc(P.hists->s2[s], 1024, false, ctl->s_rank[s], s_scan, &s_pick);
+            if (threadIdx.x == 0) {
+                const uint32_t skey = (pre[s] << 10) | s_pick.bin;
+                if (s == 0) ctl->lo_f = __uint_as_float(bits_of_key(skey));
+                else        ctl->hi_f = __uint_as_float(bits_of_key(~skey));
                 if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
             }
             __syncthreads();
@@ -253,9 +299,13 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
     if (last_block_ticket(&ctl->done[ST_COLLECT], S.nb)) {
         if (threadIdx.x == 0) {
             const uint32_t c0 = __ldcg(&ctl->cand_cnt[0]), c1 = __ldcg(&ctl->cand_cnt[1]);
-            const bool ok = c0 >= (uint32_t)P.k && c0 <= P.cap &&
-                            (MODE == kModeValues || (c1 >= (uint32_t)P.k && c1 <= P.cap));
+            // exact modes: both lists must hold at least the k wanted entries; sampled mode: the
+            // lists ARE the kept sets and only have to be non-empty; either way they must fit
+            const uint32_t need = P.sampled ? 1u : (uint32_t)P.k;
+            const bool ok = c0 >= need && c0 <= P.cap &&
+                            (MODE == kModeValues || (c1 >= need && c1 <= P.cap));
             ctl->use_fallback = ok ? 0u : 1u;
+            ctl->sampled_ok = (ok && P.sampled) ? 1u : 0u;
         }
     }
 }

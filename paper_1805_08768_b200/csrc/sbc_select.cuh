@@ -22,7 +22,7 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
-    if (ctl->status) return;
+    if (ctl->status || ctl->sampled_ok) return;  // sampled thresholds: every candidate is kept (thr = 0)
     const int s = blockIdx.z;
     if (s == 1 && P.mode == kModeValues) return;  // magnitude selection has one side only
     __shared__ uint32_t s_hist[kHistBins];
@@ -61,7 +61,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
-    if (ctl->status) return;
+    if (ctl->status || ctl->sampled_ok) return;
     const int s = blockIdx.z;
     if (s == 1 && P.mode == kModeValues) return;
     constexpr int kItems = 4;
@@ -196,7 +196,8 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     // Almost every kept value shares the exponent of the threshold value or the
     // next one up: those two bins are summed in registers, the rest goes
     // straight to the shared bins.
-    const uint32_t thr_bits = values_mode ? (uint32_t)(thr >> 32) : bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
+    const uint32_t thr_bits = ctl->sampled_ok ? __float_as_uint(s ? ctl->hi_f : ctl->lo_f)
+                            : values_mode ? (uint32_t)(thr >> 32) : bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
     const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
     const int bin_b = bin_a + 1;
     long long acc_a = 0, acc_b = 0;
@@ -252,7 +253,9 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
         __syncthreads();
         if (threadIdx.x < 2) {  // one thread per side rounds its exact sum
             const double sum = bins_to_double(reinterpret_cast<const long long*>(s_bins[threadIdx.x]));
-            ctl->mu64[threadIdx.x] = threadIdx.x ? -sum / (double)P.k : sum / (double)P.k;
+            // mean over the k selected entries, or over however many the sampled threshold let through
+            const double count = ctl->sampled_ok ? (double)min(__ldcg(&ctl->cand_cnt[threadIdx.x]), P.cap) : (double)P.k;
+            ctl->mu64[threadIdx.x] = threadIdx.x ? -sum / count : sum / count;
         }
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -263,6 +266,14 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
             ctl->side = side;
             ctl->mu32 = mu;
             if (P.out_mu) *P.out_mu = mu;
+            const uint32_t k_final = ctl->sampled_ok ? min(__ldcg(&ctl->cand_cnt[side]), P.cap) : (uint32_t)P.k;
+            ctl->k_final = k_final;
+            if (P.sampled) {  // the kernels that follow size their work from the descriptor
+                S.G->k = k_final;
+                S.G->n_len_blocks = (k_final + kLenBlock - 1) / kLenBlock;
+                S.G->n_chunks = (k_final + kChunkCodewords - 1) / kChunkCodewords;
+                S.G->payload_offset = SBC_HEADER_BYTES + (unsigned long long)S.G->n_chunks * SBC_CHUNK_ENTRY_BYTES;
+            }
         }
     }
 }

@@ -360,3 +360,58 @@ def test_values_mode_three_rounds_with_carried_residual():
         info = sbc.sbc_stream_info_get(out)
         assert np.array_equal(out[: info.total_bytes].cpu().numpy(), want)
         assert np.array_equal(r.cpu().numpy().view(np.uint32), res_cpu.view(np.uint32))
+
+
+# ---------------------------------------------------------------- subsampled thresholds
+
+def check_sampled(upd, res, p, idx):
+    n = upd.size
+    want_res = res.copy()
+    want_stream, want_mu = oracle.encode_sampled(upd, want_res, p, idx)
+    u = torch.from_numpy(upd).to(DEV)
+    r = torch.from_numpy(res).to(DEV)
+    sidx = torch.from_numpy(idx.astype(np.int32)).to(DEV)
+    cap = sbc.sbc_stream_bytes_sampled(n, p)
+    out = torch.full((cap + 64,), 0xAB, dtype=torch.uint8, device=DEV)
+    ws_bytes = sbc.sbc_workspace_bytes_sampled(n, p, idx.size)
+    ws = torch.full((ws_bytes + 256,), 0xCD, dtype=torch.uint8, device=DEV)
+    mu = torch.zeros(1, dtype=torch.float32, device=DEV)
+    sbc.sbc_encode_sampled(u, r, p, sidx, out_stream=out[:cap], out_mu=mu, workspace=ws[:ws_bytes])
+    info = sbc.sbc_stream_info_get(out)
+    torch.cuda.synchronize()
+    assert bool((out[cap:] == 0xAB).all()) and bool((ws[ws_bytes:] == 0xCD).all())
+    got = out[: info.total_bytes].cpu().numpy()
+    assert info.k == oracle.parse_header(want_stream).k
+    assert got.size == want_stream.size and np.array_equal(got, want_stream)
+    assert np.float32(mu.item()).view(np.uint32) == want_mu.view(np.uint32)
+    assert np.array_equal(r.cpu().numpy().view(np.uint32), want_res.view(np.uint32))
+    return out, info
+
+
+@pytest.mark.parametrize("n,p,m", [(1 << 21, 0.01, 20000), (3_000_001, 0.001, 100000), (1 << 22, 1e-4, 1 << 20),
+                                   (70001, 0.05, 1000), (5000, 0.01, 64)])
+def test_sampled_thresholds(n, p, m):
+    rng = np.random.default_rng(n + m)
+    upd = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
+    res = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    idx = rng.integers(0, n, m).astype(np.uint32)
+    out, info = check_sampled(upd, res, p, idx)
+    k = oracle.kept_count(n, p)
+    assert info.k != k or m == n                       # the amount of sparsity is noisy, as the paper says
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sbc.sbc_decode_accumulate([out], dense, status=status)
+    torch.cuda.synchronize()
+    assert status.item() == 0 and int((dense != 0).sum().item()) == info.k
+
+
+def test_sampled_thresholds_rejected_estimate_gives_the_exact_result():
+    n, p = 300000, 0.01
+    rng = np.random.default_rng(8)
+    upd = np.zeros(n, dtype=np.float32)
+    upd[rng.choice(n, 2000, replace=False)] = rng.standard_normal(2000).astype(np.float32)
+    res = np.zeros(n, dtype=np.float32)
+    idx = np.arange(1000, 3000, dtype=np.uint32)        # sees (almost) only zeros: threshold 0 keeps everything
+    out, info = check_sampled(upd, res, p, idx)
+    want_exact, _ = oracle.encode(upd, np.zeros(n, dtype=np.float32), p)
+    assert np.array_equal(out[: info.total_bytes].cpu().numpy(), want_exact)

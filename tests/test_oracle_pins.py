@@ -475,3 +475,59 @@ def test_bit_accounting_of_binarisation_and_golomb_coding():
     assert 1.8 < sbc_naive_bits / sbc_bits < 2.1               # 16 -> ~8.1 position bits
     assert abs(hg.nbits / k - oracle.mean_position_bits(p, hg.b)) < 0.1
     assert golomb_gd_bits < naive_gd_bits
+
+
+# ---------------------------------------------------------------- subsampled thresholds
+
+def test_sampled_thresholds_with_the_whole_tensor_as_sample_equal_the_exact_method():
+    # sample = every position, distinct values: floor(p*n) = k and the j-th order statistics are the
+    # exact thresholds, so the result must be the exact method's
+    rng = np.random.default_rng(41)
+    n, p = 20000, 0.01
+    upd = rng.standard_normal(n).astype(np.float32)
+    res = (rng.standard_normal(n) * 0.1).astype(np.float32)
+    r1, r2 = res.copy(), res.copy()
+    s1, m1 = oracle.encode(upd, r1, p)
+    s2, m2 = oracle.encode_sampled(upd, r2, p, np.arange(n, dtype=np.uint32))
+    assert np.array_equal(s1, s2) and m1 == m2 and np.array_equal(r1, r2)
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_sampled_thresholds_against_a_numpy_restatement(seed):
+    rng = np.random.default_rng(seed)
+    n, p, m = 200000, 0.01, 5000
+    upd = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
+    res = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    A = (res + upd).astype(np.float32)
+    idx = rng.integers(0, n, m).astype(np.uint32)
+    r = res.copy()
+    stream, mu = oracle.encode_sampled(upd, r, p, idx)
+    h = oracle.parse_header(stream)
+    sv = np.sort(A[idx])[::-1]
+    j = max(1, int(np.floor(p * m)))
+    t_pos, t_neg = sv[j - 1], sv[m - j]
+    P, N = np.flatnonzero(A >= t_pos), np.flatnonzero(A <= t_neg)
+    mp = math.fsum(float(v) for v in A[P]) / P.size
+    mn = -math.fsum(float(v) for v in A[N]) / N.size
+    side = 0 if mp >= mn else 1
+    kept = N if side else P
+    assert (h.side, h.k) == (side, kept.size)
+    assert mu == np.float32(-mn if side else mp)
+    dense = np.zeros(n, dtype=np.float32)
+    oracle.decode_accumulate([stream], dense)
+    assert np.array_equal(np.flatnonzero(dense), kept)
+    want_r = A.copy()
+    want_r[kept] = (A[kept] - mu).astype(np.float32)
+    assert np.array_equal(r, want_r)
+    k = oracle.kept_count(n, p)
+    assert 0.5 * k < kept.size < 2 * k             # noise in the amount of sparsity, not in its scale
+
+
+def test_sampled_thresholds_fall_back_to_the_exact_method_when_the_estimate_is_useless():
+    n, p = 5000, 0.01
+    upd = np.zeros(n, dtype=np.float32)           # threshold 0: every entry would be kept
+    upd[:10] = 1.0
+    r1, r2 = np.zeros(n, dtype=np.float32), np.zeros(n, dtype=np.float32)
+    s1, m1 = oracle.encode(upd, r1, p)
+    s2, m2 = oracle.encode_sampled(upd, r2, p, np.arange(100, 200, dtype=np.uint32))
+    assert np.array_equal(s1, s2) and m1 == m2 and np.array_equal(r1, r2)

@@ -415,3 +415,22 @@ def test_sampled_thresholds_rejected_estimate_gives_the_exact_result():
     out, info = check_sampled(upd, res, p, idx)
     want_exact, _ = oracle.encode(upd, np.zeros(n, dtype=np.float32), p)
     assert np.array_equal(out[: info.total_bytes].cpu().numpy(), want_exact)
+
+
+def test_checkpoint_and_resume_reproduces_the_streams():
+    # the residual is the only state: six rounds straight == three rounds, save/restore, three more
+    n, p = 200000, 0.01
+    updates = [workloads.normal_flat(n, 1e-3, 300 + r) for r in range(6)]
+
+    def run(rounds, residual):
+        streams = []
+        for upd in rounds:
+            stream, mu, residual, _, _ = gpu_encode(upd, residual, p)
+            streams.append((stream, mu))
+        return streams, residual
+
+    straight, _ = run(updates, np.zeros(n, dtype=np.float32))
+    first, saved = run(updates[:3], np.zeros(n, dtype=np.float32))
+    second, _ = run(updates[3:], saved.copy())            # "restore" = hand the saved tensor back
+    for (s0, m0), (s1, m1) in zip(straight, first + second):
+        assert np.array_equal(s0, s1) and m0 == m1

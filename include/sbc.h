@@ -267,6 +267,8 @@ typedef struct sbc_encode_diag {
     uint32_t capacity;      /* capacity of each candidate list */
     float bound_lo, bound_hi; /* candidates were: value >= bound_lo, value <= bound_hi */
     double mu_pos, mu_neg;  /* the two means of Algorithm 2 */
+    uint32_t certain[2];    /* of the candidates, those at or above the sample's upper bound of the
+                               threshold (kept without being looked at by the exact selection) */
 } sbc_encode_diag;
 int sbc_encode_diag_get(const void *workspace, sbc_encode_diag *host_out, sbc_cuda_stream_t stream);
 

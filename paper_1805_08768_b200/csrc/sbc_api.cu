@@ -30,7 +30,7 @@ struct Plan {
     long long n, k;
     int b, mode, sampled;
     uint32_t cap, m, n_xtiles, n_tiles, n_len_blocks, n_chunks;
-    uint32_t s_target[2];
+    uint32_t s_target, s_up;
     unsigned long long payload_offset;
     size_t stream_bytes;
     size_t zero_bytes, off_ctl, off_hists;                 // offsets inside the zero part
@@ -66,21 +66,31 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
     // deviations of a binomial count (and a little), so that the bound falls
     // below the true k-th value except with negligible probability -- and if
     // it does not, the exact route takes over.
-    uint32_t target;
+    // The same sample bounds the threshold from above (four deviations below the expected rank):
+    // candidates at or above that bound are certainly kept, so the exact selection only has to
+    // look at the band between the two bounds.  A bound that turns out too low costs time, not
+    // correctness: the selection then runs over the certain part instead.
+    uint32_t target, up = 0;
     if ((long long)pl->m == n) {
         target = (uint32_t)k;
+        up = (uint32_t)k;
     } else {
         const double expect = (double)k * (double)pl->m / (double)n;
         const double t = std::ceil(expect + 6.0 * std::sqrt(expect) + 8.0);
         target = (uint32_t)std::min<double>(t, (double)pl->m);
+        const double u = std::floor(expect - 4.0 * std::sqrt(expect) - 4.0);
+        up = u >= 1.0 ? (uint32_t)u : 0u;
     }
     pl->sampled = sampled_m > 0;
     if (pl->sampled) {  // the caller's subsample; its floor(p*m)-th order statistics ARE the thresholds
         if (sampled_m > (long long)kSampleMax) return false;
         pl->m = (uint32_t)sampled_m;
         target = (uint32_t)std::max<long long>(1, (long long)std::floor(p * (double)sampled_m));
+        up = 0;  // every candidate is kept: nothing is selected afterwards
     }
-    pl->s_target[0] = pl->s_target[1] = target;
+    if (k < 32768) up = 0;  // short lists: selecting over all of them costs less than the second bound
+    pl->s_target = target;
+    pl->s_up = up;
     pl->n_xtiles = (uint32_t)((n + kXTile - 1) / kXTile);
     pl->n_tiles = (uint32_t)((n + (1ll << kTileShift) - 1) >> kTileShift);
     const long long k_max = pl->sampled ? (long long)pl->cap : k;  // most positions a stream can carry
@@ -161,10 +171,11 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile
         P.cand[s] = reinterpret_cast<unsigned long long*>(rest + pl.off_cand[s]);
         for (int j = 0; j < 2; ++j) P.buf[s][j] = reinterpret_cast<unsigned long long*>(rest + pl.off_buf[s][j]);
         P.x_tile_cnt[s] = reinterpret_cast<uint32_t*>(rest + pl.off_xtile[s]);
-        P.s_target[s] = pl.s_target[s];
     }
     P.idx = reinterpret_cast<uint32_t*>(rest + pl.off_idx);
     P.blk_len = reinterpret_cast<unsigned long long*>(rest + pl.off_blklen);
+    P.s_target = pl.s_target;
+    P.s_up = pl.s_up;
     P.cap = pl.cap;
     P.m = pl.m;
     P.n_xtiles = pl.n_xtiles;
@@ -555,6 +566,7 @@ int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cu
     host_out->bound_hi = c.hi_f;
     host_out->mu_pos = c.mu64[0];
     host_out->mu_neg = c.mu64[1];
+    for (int s = 0; s < 2; ++s) host_out->certain[s] = c.use_fallback ? 0u : c.sure_cnt[s];
     return SBC_OK;
 }
 

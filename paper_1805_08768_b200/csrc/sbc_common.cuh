@@ -48,8 +48,12 @@ struct Ctl {
     uint32_t sampled_ok;        // sampled mode: the estimated thresholds were accepted
     uint32_t k_final;           // positions actually sent (k, or the count the sampled thresholds gave)
     float lo_f, hi_f;           // candidates: !(a < lo_f) for side 0, !(a > hi_f) for side 1
-    // candidate lists
-    uint32_t cand_cnt[2];
+    uint32_t s_bin0_up[2], s_rank_up[2];  // the same search for the upper bound of the threshold
+    uint32_t up_key[2];         // side key at and above which a candidate is certainly kept ("sure")
+    // candidate lists: sure entries grow from the front of cand[s], the rest ("band") from its back
+    unsigned long long cand_cnt2[2];  // low word: sure entries, high word: band entries
+    uint32_t cand_cnt[2];       // both together (set when the candidate pass ends)
+    uint32_t sure_cnt[2];
     // exact select over A (fallback)
     uint32_t x_prefix[2], x_rank[2], x_thr[2], x_ties_take[2], x_ties_have[2];
     // select over the candidate lists
@@ -71,7 +75,7 @@ struct Ctl {
 // Zeroed scratch that sits right behind Ctl.
 struct Hists {
     uint32_t s0[kHistBins];
-    uint32_t s1[2][kHistBins];
+    uint32_t s1[2][2][kHistBins];  // [side][0: lower bound's bin, 1: upper bound's bin]
     uint32_t s2[2][1024];
     uint32_t x[3][2][kHistBins];
     uint32_t b[6][2][kHistBins];
@@ -105,7 +109,8 @@ struct Prob {
     unsigned long long* blk_len;
     uint32_t cap;               // capacity of each candidate list
     uint32_t m;                 // sample size
-    uint32_t s_target[2];       // rank looked up in the sample, per side
+    uint32_t s_target;          // rank looked up in the sample (the same for both sides)
+    uint32_t s_up;              // rank in the sample of the upper bound (0: no upper bound)
     uint32_t n_xtiles, n_tiles, n_len_blocks, n_chunks;
     unsigned long long payload_offset;
 };
@@ -177,6 +182,32 @@ __device__ __forceinline__ unsigned long long make_composite(uint32_t skey, uint
     return ((unsigned long long)skey << 32) | (unsigned long long)(~idx);
 }
 __device__ __forceinline__ uint32_t composite_index(unsigned long long c) { return ~(uint32_t)c; }
+
+// A candidate list as the kernels after the candidate pass see it: entries [0, sure) sit at the
+// front of the buffer, entries [sure, total) at its back in reverse.  Every sure entry is larger
+// than every band entry.  The exact route rebuilds the list front to back (sure == total).
+struct CandView {
+    const unsigned long long* src;
+    uint32_t sure, total, cap;
+    __device__ __forceinline__ unsigned long long at(uint32_t i) const {
+        return i < sure ? src[i] : src[cap - 1u - (i - sure)];
+    }
+};
+__device__ __forceinline__ CandView cand_view(const Prob& P, const Ctl* ctl, int s) {
+    CandView v;
+    v.src = P.cand[s];
+    v.cap = P.cap;
+    v.total = min(ctl->cand_cnt[s], P.cap);
+    v.sure = ctl->use_fallback ? v.total : min(ctl->sure_cnt[s], v.total);
+    return v;
+}
+// The part of the list that holds the k-th largest entry, and that entry's rank inside the part:
+// the band when fewer than k entries are sure (the usual case), else the sure part.
+__device__ __forceinline__ void select_range(const CandView& v, uint32_t k, uint32_t* begin, uint32_t* count,
+                                             uint32_t* rank) {
+    if (v.sure < k) { *begin = v.sure; *count = v.total - v.sure; *rank = k - v.sure; }
+    else            { *begin = 0u;     *count = v.sure;           *rank = k; }
+}
 
 // ---------------------------------------------------------------- scans
 
@@ -287,8 +318,10 @@ struct Pick {
 // falls.  `mirror` reads bin i of the view as hist[nbins-1-i] (the same counts
 // seen from the complemented key).  All kBlock threads call; result in *out
 // (shared) after the trailing barrier.
+// `out2` (may be null) receives the same for a second rank `rank2` from the same walk.
 __device__ __forceinline__ void block_pick_desc(const uint32_t* hist, int nbins, bool mirror,
-                                                uint32_t rank, uint32_t* s_scan, Pick* out) {
+                                                uint32_t rank, uint32_t* s_scan, Pick* out,
+                                                uint32_t rank2 = 0u, Pick* out2 = nullptr) {
     const int per = (nbins + kBlock - 1) / kBlock;  // bins per thread, walked top-down
     uint32_t h[kHistBins / kBlock];
     uint32_t sum = 0;
@@ -300,7 +333,10 @@ __device__ __forceinline__ void block_pick_desc(const uint32_t* hist, int nbins,
         h[j] = v;
         sum += v;
     }
-    if (threadIdx.x == 0) out->found = 0u;
+    if (threadIdx.x == 0) {
+        out->found = 0u;
+        if (out2) out2->found = 0u;
+    }
     uint32_t total;
     uint32_t cum = block_exclusive_scan<uint32_t>(sum, s_scan, &total);
 #pragma unroll
@@ -311,6 +347,12 @@ __device__ __forceinline__ void block_pick_desc(const uint32_t* hist, int nbins,
                 out->rank = rank - cum;
                 out->count = h[j];
                 out->found = 1u;
+            }
+            if (out2 && cum < rank2 && rank2 <= cum + h[j]) {
+                out2->bin = (uint32_t)(nbins - 1 - ((int)threadIdx.x * per + j));
+                out2->rank = rank2 - cum;
+                out2->count = h[j];
+                out2->found = 1u;
             }
             cum += h[j];
         }

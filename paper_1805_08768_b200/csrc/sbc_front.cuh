@@ -26,14 +26,14 @@ __device__ __forceinline__ long long sample_element(const Prob& P, uint32_t i) {
 
 // Level 0: keys of the sampled A values, histogram of their top 11 bits; the
 // last block locates the bin of the target rank for each side.
-__global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
+__global__ void __launch_bounds__(kBlock, 8) k_sample0(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     __shared__ uint32_t s_hist[kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    __shared__ Pick s_pick;
+    __shared__ Pick s_pick, s_pick_up;
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
     for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
@@ -56,11 +56,14 @@ __global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
     }
     if (last_block_ticket(&ctl->done[ST_SAMPLE0], S.nb)) {
         for (int s = 0; s < 2; ++s) {
-            block_pick_desc(P.hists->s0, kHistBins, s == 1, P.s_target[s], s_scan, &s_pick);
+            // one walk finds the bin of the lower bound's rank and of the upper bound's (if any)
+            block_pick_desc(P.hists->s0, kHistBins, s == 1, P.s_target, s_scan, &s_pick, P.s_up, &s_pick_up);
             if (threadIdx.x == 0) {
                 ctl->s_bin0[s] = s_pick.bin;
                 ctl->s_rank[s] = s_pick.rank;
                 if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+                ctl->s_bin0_up[s] = s_pick_up.bin;
+                ctl->s_rank_up[s] = s_pick_up.found ? s_pick_up.rank : 0u;  // 0: no upper bound
             }
             __syncthreads();
         }
@@ -69,36 +72,58 @@ __global__ void __launch_bounds__(kBlock) k_sample0(const Batch B) {
 
 // Level 1: next 11 bits inside the located bins; the last block turns the
 // 22-bit prefixes into the two float bounds used by the candidate pass.
-__global__ void __launch_bounds__(kBlock) k_sample1(const Batch B) {
+__global__ void __launch_bounds__(kBlock, 8) k_sample1(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     __shared__ uint32_t s_hist[2][kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    __shared__ Pick s_pick;
-    for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) (&s_hist[0][0])[i] = 0u;
-    __syncthreads();
+    __shared__ Pick s_pick, s_pick_up;
     const uint32_t bin0[2] = {ctl->s_bin0[0], ctl->s_bin0[1]};
-    for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
-        const uint32_t i = base + threadIdx.x;
-        const bool valid = i < P.m;
-        const uint32_t key = valid ? P.sample_keys[i] : 0u;
-#pragma unroll
-        for (int s = 0; s < 2; ++s) {
-            const uint32_t sk = side_key(s, key);
-            warp_hist_add(s_hist[s], (sk >> 10) & 2047u, valid && (sk >> 21) == bin0[s]);
+    // the upper bound's top-level bin gets a histogram of its own only where it differs from the
+    // lower bound's, in a second walk over the sample keys
+    const bool has_up[2] = {ctl->s_rank_up[0] != 0u, ctl->s_rank_up[1] != 0u};
+    const uint32_t bin0_up[2] = {ctl->s_bin0_up[0], ctl->s_bin0_up[1]};
+    const bool own_up[2] = {has_up[0] && bin0_up[0] != bin0[0], has_up[1] && bin0_up[1] != bin0[1]};
+    for (int u = 0; u < ((own_up[0] || own_up[1]) ? 2 : 1); ++u) {
+        const uint32_t want0 = u ? bin0_up[0] : bin0[0], want1 = u ? bin0_up[1] : bin0[1];
+        const bool on0 = u == 0 || own_up[0], on1 = u == 0 || own_up[1];
+        for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) (&s_hist[0][0])[i] = 0u;
+        __syncthreads();
+        for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
+            const uint32_t i = base + threadIdx.x;
+            const bool valid = i < P.m;
+            const uint32_t key = valid ? P.sample_keys[i] : 0u;
+            const uint32_t sk1 = ~key;
+            warp_hist_add(s_hist[0], (key >> 10) & 2047u, valid && on0 && (key >> 21) == want0);
+            warp_hist_add(s_hist[1], (sk1 >> 10) & 2047u, valid && on1 && (sk1 >> 21) == want1);
         }
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) {
-        const uint32_t v = (&s_hist[0][0])[i];
-        if (v) atomicAdd(&P.hists->s1[0][0] + i, v);
+        __syncthreads();
+        for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) {
+            const uint32_t v = (&s_hist[0][0])[i];
+            if (v) atomicAdd(&P.hists->s1[i / kHistBins][u][i % kHistBins], v);
+        }
+        __syncthreads();
     }
     if (last_block_ticket(&ctl->done[ST_SAMPLE1], S.nb)) {
         for (int s = 0; s < 2; ++s) {
-            block_pick_desc(P.hists->s1[s], kHistBins, false, ctl->s_rank[s], s_scan, &s_pick);
+            // "sure" = at or above the lower edge of the second-level bin just above the one that
+            // holds the upper bound's rank: fewer sample entries than that rank lie there
+            const bool want_up = has_up[s] && !P.sampled;
+            if (want_up && own_up[s])
+                block_pick_desc(P.hists->s1[s][1], kHistBins, false, ctl->s_rank_up[s], s_scan, &s_pick_up);
+            // same top-level bin: both ranks come out of one walk
+            block_pick_desc(P.hists->s1[s][0], kHistBins, false, ctl->s_rank[s], s_scan, &s_pick,
+                            (want_up && !own_up[s]) ? ctl->s_rank_up[s] : 0u, own_up[s] ? nullptr : &s_pick_up);
             if (threadIdx.x == 0) {
+                uint32_t up_key = 0xffffffffu;
+                if (want_up && s_pick_up.found) {
+                    const unsigned long long edge =
+                        ((((unsigned long long)bin0_up[s] << 11) | (unsigned long long)s_pick_up.bin) + 1ull) << 10;
+                    if (edge <= 0xffffffffull) up_key = (uint32_t)edge;
+                }
+                ctl->up_key[s] = up_key;
                 const uint32_t lower = (bin0[s] << 21) | (s_pick.bin << 10);  // side key, low bits 0
                 if (P.sampled) {  // one more level follows: the exact order statistic is wanted
                     ctl->s_prefix22[s] = lower >> 10;
@@ -174,7 +199,7 @@ constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 wa
 // one atomic per hundred or so candidates.  Each thread has eight 16-byte
 // loads in flight before it touches any of them.
 template <int MODE>
-__global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
+__global__ void __launch_bounds__(kBlock, 4) k_add_collect(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -192,14 +217,44 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
     unsigned long long* const cand1 = P.cand[1];
     const bool vec_ok = P.vec_ok != 0;
 
+    const uint32_t up_key0 = ctl->up_key[0], up_key1 = ctl->up_key[1];
+
+    // Staged candidates of one side go to the list: sure entries (key at or above the upper bound
+    // of the threshold) to its front, the others to its back, with ONE atomic for both ranges.
     auto flush = [&](int s) {
-        if (wcnt[s] == 0u) return;  // warp-uniform
+        const uint32_t cnt = wcnt[s];
+        if (cnt == 0u) return;  // warp-uniform
         __syncwarp();
-        uint32_t base = 0u;
-        if (lane == 0) base = atomicAdd(&ctl->cand_cnt[s], wcnt[s]);
-        base = __shfl_sync(0xffffffffu, base, 0);
-        for (uint32_t i = lane; i < wcnt[s]; i += 32)
-            if (base + i < cap) (s ? cand1 : cand0)[base + i] = s_stage[warp][s][i];
+        const uint32_t up_key = s ? up_key1 : up_key0;
+        unsigned long long* const dst = s ? cand1 : cand0;
+        uint32_t n_sure = 0u;
+        for (uint32_t i0 = 0u; i0 < cnt; i0 += 32u) {
+            const uint32_t i = i0 + lane;
+            const bool sure = i < cnt && (uint32_t)(s_stage[warp][s][i] >> 32) >= up_key;
+            n_sure += (uint32_t)__popc(__ballot_sync(0xffffffffu, sure));
+        }
+        const uint32_t n_band = cnt - n_sure;
+        unsigned long long old = 0ull;
+        if (lane == 0)
+            old = atomicAdd(&ctl->cand_cnt2[s], (unsigned long long)n_sure | ((unsigned long long)n_band << 32));
+        old = __shfl_sync(0xffffffffu, old, 0);
+        uint32_t front = (uint32_t)old, back = (uint32_t)(old >> 32);
+        // both ranges must stay clear of each other; a list that does not fit is rebuilt by the exact route
+        if ((unsigned long long)front + n_sure + (unsigned long long)back + n_band <= (unsigned long long)cap) {
+            const unsigned lt = (1u << lane) - 1u;
+            for (uint32_t i0 = 0u; i0 < cnt; i0 += 32u) {
+                const uint32_t i = i0 + lane;
+                const bool valid = i < cnt;
+                const unsigned long long c = valid ? s_stage[warp][s][i] : 0ull;
+                const bool sure = valid && (uint32_t)(c >> 32) >= up_key;
+                const unsigned ms = __ballot_sync(0xffffffffu, sure);
+                const unsigned mb = __ballot_sync(0xffffffffu, valid && !sure);
+                if (sure) dst[front + (uint32_t)__popc(ms & lt)] = c;
+                else if (valid) dst[cap - 1u - (back + (uint32_t)__popc(mb & lt))] = c;
+                front += (uint32_t)__popc(ms);
+                back += (uint32_t)__popc(mb);
+            }
+        }
         __syncwarp();
         wcnt[s] = 0u;
     };
@@ -263,18 +318,33 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
                 const uint32_t tot_s = s ? (tot >> 16) : (tot & 0xffffu);
                 if (tot_s == 0u) continue;
                 if (wcnt[s] + tot_s > (uint32_t)kStage) flush(s);
-                // more candidates in one step than the stage holds (dense ties): straight to the list
-                const bool direct = tot_s > (uint32_t)kStage;
-                uint32_t off = s ? (excl >> 16) : (excl & 0xffffu);
-                if (direct) {
-                    uint32_t gbase = 0u;
-                    if (lane == 0) gbase = atomicAdd(&ctl->cand_cnt[s], tot_s);
-                    off += __shfl_sync(0xffffffffu, gbase, 0);
-                } else {
-                    off += wcnt[s];
-                    wcnt[s] += tot_s;
-                }
                 const unsigned mask = s ? qm : pm;
+                if (tot_s > (uint32_t)kStage) {
+                    // more candidates in one step than the stage holds (dense ties): element slot by
+                    // element slot, at most 32 at a time, each round flushed at once
+#pragma unroll 1
+                    for (int j = 0; j < kPerThread; ++j) {
+                        const bool mine = (mask >> j) & 1u;
+                        const unsigned mm = __ballot_sync(0xffffffffu, mine);
+                        if (mm == 0u) continue;
+                        if (mine) {
+                            float aj = a[0];  // a[j] without indexing the register array dynamically
+#pragma unroll
+                            for (int jj = 1; jj < kPerThread; ++jj) aj = (jj == j) ? a[jj] : aj;
+                            const uint32_t bits = __float_as_uint(aj);
+                            if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;
+                            const long long e = vec_layout ? base + (long long)(((j >> 2) * 32 + lane) * 4 + (j & 3))
+                                                           : base + j * 32 + lane;
+                            s_stage[warp][s][__popc(mm & ((1u << lane) - 1u))] =
+                                make_composite(side_key(s, select_key(MODE, bits)), (uint32_t)e);
+                        }
+                        wcnt[s] = (uint32_t)__popc(mm);
+                        flush(s);
+                    }
+                    continue;
+                }
+                uint32_t off = (s ? (excl >> 16) : (excl & 0xffffu)) + wcnt[s];
+                wcnt[s] += tot_s;
 #pragma unroll
                 for (int j = 0; j < kPerThread; ++j) {
                     if ((mask >> j) & 1u) {
@@ -282,9 +352,7 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
                         if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;
                         const long long e = vec_layout ? base + (long long)(((j >> 2) * 32 + lane) * 4 + (j & 3))
                                                        : base + j * 32 + lane;
-                        const unsigned long long c = make_composite(side_key(s, select_key(MODE, bits)), (uint32_t)e);
-                        if (direct) { if (off < cap) (s ? cand1 : cand0)[off] = c; }
-                        else s_stage[warp][s][off] = c;
+                        s_stage[warp][s][off] = make_composite(side_key(s, select_key(MODE, bits)), (uint32_t)e);
                         ++off;
                     }
                 }
@@ -298,7 +366,13 @@ __global__ void __launch_bounds__(kBlock) k_add_collect(const Batch B) {
 
     if (last_block_ticket(&ctl->done[ST_COLLECT], S.nb)) {
         if (threadIdx.x == 0) {
-            const uint32_t c0 = __ldcg(&ctl->cand_cnt[0]), c1 = __ldcg(&ctl->cand_cnt[1]);
+            const unsigned long long t0 = __ldcg(&ctl->cand_cnt2[0]), t1 = __ldcg(&ctl->cand_cnt2[1]);
+            const unsigned long long sum0 = (t0 & 0xffffffffull) + (t0 >> 32), sum1 = (t1 & 0xffffffffull) + (t1 >> 32);
+            const uint32_t c0 = (uint32_t)min(sum0, 0xffffffffull), c1 = (uint32_t)min(sum1, 0xffffffffull);
+            ctl->cand_cnt[0] = c0;
+            ctl->cand_cnt[1] = c1;
+            ctl->sure_cnt[0] = (uint32_t)t0;
+            ctl->sure_cnt[1] = (uint32_t)t1;
             // exact modes: both lists must hold at least the k wanted entries; sampled mode: the
             // lists ARE the kept sets and only have to be non-empty; either way they must fit
             const uint32_t need = P.sampled ? 1u : (uint32_t)P.k;

@@ -30,12 +30,13 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     __shared__ Pick s_pick;
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
-    const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
-    const unsigned long long* __restrict__ src = P.cand[s];
+    const CandView view = cand_view(P, ctl, s);
+    uint32_t begin, cnt, rank;
+    select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
     for (uint32_t base = S.bx * kBlock; base < cnt; base += S.nb * kBlock) {
         const uint32_t i = base + threadIdx.x;
         const bool valid = i < cnt;
-        const unsigned long long c = valid ? src[i] : 0ull;
+        const unsigned long long c = valid ? view.at(begin + i) : 0ull;
         warp_hist_add(s_hist, digit_of(c, 0), valid);
     }
     __syncthreads();
@@ -44,7 +45,7 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
         if (v) atomicAdd(&P.hists->b[0][s][i], v);
     }
     if (last_block_ticket(&ctl->done[ST_BH0_S0 + s], S.nb)) {
-        block_pick_desc(P.hists->b[0][s], kHistBins, false, (uint32_t)P.k, s_scan, &s_pick);
+        block_pick_desc(P.hists->b[0][s], kHistBins, false, rank, s_scan, &s_pick);
         if (threadIdx.x == 0) {
             ctl->b_prefix[s] = s_pick.bin;
             ctl->b_rank[s] = s_pick.rank;
@@ -71,8 +72,10 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
     __shared__ Pick s_pick;
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
-    const uint32_t cnt = (LEVEL == 0) ? min(ctl->cand_cnt[s], P.cap) : ctl->list_cnt[s][LEVEL];
-    const unsigned long long* __restrict__ src = (LEVEL == 0) ? P.cand[s] : P.buf[s][(LEVEL - 1) & 1];
+    const CandView view = cand_view(P, ctl, s);
+    uint32_t begin = 0u, cnt = ctl->list_cnt[s][LEVEL], rank0;
+    if (LEVEL == 0) select_range(view, (uint32_t)P.k, &begin, &cnt, &rank0);  // the part of the list hist0 looked at
+    const unsigned long long* __restrict__ src = P.buf[s][(LEVEL + 1) & 1];  // the previous level's output
     unsigned long long* __restrict__ dst = P.buf[s][LEVEL & 1];
     const uint32_t sel = (uint32_t)ctl->b_prefix[s] & ((1u << digit_bits(LEVEL)) - 1u);
     for (uint32_t base = S.bx * (kBlock * kItems); base < cnt; base += S.nb * (kBlock * kItems)) {
@@ -81,7 +84,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
 #pragma unroll
         for (int j = 0; j < kItems; ++j) {
             const uint32_t i = base + j * kBlock + threadIdx.x;
-            c[j] = (i < cnt) ? src[i] : 0ull;
+            c[j] = (i < cnt) ? (LEVEL == 0 ? view.at(begin + i) : src[i]) : 0ull;
             const bool m = (i < cnt) && digit_of(c[j], LEVEL) == sel;
             match |= m ? (1u << j) : 0u;
             warp_hist_add(s_hist, digit_of(c[j], LEVEL + 1), m);
@@ -190,9 +193,9 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     __shared__ unsigned long long s_bins[2][256];
     s_bins[0][threadIdx.x] = 0ull;
     __syncthreads();
-    const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
+    const CandView view = cand_view(P, ctl, s);
+    const uint32_t cnt = view.total;
     const unsigned long long thr = ctl->thr[s];
-    const unsigned long long* __restrict__ src = P.cand[s];
     // Almost every kept value shares the exponent of the threshold value or the
     // next one up: those two bins are summed in registers, the rest goes
     // straight to the shared bins.
@@ -210,11 +213,11 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     if (threadIdx.x < kTileWindow) s_win[threadIdx.x] = 0u;
     const uint32_t span = ((cnt + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
     const uint32_t lo = min(cnt, S.bx * span), hi = min(cnt, lo + span);
-    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(src[lo]) >> kTileShift : 0u);
+    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(view.at(lo)) >> kTileShift : 0u);
     __syncthreads();
     for (uint32_t base = lo; base < hi; base += kBlock) {
         const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < hi) ? src[i] : 0ull;
+        const unsigned long long c = (i < hi) ? view.at(i) : 0ull;
         const bool kept = (i < hi) && c >= thr;
         if (kept && !values_mode) {  // the means exist only for the binarised form
             const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
@@ -288,9 +291,9 @@ __global__ void __launch_bounds__(kBlock) k_scatter(const Batch B) {
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     const int s = (int)ctl->side;
-    const uint32_t cnt = min(ctl->cand_cnt[s], P.cap);
+    const CandView view = cand_view(P, ctl, s);
+    const uint32_t cnt = view.total;
     const unsigned long long thr = ctl->thr[s];
-    const unsigned long long* __restrict__ src = P.cand[s];
     const uint32_t* __restrict__ tile_base = P.tile_cnt[s];
     uint32_t* __restrict__ tile_fill = P.tile_fill;
     uint32_t* __restrict__ out = P.idx;
@@ -303,11 +306,11 @@ __global__ void __launch_bounds__(kBlock) k_scatter(const Batch B) {
     if (threadIdx.x < kTileWindow) s_win[threadIdx.x] = 0u;
     const uint32_t span = ((cnt + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
     const uint32_t lo = min(cnt, S.bx * span), hi = min(cnt, lo + span);
-    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(src[lo]) >> kTileShift : 0u);
+    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(view.at(lo)) >> kTileShift : 0u);
     __syncthreads();
     for (uint32_t base = lo; base < hi; base += kBlock) {
         const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < hi) ? src[i] : 0ull;
+        const unsigned long long c = (i < hi) ? view.at(i) : 0ull;
         const uint32_t rel = (composite_index(c) >> kTileShift) - win0;
         warp_group_add<false>(s_win, rel, (i < hi) && c >= thr && rel < (uint32_t)kTileWindow, nullptr);
     }
@@ -320,7 +323,7 @@ __global__ void __launch_bounds__(kBlock) k_scatter(const Batch B) {
     __syncthreads();
     for (uint32_t base = lo; base < hi; base += kBlock) {
         const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < hi) ? src[i] : 0ull;
+        const unsigned long long c = (i < hi) ? view.at(i) : 0ull;
         const bool kept = (i < hi) && c >= thr;
         const uint32_t idx = composite_index(c);
         const uint32_t tile = idx >> kTileShift;

@@ -133,6 +133,53 @@ def test_unrepresentative_sample_takes_the_exact_route():
     check_against_oracle(sparse, np.zeros(n, dtype=np.float32), 0.01)
 
 
+def encode_with_diag(upd, p):
+    n = upd.size
+    u = torch.from_numpy(upd).to(DEV)
+    r = torch.zeros(n, dtype=torch.float32, device=DEV)
+    ws = torch.empty(sbc.sbc_workspace_bytes(n, p), dtype=torch.uint8, device=DEV)
+    out, mu = sbc.sbc_encode(u, r, p, workspace=ws)
+    diag = sbc.sbc_encode_diag_get(ws)
+    info = sbc.sbc_stream_info_get(out)
+    return out[: info.total_bytes].cpu().numpy(), np.float32(mu.item()), r.cpu().numpy(), diag
+
+
+def test_selection_looks_only_at_the_band_between_the_two_bounds():
+    # long lists: candidates at or above the sample's upper bound are kept unseen by the
+    # selection, which then ranks the rest; the result is the oracle's all the same
+    n, p = 1 << 23, 0.01
+    k = oracle.kept_count(n, p)
+    for upd in (workloads.student_t_flat(n, 31), workloads.normal_flat(n, 1e-3, 32)):
+        want_res = np.zeros(n, dtype=np.float32)
+        want_stream, want_mu = oracle.encode(upd, want_res, p)
+        stream, mu, res, diag = encode_with_diag(upd, p)
+        assert diag.exact_route == 0
+        for s in range(2):
+            assert 0.5 * k < diag.certain[s] < k <= diag.candidates[s] <= diag.capacity
+        assert np.array_equal(stream, want_stream) and mu.view(np.uint32) == want_mu.view(np.uint32)
+        assert np.array_equal(res.view(np.uint32), want_res.view(np.uint32))
+
+
+def test_upper_bound_below_the_threshold_selects_among_the_certain_entries():
+    # large entries only where the strided sample does not look: both bounds come out too low,
+    # more than k candidates pass the upper one, and the k-th largest is found among those
+    n, p = 1 << 23, 0.01
+    k = oracle.kept_count(n, p)
+    rng = np.random.default_rng(7)
+    upd = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    hidden = np.flatnonzero((np.arange(n) // 32) % 16 != 0)        # the sample reads one 32-element line in 16
+    extra = rng.choice(hidden, k, replace=False)
+    upd[extra[: k // 2]] = (5e-3 + 1e-3 * rng.random(k // 2)).astype(np.float32)
+    upd[extra[k // 2:]] = (-5e-3 - 1e-3 * rng.random(k - k // 2)).astype(np.float32)
+    want_res = np.zeros(n, dtype=np.float32)
+    want_stream, want_mu = oracle.encode(upd, want_res, p)
+    stream, mu, res, diag = encode_with_diag(upd, p)
+    assert diag.exact_route == 0
+    assert diag.certain[0] >= k and diag.certain[1] >= k
+    assert np.array_equal(stream, want_stream) and mu.view(np.uint32) == want_mu.view(np.uint32)
+    assert np.array_equal(res.view(np.uint32), want_res.view(np.uint32))
+
+
 def test_multi_round_residual_carry():
     n, p = 250000, 0.001
     res_gpu = np.zeros(n, dtype=np.float32)

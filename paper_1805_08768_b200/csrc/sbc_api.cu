@@ -18,7 +18,7 @@ namespace {
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-constexpr size_t kProbSlotBytes = 256;  // one problem descriptor, padded
+constexpr size_t kProbSlotBytes = 512;  // one problem descriptor, padded
 static_assert(sizeof(Prob) <= kProbSlotBytes, "descriptor must fit its slot");
 
 // Host-side plan of one encode problem: scalar parameters and the layout of its scratch, which
@@ -34,13 +34,21 @@ struct Plan {
     unsigned long long payload_offset;
     size_t stream_bytes;
     size_t zero_bytes, off_ctl, off_hists;                 // offsets inside the zero part
-    size_t tile_bytes, off_tile_cnt[2], off_tile_fill;     // inside the tile part
+    size_t tile_bytes, off_tile_in, off_tile_base, off_tile_fill;  // inside the tile part
     size_t rest_bytes, off_mu, off_sample, off_cand[2], off_buf[2][2], off_xtile[2], off_idx,
-        off_blklen;                                        // inside the rest
+        off_blklen, off_blk_first;                                        // inside the rest
     size_t total;                                          // single problem: slot + zero + tile + rest
 };
 
 bool valid_p(double p) { return p > 0.0 && p < 1.0; }
+
+// Blocks that walk a candidate list to bucket its kept entries by tile: one per 1024 list slots,
+// at most kMaxScatterBlocks (the scratch that carries their slot reservations from the counting
+// kernel to the placing kernel is sized from this bound, without asking the device).
+constexpr unsigned kMaxScatterBlocks = 2048;
+unsigned scatter_blocks_bound(uint32_t cap) {
+    return (unsigned)std::min<unsigned long long>(((unsigned long long)cap + kBlock * 4 - 1) / (kBlock * 4), kMaxScatterBlocks) + 1u;
+}
 
 bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long long sampled_m = 0) {
     if (n <= 0 || n >= (1ll << 31) || !valid_p(p)) return false;
@@ -110,7 +118,8 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
     pl->off_hists = take(sizeof(Hists));
     pl->zero_bytes = off;
     off = 0;
-    for (int s = 0; s < 2; ++s) pl->off_tile_cnt[s] = take((size_t)(pl->n_tiles + 1) * 4);
+    pl->off_tile_in = take((size_t)pl->n_tiles * 4);
+    pl->off_tile_base = take((size_t)(pl->n_tiles + 1) * 4);
     pl->off_tile_fill = take((size_t)pl->n_tiles * 4);
     pl->tile_bytes = off;
     off = 0;
@@ -122,6 +131,7 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
     for (int s = 0; s < 2; ++s) pl->off_xtile[s] = take((size_t)pl->n_xtiles * 4);
     pl->off_idx = take((size_t)k_max * 4);
     pl->off_blklen = take((size_t)pl->n_len_blocks * 8);
+    pl->off_blk_first = take((size_t)scatter_blocks_bound(pl->cap) * kTileWindow * 4);
     pl->rest_bytes = off;
     pl->total = kProbSlotBytes + pl->zero_bytes + pl->tile_bytes + pl->rest_bytes;
     return true;
@@ -164,8 +174,10 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile
     P.out_mu = a.out_mu;
     P.ctl = reinterpret_cast<Ctl*>(zero + pl.off_ctl);
     P.hists = reinterpret_cast<Hists*>(zero + pl.off_hists);
-    for (int s = 0; s < 2; ++s) P.tile_cnt[s] = reinterpret_cast<uint32_t*>(tile + pl.off_tile_cnt[s]);
+    P.tile_in = reinterpret_cast<uint32_t*>(tile + pl.off_tile_in);
+    P.tile_base = reinterpret_cast<uint32_t*>(tile + pl.off_tile_base);
     P.tile_fill = reinterpret_cast<uint32_t*>(tile + pl.off_tile_fill);
+    P.blk_first = reinterpret_cast<uint32_t*>(rest + pl.off_blk_first);
     P.sample_keys = reinterpret_cast<uint32_t*>(rest + pl.off_sample);
     for (int s = 0; s < 2; ++s) {
         P.cand[s] = reinterpret_cast<unsigned long long*>(rest + pl.off_cand[s]);
@@ -213,8 +225,8 @@ void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned
     nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 8);
     nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 8);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
-    nb[WK_SCATTER] = grid_for(pl.cap, kBlock * 4, sms * 8);
-    nb[WK_MASK] = grid_for(pl.n_tiles, 1, sms * 8);
+    nb[WK_SCATTER] = grid_for(pl.cap, kBlock * 4, std::min(sms * 8, kMaxScatterBlocks));
+    nb[WK_MASK] = grid_for(pl.n_tiles, 1, sms * 6);  // one resident wave: the tile bitmask allows six blocks per SM
     nb[WK_LEN] = grid_for(pl.n_len_blocks, 1, sms * 8);
     nb[WK_ONE] = 1;
     nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
@@ -276,6 +288,7 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     mark(SBC_MARK_SELECT);
 
     // 4. ordered positions, residual write-back, Golomb payload, chunk table, header
+    k_tile_count<<<g1(WK_SCATTER), blk, 0, st>>>(B(WK_SCATTER));
     k_tile_scan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
     k_scatter<<<g1(WK_SCATTER), blk, 0, st>>>(B(WK_SCATTER));
     k_tile_sort<<<g1(WK_MASK), blk, 0, st>>>(B(WK_MASK));
@@ -540,7 +553,7 @@ int sbc_encode_static(const float* update, float* residual, int64_t numel, doubl
                       (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
 }
 
-int sbc_encode_launches(void) { return 23; }  // put_prob, 2 sample, 1 collect, 6 exact, 8 select, 5 Golomb
+int sbc_encode_launches(void) { return 24; }  // put_prob, 2 sample, 1 collect, 6 exact, 7 select, 7 ordering + Golomb
 
 int sbc_decode_launches(int n_clients) {
     return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;

@@ -102,8 +102,11 @@ struct Prob {
     uint32_t* sample_keys;
     unsigned long long* cand[2];
     unsigned long long* buf[2][2];   // ping-pong lists of the candidate select
-    uint32_t* tile_cnt[2];      // kept positions per tile and side (n_tiles + 1 entries; scanned in place)
-    uint32_t* tile_fill;        // entries already placed in each tile's bucket
+    // ordering of the kept positions of the chosen side by tile (tile = 2^kTileShift positions)
+    uint32_t* tile_in;          // per tile: entries whose bucket slots the counting blocks reserved
+    uint32_t* tile_base;        // per tile: the other entries; then scanned in place to bucket starts (n_tiles + 1)
+    uint32_t* tile_fill;        // per tile: of those other entries, how many are already placed
+    uint32_t* blk_first;        // per counting block and window tile: first reserved slot in the bucket
     uint32_t* x_tile_cnt[2];
     uint32_t* idx;              // sorted kept positions
     unsigned long long* blk_len;
@@ -264,9 +267,9 @@ __device__ __forceinline__ bool last_block_ticket(uint32_t* counter, uint32_t n_
 // Shared-memory window of per-tile counters used by blocks that walk a contiguous span of a
 // nearly position-ordered list: tiles [base, base + kTileWindow), base a little before the tile
 // of the span's first entry.
-constexpr int kTileWindow = 128;
+constexpr int kTileWindow = 1024;
 __device__ __forceinline__ uint32_t tile_window_base(uint32_t first_tile) {
-    return first_tile > 16u ? first_tile - 16u : 0u;
+    return first_tile > 256u ? first_tile - 256u : 0u;
 }
 
 // One counter update per distinct `key` among the warp's `valid` lanes; returns each valid lane's

@@ -13,8 +13,8 @@ namespace sbc {
 
 // ---------------------------------------------------------------- mask -> sorted positions
 
-// In-place exclusive scan of the chosen side's kept-position counts per tile (one block); entry
-// n_tiles receives the total.
+// Exclusive scan of the kept positions per tile (both counters of k_tile_count together) into
+// the bucket starts, in place over the second counter (one block); entry n_tiles receives the total.
 __global__ void __launch_bounds__(kBlock) k_tile_scan(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
@@ -22,7 +22,8 @@ __global__ void __launch_bounds__(kBlock) k_tile_scan(const Batch B) {
     Ctl* ctl = P.ctl;
     if (ctl->status) return;
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    uint32_t* __restrict__ cnt = P.tile_cnt[ctl->side];
+    uint32_t* __restrict__ cnt = P.tile_base;
+    const uint32_t* __restrict__ cnt_in = P.tile_in;
     const uint32_t n_tiles = P.n_tiles;
     constexpr int kPer = 8;
     uint32_t carry = 0u;
@@ -32,7 +33,7 @@ __global__ void __launch_bounds__(kBlock) k_tile_scan(const Batch B) {
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             const uint32_t t = base + threadIdx.x * kPer + j;
-            v[j] = (t < n_tiles) ? cnt[t] : 0u;
+            v[j] = (t < n_tiles) ? cnt[t] + cnt_in[t] : 0u;
             sum += v[j];
         }
         uint32_t total;
@@ -60,9 +61,13 @@ __global__ void __launch_bounds__(kBlock) k_tile_sort(const Batch B) {
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     if (P.ctl->status) return;
-    __shared__ uint32_t s_mask[kTileWords];
+    // the bitmask is stored with one pad word per 32 so that thread t's 32 consecutive words
+    // (t*32 .. t*32+31 -> slots t*33 .. t*33+31) fall into 32 different banks for every t
+    __shared__ uint32_t s_mask[kTileWords + kTileWords / 32];
     __shared__ uint32_t s_small[kBlock];
-    const uint32_t* __restrict__ tile_base = P.tile_cnt[P.ctl->side];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    static_assert(kTileWords == 32 * kBlock, "one thread reads out 32 words of the tile's bitmask");
+    const uint32_t* __restrict__ tile_base = P.tile_base;
     uint32_t* __restrict__ list = P.idx;
     const uint32_t n_tiles = P.n_tiles;
     for (uint32_t tile = S.bx; tile < n_tiles; tile += S.nb) {
@@ -79,7 +84,7 @@ __global__ void __launch_bounds__(kBlock) k_tile_sort(const Batch B) {
             __syncthreads();
             continue;
         }
-        for (int w = threadIdx.x; w < kTileWords; w += kBlock) s_mask[w] = 0u;
+        for (int w = threadIdx.x; w < kTileWords + kTileWords / 32; w += kBlock) s_mask[w] = 0u;
         __syncthreads();
         for (uint32_t base = beg; base < end; base += 4 * kBlock) {  // four loads in flight per thread
             uint32_t v[4];
@@ -92,37 +97,30 @@ __global__ void __launch_bounds__(kBlock) k_tile_sort(const Batch B) {
             for (int j = 0; j < 4; ++j) {
                 if (v[j] != 0xffffffffu) {
                     const uint32_t r = v[j] & ((1u << kTileShift) - 1u);
-                    atomicOr(&s_mask[r >> 5], 1u << (r & 31u));
+                    const uint32_t word = r >> 5;
+                    atomicOr(&s_mask[word + (word >> 5)], 1u << (r & 31u));
                 }
             }
         }
         __syncthreads();
-        // read-out: warp w owns words [w*kPerWarp, (w+1)*kPerWarp), lane l takes word it*32 + l of
-        // them in step `it` (conflict-free); order of the output = (warp, step, lane, bit)
-        constexpr int kPerWarp = kTileWords / (kBlock / 32);
-        const int warp = threadIdx.x >> 5, lane = lane_id();
+        // read-out in position order: thread t owns words t*32 .. t*32+31
+        const uint32_t* mine_words = s_mask + threadIdx.x * 33;
         uint32_t mine = 0u;
-        for (int it = 0; it < kPerWarp / 32; ++it) mine += __popc(s_mask[warp * kPerWarp + it * 32 + lane]);
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) mine += __shfl_xor_sync(0xffffffffu, mine, d);
-        if (lane == 0) s_small[warp] = mine;
-        __syncthreads();
-        uint32_t pos = beg;
-        for (int w = 0; w < warp; ++w) pos += s_small[w];
-        for (int it = 0; it < kPerWarp / 32; ++it) {
-            const int word = warp * kPerWarp + it * 32 + lane;
-            uint32_t w = s_mask[word];
-            const uint32_t c = (uint32_t)__popc(w);
-            const uint32_t incl = warp_inclusive_scan(c);
-            uint32_t at = pos + incl - c;
-            const uint32_t first = (tile << kTileShift) + ((uint32_t)word << 5);
-            while (w) {
-                const uint32_t idx = first + (__ffs(w) - 1);
-                w &= w - 1u;
-                if (at < end) list[at] = idx;
-                ++at;
+#pragma unroll 8
+        for (int j = 0; j < 32; ++j) mine += __popc(mine_words[j]);
+        uint32_t total;
+        uint32_t at = beg + block_exclusive_scan<uint32_t>(mine, s_scan, &total);
+        if (mine) {
+            const uint32_t first = (tile << kTileShift) + ((uint32_t)threadIdx.x << 10);
+            for (int j = 0; j < 32; ++j) {
+                uint32_t w = mine_words[j];
+                while (w) {
+                    const uint32_t idx = first + ((uint32_t)j << 5) + (__ffs(w) - 1);
+                    w &= w - 1u;
+                    if (at < end) list[at] = idx;
+                    ++at;
+                }
             }
-            pos += __shfl_sync(0xffffffffu, incl, 31);
         }
         __syncthreads();  // s_mask is cleared again for the next tile
     }

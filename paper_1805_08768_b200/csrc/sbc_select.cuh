@@ -194,57 +194,51 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     s_bins[0][threadIdx.x] = 0ull;
     __syncthreads();
     const CandView view = cand_view(P, ctl, s);
-    const uint32_t cnt = view.total;
     const unsigned long long thr = ctl->thr[s];
     // Almost every kept value shares the exponent of the threshold value or the
     // next one up: those two bins are summed in registers, the rest goes
     // straight to the shared bins.
     const uint32_t thr_bits = ctl->sampled_ok ? __float_as_uint(s ? ctl->hi_f : ctl->lo_f)
                             : values_mode ? (uint32_t)(thr >> 32) : bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
+    // Values within eight binades of the threshold's (nearly all of them) are summed in one
+    // register, in units of the lowest of those binades; the rest goes to the shared bins.
     const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
-    const int bin_b = bin_a + 1;
-    long long acc_a = 0, acc_b = 0;
-    // Each block walks one contiguous span of the list.  The list is nearly in position order, so
-    // a span touches few ordering tiles: their counts are kept in a shared-memory window and
-    // added to the global per-tile counts once per block (entries outside the window go straight
-    // to the global counters).
-    uint32_t* __restrict__ tile_cnt = P.tile_cnt[s];
-    __shared__ uint32_t s_win[kTileWindow];
-    if (threadIdx.x < kTileWindow) s_win[threadIdx.x] = 0u;
-    const uint32_t span = ((cnt + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
-    const uint32_t lo = min(cnt, S.bx * span), hi = min(cnt, lo + span);
-    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(view.at(lo)) >> kTileShift : 0u);
-    __syncthreads();
-    for (uint32_t base = lo; base < hi; base += kBlock) {
-        const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < hi) ? view.at(i) : 0ull;
-        const bool kept = (i < hi) && c >= thr;
-        if (kept && !values_mode) {  // the means exist only for the binarised form
-            const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
-            const uint32_t e = (bits >> 23) & 0xffu;
-            int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
-            if (bits >> 31) m = -m;
-            const int bin = e ? (int)e - 1 : 0;
-            if (bin == bin_a) acc_a += m;
-            else if (bin == bin_b) acc_b += m;
-            else atomicAdd(&s_bins[0][bin], (unsigned long long)(long long)m);
-        }
-        const uint32_t tile = composite_index(c) >> kTileShift;
-        const uint32_t rel = tile - win0;
-        warp_group_add<false>(s_win, rel, kept && rel < (uint32_t)kTileWindow, nullptr);
-        warp_group_add<false>(tile_cnt, tile, kept && rel >= (uint32_t)kTileWindow, nullptr);
-    }
-    __syncthreads();
-    if (threadIdx.x < kTileWindow && s_win[threadIdx.x]) atomicAdd(&tile_cnt[win0 + threadIdx.x], s_win[threadIdx.x]);
+    long long acc_a = 0;
+    auto add = [&](unsigned long long c) {
+        const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(c >> 32)));
+        const uint32_t e = (bits >> 23) & 0xffu;
+        int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
+        if (bits >> 31) m = -m;
+        const int bin = e ? (int)e - 1 : 0;
+        const uint32_t up = (uint32_t)(bin - bin_a);
+        if (up < 8u) acc_a += (long long)m << up;   // |m| < 2^24: at most 2^31 per entry, 2^62 over 2^31 entries
+        else atomicAdd(&s_bins[0][bin], (unsigned long long)(long long)m);
+    };
+    if (!values_mode) {  // the means exist only for the binarised form
+        constexpr int kItems = 4;  // loads in flight per thread
+        const uint32_t stride = S.nb * kBlock * kItems;
+        for (uint32_t base = S.bx * kBlock * kItems + threadIdx.x; base < view.sure; base += stride) {  // front of the list
+            unsigned long long c[kItems];
 #pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        acc_a += __shfl_down_sync(0xffffffffu, acc_a, d);
-        acc_b += __shfl_down_sync(0xffffffffu, acc_b, d);
+            for (int j = 0; j < kItems; ++j) c[j] = (base + j * kBlock < view.sure) ? view.src[base + j * kBlock] : 0ull;
+#pragma unroll
+            for (int j = 0; j < kItems; ++j)
+                if (base + j * kBlock < view.sure && c[j] >= thr) add(c[j]);
+        }
+        const unsigned long long* __restrict__ back = view.src + (view.cap - 1u);
+        const uint32_t n_back = view.total - view.sure;
+        for (uint32_t base = S.bx * kBlock * kItems + threadIdx.x; base < n_back; base += stride) {  // its back
+            unsigned long long c[kItems];
+#pragma unroll
+            for (int j = 0; j < kItems; ++j) c[j] = (base + j * kBlock < n_back) ? *(back - (base + j * kBlock)) : 0ull;
+#pragma unroll
+            for (int j = 0; j < kItems; ++j)
+                if (base + j * kBlock < n_back && c[j] >= thr) add(c[j]);
+        }
     }
-    if (lane_id() == 0) {
-        if (acc_a) atomicAdd(&s_bins[0][bin_a], (unsigned long long)acc_a);
-        if (acc_b && bin_b < kSumBins) atomicAdd(&s_bins[0][bin_b], (unsigned long long)acc_b);
-    }
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) acc_a += __shfl_down_sync(0xffffffffu, acc_a, d);
+    if (lane_id() == 0 && acc_a) atomicAdd(&s_bins[0][bin_a], (unsigned long long)acc_a);
     __syncthreads();
     {
         const unsigned long long v = s_bins[0][threadIdx.x];
@@ -281,9 +275,56 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     }
 }
 
-// Kept positions of the chosen side into per-tile buckets of the position list (tile = 65536
-// consecutive positions; bucket starts come from the scanned tile counts).  Inside a bucket the
-// order is whatever the atomics give; k_tile_sort puts each bucket in order afterwards.
+// Ordering of the kept positions, step 1: how many fall into each tile (2^kTileShift consecutive
+// positions).  Each block walks one contiguous span of the chosen side's list.  The list is nearly
+// in position order, so a span touches few tiles: their counts are kept in a shared-memory window
+// and each is added to the tile's global count with ONE atomic, whose return value is at the same
+// time the block's reserved range in the tile's bucket (kept for k_scatter).  Entries outside the
+// window are counted one warp group at a time in a second per-tile counter.
+__global__ void __launch_bounds__(kBlock) k_tile_count(const Batch B) {
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
+    Ctl* ctl = P.ctl;
+    if (ctl->status) return;
+    const int s = (int)ctl->side;
+    const CandView view = cand_view(P, ctl, s);
+    const unsigned long long thr = ctl->thr[s];
+    uint32_t* __restrict__ tile_out = P.tile_base;
+    __shared__ uint32_t s_win[kTileWindow];
+    for (int w = threadIdx.x; w < kTileWindow; w += kBlock) s_win[w] = 0u;
+    const uint32_t span = ((view.total + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
+    const uint32_t lo = min(view.total, S.bx * span), hi = min(view.total, lo + span);
+    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(view.at(lo)) >> kTileShift : 0u);
+    __syncthreads();
+    constexpr int kItems = 4;  // loads in flight per thread
+    for (uint32_t base = lo; base < hi; base += kBlock * kItems) {
+        unsigned long long cs[kItems];
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const uint32_t i = base + j * kBlock + threadIdx.x;
+            cs[j] = (i < hi) ? view.at(i) : 0ull;
+        }
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const bool kept = (base + j * kBlock + threadIdx.x < hi) && cs[j] >= thr;
+            const uint32_t tile = composite_index(cs[j]) >> kTileShift;
+            const uint32_t rel = tile - win0;
+            if (kept && rel < (uint32_t)kTileWindow) atomicAdd(&s_win[rel], 1u);
+            warp_group_add<false>(tile_out, tile, kept && rel >= (uint32_t)kTileWindow, nullptr);
+        }
+    }
+    __syncthreads();
+    for (int w = threadIdx.x; w < kTileWindow; w += kBlock) {
+        const uint32_t c = s_win[w];
+        P.blk_first[(size_t)S.bx * kTileWindow + w] = c ? atomicAdd(&P.tile_in[win0 + w], c) : 0u;
+    }
+}
+
+// Step 3 (after the scan of the tile counts): every kept position goes into its tile's bucket of
+// the position list.  A bucket holds first the ranges the counting blocks reserved, then the
+// entries that were outside their block's window.  Inside a bucket the order is arbitrary;
+// k_tile_sort puts each bucket in order afterwards.  Same spans and windows as k_tile_count.
 __global__ void __launch_bounds__(kBlock) k_scatter(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
@@ -292,49 +333,44 @@ __global__ void __launch_bounds__(kBlock) k_scatter(const Batch B) {
     if (ctl->status) return;
     const int s = (int)ctl->side;
     const CandView view = cand_view(P, ctl, s);
-    const uint32_t cnt = view.total;
     const unsigned long long thr = ctl->thr[s];
-    const uint32_t* __restrict__ tile_base = P.tile_cnt[s];
+    const uint32_t* __restrict__ tile_base = P.tile_base;
+    const uint32_t* __restrict__ tile_in = P.tile_in;
     uint32_t* __restrict__ tile_fill = P.tile_fill;
     uint32_t* __restrict__ out = P.idx;
     const uint32_t k = (uint32_t)P.k;
-    // Same span / window scheme as the counting in k_sums_decide: count the span's kept entries
-    // per tile in shared memory, reserve each tile's range of its bucket with ONE global atomic,
-    // then walk the span again and hand out slots from shared-memory counters.
     __shared__ uint32_t s_win[kTileWindow];
     __shared__ uint32_t s_first[kTileWindow];
-    if (threadIdx.x < kTileWindow) s_win[threadIdx.x] = 0u;
-    const uint32_t span = ((cnt + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
-    const uint32_t lo = min(cnt, S.bx * span), hi = min(cnt, lo + span);
+    for (int w = threadIdx.x; w < kTileWindow; w += kBlock) {
+        s_win[w] = 0u;
+        s_first[w] = P.blk_first[(size_t)S.bx * kTileWindow + w];
+    }
+    const uint32_t span = ((view.total + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
+    const uint32_t lo = min(view.total, S.bx * span), hi = min(view.total, lo + span);
     const uint32_t win0 = tile_window_base(lo < hi ? composite_index(view.at(lo)) >> kTileShift : 0u);
     __syncthreads();
-    for (uint32_t base = lo; base < hi; base += kBlock) {
-        const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < hi) ? view.at(i) : 0ull;
-        const uint32_t rel = (composite_index(c) >> kTileShift) - win0;
-        warp_group_add<false>(s_win, rel, (i < hi) && c >= thr && rel < (uint32_t)kTileWindow, nullptr);
-    }
-    __syncthreads();
-    if (threadIdx.x < kTileWindow) {
-        const uint32_t c = s_win[threadIdx.x];
-        s_first[threadIdx.x] = c ? atomicAdd(&tile_fill[win0 + threadIdx.x], c) : 0u;
-        s_win[threadIdx.x] = 0u;
-    }
-    __syncthreads();
-    for (uint32_t base = lo; base < hi; base += kBlock) {
-        const uint32_t i = base + threadIdx.x;
-        const unsigned long long c = (i < hi) ? view.at(i) : 0ull;
-        const bool kept = (i < hi) && c >= thr;
-        const uint32_t idx = composite_index(c);
-        const uint32_t tile = idx >> kTileShift;
-        const uint32_t rel = tile - win0;
-        const bool in_win = rel < (uint32_t)kTileWindow;
-        uint32_t first_w = 0u, first_g = 0u;
-        const uint32_t rank_w = warp_group_add<true>(s_win, rel, kept && in_win, &first_w);
-        const uint32_t rank_g = warp_group_add<true>(tile_fill, tile, kept && !in_win, &first_g);
-        if (kept) {
-            const uint32_t slot = tile_base[tile] + (in_win ? s_first[rel] + first_w + rank_w : first_g + rank_g);
-            if (slot < k) out[slot] = idx;
+    constexpr int kItems = 4;  // loads in flight per thread
+    for (uint32_t base = lo; base < hi; base += kBlock * kItems) {
+        unsigned long long cs[kItems];
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const uint32_t i = base + j * kBlock + threadIdx.x;
+            cs[j] = (i < hi) ? view.at(i) : 0ull;
+        }
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const bool kept = (base + j * kBlock + threadIdx.x < hi) && cs[j] >= thr;
+            const uint32_t idx = composite_index(cs[j]);
+            const uint32_t tile = idx >> kTileShift;
+            const uint32_t rel = tile - win0;
+            const bool in_win = rel < (uint32_t)kTileWindow;
+            uint32_t first_g = 0u;
+            const uint32_t rank_g = warp_group_add<true>(tile_fill, tile, kept && !in_win, &first_g);
+            if (kept) {
+                const uint32_t slot = tile_base[tile] + (in_win ? s_first[rel] + atomicAdd(&s_win[rel], 1u)
+                                                                : tile_in[tile] + first_g + rank_g);
+                if (slot < k) out[slot] = idx;
+            }
         }
     }
 }

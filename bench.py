@@ -151,11 +151,11 @@ def run_reference(args):
 # ------------------------------------------------------------------ our arm
 
 # DRAM traffic of one k_add_collect launch from an ncu capture at 2^26 elements (its summary
-# is kept with the other profile summaries): (536.91 + 225.70) MB at 2^26 elements, p = 1e-2.
+# is kept with the other profile summaries): (536.94 + 227.01) MB at 2^26 elements, p = 1e-2.
 # Traffic is proportional to the element count, so it is scaled by numel / 2^26.  Valid only for
 # the kernel source it was taken from: a different hash of the file reports null.
-NCU_TRAFFIC_BYTES_AT_2P26 = 762.61e6
-NCU_TRAFFIC_SOURCE_SHA256 = "c521829546d3db5d60a2f1cde45196742e35cc024f88ca7f7609b7745a94e4af"
+NCU_TRAFFIC_BYTES_AT_2P26 = 763.95e6
+NCU_TRAFFIC_SOURCE_SHA256 = "2babc2fdaf67fffb336aa23a1590d3317710a0d65960ac0f24d782486236eafe"
 
 
 def measured_traffic(numel: int):

@@ -226,7 +226,7 @@ void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned
     nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 8);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
     nb[WK_SCATTER] = grid_for(pl.cap, kBlock * 4, std::min(sms * 8, kMaxScatterBlocks));
-    nb[WK_MASK] = grid_for(pl.n_tiles, 1, sms * 6);  // one resident wave: the tile bitmask allows six blocks per SM
+    nb[WK_TILE] = grid_for(pl.n_tiles, 1, sms * 6);  // one resident wave: the tile bitmask allows six blocks per SM
     nb[WK_LEN] = grid_for(pl.n_len_blocks, 1, sms * 8);
     nb[WK_ONE] = 1;
     nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
@@ -291,7 +291,7 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     k_tile_count<<<g1(WK_SCATTER), blk, 0, st>>>(B(WK_SCATTER));
     k_tile_scan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
     k_scatter<<<g1(WK_SCATTER), blk, 0, st>>>(B(WK_SCATTER));
-    k_tile_sort<<<g1(WK_MASK), blk, 0, st>>>(B(WK_MASK));
+    k_tile_sort<<<g1(WK_TILE), blk, 0, st>>>(B(WK_TILE));
     k_len_sum_residual<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));
     k_len_scan_header<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
     k_pack<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));

@@ -159,7 +159,7 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
 
 // Kinds of work a kernel's grid is sized by (one prefix table per kind in a batch).
 enum WorkKind : int {
-    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_SCATTER, WK_MASK, WK_LEN, WK_ONE, WK_STREAM, WK_COUNT
+    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_SCATTER, WK_TILE, WK_LEN, WK_ONE, WK_STREAM, WK_COUNT
 };
 
 // ---------------------------------------------------------------- keys

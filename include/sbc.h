@@ -279,7 +279,14 @@ int sbc_encode_diag_get(const void *workspace, sbc_encode_diag *host_out, sbc_cu
  * `stream`.  The residual is the encoder's persistent state (Algorithm 1) and
  * stays on the device.  update_dev: device scratch of numel floats;
  * stream_dev: device scratch of out_capacity bytes.  Pinned host memory makes
- * the copies asynchronous up to the final synchronise.
+ * the copies asynchronous up to the final synchronise.  With page-locked
+ * out_stream_host the container is written to the host by a kernel instead of
+ * a copy engine (so that it does not queue behind another stream's large
+ * transfer in the same direction); sbc_decode_accumulate_host fetches
+ * page-locked containers the same way.  Two such calls on two streams, from
+ * two host threads, then use both directions of the link at once.  The first
+ * host-buffer call of a host thread page-locks a 256-byte landing pad for the
+ * header and status words it reads back (kept for the life of the thread).
  */
 int sbc_encode_host(const float *update_host, float *update_dev, float *residual_dev,
                     int64_t numel, double p, void *out_stream_host, void *stream_dev,

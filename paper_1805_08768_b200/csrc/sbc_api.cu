@@ -235,6 +235,20 @@ void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned
 // A single problem's descriptor reaches the device as a kernel argument.
 __global__ void k_put_prob(Prob* dst, const Prob src) { *dst = src; }
 
+// Plain byte copy (16 bytes per thread and step where both sides are 16-byte aligned).
+__global__ void __launch_bounds__(kBlock) k_copy_bytes(uint8_t* __restrict__ dst, const uint8_t* __restrict__ src,
+                                                       size_t bytes) {
+    const size_t tid = (size_t)blockIdx.x * kBlock + threadIdx.x, stride = (size_t)gridDim.x * kBlock;
+    if ((((uintptr_t)dst | (uintptr_t)src) & 15) == 0) {
+        const size_t vecs = bytes / 16;
+        for (size_t i = tid; i < vecs; i += stride)
+            reinterpret_cast<uint4*>(dst)[i] = reinterpret_cast<const uint4*>(src)[i];
+        for (size_t i = vecs * 16 + tid; i < bytes; i += stride) dst[i] = src[i];
+    } else {
+        for (size_t i = tid; i < bytes; i += stride) dst[i] = src[i];
+    }
+}
+
 // Zero the chunk table and payload area of every problem's output stream (batch form; a single
 // encode uses one memset instead).
 __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
@@ -583,6 +597,48 @@ int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cu
     return SBC_OK;
 }
 
+// Page-locked landing pad for the few bytes the host-buffer calls read back (a header, a status
+// word), one per host thread, allocated on the thread's first such call and kept.  A device-to-host
+// copy into ordinary (pageable) memory makes the driver wait for the stream inside the copy call,
+// which kept a second thread's transfers from being enqueued meanwhile; with the pad the calls only
+// ever wait in cudaStreamSynchronize.  Null if the allocation failed: the callers then fall back
+// to a buffer on their stack.
+static uint8_t* landing_pad() {
+    thread_local uint8_t* pad = nullptr;
+    thread_local bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* q = nullptr;
+        if (cudaHostAlloc(&q, 256, cudaHostAllocDefault) == cudaSuccess) pad = static_cast<uint8_t*>(q);
+        else (void)cudaGetLastError();
+    }
+    return pad;
+}
+
+// Small transfers between page-locked host memory and the device are done by a kernel, not by
+// the copy engines: a copy engine works through its queue in order, so a header or a container of
+// a few MB enqueued behind another stream's multi-GB transfer in the same direction would wait for
+// all of it, and two host-buffer calls running on two streams would take turns instead of using
+// both directions of the link at once.
+static bool kernel_visible(const void* p, void** dev_view) {
+    cudaPointerAttributes a;
+    if (cudaPointerGetAttributes(&a, p) != cudaSuccess) { (void)cudaGetLastError(); return false; }
+    if (a.type != cudaMemoryTypeHost && a.type != cudaMemoryTypeDevice && a.type != cudaMemoryTypeManaged) return false;
+    if (!a.devicePointer) return false;
+    *dev_view = a.devicePointer;
+    return true;
+}
+// dst <- src, `bytes` bytes, either side in device memory or page-locked host memory; falls back
+// to the copy engine when a side is ordinary host memory.
+static cudaError_t small_copy(void* dst, const void* src, size_t bytes, cudaMemcpyKind kind, cudaStream_t st) {
+    if (bytes == 0) return cudaSuccess;
+    void *d = nullptr, *s = nullptr;
+    if (!kernel_visible(dst, &d) || !kernel_visible(src, &s)) return cudaMemcpyAsync(dst, src, bytes, kind, st);
+    const unsigned blocks = (unsigned)std::min<size_t>((bytes + kBlock * 16 - 1) / (kBlock * 16), (size_t)sm_count() * 4);
+    k_copy_bytes<<<blocks, kBlock, 0, st>>>(static_cast<uint8_t*>(d), static_cast<const uint8_t*>(s), bytes);
+    return cudaGetLastError();
+}
+
 int sbc_encode_host(const float* update_host, float* update_dev, float* residual_dev, int64_t numel,
                     double p, void* out_stream_host, void* stream_dev, size_t out_capacity,
                     size_t* out_bytes_host, float* out_mu_host, void* workspace, size_t workspace_bytes,
@@ -604,20 +660,20 @@ int sbc_encode_host(const float* update_host, float* update_dev, float* residual
     const int irc = sbc_stream_info_get(stream_dev, &info, stream);  // synchronises
     if (irc != SBC_OK) return irc;
     if (info.total_bytes > out_capacity) return SBC_ECAPACITY;
-    float mu = 0.f;
-    if (cudaMemcpyAsync(out_stream_host, stream_dev, info.total_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-        cudaMemcpyAsync(&mu, mu_dev, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+    if (small_copy(out_stream_host, stream_dev, info.total_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return SBC_ECUDA;
     *out_bytes_host = info.total_bytes;
-    if (out_mu_host) *out_mu_host = mu;
+    if (out_mu_host) *out_mu_host = info.mu;  // the header carries the value out_mu received
     return SBC_OK;
 }
 
 int sbc_stream_info_get(const void* stream_dev, sbc_stream_info* host_out, sbc_cuda_stream_t stream) {
     if (!stream_dev || !host_out) return SBC_EINVAL;
-    uint8_t h[SBC_HEADER_BYTES];
-    if (cudaMemcpyAsync(h, stream_dev, SBC_HEADER_BYTES, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+    uint8_t on_stack[SBC_HEADER_BYTES];
+    uint8_t* pad = landing_pad();
+    uint8_t* h = pad ? pad : on_stack;
+    if (small_copy(h, stream_dev, SBC_HEADER_BYTES, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return SBC_ECUDA;
     sbc_stream_info& o = *host_out;
@@ -738,7 +794,7 @@ int sbc_decode_accumulate_host(const void* const* streams_host, const size_t* st
         return SBC_ECUDA;
     for (int c = 0; c < n_clients; ++c) {
         if (!streams_host[c] || stream_bytes[c] < SBC_HEADER_BYTES) return SBC_EINVAL;
-        if (cudaMemcpyAsync(base + off, streams_host[c], stream_bytes[c], cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        if (small_copy(base + off, streams_host[c], stream_bytes[c], cudaMemcpyHostToDevice, stream) != cudaSuccess)
             return SBC_ECUDA;
         dev_ptrs[c] = base + off;
         off += align_up(stream_bytes[c], 16);
@@ -746,11 +802,14 @@ int sbc_decode_accumulate_host(const void* const* streams_host, const size_t* st
     const int rc = sbc_decode_accumulate(dev_ptrs, n_clients, dense_dev, numel,
                                          reinterpret_cast<uint32_t*>(base), stream);
     if (rc != SBC_OK) return rc;
-    uint32_t status = 0;
+    uint32_t on_stack = 0;
+    uint8_t* pad = landing_pad();
+    uint32_t* landed = pad ? reinterpret_cast<uint32_t*>(pad + 128) : &on_stack;
     if (cudaMemcpyAsync(out_dense_host, dense_dev, (size_t)numel * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-        cudaMemcpyAsync(&status, base, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+        small_copy(landed, base, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
         cudaStreamSynchronize(stream) != cudaSuccess)
         return SBC_ECUDA;
+    const uint32_t status = *landed;
     if (status_host) *status_host = status;
     return status ? SBC_ECORRUPT : SBC_OK;
 }

@@ -63,6 +63,33 @@ def test_random_sizes_sparsities_and_distributions(case):
     assert_matches_oracle(upd, res, p, fetch(out, mu, r))
 
 
+@pytest.mark.parametrize("case", range(6))
+def test_long_lists_with_certain_and_band_parts(case):
+    # k >= 32768: the candidate lists are split at the sample's upper bound of the threshold
+    rng = np.random.default_rng(5000 + case)
+    n = int(rng.integers(1 << 21, 3_500_000))
+    p = float(10.0 ** rng.uniform(-1.7, -0.5))
+    if case == 0:
+        upd = rng.standard_normal(n)
+    elif case == 1:
+        upd = rng.standard_t(2, n)
+    elif case == 2:
+        upd = np.round(rng.standard_normal(n) * 8) / 8               # heavy ties around the threshold
+    elif case == 3:
+        upd = rng.standard_normal(n) * (rng.random(n) < 0.3)          # mostly zeros
+    elif case == 4:
+        upd = -np.abs(rng.standard_normal(n))                         # one-signed
+    else:
+        upd = rng.standard_normal(n)
+        upd[::7] = rng.choice([-3.0, 3.0, 2.5], size=upd[::7].size)   # blocks of equal large values
+    upd = (upd * 10.0 ** rng.integers(-5, 2)).astype(np.float32)
+    res = (rng.standard_normal(n) * float(np.abs(upd).mean())).astype(np.float32) if case % 2 else \
+        np.zeros(n, dtype=np.float32)
+    assert oracle.kept_count(n, p) >= 32768
+    _, r, out, mu = encode_on_gpu(upd, res, p)
+    assert_matches_oracle(upd, res, p, fetch(out, mu, r))
+
+
 @pytest.mark.parametrize("pattern", ["all_zero", "plus_minus_one", "two_values", "sparse_spikes"])
 def test_exact_route_at_scale(pattern):
     n, p = 1 << 22, 0.01

@@ -152,21 +152,38 @@ __global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
     float* values = (P.mode == kModeValues)
         ? reinterpret_cast<float*>(P.stream + SBC_HEADER_BYTES + (size_t)P.n_chunks * SBC_CHUNK_ENTRY_BYTES)
         : nullptr;
+    // R_j - mu as a fire-and-forget atomic add of -mu (no load round trip): the same single fp32
+    // rounding as the subtraction.  The hardware's atomic adder treats subnormal operands and
+    // results as zero, which cannot change the result while |mu| >= 2^-100: a subnormal R_j is less
+    // than a quarter ulp of mu, and a non-zero difference of two values that close is a multiple of
+    // 2^-124.  Smaller |mu| (zero included) takes the load / subtract / store path.
+    const bool by_atomic = values == nullptr && fabsf(mu) >= 7.888609052e-31f;  // 2^-100
     for (uint32_t blk = S.bx; blk < P.n_len_blocks; blk += S.nb) {
         const uint32_t i0 = blk * kLenBlock + threadIdx.x * kPer;
         uint32_t pos[kPer];
-        float r[kPer];
 #pragma unroll
         for (int j = 0; j < kPer; ++j) pos[j] = (i0 + j < k) ? P.idx[i0 + j] : 0u;
+        if (by_atomic) {
 #pragma unroll
-        for (int j = 0; j < kPer; ++j) r[j] = (i0 + j < k) ? P.residual[pos[j]] : 0.f;
+            for (int j = 0; j < kPer; ++j)
+                if (i0 + j < k) atomicAdd(P.residual + pos[j], -mu);
+        } else {
+            float r[kPer];
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) r[j] = (i0 + j < k) ? P.residual[pos[j]] : 0.f;
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                if (i0 + j < k) {
+                    if (values) values[i0 + j] = r[j];
+                    P.residual[pos[j]] = __fsub_rn(r[j], values ? r[j] : mu);
+                }
+            }
+        }
         long long prev = (i0 && i0 < k) ? (long long)P.idx[i0 - 1] : -1ll;
         unsigned long long sum = 0ull;
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             if (i0 + j < k) {
-                if (values) values[i0 + j] = r[j];
-                P.residual[pos[j]] = __fsub_rn(r[j], values ? r[j] : mu);
                 const uint32_t g = (uint32_t)((long long)pos[j] - prev - 1);
                 sum += (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
                 prev = pos[j];

@@ -290,6 +290,23 @@ def test_argument_errors_are_returned_at_once():
     assert e.value.code == sbc.SBC_EINVAL
 
 
+@pytest.mark.parametrize("exponent", [-90, -96, -98, -99, -100, -102, -120])
+def test_residual_write_back_around_the_atomic_adder_s_subnormal_limit(exponent):
+    # kept entries that are subnormal or zero next to a transmitted value near 2^-100: the
+    # hardware adder flushes subnormals, so the write-back switches to load/subtract/store below
+    # that magnitude; either way R_j = fl32(A_j - mu) exactly
+    n, p = 200000, 0.01
+    k = oracle.kept_count(n, p)
+    rng = np.random.default_rng(300 - exponent)
+    upd = (rng.integers(-(1 << 22), 1 << 22, n).astype(np.float64) * 2.0 ** -149).astype(np.float32)  # subnormals
+    upd[rng.random(n) < 0.2] = 0.0
+    big = rng.choice(n, k // 2, replace=False)                       # fewer than k large entries per side
+    upd[big[: k // 4]] = ((1.0 + rng.random(k // 4)) * 2.0 ** exponent).astype(np.float32)
+    upd[big[k // 4:]] = (-(1.0 + rng.random(k // 2 - k // 4)) * 2.0 ** exponent).astype(np.float32)
+    res = (rng.integers(-(1 << 20), 1 << 20, n).astype(np.float64) * 2.0 ** -149).astype(np.float32)
+    check_against_oracle(upd, res, p)
+
+
 def test_decode_of_a_subnormal_mu_is_exact():
     # the transmitted value itself is subnormal: the sum must not be flushed to zero
     n = 5000

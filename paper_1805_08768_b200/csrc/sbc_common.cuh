@@ -50,6 +50,7 @@ struct Ctl {
     float lo_f, hi_f;           // candidates: !(a < lo_f) for side 0, !(a > hi_f) for side 1
     uint32_t s_bin0_up[2], s_rank_up[2];  // the same search for the upper bound of the threshold
     uint32_t up_key[2];         // side key at and above which a candidate is certainly kept ("sure")
+    uint32_t lo_key[2];         // side key of the lower bound: every candidate's key is at least this
     // candidate lists: sure entries grow from the front of cand[s], the rest ("band") from its back
     unsigned long long cand_cnt2[2];  // low word: sure entries, high word: band entries
     uint32_t cand_cnt[2];       // both together (set when the candidate pass ends)

@@ -125,6 +125,7 @@ __global__ void __launch_bounds__(kBlock, 8) k_sample1(const Batch B) {
                 }
                 ctl->up_key[s] = up_key;
                 const uint32_t lower = (bin0[s] << 21) | (s_pick.bin << 10);  // side key, low bits 0
+                ctl->lo_key[s] = lower;
                 if (P.sampled) {  // one more level follows: the exact order statistic is wanted
                     ctl->s_prefix22[s] = lower >> 10;
                     ctl->s_rank[s] = s_pick.rank;

@@ -10,10 +10,28 @@
 
 namespace sbc {
 
-__device__ __forceinline__ int digit_shift(int level) { return level < 5 ? 53 - 11 * level : 0; }
-__device__ __forceinline__ int digit_bits(int level) { return level < 5 ? 11 : 9; }
-__device__ __forceinline__ uint32_t digit_of(unsigned long long c, int level) {
-    return (uint32_t)(c >> digit_shift(level)) & ((1u << digit_bits(level)) - 1u);
+// Digit schedule.  The entries being ranked agree in every composite bit above `top`, so the
+// digits run from bit `top` downwards, 11 bits each (the last one takes what is left).  For the
+// whole key range top = 63 (six levels); for the band between the two sample bounds the keys share
+// their leading bits and top is around 50 (five levels, and already the first digit tells the
+// entries apart).
+__device__ __forceinline__ int digit_bits(int level, int top) { return max(0, min(11, top + 1 - 11 * level)); }
+__device__ __forceinline__ int digit_shift(int level, int top) { return max(0, top + 1 - 11 * (level + 1)); }
+__device__ __forceinline__ int digit_levels(int top) { return (top + 1 + 10) / 11; }
+__device__ __forceinline__ uint32_t digit_of(unsigned long long c, int level, int top) {
+    return (uint32_t)(c >> digit_shift(level, top)) & ((1u << digit_bits(level, top)) - 1u);
+}
+// Highest composite bit in which the entries of the selected part of the list can differ, and
+// (through *base) the bits above it, which they all share.
+__device__ __forceinline__ int select_top(const Prob& P, const Ctl* ctl, int s, const CandView& v,
+                                          unsigned long long* base) {
+    *base = 0ull;
+    if (ctl->use_fallback || v.sure >= (uint32_t)P.k) return 63;  // exact route, or ranking the certain part
+    const uint32_t lo = ctl->lo_key[s], hi = ctl->up_key[s] - 1u;  // band keys lie in [lo, hi]
+    const uint32_t diff = lo ^ hi;
+    const int top = 32 + (diff ? 31 - __clz(diff) : -1);
+    *base = top == 63 ? 0ull : (((unsigned long long)lo << 32) & (~0ull << (top + 1)));
+    return top;
 }
 
 // Histogram of the top digit over a whole candidate list.  grid.z = side.
@@ -33,11 +51,16 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     const CandView view = cand_view(P, ctl, s);
     uint32_t begin, cnt, rank;
     select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
+    unsigned long long shared_bits;
+    const int top = select_top(P, ctl, s, view, &shared_bits);
     for (uint32_t base = S.bx * kBlock; base < cnt; base += S.nb * kBlock) {
         const uint32_t i = base + threadIdx.x;
         const bool valid = i < cnt;
         const unsigned long long c = valid ? view.at(begin + i) : 0ull;
-        warp_hist_add(s_hist, digit_of(c, 0), valid);
+        // whole key range: nearly all entries share the first digit, so one atomic per warp and
+        // bin; band: the first digit already spreads them, plain atomics collide rarely
+        if (top == 63) warp_hist_add(s_hist, digit_of(c, 0, top), valid);
+        else if (valid) atomicAdd(&s_hist[digit_of(c, 0, top)], 1u);
     }
     __syncthreads();
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) {
@@ -47,7 +70,8 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     if (last_block_ticket(&ctl->done[ST_BH0_S0 + s], S.nb)) {
         block_pick_desc(P.hists->b[0][s], kHistBins, false, rank, s_scan, &s_pick);
         if (threadIdx.x == 0) {
-            ctl->b_prefix[s] = s_pick.bin;
+            // the k-th largest composite, known down to the end of the first digit
+            ctl->b_prefix[s] = shared_bits | ((unsigned long long)s_pick.bin << digit_shift(0, top));
             ctl->b_rank[s] = s_pick.rank;
             if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
         }
@@ -73,11 +97,14 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
     const CandView view = cand_view(P, ctl, s);
+    unsigned long long shared_bits;
+    const int top = select_top(P, ctl, s, view, &shared_bits);
+    if (LEVEL + 1 >= digit_levels(top)) return;  // the previous level was the last one
     uint32_t begin = 0u, cnt = ctl->list_cnt[s][LEVEL], rank0;
     if (LEVEL == 0) select_range(view, (uint32_t)P.k, &begin, &cnt, &rank0);  // the part of the list hist0 looked at
     const unsigned long long* __restrict__ src = P.buf[s][(LEVEL + 1) & 1];  // the previous level's output
     unsigned long long* __restrict__ dst = P.buf[s][LEVEL & 1];
-    const uint32_t sel = (uint32_t)ctl->b_prefix[s] & ((1u << digit_bits(LEVEL)) - 1u);
+    const uint32_t sel = digit_of(ctl->b_prefix[s], LEVEL, top);
     for (uint32_t base = S.bx * (kBlock * kItems); base < cnt; base += S.nb * (kBlock * kItems)) {
         unsigned long long c[kItems];
         unsigned match = 0u;
@@ -85,9 +112,9 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
         for (int j = 0; j < kItems; ++j) {
             const uint32_t i = base + j * kBlock + threadIdx.x;
             c[j] = (i < cnt) ? (LEVEL == 0 ? view.at(begin + i) : src[i]) : 0ull;
-            const bool m = (i < cnt) && digit_of(c[j], LEVEL) == sel;
+            const bool m = (i < cnt) && digit_of(c[j], LEVEL, top) == sel;
             match |= m ? (1u << j) : 0u;
-            warp_hist_add(s_hist, digit_of(c[j], LEVEL + 1), m);
+            warp_hist_add(s_hist, digit_of(c[j], LEVEL + 1, top), m);
         }
         uint32_t total;
         const uint32_t excl = block_exclusive_scan<uint32_t>((uint32_t)__popc(match), s_scan, &total);
@@ -104,14 +131,14 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
         if (v) atomicAdd(&P.hists->b[LEVEL + 1][s][i], v);
     }
     if (last_block_ticket(&ctl->done[ST_BF0_S0 + 2 * LEVEL + s], S.nb)) {
-        block_pick_desc(P.hists->b[LEVEL + 1][s], 1 << digit_bits(LEVEL + 1), false,
+        block_pick_desc(P.hists->b[LEVEL + 1][s], 1 << digit_bits(LEVEL + 1, top), false,
                         ctl->b_rank[s], s_scan, &s_pick);
         if (threadIdx.x == 0) {
             const unsigned long long prefix =
-                (ctl->b_prefix[s] << digit_bits(LEVEL + 1)) | (unsigned long long)s_pick.bin;
+                ctl->b_prefix[s] | ((unsigned long long)s_pick.bin << digit_shift(LEVEL + 1, top));
             ctl->b_prefix[s] = prefix;
             ctl->b_rank[s] = s_pick.rank;
-            if (LEVEL + 1 == 5) ctl->thr[s] = prefix;  // the k-th largest composite itself
+            if (LEVEL + 2 == digit_levels(top)) ctl->thr[s] = prefix;  // last digit: the k-th largest composite itself
             if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
         }
     }

@@ -242,7 +242,7 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
         else atomicAdd(&s_bins[0][bin], (unsigned long long)(long long)m);
     };
     if (!values_mode) {  // the means exist only for the binarised form
-        constexpr int kItems = 4;  // loads in flight per thread
+        constexpr int kItems = 8;  // loads in flight per thread
         const uint32_t stride = S.nb * kBlock * kItems;
         for (uint32_t base = S.bx * kBlock * kItems + threadIdx.x; base < view.sure; base += stride) {  // front of the list
             unsigned long long c[kItems];

@@ -199,18 +199,51 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
             const bool tiny = fabsf(mu) < 7.888609052e-31f;  // 2^-100
             if (staged) {
                 // Fast path: bit positions relative to the stage fit 32 bits; every codeword
-                // is cut out of a 64-bit window rebuilt from three staged words.
+                // is cut out of a 64-bit window rebuilt from three staged words.  The common
+                // case (fewer than 32 ones, everything in range) is decided by ONE predicate per
+                // codeword and runs without any other branch; long unary runs and every kind of
+                // error take the general step below.
                 uint32_t rel = (uint32_t)(pos - (first_word << 5));
                 const uint32_t rel_end = (uint32_t)(gend - (first_word << 5));
+                const uint32_t n32 = (uint32_t)args.n;
+                const uint32_t q_max = n32 >> b;          // a larger quotient cannot stay inside the tensor
+                uint32_t nxt = (uint32_t)(prev + 1);      // first position the next codeword can name
+                float* __restrict__ out = args.out;
+                const bool plain = vals == nullptr && momentum == nullptr && !tiny;  // warp-uniform
                 for (uint32_t i = 0; i < count; ++i) {
-                    if (rel >= rel_end) { err = SBC_STATUS_CORRUPT; break; }
                     uint32_t w = rel >> 5;
-                    int sh = (int)(rel & 31u);
-                    uint32_t hi = __funnelshift_l(sw[w + 1], sw[w], sh);
-                    uint32_t lo = __funnelshift_l(sw[w + 2], sw[w + 1], sh);
+                    const int sh = (int)(rel & 31u);
+                    const uint32_t x0 = sw[w], x1 = sw[w + 1], x2 = sw[w + 2];
+                    uint32_t hi = __funnelshift_l(x1, x0, sh);
+                    uint32_t lo = __funnelshift_l(x2, x1, sh);
                     uint32_t ones = __clz(~hi);
+                    {
+                        const unsigned long long win = ((unsigned long long)hi << 32) | (unsigned long long)lo;
+                        const uint32_t r = (uint32_t)(((win << (ones & 31u) << 1) >> 1) >> (63u - b));  // b bits after the zero
+                        const uint32_t stp = (ones << b) + r;       // meaningful when ones <= q_max: no overflow then
+                        const bool ok = (rel < rel_end) & (ones < 32u) & (ones <= q_max) & (stp < n32 - nxt);
+                        if (ok) {
+                            const uint32_t at = nxt + stp;
+                            nxt = at + 1u;
+                            rel += ones + 1u + b;
+                            if (plain) {
+                                atomicAdd(out + at, mu);
+                            } else {
+                                if (vals) {
+                                    const float x = __fmul_rn(vals[i], args.scale);
+                                    err |= add_at(out + at, x, fabsf(x) < 7.888609052e-31f);
+                                } else {
+                                    err |= add_at(out + at, mu, tiny);
+                                }
+                                if (momentum) momentum[at] = 0.f;
+                            }
+                            continue;
+                        }
+                    }
+                    // general step: a run of 32 or more ones, or something is wrong
+                    if (rel >= rel_end) { err = SBC_STATUS_CORRUPT; break; }
                     unsigned long long q = ones;
-                    while (ones == 32u) {  // rare: a run of 32 or more ones
+                    while (ones == 32u) {
                         rel += 32u;
                         if (rel >= rel_end) break;
                         w = rel >> 5;
@@ -223,20 +256,22 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                     const unsigned long long win = ((unsigned long long)hi << 32) | (unsigned long long)lo;
                     const uint32_t r = b ? (uint32_t)((win << (ones + 1u)) >> (64u - b)) : 0u;
                     rel += ones + 1u + b;
-                    const unsigned long long step = (q << b) + r + 1ull;
-                    if (q > (unsigned long long)args.n || (unsigned long long)(args.n - 1 - prev) < step) {
+                    const unsigned long long step = (q << b) + r;
+                    if (q > (unsigned long long)args.n || (unsigned long long)(n32 - nxt) <= step) {
                         err = SBC_STATUS_RANGE;
                         break;
                     }
-                    prev += (long long)step;
+                    const uint32_t at = nxt + (uint32_t)step;
+                    nxt = at + 1u;
                     if (vals) {
                         const float x = __fmul_rn(vals[i], args.scale);
-                        err |= add_at(args.out + prev, x, fabsf(x) < 7.888609052e-31f);
+                        err |= add_at(out + at, x, fabsf(x) < 7.888609052e-31f);
                     } else {
-                        err |= add_at(args.out + prev, mu, tiny);
+                        err |= add_at(out + at, mu, tiny);
                     }
-                    if (momentum) momentum[prev] = 0.f;
+                    if (momentum) momentum[at] = 0.f;
                 }
+                prev = (long long)nxt - 1;
                 pos = (first_word << 5) + rel;
             } else {
                 // Long unary runs made the group larger than the stage: read global memory.

@@ -269,46 +269,62 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
                    const sbc_cuda_event_t* marks) {
     auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
     auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs}; };
-    const dim3 blk(kBlock);
     auto g1 = [&](int kind) { return dim3(grid[kind]); };
     auto g2 = [&](int kind) { return dim3(grid[kind], 1, 2); };  // z = side
+    // Every kernel is launched with programmatic stream serialisation: its blocks may be placed
+    // while the previous kernel drains; each kernel waits for its predecessor in resolve().
+    // The two long kernels (streaming pass, residual write-back) are launched the ordinary way:
+    // blocks placed early land wherever the draining kernel happens to free a slot, and the uneven
+    // spread over the SMs cost the write-back 30 % at 2^30 elements, p = 1e-2.
+    auto go = [&](void (*kernel)(Batch), dim3 g, Batch arg, bool early = true) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = g;
+        cfg.blockDim = dim3(kBlock);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = early ? 1 : 0;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, kernel, arg);
+    };
 
     // 1. bounds from the sample, then the streaming accumulate + collect pass
-    k_sample0<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
-    k_sample1<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
-    if (sampled) k_sample2<<<g1(WK_SAMPLE), blk, 0, st>>>(B(WK_SAMPLE));
+    go(k_sample0, g1(WK_SAMPLE), B(WK_SAMPLE));
+    go(k_sample1, g1(WK_SAMPLE), B(WK_SAMPLE));
+    if (sampled) go(k_sample2, g1(WK_SAMPLE), B(WK_SAMPLE));
     mark(SBC_MARK_BOUNDS);
-    if (mode == kModeValues) k_add_collect<kModeValues><<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
-    else                     k_add_collect<kModeBinary><<<g1(WK_MAIN), blk, 0, st>>>(B(WK_MAIN));
+    if (mode == kModeValues) go(k_add_collect<kModeValues>, g1(WK_MAIN), B(WK_MAIN), false);
+    else                     go(k_add_collect<kModeBinary>, g1(WK_MAIN), B(WK_MAIN), false);
     mark(SBC_MARK_COLLECT);
 
     // 2. exact route over A (returns immediately unless the bounds failed)
-    k_exact_hist<0><<<g1(WK_EXACT), blk, 0, st>>>(B(WK_EXACT));
-    k_exact_hist<1><<<g1(WK_EXACT), blk, 0, st>>>(B(WK_EXACT));
-    k_exact_hist<2><<<g1(WK_EXACT), blk, 0, st>>>(B(WK_EXACT));
-    k_exact_tiecount<<<g1(WK_XTILE), blk, 0, st>>>(B(WK_XTILE));
-    k_exact_tiescan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
-    k_exact_collect<<<g1(WK_XTILE), blk, 0, st>>>(B(WK_XTILE));
+    go(k_exact_hist<0>, g1(WK_EXACT), B(WK_EXACT));
+    go(k_exact_hist<1>, g1(WK_EXACT), B(WK_EXACT));
+    go(k_exact_hist<2>, g1(WK_EXACT), B(WK_EXACT));
+    go(k_exact_tiecount, g1(WK_XTILE), B(WK_XTILE));
+    go(k_exact_tiescan, g1(WK_ONE), B(WK_ONE));
+    go(k_exact_collect, g1(WK_XTILE), B(WK_XTILE));
     mark(SBC_MARK_EXACT);
 
     // 3. exact k-th composite of each candidate list, sums, side
-    k_select_hist0<<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
-    k_select_filter<0><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
-    k_select_filter<1><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
-    k_select_filter<2><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
-    k_select_filter<3><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
-    k_select_filter<4><<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
-    k_sums_decide<<<g2(WK_CAND), blk, 0, st>>>(B(WK_CAND));
+    go(k_select_hist0, g2(WK_CAND), B(WK_CAND));
+    go(k_select_filter<0>, g2(WK_CAND), B(WK_CAND));
+    go(k_select_filter<1>, g2(WK_CAND), B(WK_CAND));
+    go(k_select_filter<2>, g2(WK_CAND), B(WK_CAND));
+    go(k_select_filter<3>, g2(WK_CAND), B(WK_CAND));
+    go(k_select_filter<4>, g2(WK_CAND), B(WK_CAND));
+    go(k_sums_decide, g2(WK_CAND), B(WK_CAND));
     mark(SBC_MARK_SELECT);
 
     // 4. ordered positions, residual write-back, Golomb payload, chunk table, header
-    k_tile_count<<<g1(WK_SCATTER), blk, 0, st>>>(B(WK_SCATTER));
-    k_tile_scan<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
-    k_scatter<<<g1(WK_SCATTER), blk, 0, st>>>(B(WK_SCATTER));
-    k_tile_sort<<<g1(WK_TILE), blk, 0, st>>>(B(WK_TILE));
-    k_len_sum_residual<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));
-    k_len_scan_header<<<g1(WK_ONE), blk, 0, st>>>(B(WK_ONE));
-    k_pack<<<g1(WK_LEN), blk, 0, st>>>(B(WK_LEN));
+    go(k_tile_count, g1(WK_SCATTER), B(WK_SCATTER));
+    go(k_tile_scan, g1(WK_ONE), B(WK_ONE));
+    go(k_scatter, g1(WK_SCATTER), B(WK_SCATTER));
+    go(k_tile_sort, g1(WK_TILE), B(WK_TILE));
+    go(k_len_sum_residual, g1(WK_LEN), B(WK_LEN), false);
+    go(k_len_scan_header, g1(WK_ONE), B(WK_ONE));
+    go(k_pack, g1(WK_LEN), B(WK_LEN));
     mark(SBC_MARK_END);
 }
 

@@ -137,6 +137,13 @@ struct Slot {
 // kernels then read the descriptor at shared-memory cost and the compiler knows that their global
 // stores cannot change it.
 __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
+    // Programmatic dependent launch: the encode kernels are launched so that a kernel's blocks may
+    // be placed on the SMs while the kernel before it in the stream is still running.  Let the next
+    // kernel do the same as soon as every block of this one has got this far, then wait here until
+    // the previous kernel has completed and its writes are visible.  Nothing above this line reads
+    // memory another kernel writes.
+    cudaTriggerProgrammaticLaunchCompletion();
+    cudaGridDependencySynchronize();
     Slot s;
     const Prob* src;
     if (B.prefix == nullptr) {

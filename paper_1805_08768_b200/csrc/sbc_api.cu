@@ -265,7 +265,7 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
 // a single problem) say how each kind of work is spread over the problems.
 void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK_COUNT],
-                   const uint32_t* const* prefix, int mode, bool sampled, cudaStream_t st,
+                   const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, cudaStream_t st,
                    const sbc_cuda_event_t* marks) {
     auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
     auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs}; };
@@ -308,12 +308,16 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     mark(SBC_MARK_EXACT);
 
     // 3. exact k-th composite of each candidate list, sums, side
-    go(k_select_hist0, g2(WK_CAND), B(WK_CAND));
-    go(k_select_filter<0>, g2(WK_CAND), B(WK_CAND));
-    go(k_select_filter<1>, g2(WK_CAND), B(WK_CAND));
-    go(k_select_filter<2>, g2(WK_CAND), B(WK_CAND));
-    go(k_select_filter<3>, g2(WK_CAND), B(WK_CAND));
-    go(k_select_filter<4>, g2(WK_CAND), B(WK_CAND));
+    if (small_lists) {  // every list of this launch fits one block's registers: one kernel ranks them
+        go(k_select_small, g2(WK_ONE), B(WK_ONE));
+    } else {
+        go(k_select_hist0, g2(WK_CAND), B(WK_CAND));
+        go(k_select_filter<0>, g2(WK_CAND), B(WK_CAND));
+        go(k_select_filter<1>, g2(WK_CAND), B(WK_CAND));
+        go(k_select_filter<2>, g2(WK_CAND), B(WK_CAND));
+        go(k_select_filter<3>, g2(WK_CAND), B(WK_CAND));
+        go(k_select_filter<4>, g2(WK_CAND), B(WK_CAND));
+    }
     go(k_sums_decide, g2(WK_CAND), B(WK_CAND));
     mark(SBC_MARK_SELECT);
 
@@ -323,7 +327,6 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     go(k_scatter, g1(WK_SCATTER), B(WK_SCATTER));
     go(k_tile_sort, g1(WK_TILE), B(WK_TILE));
     go(k_len_sum_residual, g1(WK_LEN), B(WK_LEN), false);
-    go(k_len_scan_header, g1(WK_ONE), B(WK_ONE));
     go(k_pack, g1(WK_LEN), B(WK_LEN));
     mark(SBC_MARK_END);
 }
@@ -405,7 +408,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, 1u, grid);
-    launch_encode(d_prob, 1u, grid, nullptr, mode, pl.sampled != 0, st, marks);
+    launch_encode(d_prob, 1u, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -538,7 +541,9 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
     k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors});
-    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, false, st, nullptr);
+    bool small_lists = true;
+    for (int t = 0; t < n_tensors; ++t) small_lists = small_lists && plans[t].cap <= kSmallList;
+    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, false, small_lists, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -583,7 +588,7 @@ int sbc_encode_static(const float* update, float* residual, int64_t numel, doubl
                       (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
 }
 
-int sbc_encode_launches(void) { return 24; }  // put_prob, 2 sample, 1 collect, 6 exact, 7 select, 7 ordering + Golomb
+int sbc_encode_launches(void) { return 23; }  // put_prob, 2 sample, 1 collect, 6 exact, 7 select, 6 ordering + Golomb
 
 int sbc_decode_launches(int n_clients) {
     return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;

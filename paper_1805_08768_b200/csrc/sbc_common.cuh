@@ -27,6 +27,7 @@ constexpr int kTileWords = (1 << kTileShift) / 32;  // bitmask words covering on
 constexpr int kLenBlock = 1024;       // codewords per block in the length scan / packer
 constexpr int kChunkCodewords = 256;  // codewords per chunk-table entry
 constexpr int kSumBins = 254;         // one exact integer bin per fp32 exponent
+constexpr uint32_t kSmallList = 8192;  // candidate lists up to this capacity are ranked by one block
 
 // Stages that use the "last block to finish does the serial step" pattern.
 enum Stage : int {
@@ -34,7 +35,7 @@ enum Stage : int {
     ST_BH0_S0, ST_BH0_S1,
     ST_BF0_S0, ST_BF0_S1, ST_BF1_S0, ST_BF1_S1, ST_BF2_S0, ST_BF2_S1,
     ST_BF3_S0, ST_BF3_S1, ST_BF4_S0, ST_BF4_S1,
-    ST_SUM, ST_COUNT
+    ST_SUM, ST_LEN, ST_COUNT
 };
 
 // Device-side control block of one encode call; zeroed before the first kernel.
@@ -149,12 +150,27 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
     if (B.prefix == nullptr) {
         src = B.probs; s.bx = blockIdx.x; s.nb = gridDim.x;
     } else {
-        uint32_t lo = 0u, hi = B.n_probs;  // invariant: prefix[lo] <= blockIdx.x < prefix[hi]
-        while (hi - lo > 1u) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (B.prefix[mid] <= blockIdx.x) lo = mid; else hi = mid;
+        // The block's problem: largest i with prefix[i] <= blockIdx.x.  The first warp searches
+        // 32 ways at a time (two rounds of loads for up to 1024 problems); a binary search by one
+        // thread costs a block ten dependent loads before it can start, in every kernel of the chain.
+        __shared__ uint32_t s_slot[3];
+        if (threadIdx.x < 32u) {
+            const uint32_t lane = threadIdx.x;
+            uint32_t lo = 0u, hi = B.n_probs;  // invariant: prefix[lo] <= blockIdx.x < prefix[hi]
+            while (hi - lo > 1u) {
+                const uint32_t step = (hi - lo + 31u) / 32u;
+                const uint32_t probe = lo + lane * step;
+                const bool le = probe < hi && B.prefix[probe] <= blockIdx.x;  // true on lanes 0..j
+                const unsigned m = __ballot_sync(0xffffffffu, le);
+                const uint32_t j = 31u - (uint32_t)__clz((int)(m | 1u));
+                lo += j * step;
+                hi = min(hi, lo + step);
+            }
+            if (lane < 2u) s_slot[1 + lane] = B.prefix[lo + lane];
+            if (lane == 0u) s_slot[0] = lo;
         }
-        src = B.probs + lo; s.bx = blockIdx.x - B.prefix[lo]; s.nb = B.prefix[lo + 1] - B.prefix[lo];
+        __syncthreads();
+        src = B.probs + s_slot[0]; s.bx = blockIdx.x - s_slot[1]; s.nb = s_slot[2] - s_slot[1];
     }
     static_assert(sizeof(Prob) % 8 == 0, "copied as 8-byte words");
     for (int i = threadIdx.x; i < (int)(sizeof(Prob) / 8); i += blockDim.x)
@@ -330,6 +346,9 @@ struct Pick {
 // seen from the complemented key).  All kBlock threads call; result in *out
 // (shared) after the trailing barrier.
 // `out2` (may be null) receives the same for a second rank `rank2` from the same walk.
+// IN_SHARED: the histogram lives in the block's shared memory (plain loads) instead of global
+// memory written by other blocks (loads that bypass L1).
+template <bool IN_SHARED = false>
 __device__ __forceinline__ void block_pick_desc(const uint32_t* hist, int nbins, bool mirror,
                                                 uint32_t rank, uint32_t* s_scan, Pick* out,
                                                 uint32_t rank2 = 0u, Pick* out2 = nullptr) {
@@ -340,7 +359,10 @@ __device__ __forceinline__ void block_pick_desc(const uint32_t* hist, int nbins,
     for (int j = 0; j < kHistBins / kBlock; ++j) {
         int view = nbins - 1 - ((int)threadIdx.x * per + j);
         uint32_t v = 0;
-        if (j < per && view >= 0) v = __ldcg(hist + (mirror ? nbins - 1 - view : view));
+        if (j < per && view >= 0) {
+            const uint32_t* src = hist + (mirror ? nbins - 1 - view : view);
+            v = IN_SHARED ? *src : __ldcg(src);
+        }
         h[j] = v;
         sum += v;
     }

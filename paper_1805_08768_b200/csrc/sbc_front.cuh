@@ -26,7 +26,7 @@ __device__ __forceinline__ long long sample_element(const Prob& P, uint32_t i) {
 
 // Level 0: keys of the sampled A values, histogram of their top 11 bits; the
 // last block locates the bin of the target rank for each side.
-__global__ void __launch_bounds__(kBlock, 8) k_sample0(const Batch B) {
+__global__ void __launch_bounds__(kBlock, 4) k_sample0(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -36,18 +36,31 @@ __global__ void __launch_bounds__(kBlock, 8) k_sample0(const Batch B) {
     __shared__ Pick s_pick, s_pick_up;
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
-    for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
-        const uint32_t i = base + threadIdx.x;
-        const bool valid = i < P.m;
-        uint32_t key = 0u;
-        if (valid) {
-            long long e = P.sampled ? (long long)P.sample_idx[i] : sample_element(P, i);
-            if (e >= P.n) { e = P.n - 1; atomicOr(&ctl->status, SBC_STATUS_RANGE); }  // bad caller-given position
-            const float a = __fadd_rn(P.residual[e], P.update[e]);
-            key = select_key(P.mode, __float_as_uint(a));
-            P.sample_keys[i] = key;
+    constexpr int kItems = 8;  // sampled elements per thread and step, all loads issued before any is used
+    for (uint32_t base = S.bx * (kBlock * kItems); base < P.m; base += S.nb * (kBlock * kItems)) {
+        long long e[kItems];
+        float r[kItems], u[kItems];
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const uint32_t i = base + j * kBlock + threadIdx.x;
+            e[j] = -1;
+            if (i < P.m) {
+                e[j] = P.sampled ? (long long)P.sample_idx[i] : sample_element(P, i);
+                if (e[j] >= P.n) { e[j] = P.n - 1; atomicOr(&ctl->status, SBC_STATUS_RANGE); }  // bad caller-given position
+            }
         }
-        warp_hist_add(s_hist, key >> 21, valid);
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            r[j] = e[j] >= 0 ? P.residual[e[j]] : 0.f;
+            u[j] = e[j] >= 0 ? P.update[e[j]] : 0.f;
+        }
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const bool valid = e[j] >= 0;
+            const uint32_t key = select_key(P.mode, __float_as_uint(__fadd_rn(r[j], u[j])));
+            if (valid) P.sample_keys[base + j * kBlock + threadIdx.x] = key;
+            warp_hist_add(s_hist, key >> 21, valid);
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) {
@@ -72,7 +85,7 @@ __global__ void __launch_bounds__(kBlock, 8) k_sample0(const Batch B) {
 
 // Level 1: next 11 bits inside the located bins; the last block turns the
 // 22-bit prefixes into the two float bounds used by the candidate pass.
-__global__ void __launch_bounds__(kBlock, 8) k_sample1(const Batch B) {
+__global__ void __launch_bounds__(kBlock, 4) k_sample1(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -91,13 +104,21 @@ __global__ void __launch_bounds__(kBlock, 8) k_sample1(const Batch B) {
         const bool on0 = u == 0 || own_up[0], on1 = u == 0 || own_up[1];
         for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) (&s_hist[0][0])[i] = 0u;
         __syncthreads();
-        for (uint32_t base = S.bx * kBlock; base < P.m; base += S.nb * kBlock) {
-            const uint32_t i = base + threadIdx.x;
-            const bool valid = i < P.m;
-            const uint32_t key = valid ? P.sample_keys[i] : 0u;
-            const uint32_t sk1 = ~key;
-            warp_hist_add(s_hist[0], (key >> 10) & 2047u, valid && on0 && (key >> 21) == want0);
-            warp_hist_add(s_hist[1], (sk1 >> 10) & 2047u, valid && on1 && (sk1 >> 21) == want1);
+        constexpr int kItems = 8;  // keys per thread and step, loaded together
+        for (uint32_t base = S.bx * (kBlock * kItems); base < P.m; base += S.nb * (kBlock * kItems)) {
+            uint32_t keys[kItems];
+#pragma unroll
+            for (int j = 0; j < kItems; ++j) {
+                const uint32_t i = base + j * kBlock + threadIdx.x;
+                keys[j] = (i < P.m) ? P.sample_keys[i] : 0u;
+            }
+#pragma unroll
+            for (int j = 0; j < kItems; ++j) {
+                const bool valid = base + j * kBlock + threadIdx.x < P.m;
+                const uint32_t key = keys[j], sk1 = ~key;
+                warp_hist_add(s_hist[0], (key >> 10) & 2047u, valid && on0 && (key >> 21) == want0);
+                warp_hist_add(s_hist[1], (sk1 >> 10) & 2047u, valid && on1 && (sk1 >> 21) == want1);
+            }
         }
         __syncthreads();
         for (int i = threadIdx.x; i < 2 * kHistBins; i += kBlock) {

@@ -135,17 +135,70 @@ __device__ __forceinline__ unsigned long long codeword_len(const Prob& P, uint32
     return (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
 }
 
+__device__ __forceinline__ void store_u32(uint8_t* p, uint32_t v) { *reinterpret_cast<uint32_t*>(p) = v; }
+__device__ __forceinline__ void store_u64(uint8_t* p, unsigned long long v) {
+    *reinterpret_cast<unsigned long long*>(p) = v;
+}
+
+// Scan of the per-block bit counts (written by other blocks: read from L2) and the container
+// header, which is written always, so that a failed encode still leaves a header that says why.
+// One block.
+__device__ __forceinline__ void block_len_scan_header(const Prob& P, Ctl* ctl, unsigned long long* s_scan) {
+    const bool ok = __ldcg(&ctl->status) == 0u;  // uniform: nothing writes status while this kernel runs
+    unsigned long long total = 0ull;
+    if (ok) {
+        constexpr int kPer = 8;
+        for (uint32_t base = 0; base < P.n_len_blocks; base += kBlock * kPer) {
+            unsigned long long v[kPer];
+            unsigned long long sum = 0ull;
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const uint32_t t = base + threadIdx.x * kPer + j;
+                v[j] = (t < P.n_len_blocks) ? __ldcg(P.blk_len + t) : 0ull;
+                sum += v[j];
+            }
+            unsigned long long part;
+            unsigned long long run = total + block_exclusive_scan<unsigned long long>(sum, s_scan, &part);
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) {
+                const uint32_t t = base + threadIdx.x * kPer + j;
+                if (t < P.n_len_blocks) P.blk_len[t] = run;
+                run += v[j];
+            }
+            total += part;
+        }
+    }
+    if (threadIdx.x == 0) {
+        ctl->nbits = total;
+        uint8_t* h = P.stream;
+        store_u32(h + 0, SBC_MAGIC);
+        store_u32(h + 4, SBC_VERSION);
+        store_u64(h + 8, (unsigned long long)P.n);
+        store_u64(h + 16, ok ? (unsigned long long)P.k : 0ull);
+        store_u64(h + 24, total);
+        store_u64(h + 32, ok ? P.payload_offset : (unsigned long long)SBC_HEADER_BYTES);
+        store_u32(h + 40, (uint32_t)P.b);
+        store_u32(h + 44, ok ? (P.mode == kModeValues ? SBC_SIDE_VALUES : ctl->side) : 0u);
+        store_u32(h + 48, ok ? __float_as_uint(ctl->mu32) : 0u);
+        store_u32(h + 52, SBC_CHUNK_CODEWORDS);
+        store_u32(h + 56, ok ? P.n_chunks : 0u);
+        store_u32(h + 60, __ldcg(&ctl->status));
+    }
+}
+
 // Bits of each block of kLenBlock codewords, and -- since this is the first
 // walk over the ordered position list -- the residual write-back
-// R_j = A_j - mu at the kept positions (Algorithm 1), in address order.
+// R_j = A_j - mu at the kept positions (Algorithm 1), in address order.  The block that finishes
+// last scans the block bit counts and writes the container header.
 __global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
-    if (P.ctl->status) return;
+    Ctl* ctl = P.ctl;
+    const bool failed = ctl->status != 0u;  // uniform over the grid: no kernel of this stage sets it
     __shared__ unsigned long long s_scan[kBlock / 32 + 1];
     constexpr int kPer = kLenBlock / kBlock;
-    const float mu = P.ctl->mu32;
+    const float mu = ctl->mu32;
     const uint32_t k = (uint32_t)P.k;
     // values mode: the kept values themselves are sent (they sit between the chunk table and the
     // payload, in position order) and nothing of them stays in the residual
@@ -158,7 +211,7 @@ __global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
     // than a quarter ulp of mu, and a non-zero difference of two values that close is a multiple of
     // 2^-124.  Smaller |mu| (zero included) takes the load / subtract / store path.
     const bool by_atomic = values == nullptr && fabsf(mu) >= 7.888609052e-31f;  // 2^-100
-    for (uint32_t blk = S.bx; blk < P.n_len_blocks; blk += S.nb) {
+    for (uint32_t blk = S.bx; blk < (failed ? 0u : P.n_len_blocks); blk += S.nb) {
         const uint32_t i0 = blk * kLenBlock + threadIdx.x * kPer;
         uint32_t pos[kPer];
 #pragma unroll
@@ -193,61 +246,8 @@ __global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
         block_exclusive_scan<unsigned long long>(sum, s_scan, &total);
         if (threadIdx.x == 0) P.blk_len[blk] = total;
     }
-}
-
-__device__ __forceinline__ void store_u32(uint8_t* p, uint32_t v) { *reinterpret_cast<uint32_t*>(p) = v; }
-__device__ __forceinline__ void store_u64(uint8_t* p, unsigned long long v) {
-    *reinterpret_cast<unsigned long long*>(p) = v;
-}
-
-// Scan of the per-block bit counts; also writes the container header, always,
-// so that a failed encode still leaves a header that says why.
-__global__ void __launch_bounds__(kBlock) k_len_scan_header(const Batch B) {
-    __shared__ Prob s_prob;
-    const Slot S = resolve(B, &s_prob);
-    const Prob& P = s_prob;
-    Ctl* ctl = P.ctl;
-    __shared__ unsigned long long s_scan[kBlock / 32 + 1];
-    const bool ok = ctl->status == 0u;  // uniform: nothing writes status while this kernel runs
-    unsigned long long total = 0ull;
-    if (ok) {
-        constexpr int kPer = 8;
-        for (uint32_t base = 0; base < P.n_len_blocks; base += kBlock * kPer) {
-            unsigned long long v[kPer];
-            unsigned long long sum = 0ull;
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) {
-                const uint32_t t = base + threadIdx.x * kPer + j;
-                v[j] = (t < P.n_len_blocks) ? P.blk_len[t] : 0ull;
-                sum += v[j];
-            }
-            unsigned long long part;
-            unsigned long long run = total + block_exclusive_scan<unsigned long long>(sum, s_scan, &part);
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) {
-                const uint32_t t = base + threadIdx.x * kPer + j;
-                if (t < P.n_len_blocks) P.blk_len[t] = run;
-                run += v[j];
-            }
-            total += part;
-        }
-    }
-    if (threadIdx.x == 0) {
-        ctl->nbits = total;
-        uint8_t* h = P.stream;
-        store_u32(h + 0, SBC_MAGIC);
-        store_u32(h + 4, SBC_VERSION);
-        store_u64(h + 8, (unsigned long long)P.n);
-        store_u64(h + 16, ok ? (unsigned long long)P.k : 0ull);
-        store_u64(h + 24, total);
-        store_u64(h + 32, ok ? P.payload_offset : (unsigned long long)SBC_HEADER_BYTES);
-        store_u32(h + 40, (uint32_t)P.b);
-        store_u32(h + 44, ok ? (P.mode == kModeValues ? SBC_SIDE_VALUES : ctl->side) : 0u);
-        store_u32(h + 48, ok ? __float_as_uint(ctl->mu32) : 0u);
-        store_u32(h + 52, SBC_CHUNK_CODEWORDS);
-        store_u32(h + 56, ok ? P.n_chunks : 0u);
-        store_u32(h + 60, ctl->status);
-    }
+    // by the block that finishes last: bit offset of every block, total bits, header
+    if (last_block_ticket(&ctl->done[ST_LEN], S.nb)) block_len_scan_header(P, ctl, s_scan);
 }
 
 // ---------------------------------------------------------------- bit packer

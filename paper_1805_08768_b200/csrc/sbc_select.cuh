@@ -53,14 +53,22 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
     unsigned long long shared_bits;
     const int top = select_top(P, ctl, s, view, &shared_bits);
-    for (uint32_t base = S.bx * kBlock; base < cnt; base += S.nb * kBlock) {
-        const uint32_t i = base + threadIdx.x;
-        const bool valid = i < cnt;
-        const unsigned long long c = valid ? view.at(begin + i) : 0ull;
-        // whole key range: nearly all entries share the first digit, so one atomic per warp and
-        // bin; band: the first digit already spreads them, plain atomics collide rarely
-        if (top == 63) warp_hist_add(s_hist, digit_of(c, 0, top), valid);
-        else if (valid) atomicAdd(&s_hist[digit_of(c, 0, top)], 1u);
+    constexpr int kItems = 4;  // loads in flight per thread
+    for (uint32_t base = S.bx * (kBlock * kItems); base < cnt; base += S.nb * (kBlock * kItems)) {
+        unsigned long long c[kItems];
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const uint32_t i = base + j * kBlock + threadIdx.x;
+            c[j] = (i < cnt) ? view.at(begin + i) : 0ull;
+        }
+#pragma unroll
+        for (int j = 0; j < kItems; ++j) {
+            const bool valid = base + j * kBlock + threadIdx.x < cnt;
+            // whole key range: nearly all entries share the first digit, so one atomic per warp and
+            // bin; band: the first digit already spreads them, plain atomics collide rarely
+            if (top == 63) warp_hist_add(s_hist, digit_of(c[j], 0, top), valid);
+            else if (valid) atomicAdd(&s_hist[digit_of(c[j], 0, top)], 1u);
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) {
@@ -76,6 +84,73 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
             if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
         }
     }
+}
+
+// The whole selection of one side by ONE block, for lists of at most kSmallList entries (every
+// tensor of a ResNet-sized layer at p = 0.001): the entries sit in registers, every level is a
+// shared-memory histogram of the entries that still match the prefix, and the walk stops as soon as
+// the selected bucket holds a single entry.  Same result as k_select_hist0 + k_select_filter<0..4>;
+// the host launches this kernel instead of those when every list of the launch is that small.
+// One block per problem, grid.z = side.
+__global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
+    Ctl* ctl = P.ctl;
+    if (ctl->status || ctl->sampled_ok) return;
+    const int s = blockIdx.z;
+    if (s == 1 && P.mode == kModeValues) return;
+    constexpr int kPer = (int)(kSmallList / kBlock);
+    __shared__ uint32_t s_hist[kHistBins];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ Pick s_pick;
+    const CandView view = cand_view(P, ctl, s);
+    uint32_t begin, cnt, rank;
+    select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
+    unsigned long long prefix;
+    const int top = select_top(P, ctl, s, view, &prefix);
+    const int levels = digit_levels(top);
+    if (cnt > kSmallList) {  // cannot happen: cnt <= cap <= kSmallList is what the host checked
+        if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+        return;
+    }
+    unsigned long long c[kPer];
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) {
+        const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
+        c[j] = (i < cnt) ? view.at(begin + i) : 0ull;
+    }
+    unsigned alive = 0u;  // entries that still match the prefix
+#pragma unroll
+    for (int j = 0; j < kPer; ++j) alive |= ((uint32_t)j * kBlock + threadIdx.x < cnt) ? (1u << j) : 0u;
+    for (int level = 0; level < levels; ++level) {
+        for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < kPer; ++j)
+            if ((alive >> j) & 1u) atomicAdd(&s_hist[digit_of(c[j], level, top)], 1u);
+        __syncthreads();
+        block_pick_desc<true>(s_hist, 1 << digit_bits(level, top), false, rank, s_scan, &s_pick);
+        if (!s_pick.found) {  // uniform
+            if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            return;
+        }
+        const uint32_t sel = s_pick.bin;
+        const bool single = s_pick.count == 1u;
+        rank = s_pick.rank;
+        prefix |= (unsigned long long)sel << digit_shift(level, top);
+#pragma unroll
+        for (int j = 0; j < kPer; ++j)
+            if (((alive >> j) & 1u) && digit_of(c[j], level, top) != sel) alive &= ~(1u << j);
+        if (single) {  // the one entry left is the k-th largest composite
+#pragma unroll
+            for (int j = 0; j < kPer; ++j)
+                if ((alive >> j) & 1u) ctl->thr[s] = c[j];
+            return;
+        }
+        __syncthreads();  // s_pick and s_hist are reused
+    }
+    if (threadIdx.x == 0) ctl->thr[s] = prefix;  // every digit fixed
 }
 
 // Keep the entries whose level-L digit is the selected one, histogram their

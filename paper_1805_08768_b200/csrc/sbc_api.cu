@@ -190,6 +190,7 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile
     P.s_up = pl.s_up;
     P.cap = pl.cap;
     P.m = pl.m;
+    P.sample_step = (pl.m >> 5) ? ((unsigned long long)(pl.n >> 5) << 20) / (unsigned long long)(pl.m >> 5) : 0ull;
     P.n_xtiles = pl.n_xtiles;
     P.n_tiles = pl.n_tiles;
     P.n_len_blocks = pl.n_len_blocks;
@@ -219,9 +220,9 @@ inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsi
 // (or, for the exact route, usually just for finding out that it is not needed), and a batch of
 // hundreds of problems has parallelism to spare.
 void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned coarse_exact,
-                  unsigned nb[WK_COUNT]) {
+                  unsigned coarse_main, unsigned nb[WK_COUNT]) {
     nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8 * coarse_sample, sms * 4);
-    nb[WK_MAIN] = grid_for((unsigned long long)pl.n, kBlock * kPerThread, sms * kCollectBlocksPerSM);
+    nb[WK_MAIN] = grid_for((unsigned long long)pl.n, kBlock * kPerThread * coarse_main, sms * kCollectBlocksPerSM);
     nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 8);
     nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 8);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
@@ -407,7 +408,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
     k_put_prob<<<1, 1, 0, st>>>(d_prob, P);
 
     unsigned grid[WK_COUNT];
-    block_counts(pl, (unsigned)sm_count(), 1u, 1u, grid);
+    block_counts(pl, (unsigned)sm_count(), 1u, 1u, 1u, grid);
     launch_encode(d_prob, 1u, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
@@ -490,15 +491,20 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
 
     const unsigned sms = (unsigned)sm_count();
     // aim at about six (sample) and two (exact route) blocks per SM over the whole batch
-    unsigned long long fine_sample = 0, fine_exact = 0;
+    unsigned long long fine_sample = 0, fine_exact = 0, fine_main = 0;
     for (int t = 0; t < n_tensors; ++t) {
         fine_sample += (plans[t].m + kBlock * 8 - 1) / (kBlock * 8);
         fine_exact += (unsigned long long)(plans[t].n + kBlock * 16 - 1) / (kBlock * 16);
+        fine_main += (unsigned long long)(plans[t].n + kBlock * kPerThread - 1) / (kBlock * kPerThread);
     }
     auto factor = [&](unsigned long long fine, unsigned per_sm) {
         return (unsigned)std::min<unsigned long long>(256, std::max<unsigned long long>(1, fine / (sms * per_sm)));
     };
     const unsigned coarse_sample = factor(fine_sample, 6), coarse_exact = factor(fine_exact, 2);
+    // streaming pass: about three waves of resident blocks over the whole batch, so that a block's
+    // start-up (finding its problem, reading the bounds) and its final flush are paid for by several
+    // steps of loads
+    const unsigned coarse_main = std::min(8u, factor(fine_main, 3 * kCollectBlocksPerSM));
     const size_t row_len = (size_t)n_tensors + 1;
     std::vector<Prob> probs((size_t)n_tensors);
     std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
@@ -512,7 +518,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
             m += plans[t].tile_bytes;
             r += plans[t].rest_bytes;
             unsigned nb[WK_COUNT];
-            block_counts(plans[t], sms, coarse_sample, coarse_exact, nb);
+            block_counts(plans[t], sms, coarse_sample, coarse_exact, coarse_main, nb);
             for (int kind = 0; kind < WK_COUNT; ++kind) {
                 uint32_t* row = prefix.data() + (size_t)kind * row_len;
                 const unsigned long long next = (unsigned long long)row[t] + nb[kind];

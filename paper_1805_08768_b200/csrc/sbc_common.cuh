@@ -114,6 +114,7 @@ struct Prob {
     unsigned long long* blk_len;
     uint32_t cap;               // capacity of each candidate list
     uint32_t m;                 // sample size
+    unsigned long long sample_step;  // 128-byte lines between sampled segments, 20 fractional bits
     uint32_t s_target;          // rank looked up in the sample (the same for both sides)
     uint32_t s_up;              // rank in the sample of the upper bound (0: no upper bound)
     uint32_t n_xtiles, n_tiles, n_len_blocks, n_chunks;

@@ -16,12 +16,13 @@ namespace sbc {
 
 // ---------------------------------------------------------------- sample
 
+// Element behind sample slot i: the sample is made of whole 32-element segments spread evenly over
+// the tensor, segment g starting at line floor(g * n_lines / n_segments) (the quotient is a
+// fixed-point constant of the problem, at least 1, so the segments are distinct and in range).
 __device__ __forceinline__ long long sample_element(const Prob& P, uint32_t i) {
     if ((long long)P.m == P.n) return (long long)i;
     const uint32_t seg = i >> 5, lane = i & 31u;
-    const unsigned long long n_lines = (unsigned long long)(P.n >> 5);
-    const unsigned long long n_seg = P.m >> 5;
-    return (long long)(((unsigned long long)seg * n_lines) / n_seg) * 32 + lane;
+    return (long long)(((unsigned long long)seg * P.sample_step) >> 20) * 32 + lane;
 }
 
 // Level 0: keys of the sampled A values, histogram of their top 11 bits; the
@@ -59,7 +60,7 @@ __global__ void __launch_bounds__(kBlock, 4) k_sample0(const Batch B) {
             const bool valid = e[j] >= 0;
             const uint32_t key = select_key(P.mode, __float_as_uint(__fadd_rn(r[j], u[j])));
             if (valid) P.sample_keys[base + j * kBlock + threadIdx.x] = key;
-            warp_hist_add(s_hist, key >> 21, valid);
+            if (valid) atomicAdd(&s_hist[key >> 21], 1u);
         }
     }
     __syncthreads();
@@ -116,8 +117,8 @@ __global__ void __launch_bounds__(kBlock, 4) k_sample1(const Batch B) {
             for (int j = 0; j < kItems; ++j) {
                 const bool valid = base + j * kBlock + threadIdx.x < P.m;
                 const uint32_t key = keys[j], sk1 = ~key;
-                warp_hist_add(s_hist[0], (key >> 10) & 2047u, valid && on0 && (key >> 21) == want0);
-                warp_hist_add(s_hist[1], (sk1 >> 10) & 2047u, valid && on1 && (sk1 >> 21) == want1);
+                if (valid && on0 && (key >> 21) == want0) atomicAdd(&s_hist[0][(key >> 10) & 2047u], 1u);
+                if (valid && on1 && (sk1 >> 21) == want1) atomicAdd(&s_hist[1][(sk1 >> 10) & 2047u], 1u);
             }
         }
         __syncthreads();

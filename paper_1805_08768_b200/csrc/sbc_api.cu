@@ -12,6 +12,7 @@
 #include "sbc_front.cuh"
 #include "sbc_golomb.cuh"
 #include "sbc_select.cuh"
+#include "sbc_small.cuh"
 
 namespace sbc {
 namespace {
@@ -266,7 +267,7 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
 // a single problem) say how each kind of work is spread over the problems.
 void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK_COUNT],
-                   const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, cudaStream_t st,
+                   const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, bool small_kept, cudaStream_t st,
                    const sbc_cuda_event_t* marks) {
     auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
     auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs}; };
@@ -309,6 +310,13 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     mark(SBC_MARK_EXACT);
 
     // 3. exact k-th composite of each candidate list, sums, side
+    // 4. ordered positions, residual write-back, Golomb payload, chunk table, header
+    if (small_lists && small_kept && mode == kModeBinary && !sampled) {  // all of it by two blocks per problem
+        mark(SBC_MARK_SELECT);
+        go(k_small_finish, g2(WK_ONE), B(WK_ONE));
+        mark(SBC_MARK_END);
+        return;
+    }
     if (small_lists) {  // every list of this launch fits one block's registers: one kernel ranks them
         go(k_select_small, g2(WK_ONE), B(WK_ONE));
     } else {
@@ -322,7 +330,6 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK
     go(k_sums_decide, g2(WK_CAND), B(WK_CAND));
     mark(SBC_MARK_SELECT);
 
-    // 4. ordered positions, residual write-back, Golomb payload, chunk table, header
     go(k_tile_count, g1(WK_SCATTER), B(WK_SCATTER));
     go(k_tile_scan, g1(WK_ONE), B(WK_ONE));
     go(k_scatter, g1(WK_SCATTER), B(WK_SCATTER));
@@ -409,7 +416,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, 1u, 1u, grid);
-    launch_encode(d_prob, 1u, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, st, marks);
+    launch_encode(d_prob, 1u, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, pl.k <= (long long)kSmallKept, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -547,9 +554,12 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
     k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors});
-    bool small_lists = true;
-    for (int t = 0; t < n_tensors; ++t) small_lists = small_lists && plans[t].cap <= kSmallList;
-    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, false, small_lists, st, nullptr);
+    bool small_lists = true, small_kept = true;
+    for (int t = 0; t < n_tensors; ++t) {
+        small_lists = small_lists && plans[t].cap <= kSmallList;
+        small_kept = small_kept && plans[t].k <= (long long)kSmallKept;
+    }
+    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, false, small_lists, small_kept, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

@@ -140,6 +140,25 @@ __device__ __forceinline__ void store_u64(uint8_t* p, unsigned long long v) {
     *reinterpret_cast<unsigned long long*>(p) = v;
 }
 
+// The container header (one thread).  Written always, so that a failed encode still leaves a
+// header that says why.
+__device__ __forceinline__ void write_header(const Prob& P, Ctl* ctl, bool ok, unsigned long long nbits) {
+    ctl->nbits = nbits;
+    uint8_t* h = P.stream;
+    store_u32(h + 0, SBC_MAGIC);
+    store_u32(h + 4, SBC_VERSION);
+    store_u64(h + 8, (unsigned long long)P.n);
+    store_u64(h + 16, ok ? (unsigned long long)P.k : 0ull);
+    store_u64(h + 24, nbits);
+    store_u64(h + 32, ok ? P.payload_offset : (unsigned long long)SBC_HEADER_BYTES);
+    store_u32(h + 40, (uint32_t)P.b);
+    store_u32(h + 44, ok ? (P.mode == kModeValues ? SBC_SIDE_VALUES : __ldcg(&ctl->side)) : 0u);
+    store_u32(h + 48, ok ? __float_as_uint(__ldcg(&ctl->mu32)) : 0u);
+    store_u32(h + 52, SBC_CHUNK_CODEWORDS);
+    store_u32(h + 56, ok ? P.n_chunks : 0u);
+    store_u32(h + 60, __ldcg(&ctl->status));
+}
+
 // Scan of the per-block bit counts (written by other blocks: read from L2) and the container
 // header, which is written always, so that a failed encode still leaves a header that says why.
 // One block.
@@ -168,22 +187,7 @@ __device__ __forceinline__ void block_len_scan_header(const Prob& P, Ctl* ctl, u
             total += part;
         }
     }
-    if (threadIdx.x == 0) {
-        ctl->nbits = total;
-        uint8_t* h = P.stream;
-        store_u32(h + 0, SBC_MAGIC);
-        store_u32(h + 4, SBC_VERSION);
-        store_u64(h + 8, (unsigned long long)P.n);
-        store_u64(h + 16, ok ? (unsigned long long)P.k : 0ull);
-        store_u64(h + 24, total);
-        store_u64(h + 32, ok ? P.payload_offset : (unsigned long long)SBC_HEADER_BYTES);
-        store_u32(h + 40, (uint32_t)P.b);
-        store_u32(h + 44, ok ? (P.mode == kModeValues ? SBC_SIDE_VALUES : ctl->side) : 0u);
-        store_u32(h + 48, ok ? __float_as_uint(ctl->mu32) : 0u);
-        store_u32(h + 52, SBC_CHUNK_CODEWORDS);
-        store_u32(h + 56, ok ? P.n_chunks : 0u);
-        store_u32(h + 60, __ldcg(&ctl->status));
-    }
+    if (threadIdx.x == 0) write_header(P, ctl, ok, total);
 }
 
 // Bits of each block of kLenBlock codewords, and -- since this is the first
@@ -265,6 +269,30 @@ __device__ __forceinline__ void or_bits(uint32_t* words, unsigned long long off,
     if (lo) atomicOr(words + w + 1, __byte_perm(lo, 0u, 0x0123));
 }
 
+// Codeword i (gap g, Golomb parameter b) at stream bit `off`: q = g >> b ones, a zero, then g's low
+// b bits MSB first (Algorithm 3), ORed into the zeroed payload; the first codeword of a chunk also
+// writes the chunk's table entry (bit offset, position of the codeword before it, taken from the
+// ascending position list).
+__device__ __forceinline__ void pack_codeword(uint32_t* words, uint8_t* table, uint32_t i, unsigned long long off,
+                                              uint32_t g, int b, const uint32_t* positions) {
+    if (i % kChunkCodewords == 0) {
+        uint8_t* e = table + (size_t)(i / kChunkCodewords) * SBC_CHUNK_ENTRY_BYTES;
+        store_u64(e, off);
+        store_u64(e + 8, (unsigned long long)(i ? (long long)positions[i - 1] : -1ll));
+    }
+    unsigned long long pos = off;
+    uint32_t q = g >> b;
+    // q ones: head up to a word boundary, whole words, then the rest
+    if (q) {
+        const int head = min((uint32_t)(32 - (int)(pos & 31ull)) & 31u, q);
+        if (head) { or_bits(words, pos, head, 0xffffffffu >> (32 - head)); pos += head; q -= head; }
+        while (q >= 32u) { words[pos >> 5] = 0xffffffffu; pos += 32; q -= 32u; }
+        if (q) { or_bits(words, pos, (int)q, 0xffffffffu >> (32 - q)); pos += q; }
+    }
+    // the terminating zero and r in b bits, MSB first: 1 + b <= 31 bits
+    or_bits(words, pos, 1 + b, g & ((1u << b) - 1u));
+}
+
 __global__ void __launch_bounds__(kBlock) k_pack(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
@@ -292,22 +320,7 @@ __global__ void __launch_bounds__(kBlock) k_pack(const Batch B) {
         for (int j = 0; j < kPer; ++j) {
             const uint32_t i = blk * kLenBlock + threadIdx.x * kPer + j;
             if (i >= (uint32_t)P.k) continue;
-            if (i % kChunkCodewords == 0) {
-                uint8_t* e = table + (size_t)(i / kChunkCodewords) * SBC_CHUNK_ENTRY_BYTES;
-                store_u64(e, off);
-                store_u64(e + 8, (unsigned long long)(i ? (long long)P.idx[i - 1] : -1ll));
-            }
-            unsigned long long pos = off;
-            uint32_t q = gap[j] >> b;
-            // q ones: head up to a word boundary, whole words, then the rest
-            if (q) {
-                const int head = min((uint32_t)(32 - (int)(pos & 31ull)) & 31u, q);
-                if (head) { or_bits(words, pos, head, 0xffffffffu >> (32 - head)); pos += head; q -= head; }
-                while (q >= 32u) { words[pos >> 5] = 0xffffffffu; pos += 32; q -= 32u; }
-                if (q) { or_bits(words, pos, (int)q, 0xffffffffu >> (32 - q)); pos += q; }
-            }
-            // the terminating zero and r in b bits, MSB first: 1 + b <= 31 bits
-            or_bits(words, pos, 1 + b, gap[j] & ((1u << b) - 1u));
+            pack_codeword(words, table, i, off, gap[j], b, P.idx);
             off += len[j];
         }
     }

@@ -221,13 +221,23 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
 
 // ---------------------------------------------------------------- exact sums, means, side
 
+// Which of a block's 256 bins (bins[threadIdx.x]) are not zero, one bit each, into nonzero[0..8)
+// (shared).  All kBlock threads call; valid after the next barrier.
+__device__ __forceinline__ void bins_nonzero_masks(long long mine, uint32_t* nonzero) {
+    const unsigned m = __ballot_sync(0xffffffffu, mine != 0);
+    if (lane_id() == 0) nonzero[threadIdx.x >> 5] = m;
+}
+
 // Round the exact integer sum_s bins[s] * 2^s (units of 2^-149) to fp64,
-// nearest-even.  One thread.
-__device__ double bins_to_double(const long long* bins) {
+// nearest-even.  One thread.  `nonzero` has bit (s & 31) of word s >> 5 set for every bin that is
+// not zero (8 words, from bins_nonzero_masks): only those are visited.
+__device__ double bins_to_double(const long long* bins, const uint32_t* nonzero) {
     unsigned long long acc[6] = {0, 0, 0, 0, 0, 0};  // 384-bit two's complement
-    for (int s = 0; s < kSumBins; ++s) {
+    for (int word = 0; word < 8; ++word)
+    for (uint32_t left = nonzero[word]; left; left &= left - 1u) {
+        const int s = word * 32 + __ffs(left) - 1;
+        if (s >= kSumBins) continue;
         const long long v = bins[s];
-        if (v == 0) continue;
         const int limb = s >> 6, off = s & 63;
         unsigned long long part[3];
         part[0] = (unsigned long long)v << off;
@@ -347,11 +357,15 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
         if (v) atomicAdd(reinterpret_cast<unsigned long long*>(&ctl->bins[s][threadIdx.x]), v);
     }
     if (last_block_ticket(&ctl->done[ST_SUM], values_mode ? S.nb : S.nb * gridDim.z)) {
-        s_bins[0][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[0][threadIdx.x]);
-        s_bins[1][threadIdx.x] = (unsigned long long)__ldcg(&ctl->bins[1][threadIdx.x]);
+        __shared__ uint32_t s_nonzero[2][8];
+        const long long b0 = __ldcg(&ctl->bins[0][threadIdx.x]), b1 = __ldcg(&ctl->bins[1][threadIdx.x]);
+        s_bins[0][threadIdx.x] = (unsigned long long)b0;
+        s_bins[1][threadIdx.x] = (unsigned long long)b1;
+        bins_nonzero_masks(b0, s_nonzero[0]);
+        bins_nonzero_masks(b1, s_nonzero[1]);
         __syncthreads();
         if (threadIdx.x < 2) {  // one thread per side rounds its exact sum
-            const double sum = bins_to_double(reinterpret_cast<const long long*>(s_bins[threadIdx.x]));
+            const double sum = bins_to_double(reinterpret_cast<const long long*>(s_bins[threadIdx.x]), s_nonzero[threadIdx.x]);
             // mean over the k selected entries, or over however many the sampled threshold let through
             const double count = ctl->sampled_ok ? (double)min(__ldcg(&ctl->cand_cnt[threadIdx.x]), P.cap) : (double)P.k;
             ctl->mu64[threadIdx.x] = threadIdx.x ? -sum / count : sum / count;

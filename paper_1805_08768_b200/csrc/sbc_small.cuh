@@ -1,0 +1,320 @@
+// Back half of sbc_encode for problems whose candidate lists hold at most kSmallList entries
+// (every tensor of a ResNet-sized layer at p = 0.001): everything after the candidate pass in ONE
+// kernel, two blocks per problem (one per side).  Each block finds its side's k-th largest
+// composite and the exact sum of the kept values (Algorithm 2); the block that finishes second
+// takes the side decision and goes on alone: kept positions in ascending order, residual
+// write-back (Algorithm 1), Golomb code, chunk table and header (Algorithm 3).  Same results as the
+// general kernels, which a launch uses as soon as one of its lists is longer.
+#pragma once
+#include "sbc_common.cuh"
+#include "sbc_golomb.cuh"
+#include "sbc_select.cuh"
+#include "../../include/sbc.h"
+
+namespace sbc {
+
+constexpr uint32_t kSmallKept = 4096;  // positions one block orders in shared memory (k <= (kSmallList - 1024) / 2)
+static_assert((kSmallList - 1024u) / 2u <= kSmallKept, "a short list keeps at most kSmallKept positions");
+
+// Rank `rank` (1 = largest) among the cnt <= kSmallList composites a block holds in registers
+// (slot j of thread t = entry j * kBlock + t).  Radix selection, 11-bit digits from bit `top` down,
+// on shared-memory histograms; stops at the first bucket with a single entry.  Returns false if the
+// histogram walk failed (inconsistent counts).  All threads call; result identical in all.
+template <int PER>
+__device__ __forceinline__ bool block_select_registers(const unsigned long long (&c)[PER], uint32_t cnt, uint32_t rank,
+                                                       int top, unsigned long long prefix, uint32_t* s_hist,
+                                                       uint32_t* s_scan, Pick* s_pick, unsigned long long* s_result,
+                                                       unsigned long long* out) {
+    unsigned alive = 0u;  // entries that still match the prefix
+#pragma unroll
+    for (int j = 0; j < PER; ++j) alive |= ((uint32_t)j * kBlock + threadIdx.x < cnt) ? (1u << j) : 0u;
+    const int levels = digit_levels(top);
+    for (int level = 0; level < levels; ++level) {
+        for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
+        __syncthreads();
+        // a thread's entries mostly share their leading digits: one atomic per run of equal digits
+        uint32_t run_digit = 0u, run_len = 0u;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            if ((alive >> j) & 1u) {
+                const uint32_t d = digit_of(c[j], level, top);
+                if (run_len && d != run_digit) { atomicAdd(&s_hist[run_digit], run_len); run_len = 0u; }
+                run_digit = d;
+                ++run_len;
+            }
+        }
+        if (run_len) atomicAdd(&s_hist[run_digit], run_len);
+        __syncthreads();
+        block_pick_desc<true>(s_hist, 1 << digit_bits(level, top), false, rank, s_scan, s_pick);
+        if (!s_pick->found) return false;  // uniform
+        const uint32_t sel = s_pick->bin;
+        const bool single = s_pick->count == 1u;
+        rank = s_pick->rank;
+        prefix |= (unsigned long long)sel << digit_shift(level, top);
+#pragma unroll
+        for (int j = 0; j < PER; ++j)
+            if (((alive >> j) & 1u) && digit_of(c[j], level, top) != sel) alive &= ~(1u << j);
+        if (single) {  // the one entry left is the answer; its owner publishes it
+#pragma unroll
+            for (int j = 0; j < PER; ++j)
+                if ((alive >> j) & 1u) *s_result = c[j];
+            __syncthreads();
+            *out = *s_result;
+            return true;
+        }
+        __syncthreads();  // s_pick and s_hist are reused
+    }
+    *out = prefix;  // every digit fixed
+    return true;
+}
+
+// Compare-exchange stage of a bitonic network between registers r and r | STRIDE of one thread
+// (element index = first + r); ascending where (index & size) == 0.
+template <int STRIDE>
+__device__ __forceinline__ void bitonic_in_thread(uint32_t (&x)[16], uint32_t size, uint32_t first) {
+#pragma unroll
+    for (int r = 0; r < 16; ++r) {
+        if ((r & STRIDE) == 0) {
+            const bool ascending = ((first + (uint32_t)r) & size) == 0u;
+            const uint32_t a = x[r], b = x[r | STRIDE];
+            const bool swap = (a > b) == ascending;
+            x[r] = swap ? b : a;
+            x[r | STRIDE] = swap ? a : b;
+        }
+    }
+}
+
+// Ascending sort of kSmallKept = 16 * kBlock values, thread t holding elements 16 t .. 16 t + 15 in
+// registers (bitonic network): exchanges between threads of a warp by shuffle, between warps
+// through `s_swap` (kSmallKept words, transposed so that accesses are conflict-free), the rest in
+// registers.  All threads call.
+__device__ __forceinline__ void block_sort_16(uint32_t (&x)[16], uint32_t* s_swap) {
+    static_assert(kSmallKept == 16u * kBlock, "sixteen values per thread");
+    const uint32_t tid = threadIdx.x, first = tid * 16u;
+    for (uint32_t size = 2u; size <= kSmallKept; size <<= 1) {
+        const bool ascending = (first & size) == 0u;  // used where the partner is another thread (size >= 32)
+        for (uint32_t stride = size >> 1; stride >= 512u; stride >>= 1) {  // partner in another warp
+            const uint32_t d = stride >> 4;
+#pragma unroll
+            for (int r = 0; r < 16; ++r) s_swap[r * kBlock + tid] = x[r];
+            __syncthreads();
+            const bool take_min = ((tid & d) == 0u) == ascending;
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                const uint32_t o = s_swap[r * kBlock + (tid ^ d)];
+                x[r] = take_min ? min(x[r], o) : max(x[r], o);
+            }
+            __syncthreads();
+        }
+        for (uint32_t stride = min(size >> 1, 256u); stride >= 16u; stride >>= 1) {  // partner in this warp
+            const uint32_t d = stride >> 4;
+            const bool take_min = ((tid & d) == 0u) == ascending;
+#pragma unroll
+            for (int r = 0; r < 16; ++r) {
+                const uint32_t o = __shfl_xor_sync(0xffffffffu, x[r], (int)d);
+                x[r] = take_min ? min(x[r], o) : max(x[r], o);
+            }
+        }
+        if (size >= 16u) bitonic_in_thread<8>(x, size, first);
+        if (size >= 8u) bitonic_in_thread<4>(x, size, first);
+        if (size >= 4u) bitonic_in_thread<2>(x, size, first);
+        bitonic_in_thread<1>(x, size, first);
+    }
+}
+
+// One block per problem and side (grid.z = side).
+__global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
+    Ctl* ctl = P.ctl;
+    const int s = blockIdx.z;
+    constexpr int kPer = (int)(kSmallList / kBlock);
+    __shared__ uint32_t s_hist[kHistBins];
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ unsigned long long s_scan64[kBlock / 32 + 1];
+    __shared__ Pick s_pick;
+    __shared__ unsigned long long s_result;
+    __shared__ long long s_bins[256];
+    __shared__ uint32_t s_pos[kSmallKept];
+    __shared__ uint32_t s_count, s_status;
+    __shared__ uint32_t s_nonzero[8];
+
+    // ---- this side: threshold and exact sum (skipped when an earlier kernel reported an error;
+    // one thread reads the status word, since the other side's block may set it meanwhile)
+    if (threadIdx.x == 0) s_status = __ldcg(&ctl->status);
+    __syncthreads();
+    if (s_status == 0u) {
+        const CandView view = cand_view(P, ctl, s);
+        uint32_t begin, cnt, rank;
+        select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
+        unsigned long long prefix, thr = 0ull;
+        const int top = select_top(P, ctl, s, view, &prefix);
+        bool good = cnt <= kSmallList && view.total <= kSmallList;  // what the host checked through the capacity
+        unsigned long long c[kPer];
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) {
+            const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
+            c[j] = (good && i < cnt) ? view.at(begin + i) : 0ull;
+        }
+        good = good && block_select_registers<kPer>(c, cnt, rank, top, prefix, s_hist, s_scan, &s_pick, &s_result, &thr);
+        if (!good) {
+            if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+        } else {
+            // exact sum of the kept values: 24-bit integers into one 64-bit bin per exponent.  Nearly
+            // all kept values lie within eight binades of the threshold's: those are summed in one
+            // register per thread, in units of the lowest of these binades (a 64-bit shared-memory
+            // atomic is a compare-and-swap loop, and thousands of them on one bin take turns).
+            s_bins[threadIdx.x] = 0ll;
+            __syncthreads();
+            const uint32_t thr_bits = bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
+            const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
+            long long acc_a = 0;
+            constexpr int kLoads = 4;  // list entries in flight per thread
+            for (uint32_t base = threadIdx.x; base < view.total; base += kBlock * kLoads) {
+                unsigned long long e[kLoads];
+#pragma unroll
+                for (int j = 0; j < kLoads; ++j) e[j] = (base + j * kBlock < view.total) ? view.at(base + j * kBlock) : 0ull;
+#pragma unroll
+                for (int j = 0; j < kLoads; ++j) {
+                    if (base + j * kBlock >= view.total || e[j] < thr) continue;
+                    const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(e[j] >> 32)));
+                    const uint32_t ex = (bits >> 23) & 0xffu;
+                    int m = (int)(bits & 0x7fffffu) | (ex ? 0x800000 : 0);
+                    if (bits >> 31) m = -m;
+                    const int bin = ex ? (int)ex - 1 : 0;
+                    const uint32_t up = (uint32_t)(bin - bin_a);
+                    if (up < 8u) acc_a += (long long)m << up;  // |m| < 2^24: at most 2^31 per entry
+                    else atomicAdd(reinterpret_cast<unsigned long long*>(&s_bins[bin]), (unsigned long long)(long long)m);
+                }
+            }
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) acc_a += __shfl_down_sync(0xffffffffu, acc_a, d);
+            if (lane_id() == 0 && acc_a)
+                atomicAdd(reinterpret_cast<unsigned long long*>(&s_bins[bin_a]), (unsigned long long)acc_a);
+            __syncthreads();
+            bins_nonzero_masks(s_bins[threadIdx.x], s_nonzero);
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                const double sum = bins_to_double(s_bins, s_nonzero);
+                ctl->thr[s] = thr;
+                ctl->mu64[s] = s ? -sum / (double)P.k : sum / (double)P.k;  // val- holds the negated entries
+            }
+        }
+    }
+    // ---- the block that gets here second goes on alone
+    if (!last_block_ticket(&ctl->done[ST_SUM], 2u)) return;
+    if (__ldcg(&ctl->status) != 0u) {
+        if (threadIdx.x == 0) write_header(P, ctl, false, 0ull);
+        return;
+    }
+    const double mu_pos = __ldcg(&ctl->mu64[0]), mu_neg = __ldcg(&ctl->mu64[1]);
+    const uint32_t side = (mu_pos >= mu_neg) ? 0u : 1u;
+    const float mu = side ? (float)(-mu_neg) : (float)mu_pos;
+    const uint32_t k = (uint32_t)P.k;
+    if (threadIdx.x == 0) {
+        ctl->side = side;
+        ctl->mu32 = mu;
+        ctl->k_final = k;
+        if (P.out_mu) *P.out_mu = mu;
+        s_count = 0u;
+    }
+    // ---- kept positions of the chosen side, ascending: gathered into shared memory in any order,
+    // padded with 0xffffffff, sorted in registers (thread t ends up with positions 16 t .. 16 t + 15
+    // of the ascending list, which are the codewords it writes below)
+    for (uint32_t i = threadIdx.x; i < kSmallKept; i += kBlock) s_pos[i] = 0xffffffffu;
+    __syncthreads();
+    {
+        const CandView view = cand_view(P, ctl, (int)side);
+        const unsigned long long thr = __ldcg(&ctl->thr[side]);
+        constexpr int kLoads = 4;  // list entries in flight per thread
+        for (uint32_t base = 0; base < view.total; base += kBlock * kLoads) {
+            unsigned long long e[kLoads];
+#pragma unroll
+            for (int j = 0; j < kLoads; ++j) {
+                const uint32_t i = base + j * kBlock + threadIdx.x;
+                e[j] = (i < view.total) ? view.at(i) : 0ull;
+            }
+#pragma unroll
+            for (int j = 0; j < kLoads; ++j) {  // one slot reservation per warp and step
+                const bool kept = base + j * kBlock + threadIdx.x < view.total && e[j] >= thr;
+                const unsigned mask = __ballot_sync(0xffffffffu, kept);
+                uint32_t first = 0u;
+                if (lane_id() == 0 && mask) first = atomicAdd(&s_count, (uint32_t)__popc(mask));
+                first = __shfl_sync(0xffffffffu, first, 0);
+                const uint32_t slot = first + (uint32_t)__popc(mask & ((1u << lane_id()) - 1u));
+                if (kept && slot < kSmallKept) s_pos[slot] = composite_index(e[j]);
+            }
+        }
+    }
+    __syncthreads();
+    if (s_count != k) {  // uniform
+        if (threadIdx.x == 0) {
+            atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            write_header(P, ctl, false, 0ull);
+        }
+        return;
+    }
+    constexpr int kCw = 16;  // codewords per thread, consecutive
+    uint32_t pos[kCw];
+#pragma unroll
+    for (int r = 0; r < kCw; ++r) pos[r] = s_pos[r * kBlock + threadIdx.x];
+    __syncthreads();
+    block_sort_16(pos, s_pos);
+    const uint32_t i0 = threadIdx.x * kCw;
+#pragma unroll
+    for (int j = 0; j < kCw; ++j) s_pos[i0 + j] = pos[j];  // the ascending list, for the neighbours and the chunk table
+    __syncthreads();
+    // ---- residual write-back, code lengths, bit offsets, payload, chunk table, header
+    const int b = P.b;
+    uint32_t gap[kCw];
+    float r[kCw];
+    unsigned long long len_sum = 0ull;
+#pragma unroll
+    for (int j = 0; j < kCw; ++j) r[j] = (i0 + j < k) ? P.residual[pos[j]] : 0.f;  // all loads in flight together
+    long long prev = i0 ? (long long)s_pos[i0 - 1] : -1ll;
+#pragma unroll
+    for (int j = 0; j < kCw; ++j) {
+        const uint32_t i = i0 + j;
+        gap[j] = 0u;
+        if (i < k) {
+            P.residual[pos[j]] = __fsub_rn(r[j], mu);
+            P.idx[i] = pos[j];
+            gap[j] = (uint32_t)((long long)pos[j] - prev - 1);
+            prev = (long long)pos[j];
+            len_sum += (unsigned long long)(gap[j] >> b) + 1ull + (unsigned long long)b;
+        }
+    }
+    unsigned long long nbits;
+    unsigned long long off = block_exclusive_scan<unsigned long long>(len_sum, s_scan64, &nbits);
+    uint32_t* words = reinterpret_cast<uint32_t*>(P.stream + P.payload_offset);
+    uint8_t* table = P.stream + SBC_HEADER_BYTES;
+    // A payload of at most 2048 words is put together in shared memory (the histogram's, free by
+    // now) and stored once: thousands of atomics from one block on global memory take longer
+    // than everything else here.  Longer payloads are ORed into the zeroed stream directly.
+    const bool in_shared = nbits <= 32ull * kHistBins;  // uniform
+    if (in_shared) {
+        for (int w = threadIdx.x; w < kHistBins; w += kBlock) s_hist[w] = 0u;
+        __syncthreads();
+    }
+    uint32_t* target = in_shared ? s_hist : words;
+#pragma unroll
+    for (int j = 0; j < kCw; ++j) {
+        const uint32_t i = i0 + j;
+        if (i < k) {
+            pack_codeword(target, table, i, off, gap[j], b, s_pos);
+            off += (unsigned long long)(gap[j] >> b) + 1ull + (unsigned long long)b;
+        }
+    }
+    if (in_shared) {
+        __syncthreads();
+        const uint32_t n_words = (uint32_t)((nbits + 31ull) >> 5);
+        for (uint32_t w = threadIdx.x; w < n_words; w += kBlock) words[w] = s_hist[w];
+    }
+    if (threadIdx.x == 0) {
+        ctl->kept_total = k;
+        write_header(P, ctl, true, nbits);
+    }
+}
+
+}  // namespace sbc

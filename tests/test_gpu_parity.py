@@ -95,6 +95,30 @@ def test_encode_ragged_sizes(n, p):
     check_against_oracle(upd, res, p)
 
 
+# Problems whose candidate lists hold at most 8192 entries and that keep at most 4096 positions are
+# finished by one kernel (two blocks per problem); the cases sit on both sides of those two limits,
+# with smooth and with tie-heavy values.
+@pytest.mark.parametrize("n,p", [
+    (358400, 0.01),    # k = 3584, capacity 8192: the largest problem of the short-list form
+    (358500, 0.01),    # k = 3585, capacity 8194: just beyond it
+    (8192, 0.5),       # k = 4096 = the most positions one block orders, capacity = n
+    (8192, 0.6),       # k = 4915: short lists, but too many kept positions for one block
+    (8193, 0.45),      # capacity 8193 > 8192 with k below 4096
+    (4096, 0.999),     # nearly everything kept
+    (5000, 0.3), (70001, 0.05), (3_000_000, 0.001), (3_584_000, 0.001), (3_585_000, 0.001),
+])
+@pytest.mark.parametrize("kind", ["normal", "few_values"])
+def test_short_list_form_and_its_limits(n, p, kind):
+    rng = np.random.default_rng(zlib.crc32(f"{n}/{p}/{kind}".encode()))
+    if kind == "normal":
+        upd = rng.standard_normal(n).astype(np.float32) * np.float32(1e-3)
+        res = rng.standard_normal(n).astype(np.float32) * np.float32(1e-3)
+    else:  # a handful of distinct values: the thresholds fall inside long runs of equal entries
+        upd = rng.integers(-3, 4, size=n).astype(np.float32) * np.float32(0.25)
+        res = rng.integers(-1, 2, size=n).astype(np.float32) * np.float32(0.5)
+    check_against_oracle(upd, res, p)
+
+
 @pytest.mark.parametrize("offset", [1, 2, 3])
 def test_encode_misaligned_pointers(offset):
     rng = np.random.default_rng(offset)

@@ -266,11 +266,11 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
 
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
 // a single problem) say how each kind of work is spread over the problems.
-void launch_encode(const Prob* d_probs, uint32_t n_probs, const unsigned grid[WK_COUNT],
+void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, const unsigned grid[WK_COUNT],
                    const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, bool small_kept, cudaStream_t st,
                    const sbc_cuda_event_t* marks) {
     auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
-    auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs}; };
+    auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs, any_exact}; };
     auto g1 = [&](int kind) { return dim3(grid[kind]); };
     auto g2 = [&](int kind) { return dim3(grid[kind], 1, 2); };  // z = side
     // Every kernel is launched with programmatic stream serialisation: its blocks may be placed
@@ -416,7 +416,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, 1u, 1u, grid);
-    launch_encode(d_prob, 1u, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, pl.k <= (long long)kSmallKept, st, marks);
+    launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, pl.k <= (long long)kSmallKept, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -553,13 +553,13 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         d_rows[kind] = d_prefix + (size_t)kind * row_len;
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
-    k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors});
+    k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors, nullptr});
     bool small_lists = true, small_kept = true;
     for (int t = 0; t < n_tensors; ++t) {
         small_lists = small_lists && plans[t].cap <= kSmallList;
         small_kept = small_kept && plans[t].k <= (long long)kSmallKept;
     }
-    launch_encode(d_probs, (uint32_t)n_tensors, grid, d_rows, kModeBinary, false, small_lists, small_kept, st, nullptr);
+    launch_encode(d_probs, (uint32_t)n_tensors, &probs[0].ctl->launch_exact, grid, d_rows, kModeBinary, false, small_lists, small_kept, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

@@ -42,6 +42,7 @@ enum Stage : int {
 struct Ctl {
     uint32_t status;            // SBC_STATUS_* bits
     uint32_t use_fallback;      // 1: the candidate pass did not bracket both thresholds
+    uint32_t launch_exact;      // in the launch's first problem: some problem of the launch has use_fallback set
     uint32_t done[ST_COUNT];    // tickets for the last-block pattern
     // threshold bounds from the sample
     uint32_t s_bin0[2], s_rank[2];
@@ -128,6 +129,7 @@ struct Batch {
     const Prob* probs;
     const uint32_t* prefix;  // n_probs + 1 entries, or nullptr
     uint32_t n_probs;
+    uint32_t* any_exact;     // one word per launch: non-zero once a problem needs the exact route
 };
 struct Slot {
     const Prob* P;
@@ -180,6 +182,14 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
     s.P = s_prob;
     s.G = const_cast<Prob*>(src);
     return s;
+}
+
+// First lines of the exact-route kernels: false (for the whole grid) when no problem of the launch
+// needs them, which is the usual case, so that they end before looking for their problem.
+__device__ __forceinline__ bool launch_needs_exact_route(const Batch& B) {
+    cudaTriggerProgrammaticLaunchCompletion();
+    cudaGridDependencySynchronize();
+    return __ldcg(B.any_exact) != 0u;
 }
 
 // Kinds of work a kernel's grid is sized by (one prefix table per kind in a batch).

@@ -16,6 +16,7 @@ __device__ __forceinline__ bool exact_route_active(const Ctl* ctl) {
 // sides; the last block extends the two prefixes.
 template <int LEVEL>
 __global__ void __launch_bounds__(kBlock) k_exact_hist(const Batch B) {
+    if (B.prefix != nullptr && !launch_needs_exact_route(B)) return;  // batch: before looking for the block's problem
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -90,6 +91,7 @@ __device__ __forceinline__ bool tie_ranks_needed(const Ctl* ctl, int s) {
 
 // Entries equal to the threshold, per tile of kXTile elements.
 __global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Batch B) {
+    if (B.prefix != nullptr && !launch_needs_exact_route(B)) return;  // batch: before looking for the block's problem
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -120,6 +122,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiecount(const Batch B) {
 
 // In-place exclusive scan of the per-tile tie counts (one block).
 __global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Batch B) {
+    if (B.prefix != nullptr && !launch_needs_exact_route(B)) return;  // batch: before looking for the block's problem
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -149,6 +152,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Batch B) {
 // elements of a tile and walks them 32 at a time, so the rank of a tie is
 // (ties in earlier tiles) + (earlier warps) + (earlier steps) + (lower lanes).
 __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
+    if (B.prefix != nullptr && !launch_needs_exact_route(B)) return;  // batch: before looking for the block's problem
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;

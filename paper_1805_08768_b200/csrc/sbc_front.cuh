@@ -402,6 +402,7 @@ __global__ void __launch_bounds__(kBlock, 4) k_add_collect(const Batch B) {
             const bool ok = c0 >= need && c0 <= P.cap &&
                             (MODE == kModeValues || (c1 >= need && c1 <= P.cap));
             ctl->use_fallback = ok ? 0u : 1u;
+            if (!ok) atomicOr(B.any_exact, 1u);
             ctl->sampled_ok = (ok && P.sampled) ? 1u : 0u;
         }
     }

@@ -254,7 +254,9 @@ int sbc_encode_ex(const float *update, float *residual, int64_t numel, double p,
                   void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream,
                   const sbc_cuda_event_t *marks);
 
-/* Number of kernels one sbc_encode call launches (memsets not counted), and
+/* Number of kernels one sbc_encode call launches for a tensor whose candidate
+ * lists are longer than one thread block handles (memsets not counted; a tensor
+ * with 2*k + 1024 <= 8192 and k <= 4096 takes a shorter chain of 11), and
  * one sbc_decode_accumulate call for n_clients streams. */
 int sbc_encode_launches(void);
 int sbc_decode_launches(int n_clients);

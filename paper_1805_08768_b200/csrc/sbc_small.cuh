@@ -302,7 +302,7 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
     for (int j = 0; j < kCw; ++j) {
         const uint32_t i = i0 + j;
         if (i < k) {
-            pack_codeword(target, table, i, off, gap[j], b, s_pos);
+            pack_codeword(target, 0ull, table, i, off, gap[j], b, s_pos);
             off += (unsigned long long)(gap[j] >> b) + 1ull + (unsigned long long)b;
         }
     }

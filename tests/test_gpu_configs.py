@@ -216,3 +216,54 @@ def test_batch_and_single_tensor_calls_agree_with_mixed_sparsities():
     # a bad descriptor anywhere in the batch: nothing runs
     with pytest.raises(sbc.SbcError):
         sbc.sbc_encode_batch(d_up, d_res, ps[:-1] + [1.5], outs, mus, ws)
+
+
+@pytest.mark.parametrize("seed", [1, 2, 3])
+def test_batch_of_short_list_problems_with_ties_zeros_and_a_bad_tensor(seed):
+    # every tensor keeps at most 3584 positions, so the whole batch takes the one-kernel back half;
+    # it holds tie-heavy, one-signed and all-zero tensors and one tensor with a NaN, whose header must
+    # carry the error while its neighbours are encoded as usual
+    rng = np.random.default_rng(900 + seed)
+    n_tensors = 48
+    sizes, ps, ups, res0 = [], [], [], []
+    for t in range(n_tensors):
+        p = float(10.0 ** rng.uniform(-3.3, -0.4))
+        k_max = 3584
+        n = int(rng.integers(1, min(400000, int(k_max / p))))
+        kind = t % 6
+        if kind == 0:
+            u = rng.standard_normal(n)
+        elif kind == 1:
+            u = np.round(rng.standard_normal(n) * 2) / 2          # few distinct values
+        elif kind == 2:
+            u = np.zeros(n)                                        # exact route, mu = 0
+        elif kind == 3:
+            u = -np.abs(rng.standard_t(3, n))                      # one-signed
+        elif kind == 4:
+            u = rng.standard_normal(n) * (rng.random(n) < 0.02)    # mostly zeros
+        else:
+            u = rng.laplace(size=n)
+        sizes.append(n)
+        ps.append(p)
+        ups.append((u * 10.0 ** rng.integers(-5, 2)).astype(np.float32))
+        res0.append((rng.standard_normal(n) * 1e-4).astype(np.float32) if t % 2 else np.zeros(n, dtype=np.float32))
+    bad = 17
+    ups[bad][ups[bad].size // 2] = np.nan
+    want_res = [r.copy() for r in res0]
+    want = [None if t == bad else oracle.encode(ups[t], want_res[t], ps[t]) for t in range(n_tensors)]
+    d_up = [torch.from_numpy(u).to(DEV) for u in ups]
+    d_res = [torch.from_numpy(r).to(DEV) for r in res0]
+    outs = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=DEV) for n, p in zip(sizes, ps)]
+    mus = [torch.empty(1, dtype=torch.float32, device=DEV) for _ in sizes]
+    ws = torch.empty(sbc.sbc_workspace_bytes_batch(sizes, ps), dtype=torch.uint8, device=DEV)
+    sbc.sbc_encode_batch(d_up, d_res, ps, outs, mus, ws)
+    torch.cuda.synchronize()
+    for t in range(n_tensors):
+        if t == bad:
+            info = sbc.sbc_stream_info_get(outs[t], check=False)
+            assert info.status & sbc.STATUS_NONFINITE and info.k == 0
+            continue
+        info = sbc.sbc_stream_info_get(outs[t])
+        assert np.array_equal(outs[t][: info.total_bytes].cpu().numpy(), want[t][0]), f"tensor {t} (n={sizes[t]}, p={ps[t]})"
+        assert np.float32(mus[t].item()).view(np.uint32) == want[t][1].view(np.uint32), f"tensor {t}"
+        assert np.array_equal(d_res[t].cpu().numpy().view(np.uint32), want_res[t].view(np.uint32)), f"tensor {t}"

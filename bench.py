@@ -360,15 +360,24 @@ def run_network_shapes(torch, sbc, workloads, dev):
              workloads.resnet50_update),
             ("word_lstm_shapes_p1e-2", [int(np.prod(s)) for _, s in workloads.word_lstm_shapes()], 1e-2,
              workloads.word_lstm_update)):
-        ups = [torch.from_numpy(u).to(dev) for u in gen(1)]
+        n_clients = 8
         res = [torch.zeros(n, dtype=torch.float32, device=dev) for n in sizes]
-        outs = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=dev) for n in sizes]
         mus = [torch.empty(1, dtype=torch.float32, device=dev) for _ in sizes]
         ws = torch.empty(sbc.sbc_workspace_bytes_batch(sizes, [p] * len(sizes)), dtype=torch.uint8, device=dev)
-        enc = sbc.EncodeBatch(ups, res, [p] * len(sizes), outs, mus, ws)
+        # one message per client and tensor, from eight different seeded updates (zero residual each)
+        client_outs = []
+        for c in range(n_clients):
+            ups = [torch.from_numpy(u).to(dev) for u in gen(1 + c)]
+            for r in res:
+                r.zero_()
+            outs = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=dev) for n in sizes]
+            sbc.EncodeBatch(ups, res, [p] * len(sizes), outs, mus, ws).run()
+            torch.cuda.synchronize()
+            client_outs.append(outs)
+        enc = sbc.EncodeBatch(ups, res, [p] * len(sizes), client_outs[-1], mus, ws)  # timed: the last client's round
         dense = [torch.zeros(n, dtype=torch.float32, device=dev) for n in sizes]
         dws = torch.empty(sbc.sbc_decode_workspace_bytes_batch(len(sizes)), dtype=torch.uint8, device=dev)
-        dec = sbc.DecodeBatch([[o] * 8 for o in outs], dense, dws)
+        dec = sbc.DecodeBatch([[client_outs[c][t] for c in range(n_clients)] for t in range(len(sizes))], dense, dws)
 
         def timed(fn, reps=10):
             for _ in range(3):

@@ -59,7 +59,8 @@ __device__ __forceinline__ uint32_t add_at(float* p, float mu, bool ieee_path) {
 }
 
 constexpr int kDecodeThreads = 64;            // two warps per block
-constexpr int kDecodeWarpWords = 5632;        // staged payload words per warp (22 KB)
+constexpr int kDecodeWarpWords = 4608;        // staged payload words per warp (18 KB)
+constexpr uint32_t kInOrderChunks = 8192;     // streams from this many chunks (2 M positions) on add in list order
 
 // Sequential MSB-first bit reader over a warp's staged (byte-swapped) words, or over global memory when the group's payload did not fit the stage.
 // `cur` holds the next 64 - (32 - avail) ... bits left-aligned: bits [63, 64-avail)
@@ -103,6 +104,56 @@ struct BitReader {
     }
 };
 
+// One codeword from the warp's staged (MSB-first) words at relative bit `rel`: q ones, a zero,
+// b remainder bits (Algorithm 4).  Bit positions relative to the stage fit 32 bits and the
+// codeword is cut out of a 64-bit window rebuilt from three staged words.  The common case (fewer
+// than 32 ones, everything in range) is decided by ONE predicate and runs without any other branch;
+// long unary runs and every kind of error take the general step.  On success returns 0, advances
+// `rel`, sets *at to the decoded position and `nxt` to the position after it; else an error status.
+__device__ __forceinline__ uint32_t parse_staged(const uint32_t* sw, uint32_t& rel, uint32_t rel_end, uint32_t b,
+                                                 uint32_t n32, uint32_t& nxt, uint32_t* at) {
+    uint32_t w = rel >> 5;
+    const int sh = (int)(rel & 31u);
+    const uint32_t x0 = sw[w], x1 = sw[w + 1], x2 = sw[w + 2];
+    uint32_t hi = __funnelshift_l(x1, x0, sh);
+    uint32_t lo = __funnelshift_l(x2, x1, sh);
+    uint32_t ones = __clz(~hi);
+    const uint32_t q_max = n32 >> b;  // a larger quotient cannot stay inside the tensor
+    {
+        const unsigned long long win = ((unsigned long long)hi << 32) | (unsigned long long)lo;
+        const uint32_t r = (uint32_t)(((win << (ones & 31u) << 1) >> 1) >> (63u - b));  // b bits after the zero
+        const uint32_t stp = (ones << b) + r;       // meaningful when ones <= q_max: no overflow then
+        const bool ok = (rel < rel_end) & (ones < 32u) & (ones <= q_max) & (stp < n32 - nxt);
+        if (ok) {
+            *at = nxt + stp;
+            nxt = *at + 1u;
+            rel += ones + 1u + b;
+            return 0u;
+        }
+    }
+    // general step: a run of 32 or more ones, or something is wrong
+    if (rel >= rel_end) return SBC_STATUS_CORRUPT;
+    unsigned long long q = ones;
+    while (ones == 32u) {
+        rel += 32u;
+        if (rel >= rel_end) break;
+        w = rel >> 5;
+        hi = __funnelshift_l(sw[w + 1], sw[w], sh);
+        lo = __funnelshift_l(sw[w + 2], sw[w + 1], sh);
+        ones = __clz(~hi);
+        q += ones;
+    }
+    if (rel >= rel_end) return SBC_STATUS_CORRUPT;
+    const unsigned long long win = ((unsigned long long)hi << 32) | (unsigned long long)lo;
+    const uint32_t r = b ? (uint32_t)((win << (ones + 1u)) >> (64u - b)) : 0u;
+    rel += ones + 1u + b;
+    const unsigned long long step = (q << b) + r;
+    if (q > (unsigned long long)n32 || (unsigned long long)(n32 - nxt) <= step) return SBC_STATUS_RANGE;
+    *at = nxt + (uint32_t)step;
+    nxt = *at + 1u;
+    return 0u;
+}
+
 // One warp per group of 32 consecutive chunks: the group's payload is one
 // contiguous bit range, copied once (coalesced) into shared memory; then every
 // lane parses its chunk's kChunkCodewords codewords from there (Algorithm 4)
@@ -111,6 +162,8 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
     __shared__ StreamView s_view[kMaxClientsPerLaunch];
     __shared__ uint32_t s_first[kMaxClientsPerLaunch + 1];  // first work item (group) of each client
     __shared__ uint32_t s_words[kDecodeThreads / 32][kDecodeWarpWords];
+    __shared__ uint32_t s_at[kDecodeThreads / 32][32][33];  // decoded positions of a step, [chunk lane][codeword], padded
+    __shared__ uint32_t s_n[kDecodeThreads / 32][32];       // how many each lane decoded in the step
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     if (tid < args.n_clients) {
         const uint8_t* h = args.streams[tid];
@@ -188,86 +241,91 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
         for (uint32_t i = lane; i < n_staged; i += 32) sw[i] = __byte_perm(sw[i], 0u, 0x0123);
         if (staged && lane < 2) sw[n_staged + lane] = 0u;
         __syncwarp();
-        if (has && !err) {
+        // Plain sums (one value per stream, no second target, no tiny value) of long streams are
+        // added in list order: every lane parses 32 codewords of its chunk into shared memory, then
+        // the warp adds chunk after chunk, one instruction covering 32 neighbouring positions of the
+        // tensor.  Lanes that add as they parse send each instruction to 32 places a chunk apart,
+        // and DRAM serves neighbours that arrive together far better: 0.44 -> 0.40 ms for 10.7 M
+        // positions over 4 GiB.  Short streams are bound by the latency of a chunk's serial parse
+        // instead, which the extra step lengthens (60 -> 63 us at 1 M positions), so only streams
+        // of at least kInOrderChunks chunks are decoded this way.
+        const float mu_w = __fmul_rn(v.mu, args.scale);
+        const bool in_order = staged && v.n_chunks >= kInOrderChunks && v.values == nullptr &&
+                              args.momentum == nullptr && !(fabsf(mu_w) < 7.888609052e-31f);  // warp-uniform
+        if (in_order) {
+            uint32_t count = 0u, rel = 0u, rel_end = 0u, nxt = 0u, done = 0u;
+            const uint32_t n32 = (uint32_t)args.n;
+            bool live = has && !err;
+            if (live) {
+                const unsigned long long first_cw = (unsigned long long)chunk * kChunkCodewords;
+                count = (uint32_t)min((unsigned long long)kChunkCodewords, v.k - first_cw);
+                if (pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n) {
+                    err = SBC_STATUS_CORRUPT;
+                    live = false;
+                }
+                rel = (uint32_t)(pos - (first_word << 5));
+                rel_end = (uint32_t)(gend - (first_word << 5));
+                nxt = (uint32_t)(prev + 1);
+            }
+            const bool checked = live;  // the end of the chunk is compared with the table below
+            for (int step = 0; step < kChunkCodewords / 32; ++step) {
+                if (!__any_sync(0xffffffffu, live && done < count)) break;  // warp-uniform
+                uint32_t got = 0u;
+                if (live) {
+                    const uint32_t lim = min(32u, count - done);
+                    for (; got < lim; ++got) {
+                        uint32_t at;
+                        const uint32_t bad = parse_staged(sw, rel, rel_end, v.b, n32, nxt, &at);
+                        if (bad) { err = bad; live = false; break; }
+                        s_at[warp][lane][got] = at;
+                    }
+                    done += got;
+                }
+                s_n[warp][lane] = got;
+                __syncwarp();
+#pragma unroll 4
+                for (int c = 0; c < 32; ++c)
+                    if ((uint32_t)lane < s_n[warp][c]) atomicAdd(args.out + s_at[warp][c][lane], mu_w);
+                __syncwarp();
+            }
+            if (checked && !err) {
+                // the chunk must end exactly where the table says the next one starts
+                const unsigned long long end_pos = (first_word << 5) + rel;
+                const long long end_prev = (long long)nxt - 1;
+                if (chunk + 1u < v.n_chunks) {
+                    if (load_u64(e + SBC_CHUNK_ENTRY_BYTES) != end_pos ||
+                        (long long)load_u64(e + SBC_CHUNK_ENTRY_BYTES + 8) != end_prev)
+                        err = SBC_STATUS_CORRUPT;
+                } else if (end_pos != v.nbits) {
+                    err = SBC_STATUS_CORRUPT;
+                }
+            }
+        } else if (has && !err) {
             const unsigned long long first_cw = (unsigned long long)chunk * kChunkCodewords;
             const uint32_t count = (uint32_t)min((unsigned long long)kChunkCodewords, v.k - first_cw);
-            if (pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n) err = SBC_STATUS_CORRUPT;
+            const bool entry_ok = !(pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n);
+            if (!entry_ok) err = SBC_STATUS_CORRUPT;
             const uint32_t b = v.b;
             const float mu = __fmul_rn(v.mu, args.scale);
             float* __restrict__ momentum = args.momentum;
             const float* __restrict__ vals = v.values ? v.values + (size_t)chunk * kChunkCodewords : nullptr;
             const bool tiny = fabsf(mu) < 7.888609052e-31f;  // 2^-100
-            if (staged) {
-                // Fast path: bit positions relative to the stage fit 32 bits; every codeword
-                // is cut out of a 64-bit window rebuilt from three staged words.  The common
-                // case (fewer than 32 ones, everything in range) is decided by ONE predicate per
-                // codeword and runs without any other branch; long unary runs and every kind of
-                // error take the general step below.
+            if (!entry_ok) {
+                // nothing is decoded from a chunk whose table entry is out of range
+            } else if (staged) {
                 uint32_t rel = (uint32_t)(pos - (first_word << 5));
                 const uint32_t rel_end = (uint32_t)(gend - (first_word << 5));
                 const uint32_t n32 = (uint32_t)args.n;
-                const uint32_t q_max = n32 >> b;          // a larger quotient cannot stay inside the tensor
                 uint32_t nxt = (uint32_t)(prev + 1);      // first position the next codeword can name
-                float* __restrict__ out = args.out;
-                const bool plain = vals == nullptr && momentum == nullptr && !tiny;  // warp-uniform
                 for (uint32_t i = 0; i < count; ++i) {
-                    uint32_t w = rel >> 5;
-                    const int sh = (int)(rel & 31u);
-                    const uint32_t x0 = sw[w], x1 = sw[w + 1], x2 = sw[w + 2];
-                    uint32_t hi = __funnelshift_l(x1, x0, sh);
-                    uint32_t lo = __funnelshift_l(x2, x1, sh);
-                    uint32_t ones = __clz(~hi);
-                    {
-                        const unsigned long long win = ((unsigned long long)hi << 32) | (unsigned long long)lo;
-                        const uint32_t r = (uint32_t)(((win << (ones & 31u) << 1) >> 1) >> (63u - b));  // b bits after the zero
-                        const uint32_t stp = (ones << b) + r;       // meaningful when ones <= q_max: no overflow then
-                        const bool ok = (rel < rel_end) & (ones < 32u) & (ones <= q_max) & (stp < n32 - nxt);
-                        if (ok) {
-                            const uint32_t at = nxt + stp;
-                            nxt = at + 1u;
-                            rel += ones + 1u + b;
-                            if (plain) {
-                                atomicAdd(out + at, mu);
-                            } else {
-                                if (vals) {
-                                    const float x = __fmul_rn(vals[i], args.scale);
-                                    err |= add_at(out + at, x, fabsf(x) < 7.888609052e-31f);
-                                } else {
-                                    err |= add_at(out + at, mu, tiny);
-                                }
-                                if (momentum) momentum[at] = 0.f;
-                            }
-                            continue;
-                        }
-                    }
-                    // general step: a run of 32 or more ones, or something is wrong
-                    if (rel >= rel_end) { err = SBC_STATUS_CORRUPT; break; }
-                    unsigned long long q = ones;
-                    while (ones == 32u) {
-                        rel += 32u;
-                        if (rel >= rel_end) break;
-                        w = rel >> 5;
-                        hi = __funnelshift_l(sw[w + 1], sw[w], sh);
-                        lo = __funnelshift_l(sw[w + 2], sw[w + 1], sh);
-                        ones = __clz(~hi);
-                        q += ones;
-                    }
-                    if (rel >= rel_end) { err = SBC_STATUS_CORRUPT; break; }
-                    const unsigned long long win = ((unsigned long long)hi << 32) | (unsigned long long)lo;
-                    const uint32_t r = b ? (uint32_t)((win << (ones + 1u)) >> (64u - b)) : 0u;
-                    rel += ones + 1u + b;
-                    const unsigned long long step = (q << b) + r;
-                    if (q > (unsigned long long)args.n || (unsigned long long)(n32 - nxt) <= step) {
-                        err = SBC_STATUS_RANGE;
-                        break;
-                    }
-                    const uint32_t at = nxt + (uint32_t)step;
-                    nxt = at + 1u;
+                    uint32_t at;
+                    const uint32_t bad = parse_staged(sw, rel, rel_end, b, n32, nxt, &at);
+                    if (bad) { err = bad; break; }
                     if (vals) {
                         const float x = __fmul_rn(vals[i], args.scale);
-                        err |= add_at(out + at, x, fabsf(x) < 7.888609052e-31f);
+                        err |= add_at(args.out + at, x, fabsf(x) < 7.888609052e-31f);
                     } else {
-                        err |= add_at(out + at, mu, tiny);
+                        err |= add_at(args.out + at, mu, tiny);
                     }
                     if (momentum) momentum[at] = 0.f;
                 }

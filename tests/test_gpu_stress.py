@@ -166,3 +166,44 @@ def test_largest_tensor_the_interface_accepts():
     assert bool((dense[kept] == float(mu)).all())
     dense[kept] = 0.0
     assert not bool(dense.any())
+
+
+def test_long_stream_is_decoded_in_list_order_and_rejects_damage():
+    # 3.3 M positions (13 108 chunks): long enough for the decoder's in-order form, in which a warp
+    # parses 32 codewords per chunk into shared memory and then adds chunk after chunk
+    n, p = 1 << 25, 0.1
+    rng = np.random.default_rng(4242)
+    upd = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    u = torch.from_numpy(upd).to(DEV)
+    r = torch.zeros(n, dtype=torch.float32, device=DEV)
+    out, mu = sbc.sbc_encode(u, r, p)
+    info = sbc.sbc_stream_info_get(out)
+    assert info.n_chunks >= 8192
+    stream = out[: info.total_bytes].cpu().numpy()
+    want = np.full(n, 0.25, dtype=np.float32)
+    oracle.decode_accumulate([stream], want)         # Algorithm 4 on the CPU, onto existing contents
+    guard = 4096
+
+    def run(mutated: np.ndarray):
+        dense = torch.zeros(n + 2 * guard, dtype=torch.float32, device=DEV)
+        dense[guard:guard + n] = 0.25
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        sbc.sbc_decode_accumulate([torch.from_numpy(mutated).to(DEV)], dense[guard:guard + n], status=status)
+        torch.cuda.synchronize()
+        assert not bool(dense[:guard].any()) and not bool(dense[guard + n:].any()), "decoder wrote outside the tensor"
+        return status.item(), dense[guard:guard + n]
+
+    status, dense = run(stream)
+    assert status == 0
+    assert np.array_equal(dense.cpu().numpy().view(np.uint32), want.view(np.uint32))
+    table = 64                                          # chunk table: 16 bytes per chunk after the 64-byte header
+    bad = stream.copy(); bad[info.payload_offset + 100000] ^= 0x10      # one payload bit in the middle
+    assert run(bad)[0] != 0
+    bad = stream.copy(); bad[info.payload_offset + 5000: info.payload_offset + 5064] = 0xFF   # a long run of ones
+    assert run(bad)[0] != 0
+    bad = stream.copy(); bad[table + 16 * 777 + 8: table + 16 * 777 + 16].view("<i8")[0] = n + 5   # previous position beyond the tensor
+    assert run(bad)[0] & sbc.STATUS_CORRUPT
+    bad = stream.copy(); bad[table + 16 * 4000: table + 16 * 4000 + 8].view("<u8")[0] += 3         # chunk offset off by three bits
+    assert run(bad)[0] != 0
+    bad = stream.copy(); bad[table + 16 * 9000 + 8: table + 16 * 9000 + 16].view("<i8")[0] = 2**40  # absurd previous position
+    assert run(bad)[0] & sbc.STATUS_CORRUPT

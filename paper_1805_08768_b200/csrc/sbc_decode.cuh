@@ -317,10 +317,16 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                 const uint32_t rel_end = (uint32_t)(gend - (first_word << 5));
                 const uint32_t n32 = (uint32_t)args.n;
                 uint32_t nxt = (uint32_t)(prev + 1);      // first position the next codeword can name
+                float* __restrict__ out = args.out;
+                const bool plain = vals == nullptr && momentum == nullptr && !tiny;  // warp-uniform
                 for (uint32_t i = 0; i < count; ++i) {
                     uint32_t at;
                     const uint32_t bad = parse_staged(sw, rel, rel_end, b, n32, nxt, &at);
                     if (bad) { err = bad; break; }
+                    if (plain) {  // the usual case: nothing but the add in the loop
+                        atomicAdd(out + at, mu);
+                        continue;
+                    }
                     if (vals) {
                         const float x = __fmul_rn(vals[i], args.scale);
                         err |= add_at(args.out + at, x, fabsf(x) < 7.888609052e-31f);

@@ -296,8 +296,9 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
     go(k_sample1, g1(WK_SAMPLE), B(WK_SAMPLE));
     if (sampled) go(k_sample2, g1(WK_SAMPLE), B(WK_SAMPLE));
     mark(SBC_MARK_BOUNDS);
-    if (mode == kModeValues) go(k_add_collect<kModeValues>, g1(WK_MAIN), B(WK_MAIN), false);
-    else                     go(k_add_collect<kModeBinary>, g1(WK_MAIN), B(WK_MAIN), false);
+    // (a batch's streaming pass is made of many short blocks: there early placement helps)
+    if (mode == kModeValues) go(k_add_collect<kModeValues>, g1(WK_MAIN), B(WK_MAIN), prefix != nullptr);
+    else                     go(k_add_collect<kModeBinary>, g1(WK_MAIN), B(WK_MAIN), prefix != nullptr);
     mark(SBC_MARK_COLLECT);
 
     // 2. exact route over A (returns immediately unless the bounds failed)

@@ -64,6 +64,7 @@ struct Ctl {
     uint32_t b_rank[2];
     uint32_t list_cnt[2][6];
     unsigned long long thr[2];  // kept <=> composite >= thr[side]
+    uint32_t sel_done[2];       // thr[side] is final: the remaining selection kernels have nothing to do
     // sums and decision
     long long bins[2][256];
     double mu64[2];

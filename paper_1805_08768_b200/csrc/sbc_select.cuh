@@ -34,6 +34,62 @@ __device__ __forceinline__ int select_top(const Prob& P, const Ctl* ctl, int s, 
     return top;
 }
 
+// Rank `rank` (1 = largest) among the cnt <= PER * kBlock composites a block holds in registers
+// (slot j of thread t = entry j * kBlock + t), which agree in every digit before `first_level`
+// (`prefix` holds those digits).  Radix selection, 11-bit digits from bit `top` down, on
+// shared-memory histograms; stops at the first bucket with a single entry.  Returns false if the
+// histogram walk failed (inconsistent counts).  All threads call; result identical in all.
+template <int PER>
+__device__ __forceinline__ bool block_select_registers(const unsigned long long (&c)[PER], uint32_t cnt, uint32_t rank,
+                                                       int top, int first_level, unsigned long long prefix, uint32_t* s_hist,
+                                                       uint32_t* s_scan, Pick* s_pick, unsigned long long* s_result,
+                                                       unsigned long long* out) {
+    unsigned alive = 0u;  // entries that still match the prefix
+#pragma unroll
+    for (int j = 0; j < PER; ++j) alive |= ((uint32_t)j * kBlock + threadIdx.x < cnt) ? (1u << j) : 0u;
+    const int levels = digit_levels(top);
+    for (int level = first_level; level < levels; ++level) {
+        for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
+        __syncthreads();
+        // a thread's entries mostly share their leading digits: one atomic per run of equal digits
+        uint32_t run_digit = 0u, run_len = 0u;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            if ((alive >> j) & 1u) {
+                const uint32_t d = digit_of(c[j], level, top);
+                if (run_len && d != run_digit) { atomicAdd(&s_hist[run_digit], run_len); run_len = 0u; }
+                run_digit = d;
+                ++run_len;
+            }
+        }
+        if (run_len) atomicAdd(&s_hist[run_digit], run_len);
+        __syncthreads();
+        block_pick_desc<true>(s_hist, 1 << digit_bits(level, top), false, rank, s_scan, s_pick);
+        if (!s_pick->found) return false;  // uniform
+        const uint32_t sel = s_pick->bin;
+        const bool single = s_pick->count == 1u;
+        rank = s_pick->rank;
+        prefix |= (unsigned long long)sel << digit_shift(level, top);
+#pragma unroll
+        for (int j = 0; j < PER; ++j)
+            if (((alive >> j) & 1u) && digit_of(c[j], level, top) != sel) alive &= ~(1u << j);
+        if (single) {  // the one entry left is the answer; its owner publishes it
+#pragma unroll
+            for (int j = 0; j < PER; ++j)
+                if ((alive >> j) & 1u) *s_result = c[j];
+            __syncthreads();
+            *out = *s_result;
+            return true;
+        }
+        __syncthreads();  // s_pick and s_hist are reused
+    }
+    *out = prefix;  // every digit fixed
+    return true;
+}
+
+constexpr int kFinishPer = 8;  // entries per thread a selection kernel's last block finishes by itself
+constexpr uint32_t kFinishList = kFinishPer * kBlock;
+
 // Histogram of the top digit over a whole candidate list.  grid.z = side.
 __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     __shared__ Prob s_prob;
@@ -76,6 +132,23 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
         if (v) atomicAdd(&P.hists->b[0][s][i], v);
     }
     if (last_block_ticket(&ctl->done[ST_BH0_S0 + s], S.nb)) {
+        if (cnt <= kFinishList) {  // a short range: this block ranks it alone, the filter kernels return at once
+            __shared__ unsigned long long s_result;
+            unsigned long long c[kFinishPer], thr = 0ull;
+#pragma unroll
+            for (int j = 0; j < kFinishPer; ++j) {
+                const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
+                c[j] = (i < cnt) ? view.at(begin + i) : 0ull;
+            }
+            const bool good = block_select_registers<kFinishPer>(c, cnt, rank, top, 0, shared_bits, s_hist, s_scan, &s_pick,
+                                                                 &s_result, &thr);
+            if (threadIdx.x == 0) {
+                ctl->thr[s] = thr;
+                ctl->sel_done[s] = 1u;
+                if (!good) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            }
+            return;
+        }
         block_pick_desc(P.hists->b[0][s], kHistBins, false, rank, s_scan, &s_pick);
         if (threadIdx.x == 0) {
             // the k-th largest composite, known down to the end of the first digit
@@ -109,7 +182,6 @@ __global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
     select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
     unsigned long long prefix;
     const int top = select_top(P, ctl, s, view, &prefix);
-    const int levels = digit_levels(top);
     if (cnt > kSmallList) {  // cannot happen: cnt <= cap <= kSmallList is what the host checked
         if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
         return;
@@ -120,37 +192,13 @@ __global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
         const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
         c[j] = (i < cnt) ? view.at(begin + i) : 0ull;
     }
-    unsigned alive = 0u;  // entries that still match the prefix
-#pragma unroll
-    for (int j = 0; j < kPer; ++j) alive |= ((uint32_t)j * kBlock + threadIdx.x < cnt) ? (1u << j) : 0u;
-    for (int level = 0; level < levels; ++level) {
-        for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
-        __syncthreads();
-#pragma unroll
-        for (int j = 0; j < kPer; ++j)
-            if ((alive >> j) & 1u) atomicAdd(&s_hist[digit_of(c[j], level, top)], 1u);
-        __syncthreads();
-        block_pick_desc<true>(s_hist, 1 << digit_bits(level, top), false, rank, s_scan, &s_pick);
-        if (!s_pick.found) {  // uniform
-            if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
-            return;
-        }
-        const uint32_t sel = s_pick.bin;
-        const bool single = s_pick.count == 1u;
-        rank = s_pick.rank;
-        prefix |= (unsigned long long)sel << digit_shift(level, top);
-#pragma unroll
-        for (int j = 0; j < kPer; ++j)
-            if (((alive >> j) & 1u) && digit_of(c[j], level, top) != sel) alive &= ~(1u << j);
-        if (single) {  // the one entry left is the k-th largest composite
-#pragma unroll
-            for (int j = 0; j < kPer; ++j)
-                if ((alive >> j) & 1u) ctl->thr[s] = c[j];
-            return;
-        }
-        __syncthreads();  // s_pick and s_hist are reused
+    __shared__ unsigned long long s_result;
+    unsigned long long thr = 0ull;
+    const bool good = block_select_registers<kPer>(c, cnt, rank, top, 0, prefix, s_hist, s_scan, &s_pick, &s_result, &thr);
+    if (threadIdx.x == 0) {
+        if (good) ctl->thr[s] = thr;
+        else atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
     }
-    if (threadIdx.x == 0) ctl->thr[s] = prefix;  // every digit fixed
 }
 
 // Keep the entries whose level-L digit is the selected one, histogram their
@@ -164,6 +212,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
     if (ctl->status || ctl->sampled_ok) return;
     const int s = blockIdx.z;
     if (s == 1 && P.mode == kModeValues) return;
+    if (ctl->sel_done[s]) return;  // an earlier level's last block finished the selection
     constexpr int kItems = 4;
     __shared__ uint32_t s_hist[kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -206,6 +255,26 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
         if (v) atomicAdd(&P.hists->b[LEVEL + 1][s][i], v);
     }
     if (last_block_ticket(&ctl->done[ST_BF0_S0 + 2 * LEVEL + s], S.nb)) {
+        const uint32_t n_next = min(__ldcg(&ctl->list_cnt[s][LEVEL + 1]), P.cap);  // entries that matched this level's digit
+        if (n_next <= kFinishList && LEVEL + 2 < digit_levels(top)) {
+            // few entries left and more than one digit to go: this block ranks them alone (they
+            // agree in every digit up to this level's), and the later levels return at once
+            __shared__ unsigned long long s_result;
+            unsigned long long c[kFinishPer], thr = 0ull;
+#pragma unroll
+            for (int j = 0; j < kFinishPer; ++j) {
+                const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
+                c[j] = (i < n_next) ? __ldcg(dst + i) : 0ull;
+            }
+            const bool good = block_select_registers<kFinishPer>(c, n_next, ctl->b_rank[s], top, LEVEL + 1, ctl->b_prefix[s],
+                                                                 s_hist, s_scan, &s_pick, &s_result, &thr);
+            if (threadIdx.x == 0) {
+                ctl->thr[s] = thr;
+                ctl->sel_done[s] = 1u;
+                if (!good) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            }
+            return;
+        }
         block_pick_desc(P.hists->b[LEVEL + 1][s], 1 << digit_bits(LEVEL + 1, top), false,
                         ctl->b_rank[s], s_scan, &s_pick);
         if (threadIdx.x == 0) {

@@ -16,58 +16,6 @@ namespace sbc {
 constexpr uint32_t kSmallKept = 4096;  // positions one block orders in shared memory (k <= (kSmallList - 1024) / 2)
 static_assert((kSmallList - 1024u) / 2u <= kSmallKept, "a short list keeps at most kSmallKept positions");
 
-// Rank `rank` (1 = largest) among the cnt <= kSmallList composites a block holds in registers
-// (slot j of thread t = entry j * kBlock + t).  Radix selection, 11-bit digits from bit `top` down,
-// on shared-memory histograms; stops at the first bucket with a single entry.  Returns false if the
-// histogram walk failed (inconsistent counts).  All threads call; result identical in all.
-template <int PER>
-__device__ __forceinline__ bool block_select_registers(const unsigned long long (&c)[PER], uint32_t cnt, uint32_t rank,
-                                                       int top, unsigned long long prefix, uint32_t* s_hist,
-                                                       uint32_t* s_scan, Pick* s_pick, unsigned long long* s_result,
-                                                       unsigned long long* out) {
-    unsigned alive = 0u;  // entries that still match the prefix
-#pragma unroll
-    for (int j = 0; j < PER; ++j) alive |= ((uint32_t)j * kBlock + threadIdx.x < cnt) ? (1u << j) : 0u;
-    const int levels = digit_levels(top);
-    for (int level = 0; level < levels; ++level) {
-        for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
-        __syncthreads();
-        // a thread's entries mostly share their leading digits: one atomic per run of equal digits
-        uint32_t run_digit = 0u, run_len = 0u;
-#pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            if ((alive >> j) & 1u) {
-                const uint32_t d = digit_of(c[j], level, top);
-                if (run_len && d != run_digit) { atomicAdd(&s_hist[run_digit], run_len); run_len = 0u; }
-                run_digit = d;
-                ++run_len;
-            }
-        }
-        if (run_len) atomicAdd(&s_hist[run_digit], run_len);
-        __syncthreads();
-        block_pick_desc<true>(s_hist, 1 << digit_bits(level, top), false, rank, s_scan, s_pick);
-        if (!s_pick->found) return false;  // uniform
-        const uint32_t sel = s_pick->bin;
-        const bool single = s_pick->count == 1u;
-        rank = s_pick->rank;
-        prefix |= (unsigned long long)sel << digit_shift(level, top);
-#pragma unroll
-        for (int j = 0; j < PER; ++j)
-            if (((alive >> j) & 1u) && digit_of(c[j], level, top) != sel) alive &= ~(1u << j);
-        if (single) {  // the one entry left is the answer; its owner publishes it
-#pragma unroll
-            for (int j = 0; j < PER; ++j)
-                if ((alive >> j) & 1u) *s_result = c[j];
-            __syncthreads();
-            *out = *s_result;
-            return true;
-        }
-        __syncthreads();  // s_pick and s_hist are reused
-    }
-    *out = prefix;  // every digit fixed
-    return true;
-}
-
 // Compare-exchange stage of a bitonic network between registers r and r | STRIDE of one thread
 // (element index = first + r); ascending where (index & size) == 0.
 template <int STRIDE>
@@ -157,7 +105,7 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
             const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
             c[j] = (good && i < cnt) ? view.at(begin + i) : 0ull;
         }
-        good = good && block_select_registers<kPer>(c, cnt, rank, top, prefix, s_hist, s_scan, &s_pick, &s_result, &thr);
+        good = good && block_select_registers<kPer>(c, cnt, rank, top, 0, prefix, s_hist, s_scan, &s_pick, &s_result, &thr);
         if (!good) {
             if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
         } else {

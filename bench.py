@@ -317,6 +317,13 @@ def run_ours(args):
             "route": diags[i],
         })
 
+    # the metric's second half: achieved (algorithmic) HBM rate of the encode over the whole p sweep
+    sweep_ms = sum(enc_ms) / steps
+    sweep_gbs = ALGO_BYTES_PER_ELEM * n * len(P_SWEEP) / (sweep_ms * 1e-3) / 1e9
+    encode_sweep = {"ms": sweep_ms, "algorithmic_gbs": sweep_gbs, "frac_of_measured_peak": sweep_gbs / peak,
+                    "frac_of_nominal_8tbs": sweep_gbs / 8000.0,
+                    "decode_ms": sum(dec_ms) / steps}
+
     # ---- end to end through the host-buffer entry points (pinned host memory, copies timed)
     e2e = run_e2e(args, torch, sbc, dev, update, ws, n, world)
 
@@ -343,7 +350,7 @@ def run_ours(args):
                             "zero fill of the dense tensor is outside the intervals",
                    "parallelism": f"{world} independent client replica(s), no collective"},
         "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches,
-        "clocks": clocks, "per_p": per_p, "network_shapes": network_shapes, "wall_s": wall,
+        "clocks": clocks, "encode_sweep": encode_sweep, "per_p": per_p, "network_shapes": network_shapes, "wall_s": wall,
     }
     print(json.dumps(line), flush=True)
     if dist is not None:

@@ -11,6 +11,64 @@
 
 namespace sbc {
 
+// ---------------------------------------------------------------- block-wide sort in registers
+
+// Compare-exchange stage of a bitonic network between registers r and r | STRIDE of one thread
+// (element index = first + r); ascending where (index & size) == 0.
+template <int E, int STRIDE>
+__device__ __forceinline__ void bitonic_in_thread(uint32_t (&x)[E], uint32_t size, uint32_t first) {
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+        if ((r & STRIDE) == 0 && (r | STRIDE) < E) {
+            const bool ascending = ((first + (uint32_t)r) & size) == 0u;
+            const uint32_t a = x[r], b = x[r | STRIDE];
+            const bool swap = (a > b) == ascending;
+            x[r] = swap ? b : a;
+            x[r | STRIDE] = swap ? a : b;
+        }
+    }
+}
+
+// Ascending sort of E * kBlock values (E = 2, 4, 8 or 16), thread t holding elements E t .. E t + E - 1
+// in registers (bitonic network): exchanges between threads of a warp by shuffle, between warps
+// through `s_swap` (E * kBlock words, transposed so that accesses are conflict-free), the rest in
+// registers.  All threads call.
+template <int E>
+__device__ __forceinline__ void block_sort(uint32_t (&x)[E], uint32_t* s_swap) {
+    static_assert(E == 2 || E == 4 || E == 8 || E == 16, "power-of-two share per thread");
+    constexpr uint32_t kCount = (uint32_t)E * kBlock;
+    const uint32_t tid = threadIdx.x, first = tid * (uint32_t)E;
+    for (uint32_t size = 2u; size <= kCount; size <<= 1) {
+        const bool ascending = (first & size) == 0u;  // used where the partner is another thread (size >= 2 E)
+        for (uint32_t stride = size >> 1; stride >= 32u * E; stride >>= 1) {  // partner in another warp
+            const uint32_t d = stride / E;
+#pragma unroll
+            for (int r = 0; r < E; ++r) s_swap[r * kBlock + tid] = x[r];
+            __syncthreads();
+            const bool take_min = ((tid & d) == 0u) == ascending;
+#pragma unroll
+            for (int r = 0; r < E; ++r) {
+                const uint32_t o = s_swap[r * kBlock + (tid ^ d)];
+                x[r] = take_min ? min(x[r], o) : max(x[r], o);
+            }
+            __syncthreads();
+        }
+        for (uint32_t stride = min(size >> 1, 16u * E); stride >= (uint32_t)E; stride >>= 1) {  // partner in this warp
+            const uint32_t d = stride / E;
+            const bool take_min = ((tid & d) == 0u) == ascending;
+#pragma unroll
+            for (int r = 0; r < E; ++r) {
+                const uint32_t o = __shfl_xor_sync(0xffffffffu, x[r], (int)d);
+                x[r] = take_min ? min(x[r], o) : max(x[r], o);
+            }
+        }
+        if (E > 8 && size >= 16u) bitonic_in_thread<E, 8>(x, size, first);
+        if (E > 4 && size >= 8u) bitonic_in_thread<E, 4>(x, size, first);
+        if (E > 2 && size >= 4u) bitonic_in_thread<E, 2>(x, size, first);
+        bitonic_in_thread<E, 1>(x, size, first);
+    }
+}
+
 // ---------------------------------------------------------------- mask -> sorted positions
 
 // Exclusive scan of the kept positions per tile (both counters of k_tile_count together) into
@@ -53,9 +111,28 @@ __global__ void __launch_bounds__(kBlock) k_tile_scan(const Batch B) {
     }
 }
 
-// Put every tile's bucket of the position list in ascending order.  Small buckets: each thread
-// ranks its entry against the others in shared memory.  Large buckets: the entries set bits in a
-// shared-memory bitmask of the tile, which is then read out in order (popcount scan).
+// One bucket of up to E * kBlock positions, ordered in registers and written back.  All threads call.
+template <int E>
+__device__ __forceinline__ void sort_bucket_in_registers(uint32_t* list, uint32_t beg, uint32_t count, uint32_t* s_swap) {
+    uint32_t x[E];
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+        const uint32_t i = (uint32_t)r * kBlock + threadIdx.x;  // any assignment will do before the sort
+        x[r] = (i < count) ? list[beg + i] : 0xffffffffu;        // padding sorts to the end
+    }
+    block_sort<E>(x, s_swap);  // contains block-wide barriers: every load above precedes every store below
+#pragma unroll
+    for (int r = 0; r < E; ++r) {
+        const uint32_t i = threadIdx.x * (uint32_t)E + (uint32_t)r;
+        if (i < count) list[beg + i] = x[r];
+    }
+    __syncthreads();
+}
+
+// Put every tile's bucket of the position list in ascending order.  Up to 256 entries: each thread
+// ranks its entry against the others in shared memory.  Up to 1024: a bitonic network in
+// registers.  More: the entries set bits in a shared-memory bitmask of the tile, which is then read
+// out in order (popcount scan).
 __global__ void __launch_bounds__(kBlock) k_tile_sort(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
@@ -82,6 +159,11 @@ __global__ void __launch_bounds__(kBlock) k_tile_sort(const Batch B) {
             for (uint32_t j = 0; j < count; ++j) rank += (s_small[j] < x) ? 1u : 0u;
             if (threadIdx.x < count) list[beg + rank] = x;
             __syncthreads();
+            continue;
+        }
+        if (count <= 4u * kBlock) {  // block-uniform: a bitonic network in registers (larger ones lose to the bitmask)
+            if (count <= 2u * kBlock) sort_bucket_in_registers<2>(list, beg, count, s_mask);
+            else sort_bucket_in_registers<4>(list, beg, count, s_mask);
             continue;
         }
         for (int w = threadIdx.x; w < kTileWords + kTileWords / 32; w += kBlock) s_mask[w] = 0u;

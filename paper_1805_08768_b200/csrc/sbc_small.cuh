@@ -13,62 +13,8 @@
 
 namespace sbc {
 
-constexpr uint32_t kSmallKept = 4096;  // positions one block orders in shared memory (k <= (kSmallList - 1024) / 2)
+constexpr uint32_t kSmallKept = 16 * kBlock;  // positions one block orders in registers (k <= (kSmallList - 1024) / 2)
 static_assert((kSmallList - 1024u) / 2u <= kSmallKept, "a short list keeps at most kSmallKept positions");
-
-// Compare-exchange stage of a bitonic network between registers r and r | STRIDE of one thread
-// (element index = first + r); ascending where (index & size) == 0.
-template <int STRIDE>
-__device__ __forceinline__ void bitonic_in_thread(uint32_t (&x)[16], uint32_t size, uint32_t first) {
-#pragma unroll
-    for (int r = 0; r < 16; ++r) {
-        if ((r & STRIDE) == 0) {
-            const bool ascending = ((first + (uint32_t)r) & size) == 0u;
-            const uint32_t a = x[r], b = x[r | STRIDE];
-            const bool swap = (a > b) == ascending;
-            x[r] = swap ? b : a;
-            x[r | STRIDE] = swap ? a : b;
-        }
-    }
-}
-
-// Ascending sort of kSmallKept = 16 * kBlock values, thread t holding elements 16 t .. 16 t + 15 in
-// registers (bitonic network): exchanges between threads of a warp by shuffle, between warps
-// through `s_swap` (kSmallKept words, transposed so that accesses are conflict-free), the rest in
-// registers.  All threads call.
-__device__ __forceinline__ void block_sort_16(uint32_t (&x)[16], uint32_t* s_swap) {
-    static_assert(kSmallKept == 16u * kBlock, "sixteen values per thread");
-    const uint32_t tid = threadIdx.x, first = tid * 16u;
-    for (uint32_t size = 2u; size <= kSmallKept; size <<= 1) {
-        const bool ascending = (first & size) == 0u;  // used where the partner is another thread (size >= 32)
-        for (uint32_t stride = size >> 1; stride >= 512u; stride >>= 1) {  // partner in another warp
-            const uint32_t d = stride >> 4;
-#pragma unroll
-            for (int r = 0; r < 16; ++r) s_swap[r * kBlock + tid] = x[r];
-            __syncthreads();
-            const bool take_min = ((tid & d) == 0u) == ascending;
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-                const uint32_t o = s_swap[r * kBlock + (tid ^ d)];
-                x[r] = take_min ? min(x[r], o) : max(x[r], o);
-            }
-            __syncthreads();
-        }
-        for (uint32_t stride = min(size >> 1, 256u); stride >= 16u; stride >>= 1) {  // partner in this warp
-            const uint32_t d = stride >> 4;
-            const bool take_min = ((tid & d) == 0u) == ascending;
-#pragma unroll
-            for (int r = 0; r < 16; ++r) {
-                const uint32_t o = __shfl_xor_sync(0xffffffffu, x[r], (int)d);
-                x[r] = take_min ? min(x[r], o) : max(x[r], o);
-            }
-        }
-        if (size >= 16u) bitonic_in_thread<8>(x, size, first);
-        if (size >= 8u) bitonic_in_thread<4>(x, size, first);
-        if (size >= 4u) bitonic_in_thread<2>(x, size, first);
-        bitonic_in_thread<1>(x, size, first);
-    }
-}
 
 // One block per problem and side (grid.z = side).
 __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
@@ -208,7 +154,7 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
 #pragma unroll
     for (int r = 0; r < kCw; ++r) pos[r] = s_pos[r * kBlock + threadIdx.x];
     __syncthreads();
-    block_sort_16(pos, s_pos);
+    block_sort<16>(pos, s_pos);
     const uint32_t i0 = threadIdx.x * kCw;
 #pragma unroll
     for (int j = 0; j < kCw; ++j) s_pos[i0 + j] = pos[j];  // the ascending list, for the neighbours and the chunk table

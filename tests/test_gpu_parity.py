@@ -119,6 +119,27 @@ def test_short_list_form_and_its_limits(n, p, kind):
     check_against_oracle(upd, res, p)
 
 
+# The kept positions are ordered bucket by bucket (2^18 positions each): up to 256 per bucket by
+# comparison counting, up to 512 and up to 1024 by register sorting networks of two sizes, more
+# through a bitmask of the bucket.  One case per form, plus uneven buckets (all kept entries in the
+# first tenth of the tensor), where neighbouring buckets take different forms.
+@pytest.mark.parametrize("n,p,clustered", [
+    (1 << 21, 0.0005, False),   # ~131 per bucket
+    (1 << 21, 0.0015, False),   # ~393
+    (1 << 21, 0.003, False),    # ~786
+    (3_000_001, 0.0039, False), # ~1020: around the upper limit of the larger network
+    (1 << 21, 0.006, False),    # ~1573: bitmask
+    (1 << 22, 0.0004, True),    # all 1677 kept entries in two buckets
+    (1 << 22, 0.0001, True),    # 419 kept entries in two buckets
+])
+def test_bucket_ordering_forms(n, p, clustered):
+    rng = np.random.default_rng(zlib.crc32(f"buckets/{n}/{p}/{clustered}".encode()))
+    upd = rng.standard_normal(n).astype(np.float32) * np.float32(1e-3)
+    if clustered:
+        upd[n // 10:] *= np.float32(1e-3)   # large magnitudes only at the front
+    check_against_oracle(upd, np.zeros(n, dtype=np.float32), p)
+
+
 @pytest.mark.parametrize("offset", [1, 2, 3])
 def test_encode_misaligned_pointers(offset):
     rng = np.random.default_rng(offset)

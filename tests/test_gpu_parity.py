@@ -124,13 +124,13 @@ def test_short_list_form_and_its_limits(n, p, kind):
 # through a bitmask of the bucket.  One case per form, plus uneven buckets (all kept entries in the
 # first tenth of the tensor), where neighbouring buckets take different forms.
 @pytest.mark.parametrize("n,p,clustered", [
-    (1 << 21, 0.0005, False),   # ~131 per bucket
-    (1 << 21, 0.0015, False),   # ~393
+    (1 << 23, 0.0005, False),   # ~131 per bucket (k = 4194: beyond the one-kernel form for short lists)
+    (1 << 22, 0.0015, False),   # ~393
     (1 << 21, 0.003, False),    # ~786
     (3_000_001, 0.0039, False), # ~1020: around the upper limit of the larger network
     (1 << 21, 0.006, False),    # ~1573: bitmask
-    (1 << 22, 0.0004, True),    # all 1677 kept entries in two buckets
-    (1 << 22, 0.0001, True),    # 419 kept entries in two buckets
+    (1 << 24, 0.0004, True),    # 6710 kept entries in the first seven buckets
+    (1 << 24, 0.00025, True),   # 4194 kept entries in the first seven buckets
 ])
 def test_bucket_ordering_forms(n, p, clustered):
     rng = np.random.default_rng(zlib.crc32(f"buckets/{n}/{p}/{clustered}".encode()))

@@ -234,8 +234,18 @@ void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned
     nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
 }
 
-// A single problem's descriptor reaches the device as a kernel argument.
-__global__ void k_put_prob(Prob* dst, const Prob src) { *dst = src; }
+// Set-up of a single encode in one launch instead of two memsets and a descriptor kernel: the
+// descriptor (a kernel argument) goes to the head of the workspace, the scratch that must start at zero (control
+// block, histograms, tile counters: `zero_words` 16-byte words at `zero`) and the chunk table and
+// payload area the packer ORs into (`stream_words` at `stream_zero`) are cleared.
+__global__ void __launch_bounds__(kBlock) k_prepare(Prob* dst, const Prob src, uint4* zero, size_t zero_words,
+                                                    uint4* stream_zero, size_t stream_words) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) *dst = src;
+    const size_t tid = (size_t)blockIdx.x * kBlock + threadIdx.x, stride = (size_t)gridDim.x * kBlock;
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    for (size_t i = tid; i < zero_words; i += stride) zero[i] = z;
+    for (size_t i = tid; i < stream_words; i += stride) stream_zero[i] = z;
+}
 
 // Plain byte copy (16 bytes per thread and step where both sides are 16-byte aligned).
 __global__ void __launch_bounds__(kBlock) k_copy_bytes(uint8_t* __restrict__ dst, const uint8_t* __restrict__ src,
@@ -410,10 +420,14 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
     if (marks && marks[SBC_MARK_BEGIN]) cudaEventRecord(marks[SBC_MARK_BEGIN], st);
     // scratch that must start at zero: control block + histograms, tile counters (adjacent),
     // and the chunk table + payload area the packer ORs into
-    if (cudaMemsetAsync(zero, 0, pl.zero_bytes + pl.tile_bytes, st) != cudaSuccess ||
-        cudaMemsetAsync(P.stream + SBC_HEADER_BYTES, 0, pl.stream_bytes - SBC_HEADER_BYTES, st) != cudaSuccess)
-        return SBC_ECUDA;
-    k_put_prob<<<1, 1, 0, st>>>(d_prob, P);
+    {
+        // all three regions are 16-byte aligned and whole multiples of 16 bytes (workspace parts are
+        // 256-byte aligned, the stream pointer 16-byte aligned, header and stream size multiples of 16)
+        const size_t zero_words = (pl.zero_bytes + pl.tile_bytes) / 16, stream_words = (pl.stream_bytes - SBC_HEADER_BYTES) / 16;
+        const unsigned blocks = grid_for(zero_words + stream_words, kBlock * 4, (unsigned)sm_count() * 4u);
+        k_prepare<<<blocks, kBlock, 0, st>>>(d_prob, P, reinterpret_cast<uint4*>(zero), zero_words,
+                                            reinterpret_cast<uint4*>(P.stream + SBC_HEADER_BYTES), stream_words);
+    }
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, 1u, 1u, grid);
@@ -605,7 +619,7 @@ int sbc_encode_static(const float* update, float* residual, int64_t numel, doubl
                       (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
 }
 
-int sbc_encode_launches(void) { return 23; }  // put_prob, 2 sample, 1 collect, 6 exact, 7 select, 6 ordering + Golomb
+int sbc_encode_launches(void) { return 23; }  // set-up, 2 sample, 1 collect, 6 exact, 7 select, 6 ordering + Golomb
 
 int sbc_decode_launches(int n_clients) {
     return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;

@@ -226,7 +226,7 @@ void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned
     nb[WK_MAIN] = grid_for((unsigned long long)pl.n, kBlock * kPerThread * coarse_main, sms * kCollectBlocksPerSM);
     nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 8);
     nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 8);
-    nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 4);
+    nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 2);  // x 2 sides: one resident wave at four blocks per SM
     nb[WK_SCATTER] = grid_for(pl.cap, kBlock * 4, std::min(sms * 8, kMaxScatterBlocks));
     nb[WK_TILE] = grid_for(pl.n_tiles, 1, sms * 6);  // one resident wave: the tile bitmask allows six blocks per SM
     nb[WK_LEN] = grid_for(pl.n_len_blocks, 1, sms * 8);

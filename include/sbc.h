@@ -365,6 +365,27 @@ int sbc_decode_accumulate(const void *const *streams, int n_clients,
                           sbc_cuda_stream_t stream);
 
 /*
+ * sbc_decode_accumulate for messages the caller does not vouch for (received
+ * from another process or machine): Algorithm 4 reads "while i < size(msg)",
+ * and this form is told size(msg).
+ *
+ * stream_bytes  HOST array of n_clients sizes: stream_bytes[c] bytes are
+ *               readable behind streams[c] (the received length, or the
+ *               capacity of the slot the message sits in); each >= 64.
+ * A header whose size fields (k, n_chunks, payload_offset, nbits) describe a
+ * container longer than stream_bytes[c] fails validation BEFORE any chunk-table
+ * entry or payload word is read: the stream contributes nothing and
+ * SBC_STATUS_CORRUPT is set.  sbc_decode_accumulate itself checks the size
+ * fields only against each other and against numel, i.e. it trusts that the
+ * buffer is as long as its header says -- true for a container sbc_encode
+ * wrote into a buffer of sbc_stream_bytes(numel, p) bytes.
+ * Everything else as sbc_decode_accumulate.
+ */
+int sbc_decode_accumulate_sized(const void *const *streams, const size_t *stream_bytes,
+                                int n_clients, float *out_dense, int64_t numel,
+                                uint32_t *status_dev, sbc_cuda_stream_t stream);
+
+/*
  * Decode, scale and apply in one pass (Algorithm 1: server lines
  * "dW <- 1/|I_t| sum dW_i*" and "W <- W + dW", equally the client line
  * "W_i <- W_i + dW"; momentum masking, Supplement "Momentum Correction, Warm-up
@@ -384,6 +405,11 @@ int sbc_decode_accumulate(const void *const *streams, int n_clients,
 int sbc_decode_apply(const void *const *streams, int n_clients, float scale, float *weights,
                      float *momentum, int64_t numel, uint32_t *status_dev,
                      sbc_cuda_stream_t stream);
+/* sbc_decode_apply with the readable size of every message stated, as
+ * sbc_decode_accumulate_sized. */
+int sbc_decode_apply_sized(const void *const *streams, const size_t *stream_bytes, int n_clients,
+                           float scale, float *weights, float *momentum, int64_t numel,
+                           uint32_t *status_dev, sbc_cuda_stream_t stream);
 
 /*
  * sbc_decode_accumulate for many tensors at once: for every tensor t,
@@ -400,6 +426,8 @@ typedef struct sbc_decode_desc {
     const void *const *streams;
     float *out_dense;
     int64_t numel;
+    const size_t *stream_bytes; /* HOST array of n_clients readable sizes as in
+                                   sbc_decode_accumulate_sized, or NULL (not stated) */
 } sbc_decode_desc;
 size_t sbc_decode_workspace_bytes_batch(int n_tensors);
 int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_desc *descs,
@@ -413,6 +441,11 @@ int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_d
  * dense_dev (device, numel floats), decodes and sums into it, copies the
  * result to out_dense_host and the status word to *status_host, and
  * synchronises `stream`.  Returns SBC_ECORRUPT if the status word is non-zero.
+ * The headers are first checked on the host against stream_bytes[c] (magic,
+ * version, numel, and that the container they describe ends inside the bytes
+ * given): if one fails, SBC_ECORRUPT is returned, *status_host gets
+ * SBC_STATUS_CORRUPT, nothing is enqueued and out_dense_host is not touched.
+ * The device decode is the _sized form with the same lengths.
  */
 int sbc_decode_accumulate_host(const void *const *streams_host, const size_t *stream_bytes,
                                int n_clients, float *out_dense_host, float *dense_dev,

@@ -27,7 +27,7 @@ EXPORTS = [
     "sbc_encode_diag_get", "sbc_encode_host", "sbc_stream_info_get", "sbc_decode_accumulate",
     "sbc_decode_accumulate_host", "sbc_encode_static", "sbc_workspace_bytes_batch", "sbc_encode_batch",
     "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch", "sbc_decode_apply", "sbc_stream_bytes_values", "sbc_encode_values", "sbc_stream_bytes_sampled",
-    "sbc_workspace_bytes_sampled", "sbc_encode_sampled",
+    "sbc_workspace_bytes_sampled", "sbc_encode_sampled", "sbc_decode_accumulate_sized", "sbc_decode_apply_sized",
 ]
 SIDE_VALUES = 2
 STATIC_WORKSPACE_BYTES = 8 << 20
@@ -65,7 +65,8 @@ class TensorDesc(C.Structure):
 
 
 class DecodeDesc(C.Structure):
-    _fields_ = [("streams", C.POINTER(C.c_void_p)), ("out_dense", C.c_void_p), ("numel", C.c_int64)]
+    _fields_ = [("streams", C.POINTER(C.c_void_p)), ("out_dense", C.c_void_p), ("numel", C.c_int64),
+                ("stream_bytes", C.POINTER(C.c_size_t))]
 
 
 _lib = None
@@ -141,6 +142,12 @@ def lib() -> C.CDLL:
         L.sbc_decode_accumulate.restype = C.c_int
         L.sbc_decode_accumulate.argtypes = [C.POINTER(C.c_void_p), C.c_int, C.c_void_p, C.c_int64,
                                             C.c_void_p, C.c_void_p]
+        L.sbc_decode_accumulate_sized.restype = C.c_int
+        L.sbc_decode_accumulate_sized.argtypes = [C.POINTER(C.c_void_p), C.POINTER(C.c_size_t), C.c_int, C.c_void_p,
+                                                  C.c_int64, C.c_void_p, C.c_void_p]
+        L.sbc_decode_apply_sized.restype = C.c_int
+        L.sbc_decode_apply_sized.argtypes = [C.POINTER(C.c_void_p), C.POINTER(C.c_size_t), C.c_int, C.c_float,
+                                             C.c_void_p, C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
 
@@ -211,6 +218,41 @@ def sbc_encode(update: torch.Tensor, residual: torch.Tensor, p: float,
     return out_stream, out_mu
 
 
+def _tensor_descs(updates, residuals, ps, out_streams, out_mus):
+    """One sbc_tensor_desc per tensor of a batch (the only place they are marshalled)."""
+    n = len(updates)
+    descs = (TensorDesc * n)()
+    for t in range(n):
+        _dev_f32(updates[t], "update")
+        _dev_f32(residuals[t], "residual")
+        d = descs[t]
+        d.update, d.residual, d.numel, d.p = updates[t].data_ptr(), residuals[t].data_ptr(), updates[t].numel(), float(ps[t])
+        d.out_stream, d.out_capacity, d.out_mu = out_streams[t].data_ptr(), out_streams[t].numel(), out_mus[t].data_ptr()
+    return descs
+
+
+def _decode_descs(streams_per_tensor, out_denses, sizes_per_tensor=None):
+    """One sbc_decode_desc per tensor; returns (descs, n_clients, objects the descs point into)."""
+    n = len(out_denses)
+    n_clients = len(streams_per_tensor[0])
+    descs = (DecodeDesc * n)()
+    keep = []
+    for t in range(n):
+        if len(streams_per_tensor[t]) != n_clients:
+            raise ValueError("every tensor needs the same number of client streams")
+        _dev_f32(out_denses[t], "out_dense")
+        ptrs = (C.c_void_p * n_clients)(*[s.data_ptr() for s in streams_per_tensor[t]])
+        keep.append(ptrs)
+        descs[t].streams = ptrs
+        descs[t].out_dense = out_denses[t].data_ptr()
+        descs[t].numel = out_denses[t].numel()
+        if sizes_per_tensor is not None:
+            lens = (C.c_size_t * n_clients)(*[int(x) for x in sizes_per_tensor[t]])
+            keep.append(lens)
+            descs[t].stream_bytes = lens
+    return descs, n_clients, keep
+
+
 def sbc_workspace_bytes_batch(numels: Sequence[int], ps: Sequence[float]) -> int:
     n = len(numels)
     descs = (TensorDesc * n)()
@@ -220,39 +262,13 @@ def sbc_workspace_bytes_batch(numels: Sequence[int], ps: Sequence[float]) -> int
     return int(lib().sbc_workspace_bytes_batch(n, descs))
 
 
-def sbc_encode_batch(updates: Sequence[torch.Tensor], residuals: Sequence[torch.Tensor], ps: Sequence[float],
-                     out_streams: Sequence[torch.Tensor], out_mus: Sequence[torch.Tensor],
-                     workspace: torch.Tensor, stream=None) -> None:
-    """sbc_encode of every tensor of a round with one launch sequence for the whole batch."""
-    n = len(updates)
-    descs = (TensorDesc * n)()
-    for t in range(n):
-        _dev_f32(updates[t], "update")
-        _dev_f32(residuals[t], "residual")
-        descs[t].update = updates[t].data_ptr()
-        descs[t].residual = residuals[t].data_ptr()
-        descs[t].numel = updates[t].numel()
-        descs[t].p = float(ps[t])
-        descs[t].out_stream = out_streams[t].data_ptr()
-        descs[t].out_capacity = out_streams[t].numel()
-        descs[t].out_mu = out_mus[t].data_ptr()
-    code = lib().sbc_encode_batch(n, descs, workspace.data_ptr(), workspace.numel(), _cuda_stream(stream))
-    _check(code, "sbc_encode_batch")
-
-
 class EncodeBatch:
     """The marshalled descriptors of a batch, built once and reused every round (same tensors)."""
 
     def __init__(self, updates, residuals, ps, out_streams, out_mus, workspace):
         self.n = len(updates)
-        self.descs = (TensorDesc * self.n)()
+        self.descs = _tensor_descs(updates, residuals, ps, out_streams, out_mus)
         self.keep = (list(updates), list(residuals), list(out_streams), list(out_mus), workspace)
-        for t in range(self.n):
-            _dev_f32(updates[t], "update")
-            _dev_f32(residuals[t], "residual")
-            d = self.descs[t]
-            d.update, d.residual, d.numel, d.p = updates[t].data_ptr(), residuals[t].data_ptr(), updates[t].numel(), float(ps[t])
-            d.out_stream, d.out_capacity, d.out_mu = out_streams[t].data_ptr(), out_streams[t].numel(), out_mus[t].data_ptr()
         self.ws_ptr, self.ws_bytes = workspace.data_ptr(), workspace.numel()
 
     def run(self, stream=None) -> None:
@@ -260,23 +276,21 @@ class EncodeBatch:
                "sbc_encode_batch")
 
 
-class DecodeBatch:
-    """The marshalled descriptors of a batched decode, built once and reused."""
+def sbc_encode_batch(updates: Sequence[torch.Tensor], residuals: Sequence[torch.Tensor], ps: Sequence[float],
+                     out_streams: Sequence[torch.Tensor], out_mus: Sequence[torch.Tensor],
+                     workspace: torch.Tensor, stream=None) -> None:
+    """sbc_encode of every tensor of a round with one launch sequence for the whole batch."""
+    EncodeBatch(updates, residuals, ps, out_streams, out_mus, workspace).run(stream)
 
-    def __init__(self, streams_per_tensor, out_denses, workspace, status=None):
+
+class DecodeBatch:
+    """The marshalled descriptors of a batched decode, built once and reused.  ``sizes_per_tensor``
+    (readable bytes behind every stream) makes the decoder check each header against them."""
+
+    def __init__(self, streams_per_tensor, out_denses, workspace, status=None, sizes_per_tensor=None):
         self.n = len(out_denses)
-        self.n_clients = len(streams_per_tensor[0])
-        self.descs = (DecodeDesc * self.n)()
-        self.keep = [streams_per_tensor, out_denses, workspace, status]
-        for t in range(self.n):
-            if len(streams_per_tensor[t]) != self.n_clients:
-                raise ValueError("every tensor needs the same number of client streams")
-            _dev_f32(out_denses[t], "out_dense")
-            ptrs = (C.c_void_p * self.n_clients)(*[s.data_ptr() for s in streams_per_tensor[t]])
-            self.keep.append(ptrs)
-            self.descs[t].streams = ptrs
-            self.descs[t].out_dense = out_denses[t].data_ptr()
-            self.descs[t].numel = out_denses[t].numel()
+        self.descs, self.n_clients, keep = _decode_descs(streams_per_tensor, out_denses, sizes_per_tensor)
+        self.keep = [streams_per_tensor, out_denses, workspace, status, keep]
         self.status_ptr = status.data_ptr() if status is not None else None
         self.ws_ptr, self.ws_bytes = workspace.data_ptr(), workspace.numel()
 
@@ -292,25 +306,9 @@ def sbc_decode_workspace_bytes_batch(n_tensors: int) -> int:
 
 def sbc_decode_accumulate_batch(streams_per_tensor: Sequence[Sequence[torch.Tensor]],
                                 out_denses: Sequence[torch.Tensor], workspace: torch.Tensor,
-                                status: Optional[torch.Tensor] = None, stream=None) -> None:
+                                status: Optional[torch.Tensor] = None, stream=None, sizes_per_tensor=None) -> None:
     """out_denses[t][j] += mu for every client stream of every tensor t; one launch for the batch."""
-    n = len(out_denses)
-    n_clients = len(streams_per_tensor[0])
-    descs = (DecodeDesc * n)()
-    keep = []
-    for t in range(n):
-        if len(streams_per_tensor[t]) != n_clients:
-            raise ValueError("every tensor needs the same number of client streams")
-        _dev_f32(out_denses[t], "out_dense")
-        ptrs = (C.c_void_p * n_clients)(*[s.data_ptr() for s in streams_per_tensor[t]])
-        keep.append(ptrs)
-        descs[t].streams = ptrs
-        descs[t].out_dense = out_denses[t].data_ptr()
-        descs[t].numel = out_denses[t].numel()
-    code = lib().sbc_decode_accumulate_batch(n, n_clients, descs,
-                                             status.data_ptr() if status is not None else None,
-                                             workspace.data_ptr(), workspace.numel(), _cuda_stream(stream))
-    _check(code, "sbc_decode_accumulate_batch")
+    DecodeBatch(streams_per_tensor, out_denses, workspace, status, sizes_per_tensor).run(stream)
 
 
 def sbc_encode_static(update: torch.Tensor, residual: torch.Tensor, p: float, out_stream: torch.Tensor,
@@ -395,28 +393,42 @@ def sbc_stream_info_get(out_stream: torch.Tensor, stream=None, check: bool = Tru
 
 
 def sbc_decode_accumulate(streams: Sequence[torch.Tensor], out_dense: torch.Tensor,
-                          status: Optional[torch.Tensor] = None, stream=None) -> None:
-    """Enqueue out_dense[j] += mu_c for every position j of every client stream c."""
-    _dev_f32(out_dense, "out_dense")
-    ptrs = (C.c_void_p * max(len(streams), 1))(*[s.data_ptr() for s in streams])
-    code = lib().sbc_decode_accumulate(ptrs, len(streams), out_dense.data_ptr(), out_dense.numel(),
-                                       status.data_ptr() if status is not None else None,
-                                       _cuda_stream(stream))
-    _check(code, "sbc_decode_accumulate")
+                          status: Optional[torch.Tensor] = None, stream=None,
+                          sizes: Optional[Sequence[int]] = None) -> None:
+    """Enqueue out_dense[j] += mu_c for every position j of every client stream c.  With ``sizes``
+    (readable bytes behind every stream) the _sized entry point checks each header against them."""
+    sbc_decode_apply(streams, 1.0, out_dense, None, status, stream, sizes, _plain=True)
 
 
 def sbc_decode_apply(streams: Sequence[torch.Tensor], scale: float, weights: torch.Tensor,
                      momentum: Optional[torch.Tensor] = None, status: Optional[torch.Tensor] = None,
-                     stream=None) -> None:
+                     stream=None, sizes: Optional[Sequence[int]] = None, _plain: bool = False) -> None:
     """Enqueue weights[j] += scale * mu_c at every decoded position; momentum[j] = 0 there."""
     _dev_f32(weights, "weights")
     if momentum is not None:
         _dev_f32(momentum, "momentum")
-    ptrs = (C.c_void_p * max(len(streams), 1))(*[s.data_ptr() for s in streams])
-    code = lib().sbc_decode_apply(ptrs, len(streams), float(scale), weights.data_ptr(),
-                                  momentum.data_ptr() if momentum is not None else None, weights.numel(),
-                                  status.data_ptr() if status is not None else None, _cuda_stream(stream))
-    _check(code, "sbc_decode_apply")
+    nc = len(streams)
+    ptrs = (C.c_void_p * max(nc, 1))(*[s.data_ptr() for s in streams])
+    st = status.data_ptr() if status is not None else None
+    L = lib()
+    if sizes is not None:
+        if len(sizes) != nc:
+            raise ValueError("one size per stream")
+        lens = (C.c_size_t * max(nc, 1))(*[int(x) for x in sizes])
+        if _plain:
+            code = L.sbc_decode_accumulate_sized(ptrs, lens, nc, weights.data_ptr(), weights.numel(), st,
+                                                 _cuda_stream(stream))
+        else:
+            code = L.sbc_decode_apply_sized(ptrs, lens, nc, float(scale), weights.data_ptr(),
+                                            momentum.data_ptr() if momentum is not None else None,
+                                            weights.numel(), st, _cuda_stream(stream))
+    elif _plain:
+        code = L.sbc_decode_accumulate(ptrs, nc, weights.data_ptr(), weights.numel(), st, _cuda_stream(stream))
+    else:
+        code = L.sbc_decode_apply(ptrs, nc, float(scale), weights.data_ptr(),
+                                  momentum.data_ptr() if momentum is not None else None, weights.numel(), st,
+                                  _cuda_stream(stream))
+    _check(code, "sbc_decode_accumulate" if _plain else "sbc_decode_apply")
 
 
 def sbc_stream_bytes_values(numel: int, p: float) -> int:

@@ -697,12 +697,18 @@ int sbc_encode_host(const float* update_host, float* update_dev, float* residual
                     sbc_cuda_stream_t stream) {
     if (!update_host || !update_dev || !out_stream_host || !stream_dev || !out_bytes_host || numel <= 0)
         return SBC_EINVAL;
-    if (!workspace) return SBC_EINVAL;
-    if (cudaMemcpyAsync(update_dev, update_host, (size_t)numel * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-        return SBC_ECUDA;
+    // every check the host can make comes before the first copy is enqueued
+    if (!workspace || ((uintptr_t)workspace & 255)) return SBC_EINVAL;
     Plan pl;
     if (!make_plan(numel, p, &pl)) return SBC_EINVAL;
+    {
+        const TensorArgs a = {update_dev, residual_dev, stream_dev, out_capacity, nullptr};
+        const int arc = check_tensor(a, pl);
+        if (arc != SBC_OK) return arc;
+    }
     if (workspace_bytes < pl.total) return SBC_ECAPACITY;
+    if (cudaMemcpyAsync(update_dev, update_host, (size_t)numel * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return SBC_ECUDA;
     float* mu_dev = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kProbSlotBytes + pl.zero_bytes +
                                              pl.tile_bytes + pl.off_mu);
     const int rc = sbc_encode(update_dev, residual_dev, numel, p, stream_dev, out_capacity, mu_dev,
@@ -748,25 +754,27 @@ int sbc_stream_info_get(const void* stream_dev, sbc_stream_info* host_out, sbc_c
     return SBC_OK;
 }
 
-int sbc_decode_accumulate(const void* const* streams, int n_clients, float* out_dense, int64_t numel,
-                          uint32_t* status_dev, sbc_cuda_stream_t stream) {
-    return sbc_decode_apply(streams, n_clients, 1.0f, out_dense, nullptr, numel, status_dev, stream);
-}
-
-int sbc_decode_apply(const void* const* streams, int n_clients, float scale, float* out_dense, float* momentum,
-                     int64_t numel, uint32_t* status_dev, sbc_cuda_stream_t stream) {
+// Common body of the decode entry points.  `stream_bytes` may be null (sizes not stated).
+static int decode_impl(const void* const* streams, const size_t* stream_bytes, int n_clients, float scale,
+                       float* out_dense, float* momentum, int64_t numel, uint32_t* status_dev,
+                       sbc_cuda_stream_t stream) {
     if (!(scale == scale) || std::isinf(scale) || ((uintptr_t)momentum & 3)) return SBC_EINVAL;
     if (n_clients < 0 || numel <= 0 || numel >= (1ll << 31) || !out_dense) return SBC_EINVAL;
     if (n_clients > 0 && !streams) return SBC_EINVAL;
     if (((uintptr_t)out_dense & 3) || ((uintptr_t)status_dev & 3)) return SBC_EINVAL;
-    for (int c = 0; c < n_clients; ++c)
+    for (int c = 0; c < n_clients; ++c) {
         if (!streams[c] || ((uintptr_t)streams[c] & 15)) return SBC_EINVAL;
+        if (stream_bytes && stream_bytes[c] < SBC_HEADER_BYTES) return SBC_EINVAL;  // not even a header
+    }
     const unsigned sms = (unsigned)sm_count();
     for (int first = 0; first < n_clients; first += kMaxClientsPerLaunch) {
         DecodeArgs a;
         std::memset(&a, 0, sizeof(a));
         a.n_clients = std::min(kMaxClientsPerLaunch, n_clients - first);
-        for (int c = 0; c < a.n_clients; ++c) a.streams[c] = static_cast<const uint8_t*>(streams[first + c]);
+        for (int c = 0; c < a.n_clients; ++c) {
+            a.streams[c] = static_cast<const uint8_t*>(streams[first + c]);
+            a.bytes[c] = stream_bytes ? (unsigned long long)stream_bytes[first + c] : 0ull;
+        }
         a.out = out_dense;
         a.n = numel;
         a.status = status_dev;
@@ -780,6 +788,29 @@ int sbc_decode_apply(const void* const* streams, int n_clients, float scale, flo
         k_decode_accumulate<<<grid, kDecodeThreads, 0, stream>>>(a);
     }
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
+}
+
+int sbc_decode_accumulate(const void* const* streams, int n_clients, float* out_dense, int64_t numel,
+                          uint32_t* status_dev, sbc_cuda_stream_t stream) {
+    return decode_impl(streams, nullptr, n_clients, 1.0f, out_dense, nullptr, numel, status_dev, stream);
+}
+
+int sbc_decode_accumulate_sized(const void* const* streams, const size_t* stream_bytes, int n_clients,
+                                float* out_dense, int64_t numel, uint32_t* status_dev, sbc_cuda_stream_t stream) {
+    if (n_clients > 0 && !stream_bytes) return SBC_EINVAL;
+    return decode_impl(streams, stream_bytes, n_clients, 1.0f, out_dense, nullptr, numel, status_dev, stream);
+}
+
+int sbc_decode_apply(const void* const* streams, int n_clients, float scale, float* out_dense, float* momentum,
+                     int64_t numel, uint32_t* status_dev, sbc_cuda_stream_t stream) {
+    return decode_impl(streams, nullptr, n_clients, scale, out_dense, momentum, numel, status_dev, stream);
+}
+
+int sbc_decode_apply_sized(const void* const* streams, const size_t* stream_bytes, int n_clients, float scale,
+                           float* out_dense, float* momentum, int64_t numel, uint32_t* status_dev,
+                           sbc_cuda_stream_t stream) {
+    if (n_clients > 0 && !stream_bytes) return SBC_EINVAL;
+    return decode_impl(streams, stream_bytes, n_clients, scale, out_dense, momentum, numel, status_dev, stream);
 }
 
 size_t sbc_decode_workspace_bytes_batch(int n_tensors) {
@@ -797,8 +828,10 @@ int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_d
         const sbc_decode_desc& d = descs[t];
         if (!d.streams || !d.out_dense || ((uintptr_t)d.out_dense & 3) || d.numel <= 0 || d.numel >= (1ll << 31))
             return SBC_EINVAL;
-        for (int c = 0; c < n_clients; ++c)
+        for (int c = 0; c < n_clients; ++c) {
             if (!d.streams[c] || ((uintptr_t)d.streams[c] & 15)) return SBC_EINVAL;
+            if (d.stream_bytes && d.stream_bytes[c] < SBC_HEADER_BYTES) return SBC_EINVAL;
+        }
         max_numel = std::max<long long>(max_numel, d.numel);
     }
     // one copy of all argument blocks from an ordinary host buffer (read out before the call returns)
@@ -808,7 +841,10 @@ int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_d
         std::memset(static_cast<void*>(args.data()), 0, args.size() * sizeof(DecodeArgs));
         for (int t = 0; t < n_tensors; ++t) {
             args[t].n_clients = n_clients;
-            for (int c = 0; c < n_clients; ++c) args[t].streams[c] = static_cast<const uint8_t*>(descs[t].streams[c]);
+            for (int c = 0; c < n_clients; ++c) {
+                args[t].streams[c] = static_cast<const uint8_t*>(descs[t].streams[c]);
+                args[t].bytes[c] = descs[t].stream_bytes ? (unsigned long long)descs[t].stream_bytes[c] : 0ull;
+            }
             args[t].out = descs[t].out_dense;
             args[t].n = descs[t].numel;
             args[t].status = status_dev;
@@ -830,29 +866,50 @@ int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_d
 int sbc_decode_accumulate_host(const void* const* streams_host, const size_t* stream_bytes, int n_clients,
                                float* out_dense_host, float* dense_dev, int64_t numel, void* staging_dev,
                                size_t staging_bytes, uint32_t* status_host, sbc_cuda_stream_t stream) {
-    if (n_clients < 0 || n_clients > 4096 || numel <= 0 || !out_dense_host || !dense_dev || !staging_dev)
+    if (n_clients < 0 || n_clients > 4096 || numel <= 0 || numel >= (1ll << 31) || !out_dense_host || !dense_dev ||
+        !staging_dev)
         return SBC_EINVAL;
     if (n_clients > 0 && (!streams_host || !stream_bytes)) return SBC_EINVAL;
-    if ((uintptr_t)staging_dev & 15) return SBC_EINVAL;
+    if (((uintptr_t)staging_dev & 15) || ((uintptr_t)dense_dev & 3)) return SBC_EINVAL;
     // staging layout: one status word (16 bytes), then the containers
     size_t need = 16;
-    for (int c = 0; c < n_clients; ++c) need += align_up(stream_bytes[c], 16);
+    for (int c = 0; c < n_clients; ++c) {
+        if (!streams_host[c] || stream_bytes[c] < SBC_HEADER_BYTES) return SBC_EINVAL;
+        need += align_up(stream_bytes[c], 16);
+    }
     if (staging_bytes < need) return SBC_ECAPACITY;
+    // The containers are in host memory: what their headers claim is compared with the bytes the
+    // caller received, here, before anything is enqueued (the device repeats the check on its copy).
+    for (int c = 0; c < n_clients; ++c) {
+        const uint8_t* h = static_cast<const uint8_t*>(streams_host[c]);
+        uint32_t magic, version;
+        unsigned long long hdr_numel, nbits, payload_offset;
+        std::memcpy(&magic, h + 0, 4);
+        std::memcpy(&version, h + 4, 4);
+        std::memcpy(&hdr_numel, h + 8, 8);
+        std::memcpy(&nbits, h + 24, 8);
+        std::memcpy(&payload_offset, h + 32, 8);
+        const bool fits = nbits <= (1ull << 40) && payload_offset <= (unsigned long long)stream_bytes[c] &&
+                          payload_offset + align_up((size_t)((nbits + 7) / 8), 16) <= (unsigned long long)stream_bytes[c];
+        if (magic != SBC_MAGIC || version != SBC_VERSION || hdr_numel != (unsigned long long)numel || !fits) {
+            if (status_host) *status_host = SBC_STATUS_CORRUPT;
+            return SBC_ECORRUPT;
+        }
+    }
     uint8_t* base = static_cast<uint8_t*>(staging_dev);
-    const void* dev_ptrs[4096];
+    std::vector<const void*> dev_ptrs((size_t)std::max(n_clients, 1));
     size_t off = 16;
     if (cudaMemsetAsync(base, 0, 16, stream) != cudaSuccess ||
         cudaMemsetAsync(dense_dev, 0, (size_t)numel * 4, stream) != cudaSuccess)
         return SBC_ECUDA;
     for (int c = 0; c < n_clients; ++c) {
-        if (!streams_host[c] || stream_bytes[c] < SBC_HEADER_BYTES) return SBC_EINVAL;
         if (small_copy(base + off, streams_host[c], stream_bytes[c], cudaMemcpyHostToDevice, stream) != cudaSuccess)
             return SBC_ECUDA;
         dev_ptrs[c] = base + off;
         off += align_up(stream_bytes[c], 16);
     }
-    const int rc = sbc_decode_accumulate(dev_ptrs, n_clients, dense_dev, numel,
-                                         reinterpret_cast<uint32_t*>(base), stream);
+    const int rc = sbc_decode_accumulate_sized(dev_ptrs.data(), stream_bytes, n_clients, dense_dev, numel,
+                                               reinterpret_cast<uint32_t*>(base), stream);
     if (rc != SBC_OK) return rc;
     uint32_t on_stack = 0;
     uint8_t* pad = landing_pad();

@@ -11,6 +11,8 @@ constexpr int kMaxClientsPerLaunch = 32;
 
 struct DecodeArgs {
     const uint8_t* streams[kMaxClientsPerLaunch];
+    // bytes the caller vouches for behind streams[c]; 0: not stated (the header's own size fields are trusted)
+    unsigned long long bytes[kMaxClientsPerLaunch];
     int n_clients;
     float* out;
     long long n;
@@ -190,7 +192,12 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
             side <= SBC_SIDE_VALUES &&
             payload_offset == SBC_HEADER_BYTES + (unsigned long long)v.n_chunks * SBC_CHUNK_ENTRY_BYTES + values_bytes &&
             v.nbits >= v.k * (1ull + v.b) &&
-            v.nbits <= v.k * (1ull + v.b) + ((unsigned long long)args.n >> v.b);
+            v.nbits <= v.k * (1ull + v.b) + ((unsigned long long)args.n >> v.b) &&
+            // the whole container (chunk table, values, payload padded to 16 bytes) lies inside the bytes the
+            // caller stated: checked before any table entry or payload word is read (k <= n < 2^31 and
+            // nbits < 2^37 by the lines above, so nothing here overflows)
+            (args.bytes[tid] == 0ull ||
+             payload_offset + ((((v.nbits + 7ull) >> 3) + 15ull) & ~15ull) <= args.bytes[tid]);
         if (!good) {
             v.n_chunks = 0u;  // contributes nothing
             if (args.status && blockIdx.x == 0) atomicOr(args.status, SBC_STATUS_CORRUPT);

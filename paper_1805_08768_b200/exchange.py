@@ -74,11 +74,13 @@ class StreamExchange:
         client per launch in rank order, so that every rank adds in the same order."""
         from . import binding
         s = (1.0 / self.world) if scale is None else float(scale)
+        # the messages come from other ranks: every header is checked against its slot's capacity
         if ordered:
             for slot in self.slots:
-                binding.sbc_decode_apply([slot], s, weights, momentum, status, stream=stream)
+                binding.sbc_decode_apply([slot], s, weights, momentum, status, stream=stream, sizes=[self.capacity])
         else:
-            binding.sbc_decode_apply(self.slots, s, weights, momentum, status, stream=stream)
+            binding.sbc_decode_apply(self.slots, s, weights, momentum, status, stream=stream,
+                                     sizes=[self.capacity] * self.world)
 
 
 def exchange_round(update: torch.Tensor, residual: torch.Tensor, p: float, weights: torch.Tensor,

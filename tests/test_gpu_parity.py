@@ -319,6 +319,63 @@ def test_corrupt_streams_set_status_and_stay_in_bounds():
     assert run(bad) & sbc.STATUS_CORRUPT
 
 
+def test_inflated_size_fields_are_refused_when_the_length_is_stated():
+    """A header whose k, n_chunks, payload_offset and nbits are inflated *consistently* passes every
+    check the header allows on its own; told the received length, the decoder must refuse it before
+    it reads a table entry or a payload word.  The message sits inside a larger zero-filled buffer
+    the test owns, so that even an unchecked read would stay inside the test's memory."""
+    n, p = 200000, 0.01
+    upd = workloads.normal_flat(n, 1e-3, 6)
+    stream, _, _, info, _ = gpu_encode(upd, np.zeros(n, dtype=np.float32), p)
+    true_len = stream.size
+    b = int(info.b)
+
+    def header(k, nbits=None, n_chunks=None, payload_offset=None):
+        bad = stream.copy()
+        n_chunks = -(-k // int(info.chunk_codewords)) if n_chunks is None else n_chunks
+        payload_offset = 64 + 16 * n_chunks if payload_offset is None else payload_offset
+        nbits = k * (1 + b) + ((n - k) >> b) if nbits is None else nbits
+        bad[16:24].view("<u8")[0] = k
+        bad[24:32].view("<u8")[0] = nbits
+        bad[32:40].view("<u8")[0] = payload_offset
+        bad[56:60].view("<u4")[0] = n_chunks
+        return bad
+
+    def run(mutated, sizes):
+        arena = torch.zeros(8 << 20, dtype=torch.uint8, device=DEV)      # 8 MiB >= any container for this n
+        arena[: mutated.size] = torch.from_numpy(mutated).to(DEV)
+        dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+        status = torch.zeros(1, dtype=torch.int32, device=DEV)
+        sbc.sbc_decode_accumulate([arena], dense, status=status, sizes=sizes)
+        torch.cuda.synchronize()
+        return status.item(), bool(dense.any())
+
+    assert run(stream, [true_len]) == (0, True)                      # the genuine message, exact length
+    assert run(stream, [true_len + 4096])[0] == 0                    # a slot larger than the message
+    st, touched = run(stream, [true_len - 16])                       # cut short
+    assert st & sbc.STATUS_CORRUPT and not touched
+    for bad in (header(10 * int(info.k)),                            # everything inflated together
+                header(n),                                           # the largest k the tensor allows
+                header(int(info.k)),                                 # only the payload length (the most the header's own checks allow)
+                header(int(info.k) + 4096)):                         # a few more chunks
+        assert 64 + 16 * int(bad[56:60].view("<u4")[0]) + (int(bad[24:32].view("<u8")[0]) + 7) // 8 <= 8 << 20
+        st, touched = run(bad, [true_len])
+        assert st & sbc.STATUS_CORRUPT and not touched, "an over-long header was decoded"
+    with pytest.raises(sbc.SbcError) as e:                           # a length that cannot hold a header
+        run(stream, [32])
+    assert e.value.code == sbc.SBC_EINVAL
+    # the batched form carries the lengths in its descriptors
+    arena = torch.zeros(8 << 20, dtype=torch.uint8, device=DEV)
+    bad = header(10 * int(info.k))
+    arena[: bad.size] = torch.from_numpy(bad).to(DEV)
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    dws = torch.empty(sbc.sbc_decode_workspace_bytes_batch(1), dtype=torch.uint8, device=DEV)
+    sbc.sbc_decode_accumulate_batch([[arena]], [dense], dws, status=status, sizes_per_tensor=[[true_len]])
+    torch.cuda.synchronize()
+    assert status.item() & sbc.STATUS_CORRUPT and not bool(dense.any())
+
+
 def test_argument_errors_are_returned_at_once():
     n = 1000
     u = torch.zeros(n, dtype=torch.float32, device=DEV)

@@ -254,26 +254,6 @@ int sbc_encode_ex(const float *update, float *residual, int64_t numel, double p,
                   void *workspace, size_t workspace_bytes, sbc_cuda_stream_t stream,
                   const sbc_cuda_event_t *marks);
 
-/* Number of kernels one sbc_encode call launches for a tensor whose candidate
- * lists are longer than one thread block handles (memsets not counted; a tensor
- * with 2*k + 1024 <= 8192 and k <= 4096 takes a shorter chain of 11), and
- * one sbc_decode_accumulate call for n_clients streams. */
-int sbc_encode_launches(void);
-int sbc_decode_launches(int n_clients);
-
-/* What the last sbc_encode that used `workspace` did; synchronises `stream`. */
-typedef struct sbc_encode_diag {
-    uint32_t status;        /* SBC_STATUS_* bits */
-    uint32_t exact_route;   /* 1 if the bounds from the sample failed and the exact route ran */
-    uint32_t candidates[2]; /* entries gathered per side (>= k) */
-    uint32_t capacity;      /* capacity of each candidate list */
-    float bound_lo, bound_hi; /* candidates were: value >= bound_lo, value <= bound_hi */
-    double mu_pos, mu_neg;  /* the two means of Algorithm 2 */
-    uint32_t certain[2];    /* of the candidates, those at or above the sample's upper bound of the
-                               threshold (kept without being looked at by the exact selection) */
-} sbc_encode_diag;
-int sbc_encode_diag_get(const void *workspace, sbc_encode_diag *host_out, sbc_cuda_stream_t stream);
-
 /*
  * Host-buffer form of sbc_encode for callers whose update lives in host
  * memory: copies update_host to update_dev, encodes, copies the finished

@@ -55,7 +55,7 @@ class EncodeDiag(C.Structure):
     _fields_ = [
         ("status", C.c_uint32), ("exact_route", C.c_uint32), ("candidates", C.c_uint32 * 2),
         ("capacity", C.c_uint32), ("bound_lo", C.c_float), ("bound_hi", C.c_float),
-        ("mu_pos", C.c_double), ("mu_neg", C.c_double), ("certain", C.c_uint32 * 2),
+        ("mu_pos", C.c_double), ("mu_neg", C.c_double), ("certain", C.c_uint32 * 2), ("regathered", C.c_uint32),
     ]
 
 

@@ -6,6 +6,7 @@
 #include <vector>
 
 #include "../../include/sbc.h"
+#include "../../include/sbc_debug.h"
 #include "sbc_common.cuh"
 #include "sbc_decode.cuh"
 #include "sbc_exact.cuh"
@@ -23,35 +24,37 @@ constexpr size_t kProbSlotBytes = 512;  // one problem descriptor, padded
 static_assert(sizeof(Prob) <= kProbSlotBytes, "descriptor must fit its slot");
 
 // Host-side plan of one encode problem: scalar parameters and the layout of its scratch, which
-// comes in three parts so that a batch can keep each part contiguous across problems:
+// comes in two parts so that a batch can keep each part contiguous across problems:
 //   zero part  control block + radix histograms (cleared before every call)
-//   tile part  per-tile counts of kept positions, both sides, and bucket fill counters (cleared)
 //   rest       everything that needs no clearing
 struct Plan {
     long long n, k;
     int b, mode, sampled;
-    uint32_t cap, m, n_xtiles, n_tiles, n_len_blocks, n_chunks;
+    uint32_t cap, m, n_xtiles, n_chunks, chunk_cw;
     uint32_t s_target, s_up;
+    uint32_t main_blocks, main_warps, span_steps, n_spans, cap_w, list_cap, use_runs, order_blocks;
     unsigned long long payload_offset;
     size_t stream_bytes;
     size_t zero_bytes, off_ctl, off_hists;                 // offsets inside the zero part
-    size_t tile_bytes, off_tile_in, off_tile_base, off_tile_fill;  // inside the tile part
-    size_t rest_bytes, off_mu, off_sample, off_cand[2], off_buf[2][2], off_xtile[2], off_idx,
-        off_blklen, off_blk_first;                                        // inside the rest
-    size_t total;                                          // single problem: slot + zero + tile + rest
+    size_t rest_bytes, off_mu, off_sample, off_list[2], off_band[2], off_buf[2][2], off_xtile[2], off_span[2],
+        off_rng_sum, off_blk_sum, off_blk_base;            // inside the rest
+    size_t total;                                          // single problem: slot + zero + rest
 };
+
+// The layout of the ordered candidate lists depends on how many warps the streaming pass runs, so
+// the grids that shape it are planned for the B200's 148 SMs whatever device is current (on
+// another device the plan is still valid, only not tuned).
+constexpr unsigned kPlanSMs = 148;
 
 bool valid_p(double p) { return p > 0.0 && p < 1.0; }
 
-// Blocks that walk a candidate list to bucket its kept entries by tile: one per 1024 list slots,
-// at most kMaxScatterBlocks (the scratch that carries their slot reservations from the counting
-// kernel to the placing kernel is sized from this bound, without asking the device).
-constexpr unsigned kMaxScatterBlocks = 2048;
-unsigned scatter_blocks_bound(uint32_t cap) {
-    return (unsigned)std::min<unsigned long long>(((unsigned long long)cap + kBlock * 4 - 1) / (kBlock * 4), kMaxScatterBlocks) + 1u;
-}
+inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsigned max_blocks);
 
-bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long long sampled_m = 0) {
+// coarse_main: elements per streaming block, in units of 4096 (a batch gives its blocks several
+// steps each).  force_runs: the launch this problem is part of takes the general chain of kernels
+// even if this problem alone would fit the short-list form.
+bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long long sampled_m = 0, unsigned coarse_main = 1,
+               bool force_runs = false) {
     if (n <= 0 || n >= (1ll << 31) || !valid_p(p)) return false;
     const int b = sbc_golomb_b(p);
     if (b < 0 || b > 30) return false;
@@ -101,10 +104,10 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
     pl->s_target = target;
     pl->s_up = up;
     pl->n_xtiles = (uint32_t)((n + kXTile - 1) / kXTile);
-    pl->n_tiles = (uint32_t)((n + (1ll << kTileShift) - 1) >> kTileShift);
     const long long k_max = pl->sampled ? (long long)pl->cap : k;  // most positions a stream can carry
-    pl->n_len_blocks = (uint32_t)((k_max + kLenBlock - 1) / kLenBlock);
-    pl->n_chunks = (uint32_t)((k_max + kChunkCodewords - 1) / kChunkCodewords);
+    pl->chunk_cw = chunk_codewords_for((unsigned long long)k);
+    // table entries for the most positions at the smallest chunk size a stream of that many could get
+    pl->n_chunks = (uint32_t)((k_max + pl->chunk_cw - 1) / pl->chunk_cw);
     pl->payload_offset = SBC_HEADER_BYTES + (unsigned long long)pl->n_chunks * SBC_CHUNK_ENTRY_BYTES;
     if (mode == kModeValues) pl->payload_offset += align_up((size_t)k * 4, 16);  // the values sit before the payload
     pl->mode = mode;
@@ -113,28 +116,52 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
         (pl->sampled ? ((unsigned long long)n >> b) : 0ull);
     pl->stream_bytes = (size_t)pl->payload_offset + align_up((size_t)((bits_bound + 7) / 8), 16);
 
+    // Streaming pass: blocks, warps, spans, and each warp's region of the ordered lists.
+    pl->main_blocks = grid_for((unsigned long long)n, kBlock * kPerThread * coarse_main, kPlanSMs * kCollectBlocksPerSM);
+    pl->main_warps = pl->main_blocks * (kBlock / 32);
+    const unsigned long long n_steps = ((unsigned long long)n + kWarpChunk - 1) / kWarpChunk;
+    // the longest span (8, 4, 2 or 1 steps) that still leaves every warp at least two spans
+    pl->span_steps = 1;
+    for (uint32_t steps = kMaxSpanSteps; steps > 1; steps >>= 1)
+        if ((n_steps + steps - 1) / steps >= 2ull * pl->main_warps) { pl->span_steps = steps; break; }
+    pl->n_spans = (uint32_t)((n_steps + pl->span_steps - 1) / pl->span_steps);
+    // the short-list form (one kernel after the candidate pass, which orders the positions itself)
+    // needs no ordered lists; everything else walks them
+    pl->use_runs = force_runs || !(pl->cap <= kSmallList && k <= (long long)kSmallKept && mode == kModeBinary && !pl->sampled);
+    {
+        // candidates a warp expects per side: its share of the spans times the density the lower
+        // bound lets through (about k/n and a margin); twice that, eight deviations and a floor
+        const unsigned long long spans_per_warp = (pl->n_spans + pl->main_warps - 1) / pl->main_warps;
+        const double elems = (double)std::min<unsigned long long>((unsigned long long)n, spans_per_warp * pl->span_steps * kWarpChunk);
+        const double expect = (double)k_max * elems / (double)n;
+        double slots = std::ceil(2.0 * expect + 8.0 * std::sqrt(expect) + 64.0);
+        slots = std::min(slots, elems);                 // a warp cannot see more candidates than elements
+        pl->cap_w = (uint32_t)((unsigned long long)slots + 15ull) / 16u * 16u;   // whole 128-byte lines
+        const unsigned long long regions = pl->use_runs ? (unsigned long long)pl->main_warps * pl->cap_w : 0ull;
+        pl->list_cap = (uint32_t)std::min<unsigned long long>(std::max<unsigned long long>(regions, pl->cap), 0xfffffff0ull);
+        if (regions > 0xfffffff0ull) return false;      // cannot happen below 2^31 elements
+    }
+    pl->order_blocks = grid_for(pl->n_spans, (kBlock / 32) * 4, kOrderBlocksMax);   // four spans or more per warp
+
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
     pl->off_ctl = take(sizeof(Ctl));
     pl->off_hists = take(sizeof(Hists));
     pl->zero_bytes = off;
     off = 0;
-    pl->off_tile_in = take((size_t)pl->n_tiles * 4);
-    pl->off_tile_base = take((size_t)(pl->n_tiles + 1) * 4);
-    pl->off_tile_fill = take((size_t)pl->n_tiles * 4);
-    pl->tile_bytes = off;
-    off = 0;
     pl->off_mu = take(sizeof(float));  // where the host-buffer form parks mu
     pl->off_sample = take((size_t)pl->m * 4);
-    for (int s = 0; s < 2; ++s) pl->off_cand[s] = take((size_t)pl->cap * 8);
+    for (int s = 0; s < 2; ++s) pl->off_list[s] = take((size_t)pl->list_cap * 8);
+    for (int s = 0; s < 2; ++s) pl->off_band[s] = take((size_t)pl->cap * 8);
     for (int s = 0; s < 2; ++s)
         for (int j = 0; j < 2; ++j) pl->off_buf[s][j] = take((size_t)pl->cap * 8);
     for (int s = 0; s < 2; ++s) pl->off_xtile[s] = take((size_t)pl->n_xtiles * 4);
-    pl->off_idx = take((size_t)k_max * 4);
-    pl->off_blklen = take((size_t)pl->n_len_blocks * 8);
-    pl->off_blk_first = take((size_t)scatter_blocks_bound(pl->cap) * kTileWindow * 4);
+    for (int s = 0; s < 2; ++s) pl->off_span[s] = take(pl->use_runs ? (size_t)pl->n_spans * sizeof(uint2) : 0);
+    pl->off_rng_sum = take(pl->use_runs ? (size_t)pl->order_blocks * (kBlock / 32) * sizeof(RangeSum) : 0);
+    pl->off_blk_sum = take(pl->use_runs ? (size_t)pl->order_blocks * sizeof(RangeSum) : 0);
+    pl->off_blk_base = take(pl->use_runs ? (size_t)pl->order_blocks * sizeof(RangeBase) : 0);
     pl->rest_bytes = off;
-    pl->total = kProbSlotBytes + pl->zero_bytes + pl->tile_bytes + pl->rest_bytes;
+    pl->total = kProbSlotBytes + pl->zero_bytes + pl->rest_bytes;
     return true;
 }
 
@@ -158,7 +185,7 @@ int check_tensor(const TensorArgs& a, const Plan& pl) {
     return SBC_OK;
 }
 
-Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile, uint8_t* rest) {
+Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* rest) {
     Prob P;
     std::memset(&P, 0, sizeof(P));
     P.update = a.update;
@@ -175,26 +202,30 @@ Prob make_prob(const TensorArgs& a, const Plan& pl, uint8_t* zero, uint8_t* tile
     P.out_mu = a.out_mu;
     P.ctl = reinterpret_cast<Ctl*>(zero + pl.off_ctl);
     P.hists = reinterpret_cast<Hists*>(zero + pl.off_hists);
-    P.tile_in = reinterpret_cast<uint32_t*>(tile + pl.off_tile_in);
-    P.tile_base = reinterpret_cast<uint32_t*>(tile + pl.off_tile_base);
-    P.tile_fill = reinterpret_cast<uint32_t*>(tile + pl.off_tile_fill);
-    P.blk_first = reinterpret_cast<uint32_t*>(rest + pl.off_blk_first);
     P.sample_keys = reinterpret_cast<uint32_t*>(rest + pl.off_sample);
     for (int s = 0; s < 2; ++s) {
-        P.cand[s] = reinterpret_cast<unsigned long long*>(rest + pl.off_cand[s]);
+        P.list[s] = reinterpret_cast<unsigned long long*>(rest + pl.off_list[s]);
+        P.band[s] = reinterpret_cast<unsigned long long*>(rest + pl.off_band[s]);
+        P.span_rec[s] = reinterpret_cast<uint2*>(rest + pl.off_span[s]);
         for (int j = 0; j < 2; ++j) P.buf[s][j] = reinterpret_cast<unsigned long long*>(rest + pl.off_buf[s][j]);
         P.x_tile_cnt[s] = reinterpret_cast<uint32_t*>(rest + pl.off_xtile[s]);
     }
-    P.idx = reinterpret_cast<uint32_t*>(rest + pl.off_idx);
-    P.blk_len = reinterpret_cast<unsigned long long*>(rest + pl.off_blklen);
+    P.rng_sum = reinterpret_cast<RangeSum*>(rest + pl.off_rng_sum);
+    P.blk_sum = reinterpret_cast<RangeSum*>(rest + pl.off_blk_sum);
+    P.blk_base = reinterpret_cast<RangeBase*>(rest + pl.off_blk_base);
     P.s_target = pl.s_target;
     P.s_up = pl.s_up;
     P.cap = pl.cap;
+    P.list_cap = pl.list_cap;
+    P.cap_w = pl.cap_w;
+    P.main_warps = pl.main_warps;
+    P.span_steps = pl.span_steps;
+    P.n_spans = pl.n_spans;
+    P.use_runs = pl.use_runs;
+    P.chunk_cw = pl.chunk_cw;
     P.m = pl.m;
     P.sample_step = (pl.m >> 5) ? ((unsigned long long)(pl.n >> 5) << 20) / (unsigned long long)(pl.m >> 5) : 0ull;
     P.n_xtiles = pl.n_xtiles;
-    P.n_tiles = pl.n_tiles;
-    P.n_len_blocks = pl.n_len_blocks;
     P.n_chunks = pl.n_chunks;
     P.payload_offset = pl.payload_offset;
     return P;
@@ -219,17 +250,15 @@ inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsi
 // problem) make the blocks of the sample kernels and of the exact-route kernels that many times
 // larger: every block of those kernels pays for clearing and flushing a shared-memory histogram
 // (or, for the exact route, usually just for finding out that it is not needed), and a batch of
-// hundreds of problems has parallelism to spare.
-void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned coarse_exact,
-                  unsigned coarse_main, unsigned nb[WK_COUNT]) {
+// hundreds of problems has parallelism to spare.  The streaming pass and the ordering kernels take
+// their grids from the plan (the layout of the ordered lists depends on them).
+void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned coarse_exact, unsigned nb[WK_COUNT]) {
     nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8 * coarse_sample, sms * 4);
-    nb[WK_MAIN] = grid_for((unsigned long long)pl.n, kBlock * kPerThread * coarse_main, sms * kCollectBlocksPerSM);
+    nb[WK_MAIN] = pl.main_blocks;
     nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 8);
     nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 8);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 2);  // x 2 sides: one resident wave at four blocks per SM
-    nb[WK_SCATTER] = grid_for(pl.cap, kBlock * 4, std::min(sms * 8, kMaxScatterBlocks));
-    nb[WK_TILE] = grid_for(pl.n_tiles, 1, sms * 6);  // one resident wave: the tile bitmask allows six blocks per SM
-    nb[WK_LEN] = grid_for(pl.n_len_blocks, 1, sms * 8);
+    nb[WK_ORDER] = pl.order_blocks;
     nb[WK_ONE] = 1;
     nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
 }
@@ -277,7 +306,7 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
 // a single problem) say how each kind of work is spread over the problems.
 void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, const unsigned grid[WK_COUNT],
-                   const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, bool small_kept, cudaStream_t st,
+                   const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, bool small_form, cudaStream_t st,
                    const sbc_cuda_event_t* marks) {
     auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
     auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs, any_exact}; };
@@ -285,7 +314,7 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
     auto g2 = [&](int kind) { return dim3(grid[kind], 1, 2); };  // z = side
     // Every kernel is launched with programmatic stream serialisation: its blocks may be placed
     // while the previous kernel drains; each kernel waits for its predecessor in resolve().
-    // The two long kernels (streaming pass, residual write-back) are launched the ordinary way:
+    // The two long kernels (streaming pass, second ordering walk with the residual write-back) are launched the ordinary way:
     // blocks placed early land wherever the draining kernel happens to free a slot, and the uneven
     // spread over the SMs cost the write-back 30 % at 2^30 elements, p = 1e-2.
     auto go = [&](void (*kernel)(Batch), dim3 g, Batch arg, bool early = true) {
@@ -322,7 +351,7 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
 
     // 3. exact k-th composite of each candidate list, sums, side
     // 4. ordered positions, residual write-back, Golomb payload, chunk table, header
-    if (small_lists && small_kept && mode == kModeBinary && !sampled) {  // all of it by two blocks per problem
+    if (small_form) {  // every problem of the launch is short: all of it by two blocks per problem
         mark(SBC_MARK_SELECT);
         go(k_small_finish, g2(WK_ONE), B(WK_ONE));
         mark(SBC_MARK_END);
@@ -341,12 +370,8 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
     go(k_sums_decide, g2(WK_CAND), B(WK_CAND));
     mark(SBC_MARK_SELECT);
 
-    go(k_tile_count, g1(WK_SCATTER), B(WK_SCATTER));
-    go(k_tile_scan, g1(WK_ONE), B(WK_ONE));
-    go(k_scatter, g1(WK_SCATTER), B(WK_SCATTER));
-    go(k_tile_sort, g1(WK_TILE), B(WK_TILE));
-    go(k_len_sum_residual, g1(WK_LEN), B(WK_LEN), false);
-    go(k_pack, g1(WK_LEN), B(WK_LEN));
+    go(k_span_count, g1(WK_ORDER), B(WK_ORDER));
+    go(k_span_emit, g1(WK_ORDER), B(WK_ORDER), false);
     mark(SBC_MARK_END);
 }
 
@@ -383,8 +408,10 @@ size_t sbc_stream_bytes(int64_t numel, double p) {
 }
 
 size_t sbc_workspace_bytes(int64_t numel, double p) {
+    // the same figure serves sbc_encode and sbc_encode_values: sized for the general chain of
+    // kernels, which the short-list form of sbc_encode needs only a part of
     Plan pl;
-    return make_plan(numel, p, &pl) ? pl.total : 0;
+    return make_plan(numel, p, &pl, kModeBinary, 0, 1, true) ? pl.total : 0;
 }
 
 int sbc_encode(const float* update, float* residual, int64_t numel, double p, void* out_stream,
@@ -407,31 +434,30 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
     if (rc != SBC_OK) return rc;
     if (workspace_bytes < pl.total) return SBC_ECAPACITY;
 
-    // workspace: [descriptor][zero part][tile part][rest]
+    // workspace: [descriptor][zero part][rest]
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     uint8_t* zero = ws + kProbSlotBytes;
-    uint8_t* tile = zero + pl.zero_bytes;
-    uint8_t* rest = tile + pl.tile_bytes;
-    Prob P = make_prob(a, pl, zero, tile, rest);
+    uint8_t* rest = zero + pl.zero_bytes;
+    Prob P = make_prob(a, pl, zero, rest);
     P.sample_idx = sample_idx;
     Prob* d_prob = reinterpret_cast<Prob*>(ws);
 
     cudaStream_t st = stream;
     if (marks && marks[SBC_MARK_BEGIN]) cudaEventRecord(marks[SBC_MARK_BEGIN], st);
-    // scratch that must start at zero: control block + histograms, tile counters (adjacent),
+    // scratch that must start at zero: control block + histograms,
     // and the chunk table + payload area the packer ORs into
     {
-        // all three regions are 16-byte aligned and whole multiples of 16 bytes (workspace parts are
+        // both regions are 16-byte aligned and whole multiples of 16 bytes (workspace parts are
         // 256-byte aligned, the stream pointer 16-byte aligned, header and stream size multiples of 16)
-        const size_t zero_words = (pl.zero_bytes + pl.tile_bytes) / 16, stream_words = (pl.stream_bytes - SBC_HEADER_BYTES) / 16;
+        const size_t zero_words = pl.zero_bytes / 16, stream_words = (pl.stream_bytes - SBC_HEADER_BYTES) / 16;
         const unsigned blocks = grid_for(zero_words + stream_words, kBlock * 4, (unsigned)sm_count() * 4u);
         k_prepare<<<blocks, kBlock, 0, st>>>(d_prob, P, reinterpret_cast<uint4*>(zero), zero_words,
                                             reinterpret_cast<uint4*>(P.stream + SBC_HEADER_BYTES), stream_words);
     }
 
     unsigned grid[WK_COUNT];
-    block_counts(pl, (unsigned)sm_count(), 1u, 1u, 1u, grid);
-    launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, pl.k <= (long long)kSmallKept, st, marks);
+    block_counts(pl, (unsigned)sm_count(), 1u, 1u, grid);
+    launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, !pl.use_runs, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -471,15 +497,37 @@ int sbc_encode_values(const float* update, float* residual, int64_t numel, doubl
                        workspace_bytes, stream, nullptr);
 }
 
+// Plans of all tensors of a batch.  Two things are decided over the whole batch: how many steps a
+// streaming block gets (about three waves of resident blocks over the batch, so that a block's
+// start-up -- finding its problem, reading the bounds -- and its final flush are paid for by
+// several steps of loads), and whether the launch can use the short-list form (only if every
+// tensor fits it).
+static bool plan_batch(int n_tensors, const sbc_tensor_desc* descs, std::vector<Plan>* plans, bool* all_small) {
+    unsigned long long fine_main = 0;
+    bool small = true;
+    Plan pl;
+    for (int t = 0; t < n_tensors; ++t) {
+        if (!make_plan(descs[t].numel, descs[t].p, &pl)) return false;
+        fine_main += (unsigned long long)(pl.n + kBlock * kPerThread - 1) / (kBlock * kPerThread);
+        small = small && !pl.use_runs;
+    }
+    const unsigned coarse_main = (unsigned)std::min<unsigned long long>(
+        8, std::max<unsigned long long>(1, fine_main / (kPlanSMs * 3 * kCollectBlocksPerSM)));
+    plans->resize((size_t)n_tensors);
+    for (int t = 0; t < n_tensors; ++t)
+        if (!make_plan(descs[t].numel, descs[t].p, &(*plans)[t], kModeBinary, 0, coarse_main, !small)) return false;
+    *all_small = small;
+    return true;
+}
+
 size_t sbc_workspace_bytes_batch(int n_tensors, const sbc_tensor_desc* descs) {
-    if (n_tensors <= 0 || !descs) return 0;
+    if (n_tensors <= 0 || n_tensors > (1 << 20) || !descs) return 0;
+    std::vector<Plan> plans;
+    bool all_small;
+    if (!plan_batch(n_tensors, descs, &plans, &all_small)) return 0;
     size_t total = align_up((size_t)n_tensors * sizeof(Prob), 256) +
                    align_up((size_t)WK_COUNT * (size_t)(n_tensors + 1) * 4, 256);
-    for (int t = 0; t < n_tensors; ++t) {
-        Plan pl;
-        if (!make_plan(descs[t].numel, descs[t].p, &pl)) return 0;
-        total += pl.zero_bytes + pl.tile_bytes + pl.rest_bytes;
-    }
+    for (int t = 0; t < n_tensors; ++t) total += plans[t].zero_bytes + plans[t].rest_bytes;
     return total;
 }
 
@@ -487,60 +535,53 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
                      sbc_cuda_stream_t stream) {
     if (n_tensors <= 0 || !descs || !workspace || ((uintptr_t)workspace & 255)) return SBC_EINVAL;
     if (n_tensors > (1 << 20)) return SBC_EINVAL;
-    std::vector<Plan> plans((size_t)n_tensors);
-    size_t zero_total = 0, tile_total = 0, rest_total = 0;
+    std::vector<Plan> plans;
+    bool all_small;
+    if (!plan_batch(n_tensors, descs, &plans, &all_small)) return SBC_EINVAL;
+    size_t zero_total = 0, rest_total = 0;
     for (int t = 0; t < n_tensors; ++t) {
-        if (!make_plan(descs[t].numel, descs[t].p, &plans[t])) return SBC_EINVAL;
         const TensorArgs a = {descs[t].update, descs[t].residual, descs[t].out_stream, descs[t].out_capacity,
                               descs[t].out_mu};
         const int rc = check_tensor(a, plans[t]);
         if (rc != SBC_OK) return rc;
         zero_total += plans[t].zero_bytes;
-        tile_total += plans[t].tile_bytes;
         rest_total += plans[t].rest_bytes;
     }
     const size_t probs_bytes = align_up((size_t)n_tensors * sizeof(Prob), 256);
     const size_t prefix_bytes = align_up((size_t)WK_COUNT * (size_t)(n_tensors + 1) * 4, 256);
-    if (workspace_bytes < probs_bytes + prefix_bytes + zero_total + tile_total + rest_total) return SBC_ECAPACITY;
+    if (workspace_bytes < probs_bytes + prefix_bytes + zero_total + rest_total) return SBC_ECAPACITY;
 
-    // workspace: [descriptors][prefix tables][zero parts][tile parts][rests]
+    // workspace: [descriptors][prefix tables][zero parts][rests]
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     Prob* d_probs = reinterpret_cast<Prob*>(ws);
     uint32_t* d_prefix = reinterpret_cast<uint32_t*>(ws + probs_bytes);
     uint8_t* zero = ws + probs_bytes + prefix_bytes;
-    uint8_t* tile = zero + zero_total;
-    uint8_t* rest = tile + tile_total;
+    uint8_t* rest = zero + zero_total;
 
     const unsigned sms = (unsigned)sm_count();
     // aim at about six (sample) and two (exact route) blocks per SM over the whole batch
-    unsigned long long fine_sample = 0, fine_exact = 0, fine_main = 0;
+    unsigned long long fine_sample = 0, fine_exact = 0;
     for (int t = 0; t < n_tensors; ++t) {
         fine_sample += (plans[t].m + kBlock * 8 - 1) / (kBlock * 8);
         fine_exact += (unsigned long long)(plans[t].n + kBlock * 16 - 1) / (kBlock * 16);
-        fine_main += (unsigned long long)(plans[t].n + kBlock * kPerThread - 1) / (kBlock * kPerThread);
     }
     auto factor = [&](unsigned long long fine, unsigned per_sm) {
         return (unsigned)std::min<unsigned long long>(256, std::max<unsigned long long>(1, fine / (sms * per_sm)));
     };
     const unsigned coarse_sample = factor(fine_sample, 6), coarse_exact = factor(fine_exact, 2);
-    // streaming pass: about three waves of resident blocks over the whole batch, so that a block's
-    // start-up (finding its problem, reading the bounds) and its final flush are paid for by several
-    // steps of loads
-    const unsigned coarse_main = std::min(8u, factor(fine_main, 3 * kCollectBlocksPerSM));
     const size_t row_len = (size_t)n_tensors + 1;
     std::vector<Prob> probs((size_t)n_tensors);
     std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
     {
-        uint8_t *z = zero, *m = tile, *r = rest;
+        uint8_t *z = zero, *r = rest;
         for (int t = 0; t < n_tensors; ++t) {
             const TensorArgs a = {descs[t].update, descs[t].residual, descs[t].out_stream,
                                   descs[t].out_capacity, descs[t].out_mu};
-            probs[t] = make_prob(a, plans[t], z, m, r);
+            probs[t] = make_prob(a, plans[t], z, r);
             z += plans[t].zero_bytes;
-            m += plans[t].tile_bytes;
             r += plans[t].rest_bytes;
             unsigned nb[WK_COUNT];
-            block_counts(plans[t], sms, coarse_sample, coarse_exact, coarse_main, nb);
+            block_counts(plans[t], sms, coarse_sample, coarse_exact, nb);
             for (int kind = 0; kind < WK_COUNT; ++kind) {
                 uint32_t* row = prefix.data() + (size_t)kind * row_len;
                 const unsigned long long next = (unsigned long long)row[t] + nb[kind];
@@ -551,7 +592,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     }
 
     cudaStream_t st = stream;
-    if (cudaMemsetAsync(zero, 0, zero_total + tile_total, st) != cudaSuccess) return SBC_ECUDA;
+    if (cudaMemsetAsync(zero, 0, zero_total, st) != cudaSuccess) return SBC_ECUDA;
     // Descriptors and tables are adjacent in the workspace: one copy from a host buffer laid out
     // the same way.  The source is ordinary (pageable) memory, which the runtime reads out before
     // cudaMemcpyAsync returns, so the buffer may die with this call.
@@ -569,12 +610,9 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
     k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors, nullptr});
-    bool small_lists = true, small_kept = true;
-    for (int t = 0; t < n_tensors; ++t) {
-        small_lists = small_lists && plans[t].cap <= kSmallList;
-        small_kept = small_kept && plans[t].k <= (long long)kSmallKept;
-    }
-    launch_encode(d_probs, (uint32_t)n_tensors, &probs[0].ctl->launch_exact, grid, d_rows, kModeBinary, false, small_lists, small_kept, st, nullptr);
+    bool small_lists = true;
+    for (int t = 0; t < n_tensors; ++t) small_lists = small_lists && plans[t].cap <= kSmallList;
+    launch_encode(d_probs, (uint32_t)n_tensors, &probs[0].ctl->launch_exact, grid, d_rows, kModeBinary, false, small_lists, all_small, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -619,7 +657,7 @@ int sbc_encode_static(const float* update, float* residual, int64_t numel, doubl
                       (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
 }
 
-int sbc_encode_launches(void) { return 23; }  // set-up, 2 sample, 1 collect, 6 exact, 7 select, 6 ordering + Golomb
+int sbc_encode_launches(void) { return 19; }  // set-up, 2 sample, 1 collect, 6 exact, 7 select, 2 ordering + Golomb
 
 int sbc_decode_launches(int n_clients) {
     return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;
@@ -646,6 +684,7 @@ int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cu
     host_out->mu_pos = c.mu64[0];
     host_out->mu_neg = c.mu64[1];
     for (int s = 0; s < 2; ++s) host_out->certain[s] = c.use_fallback ? 0u : c.sure_cnt[s];
+    host_out->regathered = (c.use_fallback && c.x_known) ? 1u : 0u;
     return SBC_OK;
 }
 
@@ -709,8 +748,7 @@ int sbc_encode_host(const float* update_host, float* update_dev, float* residual
     if (workspace_bytes < pl.total) return SBC_ECAPACITY;
     if (cudaMemcpyAsync(update_dev, update_host, (size_t)numel * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return SBC_ECUDA;
-    float* mu_dev = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kProbSlotBytes + pl.zero_bytes +
-                                             pl.tile_bytes + pl.off_mu);
+    float* mu_dev = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + kProbSlotBytes + pl.zero_bytes + pl.off_mu);
     const int rc = sbc_encode(update_dev, residual_dev, numel, p, stream_dev, out_capacity, mu_dev,
                               workspace, workspace_bytes, stream);
     if (rc != SBC_OK) return rc;

@@ -22,10 +22,10 @@ constexpr int kBlock = 256;           // threads per block for every kernel here
 constexpr int kHistBins = 2048;       // 11-bit radix digits
 constexpr uint32_t kSampleMax = 1u << 20;  // elements looked at to bound the thresholds
 constexpr int kXTile = 4096;          // elements per tile in the exact-select fallback
-constexpr int kTileShift = 18;         // positions per ordering tile = 262144
-constexpr int kTileWords = (1 << kTileShift) / 32;  // bitmask words covering one tile
-constexpr int kLenBlock = 1024;       // codewords per block in the length scan / packer
+constexpr int kWarpChunk = 512;       // elements one warp handles per step of the streaming pass
+constexpr int kMaxSpanSteps = kXTile / kWarpChunk;  // a span is 1, 2, 4 or 8 steps and never straddles a tile
 constexpr int kChunkCodewords = 256;  // codewords per chunk-table entry
+constexpr uint32_t kOrderBlocksMax = 148 * 8;  // ordering kernels: at most one resident wave of 8-warp blocks on 148 SMs
 constexpr int kSumBins = 254;         // one exact integer bin per fp32 exponent
 constexpr uint32_t kSmallList = 8192;  // candidate lists up to this capacity are ranked by one block
 
@@ -35,7 +35,7 @@ enum Stage : int {
     ST_BH0_S0, ST_BH0_S1,
     ST_BF0_S0, ST_BF0_S1, ST_BF1_S0, ST_BF1_S1, ST_BF2_S0, ST_BF2_S1,
     ST_BF3_S0, ST_BF3_S1, ST_BF4_S0, ST_BF4_S1,
-    ST_SUM, ST_LEN, ST_COUNT
+    ST_SUM, ST_ORDER, ST_COUNT
 };
 
 // Device-side control block of one encode call; zeroed before the first kernel.
@@ -53,10 +53,13 @@ struct Ctl {
     uint32_t s_bin0_up[2], s_rank_up[2];  // the same search for the upper bound of the threshold
     uint32_t up_key[2];         // side key at and above which a candidate is certainly kept ("sure")
     uint32_t lo_key[2];         // side key of the lower bound: every candidate's key is at least this
-    // candidate lists: sure entries grow from the front of cand[s], the rest ("band") from its back
-    unsigned long long cand_cnt2[2];  // low word: sure entries, high word: band entries
-    uint32_t cand_cnt[2];       // both together (set when the candidate pass ends)
+    // candidates per side: all of them, those at or above up_key ("sure"), and the cursor of the band list
+    uint32_t cand_cnt[2];
     uint32_t sure_cnt[2];
+    uint32_t band_cnt[2];
+    uint32_t overflow;          // a warp's region of the ordered list, or a band list, did not hold its entries
+    uint32_t x_known;           // exact route: the thresholds are already known (x_thr), only the gathering is redone
+    long long pre_bins[2][256]; // exact sums of the sure entries, gathered while they were flushed
     // exact select over A (fallback)
     uint32_t x_prefix[2], x_rank[2], x_thr[2], x_ties_take[2], x_ties_have[2];
     // select over the candidate lists
@@ -104,22 +107,33 @@ struct Prob {
     Ctl* ctl;
     Hists* hists;
     uint32_t* sample_keys;
-    unsigned long long* cand[2];
+    // Candidates in position order: the tensor is cut into spans of span_steps * 512 elements; the
+    // entries of a span sit together in list[s], ascending, at span_rec[s][span] = {offset, count}.
+    // The streaming pass gives each of its warps a private region of cap_w slots (no atomics, no
+    // waits); the exact route reserves space tile by tile.
+    unsigned long long* list[2];
+    uint2* span_rec[2];
+    // Candidates below the sample's upper bound of the threshold ("band"), in any order: the part
+    // of the candidates the exact selection has to rank.  Without an upper bound: all of them.
+    unsigned long long* band[2];
     unsigned long long* buf[2][2];   // ping-pong lists of the candidate select
-    // ordering of the kept positions of the chosen side by tile (tile = 2^kTileShift positions)
-    uint32_t* tile_in;          // per tile: entries whose bucket slots the counting blocks reserved
-    uint32_t* tile_base;        // per tile: the other entries; then scanned in place to bucket starts (n_tiles + 1)
-    uint32_t* tile_fill;        // per tile: of those other entries, how many are already placed
-    uint32_t* blk_first;        // per counting block and window tile: first reserved slot in the bucket
     uint32_t* x_tile_cnt[2];
-    uint32_t* idx;              // sorted kept positions
-    unsigned long long* blk_len;
-    uint32_t cap;               // capacity of each candidate list
+    struct RangeSum* rng_sum;        // per warp range of the ordering kernels: what its kept entries add up to
+    struct RangeSum* blk_sum;        // the same per block (eight ranges)
+    struct RangeBase* blk_base;      // where each block starts (rank, bit offset, previous position)
+    uint32_t cap;               // capacity of each band list
+    uint32_t list_cap;          // slots of each ordered list
+    uint32_t cap_w;             // slots of one streaming warp's region
+    uint32_t main_warps;        // warps of the streaming pass that share this problem
+    uint32_t span_steps;        // steps (512 elements each) per span: 1, 2, 4 or 8
+    uint32_t n_spans;
+    uint32_t use_runs;          // 0: short-list form, only the band lists are needed
+    uint32_t chunk_cw;          // codewords per chunk-table entry
     uint32_t m;                 // sample size
     unsigned long long sample_step;  // 128-byte lines between sampled segments, 20 fractional bits
     uint32_t s_target;          // rank looked up in the sample (the same for both sides)
     uint32_t s_up;              // rank in the sample of the upper bound (0: no upper bound)
-    uint32_t n_xtiles, n_tiles, n_len_blocks, n_chunks;
+    uint32_t n_xtiles, n_chunks;
     unsigned long long payload_offset;
 };
 
@@ -195,7 +209,20 @@ __device__ __forceinline__ bool launch_needs_exact_route(const Batch& B) {
 
 // Kinds of work a kernel's grid is sized by (one prefix table per kind in a batch).
 enum WorkKind : int {
-    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_SCATTER, WK_TILE, WK_LEN, WK_ONE, WK_STREAM, WK_COUNT
+    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_ORDER, WK_ONE, WK_STREAM, WK_COUNT
+};
+
+// What the kept entries of one warp range of the ordering kernels add up to (see k_span_count).
+struct RangeSum {
+    uint32_t cnt;            // kept entries in the range
+    uint32_t first, last;    // position of the first and the last of them (cnt > 0)
+    uint32_t pad_;
+    unsigned long long inner_bits;  // code lengths of all of them but the first (whose gap reaches into an earlier range)
+};
+struct RangeBase {
+    uint32_t rank;           // kept entries before the range
+    uint32_t prev_plus1;     // position of the last of those, plus one (0: none)
+    unsigned long long bit;  // payload bits before the range
 };
 
 // ---------------------------------------------------------------- keys
@@ -222,30 +249,33 @@ __device__ __forceinline__ unsigned long long make_composite(uint32_t skey, uint
 }
 __device__ __forceinline__ uint32_t composite_index(unsigned long long c) { return ~(uint32_t)c; }
 
-// A candidate list as the kernels after the candidate pass see it: entries [0, sure) sit at the
-// front of the buffer, entries [sure, total) at its back in reverse.  Every sure entry is larger
-// than every band entry.  The exact route rebuilds the list front to back (sure == total).
-struct CandView {
+// What the exact selection ranks and the exact sums read.  Fast route: the band list (every
+// candidate below the sample's upper bound of the threshold; all `sure` entries above it are kept
+// and already summed), with the rank reduced by the sure entries.  Exact route: the rebuilt list
+// itself, which then holds nothing else (densely packed from slot 0).
+struct BandView {
     const unsigned long long* src;
-    uint32_t sure, total, cap;
-    __device__ __forceinline__ unsigned long long at(uint32_t i) const {
-        return i < sure ? src[i] : src[cap - 1u - (i - sure)];
-    }
+    uint32_t count;  // entries
+    uint32_t rank;   // the k-th largest candidate is the rank-th largest of these
 };
-__device__ __forceinline__ CandView cand_view(const Prob& P, const Ctl* ctl, int s) {
-    CandView v;
-    v.src = P.cand[s];
-    v.cap = P.cap;
-    v.total = min(ctl->cand_cnt[s], P.cap);
-    v.sure = ctl->use_fallback ? v.total : min(ctl->sure_cnt[s], v.total);
+__device__ __forceinline__ BandView band_view(const Prob& P, const Ctl* ctl, int s) {
+    BandView v;
+    if (ctl->use_fallback) {
+        v.src = P.list[s];
+        v.count = min(ctl->cand_cnt[s], P.list_cap);
+        v.rank = (uint32_t)P.k;
+    } else {
+        v.src = P.band[s];
+        v.count = min(ctl->band_cnt[s], P.cap);
+        v.rank = (uint32_t)P.k - min(ctl->sure_cnt[s], (uint32_t)P.k - 1u);  // sure < k on this route
+    }
     return v;
 }
-// The part of the list that holds the k-th largest entry, and that entry's rank inside the part:
-// the band when fewer than k entries are sure (the usual case), else the sure part.
-__device__ __forceinline__ void select_range(const CandView& v, uint32_t k, uint32_t* begin, uint32_t* count,
-                                             uint32_t* rank) {
-    if (v.sure < k) { *begin = v.sure; *count = v.total - v.sure; *rank = k - v.sure; }
-    else            { *begin = 0u;     *count = v.sure;           *rank = k; }
+
+// Codewords per chunk-table entry of a stream that carries k positions.
+__host__ __device__ __forceinline__ uint32_t chunk_codewords_for(unsigned long long k) {
+    (void)k;
+    return (uint32_t)kChunkCodewords;
 }
 
 // ---------------------------------------------------------------- scans
@@ -298,50 +328,6 @@ __device__ __forceinline__ bool last_block_ticket(uint32_t* counter, uint32_t n_
     bool last = s_is_last != 0u;
     if (last) __threadfence();
     return last;
-}
-
-// Shared-memory window of per-tile counters used by blocks that walk a contiguous span of a
-// nearly position-ordered list: tiles [base, base + kTileWindow), base a little before the tile
-// of the span's first entry.
-constexpr int kTileWindow = 1024;
-__device__ __forceinline__ uint32_t tile_window_base(uint32_t first_tile) {
-    return first_tile > 256u ? first_tile - 256u : 0u;
-}
-
-// One counter update per distinct `key` among the warp's `valid` lanes; returns each valid lane's
-// rank within its key group and, through *first, the counter value before the group's update (only
-// meaningful when WANT_OLD).  Fast path: every valid lane has the same key (the common case when
-// neighbouring list entries are neighbours in the tensor).  All 32 lanes must call.
-template <bool WANT_OLD>
-__device__ __forceinline__ uint32_t warp_group_add(uint32_t* counters, uint32_t key, bool valid, uint32_t* first) {
-    const unsigned active = __ballot_sync(0xffffffffu, valid);
-    if (active == 0u) return 0u;
-    const int lead = __ffs(active) - 1;
-    const uint32_t lead_key = __shfl_sync(0xffffffffu, key, lead);
-    const bool uniform = __all_sync(0xffffffffu, !valid || key == lead_key);
-    const unsigned lt = (1u << lane_id()) - 1u;
-    if (uniform) {
-        uint32_t old = 0u;
-        if ((int)lane_id() == lead) {
-            if (WANT_OLD) old = atomicAdd(&counters[key], (uint32_t)__popc(active));
-            else atomicAdd(&counters[key], (uint32_t)__popc(active));
-        }
-        if (WANT_OLD) *first = __shfl_sync(0xffffffffu, old, lead);
-        return (uint32_t)__popc(active & lt);
-    }
-    uint32_t rank = 0u, old = 0u;
-    if (valid) {
-        const unsigned peers = __match_any_sync(active, key);
-        const int leader = __ffs(peers) - 1;
-        if ((int)lane_id() == leader) {
-            if (WANT_OLD) old = atomicAdd(&counters[key], (uint32_t)__popc(peers));
-            else atomicAdd(&counters[key], (uint32_t)__popc(peers));
-        }
-        if (WANT_OLD) old = __shfl_sync(peers, old, leader);
-        rank = (uint32_t)__popc(peers & lt);
-    }
-    if (WANT_OLD) *first = old;
-    return rank;
 }
 
 // ---------------------------------------------------------------- histogram pick

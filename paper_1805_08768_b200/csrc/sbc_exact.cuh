@@ -21,7 +21,7 @@ __global__ void __launch_bounds__(kBlock) k_exact_hist(const Batch B) {
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
-    if (!exact_route_active(ctl)) return;
+    if (!exact_route_active(ctl) || ctl->x_known) return;  // thresholds already known: only the gathering is redone
     constexpr int kBins = (LEVEL == 2) ? 1024 : kHistBins;
     __shared__ uint32_t s_hist[2][kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
@@ -147,10 +147,13 @@ __global__ void __launch_bounds__(kBlock) k_exact_tiescan(const Batch B) {
     }
 }
 
-// Gather exactly k composites per side: everything strictly beyond the
-// threshold plus the lowest-index ties.  Each warp owns 512 consecutive
-// elements of a tile and walks them 32 at a time, so the rank of a tie is
-// (ties in earlier tiles) + (earlier warps) + (earlier steps) + (lower lanes).
+// Gather the composites of each side: everything strictly beyond the threshold plus the
+// lowest-index ties (exactly k when the route found the thresholds itself; everything at or beyond
+// the known bounds when only the gathering is redone).  A block takes a tile of kXTile elements,
+// its warps 512 consecutive elements each, walked 32 at a time, so the rank of a tie is
+// (ties in earlier tiles) + (earlier warps) + (earlier steps) + (lower lanes), and the entries of a
+// tile leave in position order: space for them is reserved with one atomic per tile and side, and
+// every span of the tile gets its record (offset, count) as in the streaming pass.
 __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
     if (B.prefix != nullptr && !launch_needs_exact_route(B)) return;  // batch: before looking for the block's problem
     __shared__ Prob s_prob;
@@ -159,17 +162,21 @@ __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
     Ctl* ctl = P.ctl;
     if (!exact_route_active(ctl)) return;
     constexpr int kSteps = kXTile / kBlock;  // 16 steps of 32 lanes per warp
-    __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    __shared__ uint32_t s_warp_ties[2][kBlock / 32];
+    constexpr int kWarps = kBlock / 32;
+    static_assert(kXTile / kWarps == kWarpChunk, "a warp of this kernel covers one step of the streaming pass");
+    __shared__ uint32_t s_warp_ties[2][kWarps];
+    __shared__ uint32_t s_warp_emit[2][kWarps + 1];
     __shared__ uint32_t s_base[2];
     const int warp = threadIdx.x >> 5, lane = lane_id();
+    const unsigned lt = (1u << lane) - 1u;
     const uint32_t thr[2] = {ctl->x_thr[0], ctl->x_thr[1]};
     const uint32_t take[2] = {ctl->x_ties_take[0], ctl->x_ties_take[1]};
     const bool ranked[2] = {tie_ranks_needed(ctl, 0), tie_ranks_needed(ctl, 1)};
     const bool one_sided = P.mode == kModeValues;  // magnitude selection has no second side
     const float* __restrict__ A = P.residual;
+    const uint32_t span_steps = P.span_steps;
     for (uint32_t tile = S.bx; tile < P.n_xtiles; tile += S.nb) {
-        const long long wbase = (long long)tile * kXTile + (long long)warp * (kXTile / (kBlock / 32));
+        const long long wbase = (long long)tile * kXTile + (long long)warp * kWarpChunk;
         uint32_t key[kSteps];
         unsigned inb = 0u;
 #pragma unroll
@@ -209,33 +216,54 @@ __global__ void __launch_bounds__(kBlock) k_exact_collect(const Batch B) {
                 const bool in = (inb >> j) & 1u;
                 const uint32_t sk = side_key(s, key[j]);
                 const unsigned tb = __ballot_sync(0xffffffffu, in && sk == thr[s]);
-                const uint32_t my_rank = run + __popc(tb & ((1u << lane) - 1u));
+                const uint32_t my_rank = run + __popc(tb & lt);
                 const bool keep = in && (sk > thr[s] || (sk == thr[s] && my_rank < take[s]));
                 emit[s] |= keep ? (1u << j) : 0u;
                 run += __popc(tb);
             }
         }
-        const uint32_t packed = (uint32_t)__popc(emit[0]) | ((uint32_t)__popc(emit[1]) << 16);
-        uint32_t total;
-        const uint32_t excl = block_exclusive_scan<uint32_t>(packed, s_scan, &total);
-        if (threadIdx.x == 0) {
-            s_base[0] = (total & 0xffffu) ? atomicAdd(&ctl->cand_cnt[0], total & 0xffffu) : 0u;
-            s_base[1] = (total >> 16) ? atomicAdd(&ctl->cand_cnt[1], total >> 16) : 0u;
+        // entries per warp and side; position order inside a warp is (step, lane)
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            uint32_t wt = 0u;
+#pragma unroll
+            for (int j = 0; j < kSteps; ++j) wt += __popc(__ballot_sync(0xffffffffu, (emit[s] >> j) & 1u));
+            if (lane == 0) s_warp_emit[s][warp] = wt;
+        }
+        __syncthreads();
+        if (threadIdx.x < 2) {  // one thread per side: exclusive scan over the warps, then the tile's reservation
+            const int s = threadIdx.x;
+            uint32_t run = 0u;
+            for (int w = 0; w < kWarps; ++w) { const uint32_t v = s_warp_emit[s][w]; s_warp_emit[s][w] = run; run += v; }
+            s_warp_emit[s][kWarps] = run;
+            s_base[s] = run ? atomicAdd(&ctl->cand_cnt[s], run) : 0u;
         }
         __syncthreads();
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
-            uint32_t pos = s_base[s] + (s ? (excl >> 16) : (excl & 0xffffu));
+            if (s == 1 && one_sided) continue;
+            const uint32_t first = s_base[s] + s_warp_emit[s][warp];
+            uint32_t pos = first;
 #pragma unroll
             for (int j = 0; j < kSteps; ++j) {
-                if ((emit[s] >> j) & 1u) {
-                    const long long i = wbase + j * 32 + lane;
-                    if (pos < P.cap) P.cand[s][pos] = make_composite(side_key(s, key[j]), (uint32_t)i);
-                    ++pos;
+                const bool mine = (emit[s] >> j) & 1u;
+                const unsigned mm = __ballot_sync(0xffffffffu, mine);
+                if (mine) {
+                    const uint32_t slot = pos + (uint32_t)__popc(mm & lt);
+                    if (slot < P.list_cap)
+                        P.list[s][slot] = make_composite(side_key(s, key[j]), (uint32_t)(wbase + j * 32 + lane));
                 }
+                pos += (uint32_t)__popc(mm);
+            }
+            // the span that starts with this warp's 512 elements: its warps' entries follow one another
+            if (P.use_runs && lane == 0 && (uint32_t)warp % span_steps == 0u) {
+                const uint32_t span = (tile * (uint32_t)kWarps + (uint32_t)warp) / span_steps;
+                const uint32_t end_warp = min((uint32_t)warp + span_steps, (uint32_t)kWarps);
+                if (span < P.n_spans)
+                    P.span_rec[s][span] = make_uint2(first, s_base[s] + s_warp_emit[s][end_warp] - first);
             }
         }
-        __syncthreads();  // s_base / s_warp_ties are reused by the next tile
+        __syncthreads();  // the shared arrays are reused by the next tile
     }
 }
 

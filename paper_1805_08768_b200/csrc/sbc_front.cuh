@@ -199,6 +199,7 @@ __global__ void __launch_bounds__(kBlock) k_sample2(const Batch B) {
             block_pick_desc(P.hists->s2[s], 1024, false, ctl->s_rank[s], s_scan, &s_pick);
             if (threadIdx.x == 0) {
                 const uint32_t skey = (pre[s] << 10) | s_pick.bin;
+                ctl->lo_key[s] = skey;  // the threshold itself: candidates are exactly the entries at or beyond it
                 if (s == 0) ctl->lo_f = __uint_as_float(bits_of_key(skey));
                 else        ctl->hi_f = __uint_as_float(bits_of_key(~skey));
                 if (!s_pick.found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
@@ -212,198 +213,332 @@ __global__ void __launch_bounds__(kBlock) k_sample2(const Batch B) {
 
 constexpr int kUnroll = 4;                    // float4 loads per array per thread per step
 constexpr int kPerThread = 4 * kUnroll;       // elements per thread per step
-constexpr int kWarpChunk = 32 * kPerThread;   // elements per warp per step
+static_assert(32 * kPerThread == kWarpChunk, "one warp step covers kWarpChunk elements");
 constexpr int kStage = 128;                   // staged candidates per warp per side
+constexpr int kBandStage = 64;                // staged band entries per warp per side (flushed from 32 on)
 constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 warps, 128 B in flight per thread)
 
-// The streaming pass: A = R + dW written over R (12 bytes per element), two
-// float compares per element, and a rare append of (key, index) composites
-// through per-warp shared-memory staging so that the global list counters see
-// one atomic per hundred or so candidates.  Each thread has eight 16-byte
-// loads in flight before it touches any of them.
+// The streaming pass: A = R + dW written over R (12 bytes per element), two float compares per
+// element, and a rare append of (key, index) composites.  Each thread has eight 16-byte loads in
+// flight before it touches any of them.
+//
+// A warp works through whole spans (span_steps consecutive steps of 512 elements), span after
+// span in ascending order, and appends each side's candidates, in position order, to a region of
+// the ordered list that belongs to this warp alone: no atomics, nothing to wait for.  Where a
+// span's entries start in the region and how many they are goes into the span's record, which is
+// all a later kernel needs to walk the candidates of the whole tensor in position order.
+// Candidates pass through a per-warp shared-memory stage so that the region is written in full
+// lines.  While a stage is flushed, entries at or above the sample's upper bound of the threshold
+// ("sure": known to be kept) are added to the exact sums right away; the others ("band") are also
+// copied to the unordered band list the exact selection works on (one atomic per 32 or more).
 template <int MODE>
-__global__ void __launch_bounds__(kBlock, 4) k_add_collect(const Batch B) {
+__global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
-    __shared__ unsigned long long s_stage[kBlock / 32][2][kStage];
+    constexpr int kSides = (MODE == kModeValues) ? 1 : 2;
+    // A staged candidate is the pair (bit pattern of A_i, i): everything else (key, composite,
+    // checks, sums) is done when the stage is flushed, by 32 lanes at a time, and not when the
+    // candidate is found, by the one lane that holds it.
+    __shared__ uint2 s_stage[kBlock / 32][2][kStage];
+    __shared__ unsigned long long s_bstage[kBlock / 32][2][kBandStage];
+    __shared__ unsigned long long s_bins[2][256];
     const int warp = threadIdx.x >> 5, lane = lane_id();
+    const unsigned lt = (1u << lane) - 1u;
     const float lo = ctl->lo_f, hi = ctl->hi_f;
     const long long n = P.n;
     const float* __restrict__ U = P.update;
     float* __restrict__ R = P.residual;
-    uint32_t wcnt[2] = {0u, 0u};
-    bool bad = false;
-    const uint32_t cap = P.cap;
-    unsigned long long* const cand0 = P.cand[0];
-    unsigned long long* const cand1 = P.cand[1];
     const bool vec_ok = P.vec_ok != 0;
-
+    const bool use_runs = P.use_runs != 0u;
+    const uint32_t cap_w = P.cap_w, band_cap = P.cap;
     const uint32_t up_key0 = ctl->up_key[0], up_key1 = ctl->up_key[1];
+    // the exact sums of the sure entries: values within eight binades of the upper bound's are added
+    // in one register per side (units of the lowest of those binades), the rest in shared bins
+    int bin_a[2];
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+        const uint32_t ub = bits_of_key(side_key(s, s ? up_key1 : up_key0));
+        bin_a[s] = max((int)((ub >> 23) & 0xffu) - 1, 0);
+    }
+    long long acc[2] = {0, 0};
+    s_bins[0][threadIdx.x] = 0ull;
+    s_bins[1][threadIdx.x] = 0ull;
+    __syncthreads();
 
-    // Staged candidates of one side go to the list: sure entries (key at or above the upper bound
-    // of the threshold) to its front, the others to its back, with ONE atomic for both ranges.
+    const uint32_t total_warps = S.nb * (kBlock / 32);
+    const uint32_t gw = S.bx * (kBlock / 32) + (uint32_t)warp;   // < P.main_warps: the grid is sized from the same plan
+    unsigned long long* const region0 = P.list[0] + (size_t)gw * cap_w;
+    unsigned long long* const region1 = P.list[1] + (size_t)gw * cap_w;
+    uint32_t wcnt[2] = {0u, 0u};   // staged, not yet in the region
+    uint32_t fill[2] = {0u, 0u};   // already in the region (or dropped, once it overflowed)
+    uint32_t bcnt[2] = {0u, 0u};   // staged band entries
+    uint32_t n_cand[2] = {0u, 0u}, n_sure[2] = {0u, 0u};
+    bool bad = false, overflow = false;
+
+    // Staged band entries of one side go to the band list (one atomic for all of them).
+    auto flush_band = [&](int s) {
+        const uint32_t cnt = bcnt[s];
+        if (cnt == 0u) return;  // warp-uniform
+        __syncwarp();
+        uint32_t first = 0u;
+        if (lane == 0) first = atomicAdd(&ctl->band_cnt[s], cnt);
+        first = __shfl_sync(0xffffffffu, first, 0);
+        unsigned long long* const dst = P.band[s];
+        if (first <= band_cap && cnt <= band_cap - first) {
+            for (uint32_t i = lane; i < cnt; i += 32u) dst[first + i] = s_bstage[warp][s][i];
+        } else {
+            overflow = true;
+        }
+        __syncwarp();
+        bcnt[s] = 0u;
+    };
+    // Staged candidates of one side go to the warp's region, in the order they were staged.
     auto flush = [&](int s) {
         const uint32_t cnt = wcnt[s];
         if (cnt == 0u) return;  // warp-uniform
         __syncwarp();
         const uint32_t up_key = s ? up_key1 : up_key0;
-        unsigned long long* const dst = s ? cand1 : cand0;
-        uint32_t n_sure = 0u;
+        unsigned long long* const dst = s ? region1 : region0;
+        const bool room = use_runs && fill[s] <= cap_w && cnt <= cap_w - fill[s];
+        if (use_runs && !room) overflow = true;
         for (uint32_t i0 = 0u; i0 < cnt; i0 += 32u) {
             const uint32_t i = i0 + lane;
-            const bool sure = i < cnt && (uint32_t)(s_stage[warp][s][i] >> 32) >= up_key;
-            n_sure += (uint32_t)__popc(__ballot_sync(0xffffffffu, sure));
-        }
-        const uint32_t n_band = cnt - n_sure;
-        unsigned long long old = 0ull;
-        if (lane == 0)
-            old = atomicAdd(&ctl->cand_cnt2[s], (unsigned long long)n_sure | ((unsigned long long)n_band << 32));
-        old = __shfl_sync(0xffffffffu, old, 0);
-        uint32_t front = (uint32_t)old, back = (uint32_t)(old >> 32);
-        // both ranges must stay clear of each other; a list that does not fit is rebuilt by the exact route
-        if ((unsigned long long)front + n_sure + (unsigned long long)back + n_band <= (unsigned long long)cap) {
-            const unsigned lt = (1u << lane) - 1u;
-            for (uint32_t i0 = 0u; i0 < cnt; i0 += 32u) {
-                const uint32_t i = i0 + lane;
-                const bool valid = i < cnt;
-                const unsigned long long c = valid ? s_stage[warp][s][i] : 0ull;
-                const bool sure = valid && (uint32_t)(c >> 32) >= up_key;
-                const unsigned ms = __ballot_sync(0xffffffffu, sure);
-                const unsigned mb = __ballot_sync(0xffffffffu, valid && !sure);
-                if (sure) dst[front + (uint32_t)__popc(ms & lt)] = c;
-                else if (valid) dst[cap - 1u - (back + (uint32_t)__popc(mb & lt))] = c;
-                front += (uint32_t)__popc(ms);
-                back += (uint32_t)__popc(mb);
+            const bool valid = i < cnt;
+            const uint2 e = valid ? s_stage[warp][s][i] : make_uint2(0u, 0u);
+            const uint32_t bits = e.x;
+            if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;   // padding lanes hold 0
+            const uint32_t skey = side_key(s, select_key(MODE, bits));
+            const unsigned long long c = make_composite(skey, e.y);
+            if (valid && room) dst[fill[s] + i] = c;
+            const bool sure = valid && skey >= up_key;
+            const unsigned mb = __ballot_sync(0xffffffffu, valid && !sure);
+            n_sure[s] += (uint32_t)__popc(__ballot_sync(0xffffffffu, sure));
+            if (MODE == kModeBinary && sure) {
+                const uint32_t ex = (bits >> 23) & 0xffu;
+                int m = (int)(bits & 0x7fffffu) | (ex ? 0x800000 : 0);
+                if (bits >> 31) m = -m;
+                const int bin = ex ? (int)ex - 1 : 0;
+                const uint32_t up = (uint32_t)(bin - bin_a[s]);
+                if (up < 8u) acc[s] += (long long)m << up;  // |m| < 2^24: at most 2^31 per entry, 2^62 over 2^31 entries
+                else atomicAdd(&s_bins[s][bin], (unsigned long long)(long long)m);
+            }
+            if (mb) {
+                if (valid && !sure) s_bstage[warp][s][bcnt[s] + (uint32_t)__popc(mb & lt)] = c;
+                bcnt[s] += (uint32_t)__popc(mb);
+                if (bcnt[s] >= 32u) flush_band(s);   // room for another round of 32 is kept at all times
             }
         }
         __syncwarp();
+        fill[s] += cnt;
         wcnt[s] = 0u;
     };
 
     const long long n_chunks = (n + kWarpChunk - 1) / kWarpChunk;
-    const long long total_warps = (long long)S.nb * (kBlock / 32);
-    for (long long chunk = (long long)S.bx * (kBlock / 32) + warp; chunk < n_chunks;
-         chunk += total_warps) {
-        const long long base = chunk * kWarpChunk;
-        float a[kPerThread];
-        unsigned inb = 0u;
-        const bool vec_layout = vec_ok && (base + kWarpChunk <= n);  // warp-uniform
-        if (vec_layout) {
-            // thread owns elements base + (u*32 + lane)*4 + {0..3}, u = 0..kUnroll-1
-            const float4* __restrict__ u4 = reinterpret_cast<const float4*>(U + base) + lane;
-            float4* __restrict__ r4 = reinterpret_cast<float4*>(R + base) + lane;
-            float4 x[kUnroll], r[kUnroll];
+    const uint32_t span_steps = P.span_steps, n_spans = P.n_spans;
+    for (uint32_t span = gw; span < n_spans; span += total_warps) {
+        const uint32_t span_first[2] = {fill[0] + wcnt[0], fill[1] + wcnt[1]};
+        for (uint32_t st = 0u; st < span_steps; ++st) {
+            const long long chunk = (long long)span * span_steps + st;
+            if (chunk >= n_chunks) break;
+            const long long base = chunk * kWarpChunk;
+            float a[kPerThread];
+            unsigned inb = 0u;
+            const bool vec_layout = vec_ok && (base + kWarpChunk <= n);  // warp-uniform
+            if (vec_layout) {
+                // thread owns elements base + (u*32 + lane)*4 + {0..3}, u = 0..kUnroll-1
+                const float4* __restrict__ u4 = reinterpret_cast<const float4*>(U + base) + lane;
+                float4* __restrict__ r4 = reinterpret_cast<float4*>(R + base) + lane;
+                float4 x[kUnroll], r[kUnroll];
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) { x[u] = __ldcs(u4 + u * 32); r[u] = __ldcs(r4 + u * 32); }
+                for (int u = 0; u < kUnroll; ++u) { x[u] = __ldcs(u4 + u * 32); r[u] = __ldcs(r4 + u * 32); }
 #pragma unroll
-            for (int u = 0; u < kUnroll; ++u) {
-                float4 y;
-                y.x = __fadd_rn(r[u].x, x[u].x); y.y = __fadd_rn(r[u].y, x[u].y);
-                y.z = __fadd_rn(r[u].z, x[u].z); y.w = __fadd_rn(r[u].w, x[u].w);
-                __stcs(r4 + u * 32, y);
-                a[4 * u + 0] = y.x; a[4 * u + 1] = y.y; a[4 * u + 2] = y.z; a[4 * u + 3] = y.w;
-            }
-            inb = (1u << kPerThread) - 1u;
-        } else {
-            // ragged tail or unaligned pointers: thread owns elements base + j*32 + lane
+                for (int u = 0; u < kUnroll; ++u) {
+                    float4 y;
+                    y.x = __fadd_rn(r[u].x, x[u].x); y.y = __fadd_rn(r[u].y, x[u].y);
+                    y.z = __fadd_rn(r[u].z, x[u].z); y.w = __fadd_rn(r[u].w, x[u].w);
+                    __stcs(r4 + u * 32, y);
+                    a[4 * u + 0] = y.x; a[4 * u + 1] = y.y; a[4 * u + 2] = y.z; a[4 * u + 3] = y.w;
+                }
+                inb = (1u << kPerThread) - 1u;
+            } else {
+                // ragged tail or unaligned pointers: thread owns elements base + j*32 + lane
 #pragma unroll
-            for (int j = 0; j < kPerThread; ++j) {
-                const long long e = base + j * 32 + lane;
-                a[j] = 0.f;
-                if (e < n) {
-                    a[j] = __fadd_rn(R[e], U[e]);
-                    R[e] = a[j];
-                    inb |= 1u << j;
+                for (int j = 0; j < kPerThread; ++j) {
+                    const long long e = base + j * 32 + lane;
+                    a[j] = 0.f;
+                    if (e < n) {
+                        a[j] = __fadd_rn(R[e], U[e]);
+                        R[e] = a[j];
+                        inb |= 1u << j;
+                    }
                 }
             }
-        }
-        unsigned pm = 0u, qm = 0u;
+            unsigned mask[2] = {0u, 0u};
 #pragma unroll
-        for (int j = 0; j < kPerThread; ++j) {
-            if (MODE == kModeValues) {
-                pm |= (!(fabsf(a[j]) < lo) ? 1u : 0u) << j;   // also true for NaN
-            } else {
-                pm |= (!(a[j] < lo) ? 1u : 0u) << j;          // also true for NaN
-                qm |= (!(a[j] > hi) ? 1u : 0u) << j;
+            for (int j = 0; j < kPerThread; ++j) {
+                if (MODE == kModeValues) {
+                    mask[0] |= (!(fabsf(a[j]) < lo) ? 1u : 0u) << j;   // also true for NaN
+                } else {
+                    mask[0] |= (!(a[j] < lo) ? 1u : 0u) << j;          // also true for NaN
+                    mask[1] |= (!(a[j] > hi) ? 1u : 0u) << j;
+                }
             }
-        }
-        pm &= inb;
-        qm &= inb;
-        if (__any_sync(0xffffffffu, (pm | qm) != 0u)) {
-            const uint32_t packed = (uint32_t)__popc(pm) | ((uint32_t)__popc(qm) << 16);
-            const uint32_t incl = warp_inclusive_scan(packed);
-            const uint32_t tot = __shfl_sync(0xffffffffu, incl, 31);
-            const uint32_t excl = incl - packed;
+            mask[0] &= inb;
+            mask[1] &= inb;
+            if (!__any_sync(0xffffffffu, (mask[0] | mask[1]) != 0u)) continue;
+            if (vec_layout) {
+                // Position order inside the step is (u, lane, element of the float4).  Per side and u,
+                // the number of candidates of every lane goes into one byte of a 64-bit word; one warp
+                // scan gives every (side, u, lane) its slot.
+                unsigned long long packed = 0ull;
 #pragma unroll
-            for (int s = 0; s < 2; ++s) {
-                const uint32_t tot_s = s ? (tot >> 16) : (tot & 0xffffu);
-                if (tot_s == 0u) continue;
-                if (wcnt[s] + tot_s > (uint32_t)kStage) flush(s);
-                const unsigned mask = s ? qm : pm;
-                if (tot_s > (uint32_t)kStage) {
-                    // more candidates in one step than the stage holds (dense ties): element slot by
-                    // element slot, at most 32 at a time, each round flushed at once
+                for (int s = 0; s < kSides; ++s)
+#pragma unroll
+                    for (int u = 0; u < kUnroll; ++u)
+                        packed |= (unsigned long long)__popc((mask[s] >> (4 * u)) & 0xfu) << (8 * (4 * s + u));
+                const unsigned long long incl = warp_inclusive_scan(packed);   // at most 128 per byte: no carries
+                const unsigned long long tot = __shfl_sync(0xffffffffu, incl, 31);
+                const unsigned long long excl = incl - packed;
+                const uint32_t idx0 = (uint32_t)base + (uint32_t)lane * 4u;
+#pragma unroll
+                for (int s = 0; s < kSides; ++s) {
+                    const uint32_t tot4 = (uint32_t)(tot >> (32 * s)), excl4 = (uint32_t)(excl >> (32 * s));
+                    const uint32_t tot_s = __dp4a(tot4, 0x01010101u, 0u);   // the four bytes added up
+                    if (tot_s == 0u) continue;  // warp-uniform
+                    n_cand[s] += tot_s;
+                    if (tot_s > (uint32_t)kStage) {
+                        // more candidates in one step than the stage holds (dense ties): row by row
+                        // (a row is one u, at most 128 candidates), the stage flushed in between
+#pragma unroll
+                        for (int u = 0; u < kUnroll; ++u) {
+                            const uint32_t t = (tot4 >> (8 * u)) & 0xffu;
+                            if (wcnt[s] + t > (uint32_t)kStage) flush(s);
+                            uint32_t slot = wcnt[s] + ((excl4 >> (8 * u)) & 0xffu);
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                if ((mask[s] >> (4 * u + q)) & 1u) {
+                                    s_stage[warp][s][slot] = make_uint2(__float_as_uint(a[4 * u + q]), idx0 + (uint32_t)(u * 128 + q));
+                                    ++slot;
+                                }
+                            }
+                            wcnt[s] += t;
+                        }
+                        continue;
+                    }
+                    if (wcnt[s] + tot_s > (uint32_t)kStage) flush(s);
+                    // element slots that hold a candidate in some lane: the others are skipped by the whole warp
+                    const unsigned any_lane = __reduce_or_sync(0xffffffffu, mask[s]);
+                    uint32_t row = wcnt[s];
+#pragma unroll
+                    for (int u = 0; u < kUnroll; ++u) {
+                        if (((any_lane >> (4 * u)) & 0xfu) == 0u) continue;  // warp-uniform
+                        uint32_t slot = row + ((excl4 >> (8 * u)) & 0xffu);
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            if (!((any_lane >> (4 * u + q)) & 1u)) continue;  // warp-uniform
+                            if ((mask[s] >> (4 * u + q)) & 1u) {
+                                s_stage[warp][s][slot] = make_uint2(__float_as_uint(a[4 * u + q]), idx0 + (uint32_t)(u * 128 + q));
+                                ++slot;
+                            }
+                        }
+                        row += (tot4 >> (8 * u)) & 0xffu;
+                    }
+                    wcnt[s] += tot_s;
+                }
+            } else {
+                // position order is (j, lane): one ballot per element slot
+#pragma unroll
+                for (int s = 0; s < kSides; ++s) {
 #pragma unroll 1
                     for (int j = 0; j < kPerThread; ++j) {
-                        const bool mine = (mask >> j) & 1u;
+                        const bool mine = (mask[s] >> j) & 1u;
                         const unsigned mm = __ballot_sync(0xffffffffu, mine);
                         if (mm == 0u) continue;
+                        const uint32_t t = (uint32_t)__popc(mm);
+                        if (wcnt[s] + t > (uint32_t)kStage) flush(s);
                         if (mine) {
                             float aj = a[0];  // a[j] without indexing the register array dynamically
 #pragma unroll
                             for (int jj = 1; jj < kPerThread; ++jj) aj = (jj == j) ? a[jj] : aj;
-                            const uint32_t bits = __float_as_uint(aj);
-                            if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;
-                            const long long e = vec_layout ? base + (long long)(((j >> 2) * 32 + lane) * 4 + (j & 3))
-                                                           : base + j * 32 + lane;
-                            s_stage[warp][s][__popc(mm & ((1u << lane) - 1u))] =
-                                make_composite(side_key(s, select_key(MODE, bits)), (uint32_t)e);
+                            s_stage[warp][s][wcnt[s] + (uint32_t)__popc(mm & lt)] =
+                                make_uint2(__float_as_uint(aj), (uint32_t)(base + j * 32 + lane));
                         }
-                        wcnt[s] = (uint32_t)__popc(mm);
-                        flush(s);
-                    }
-                    continue;
-                }
-                uint32_t off = (s ? (excl >> 16) : (excl & 0xffffu)) + wcnt[s];
-                wcnt[s] += tot_s;
-#pragma unroll
-                for (int j = 0; j < kPerThread; ++j) {
-                    if ((mask >> j) & 1u) {
-                        const uint32_t bits = __float_as_uint(a[j]);
-                        if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;
-                        const long long e = vec_layout ? base + (long long)(((j >> 2) * 32 + lane) * 4 + (j & 3))
-                                                       : base + j * 32 + lane;
-                        s_stage[warp][s][off] = make_composite(side_key(s, select_key(MODE, bits)), (uint32_t)e);
-                        ++off;
+                        wcnt[s] += t;
+                        n_cand[s] += t;
                     }
                 }
             }
             __syncwarp();
         }
+        // where this span's candidates sit (staged entries keep their order and follow the flushed ones)
+        if (use_runs && lane < kSides) {
+            const int s = lane;
+            P.span_rec[s][span] = make_uint2(gw * cap_w + (s ? span_first[1] : span_first[0]),
+                                             (s ? fill[1] + wcnt[1] - span_first[1] : fill[0] + wcnt[0] - span_first[0]));
+        }
     }
-    flush(0);
-    flush(1);
+#pragma unroll
+    for (int s = 0; s < kSides; ++s) {
+        flush(s);
+        flush_band(s);
+    }
     if (bad) atomicOr(&ctl->status, SBC_STATUS_NONFINITE);
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kSides; ++s) {
+            if (n_cand[s]) atomicAdd(&ctl->cand_cnt[s], n_cand[s]);
+            if (n_sure[s]) atomicAdd(&ctl->sure_cnt[s], n_sure[s]);
+        }
+        if (overflow) atomicOr(&ctl->overflow, 1u);
+    }
+    if (MODE == kModeBinary) {
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            long long v = acc[s];
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xffffffffu, v, d);
+            if (lane == 0 && v) atomicAdd(&s_bins[s][bin_a[s]], (unsigned long long)v);
+        }
+        __syncthreads();
+#pragma unroll
+        for (int s = 0; s < 2; ++s) {
+            const unsigned long long v = s_bins[s][threadIdx.x];
+            if (v) atomicAdd(reinterpret_cast<unsigned long long*>(&ctl->pre_bins[s][threadIdx.x]), v);
+        }
+    }
 
     if (last_block_ticket(&ctl->done[ST_COLLECT], S.nb)) {
         if (threadIdx.x == 0) {
-            const unsigned long long t0 = __ldcg(&ctl->cand_cnt2[0]), t1 = __ldcg(&ctl->cand_cnt2[1]);
-            const unsigned long long sum0 = (t0 & 0xffffffffull) + (t0 >> 32), sum1 = (t1 & 0xffffffffull) + (t1 >> 32);
-            const uint32_t c0 = (uint32_t)min(sum0, 0xffffffffull), c1 = (uint32_t)min(sum1, 0xffffffffull);
-            ctl->cand_cnt[0] = c0;
-            ctl->cand_cnt[1] = c1;
-            ctl->sure_cnt[0] = (uint32_t)t0;
-            ctl->sure_cnt[1] = (uint32_t)t1;
-            // exact modes: both lists must hold at least the k wanted entries; sampled mode: the
-            // lists ARE the kept sets and only have to be non-empty; either way they must fit
+            const uint32_t c0 = __ldcg(&ctl->cand_cnt[0]), c1 = __ldcg(&ctl->cand_cnt[1]);
+            const uint32_t u0 = __ldcg(&ctl->sure_cnt[0]), u1 = __ldcg(&ctl->sure_cnt[1]);
+            const bool spilled = __ldcg(&ctl->overflow) != 0u;
+            // exact modes: both lists must hold at least the k wanted entries, of which fewer than
+            // k may lie above the upper bound (else the bound was too low and says nothing);
+            // sampled mode: the lists ARE the kept sets and only have to be non-empty; either way
+            // they must fit
             const uint32_t need = P.sampled ? 1u : (uint32_t)P.k;
-            const bool ok = c0 >= need && c0 <= P.cap &&
-                            (MODE == kModeValues || (c1 >= need && c1 <= P.cap));
+            const bool counts_ok = c0 >= need && c0 <= P.cap && (MODE == kModeValues || (c1 >= need && c1 <= P.cap));
+            const bool bounds_ok = P.sampled || (u0 < (uint32_t)P.k && (MODE == kModeValues || u1 < (uint32_t)P.k));
+            const bool ok = counts_ok && bounds_ok && !spilled;
             ctl->use_fallback = ok ? 0u : 1u;
-            if (!ok) atomicOr(B.any_exact, 1u);
-            ctl->sampled_ok = (ok && P.sampled) ? 1u : 0u;
+            if (!ok) {
+                atomicOr(B.any_exact, 1u);
+                // The exact route rebuilds the lists.  If only the placement failed (a warp's region
+                // or a band list too small for unevenly spread candidates) the bounds still hold:
+                // everything at or beyond them is gathered again, this time with space reserved tile by tile.
+                if (counts_ok && bounds_ok) {
+                    ctl->x_known = 1u;
+                    ctl->x_thr[0] = ctl->lo_key[0];
+                    ctl->x_thr[1] = ctl->lo_key[1];
+                }
+                ctl->cand_cnt[0] = 0u;
+                ctl->cand_cnt[1] = 0u;
+                ctl->sure_cnt[0] = 0u;
+                ctl->sure_cnt[1] = 0u;
+            }
+            ctl->sampled_ok = (counts_ok && P.sampled) ? 1u : 0u;
         }
     }
 }

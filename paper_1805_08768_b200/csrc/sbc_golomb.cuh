@@ -1,10 +1,12 @@
-// Golomb position coding (Algorithm 3) and decoding (Algorithm 4).
+// Golomb position coding (Algorithm 3) of the kept positions, and the residual write-back at
+// those positions (Algorithm 1).
 //
-// Encode: kept positions bucketed by tile and ordered inside each tile -> ascending position list
-// -> per-codeword lengths q + 1 + b -> exclusive scan = bit offsets ->
-// every codeword ORs its own bits into the pre-zeroed payload.
-// Decode: one thread per chunk of kChunkCodewords codewords, started from the
-// chunk table (bit offset, previous position), adds mu into the dense tensor.
+// The candidates of the chosen side lie in position order, span by span (see k_add_collect).  Two
+// kernels walk them with the same split into warp ranges: k_span_count adds up, per range, how
+// many entries are kept and how many payload bits they take, and its last block turns the range
+// sums into the rank, bit offset and previous position every range starts from (and writes the
+// header); k_span_emit walks again and, for every kept entry, subtracts mu from the residual,
+// ORs the codeword into the pre-zeroed payload and writes the chunk-table entries.
 #pragma once
 #include "sbc_common.cuh"
 #include "../../include/sbc.h"
@@ -69,153 +71,7 @@ __device__ __forceinline__ void block_sort(uint32_t (&x)[E], uint32_t* s_swap) {
     }
 }
 
-// ---------------------------------------------------------------- mask -> sorted positions
-
-// Exclusive scan of the kept positions per tile (both counters of k_tile_count together) into
-// the bucket starts, in place over the second counter (one block); entry n_tiles receives the total.
-__global__ void __launch_bounds__(kBlock) k_tile_scan(const Batch B) {
-    __shared__ Prob s_prob;
-    const Slot S = resolve(B, &s_prob);
-    const Prob& P = s_prob;
-    Ctl* ctl = P.ctl;
-    if (ctl->status) return;
-    __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    uint32_t* __restrict__ cnt = P.tile_base;
-    const uint32_t* __restrict__ cnt_in = P.tile_in;
-    const uint32_t n_tiles = P.n_tiles;
-    constexpr int kPer = 8;
-    uint32_t carry = 0u;
-    for (uint32_t base = 0; base < n_tiles; base += kBlock * kPer) {
-        uint32_t v[kPer];
-        uint32_t sum = 0u;
-#pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            const uint32_t t = base + threadIdx.x * kPer + j;
-            v[j] = (t < n_tiles) ? cnt[t] + cnt_in[t] : 0u;
-            sum += v[j];
-        }
-        uint32_t total;
-        uint32_t run = carry + block_exclusive_scan<uint32_t>(sum, s_scan, &total);
-#pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            const uint32_t t = base + threadIdx.x * kPer + j;
-            if (t < n_tiles) cnt[t] = run;
-            run += v[j];
-        }
-        carry += total;
-    }
-    if (threadIdx.x == 0) {
-        cnt[n_tiles] = carry;
-        ctl->kept_total = carry;
-        if (carry != (uint32_t)P.k) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
-    }
-}
-
-// One bucket of up to E * kBlock positions, ordered in registers and written back.  All threads call.
-template <int E>
-__device__ __forceinline__ void sort_bucket_in_registers(uint32_t* list, uint32_t beg, uint32_t count, uint32_t* s_swap) {
-    uint32_t x[E];
-#pragma unroll
-    for (int r = 0; r < E; ++r) {
-        const uint32_t i = (uint32_t)r * kBlock + threadIdx.x;  // any assignment will do before the sort
-        x[r] = (i < count) ? list[beg + i] : 0xffffffffu;        // padding sorts to the end
-    }
-    block_sort<E>(x, s_swap);  // contains block-wide barriers: every load above precedes every store below
-#pragma unroll
-    for (int r = 0; r < E; ++r) {
-        const uint32_t i = threadIdx.x * (uint32_t)E + (uint32_t)r;
-        if (i < count) list[beg + i] = x[r];
-    }
-    __syncthreads();
-}
-
-// Put every tile's bucket of the position list in ascending order.  Up to 256 entries: each thread
-// ranks its entry against the others in shared memory.  Up to 1024: a bitonic network in
-// registers.  More: the entries set bits in a shared-memory bitmask of the tile, which is then read
-// out in order (popcount scan).
-__global__ void __launch_bounds__(kBlock) k_tile_sort(const Batch B) {
-    __shared__ Prob s_prob;
-    const Slot S = resolve(B, &s_prob);
-    const Prob& P = s_prob;
-    if (P.ctl->status) return;
-    // the bitmask is stored with one pad word per 32 so that thread t's 32 consecutive words
-    // (t*32 .. t*32+31 -> slots t*33 .. t*33+31) fall into 32 different banks for every t
-    __shared__ uint32_t s_mask[kTileWords + kTileWords / 32];
-    __shared__ uint32_t s_small[kBlock];
-    __shared__ uint32_t s_scan[kBlock / 32 + 1];
-    static_assert(kTileWords == 32 * kBlock, "one thread reads out 32 words of the tile's bitmask");
-    const uint32_t* __restrict__ tile_base = P.tile_base;
-    uint32_t* __restrict__ list = P.idx;
-    const uint32_t n_tiles = P.n_tiles;
-    for (uint32_t tile = S.bx; tile < n_tiles; tile += S.nb) {
-        const uint32_t beg = tile_base[tile], end = tile_base[tile + 1];
-        const uint32_t count = end - beg;
-        if (count <= 1u) continue;  // block-uniform
-        if (count <= (uint32_t)kBlock) {
-            const uint32_t x = (threadIdx.x < count) ? list[beg + threadIdx.x] : 0xffffffffu;
-            s_small[threadIdx.x] = x;
-            __syncthreads();
-            uint32_t rank = 0u;
-            for (uint32_t j = 0; j < count; ++j) rank += (s_small[j] < x) ? 1u : 0u;
-            if (threadIdx.x < count) list[beg + rank] = x;
-            __syncthreads();
-            continue;
-        }
-        if (count <= 4u * kBlock) {  // block-uniform: a bitonic network in registers (larger ones lose to the bitmask)
-            if (count <= 2u * kBlock) sort_bucket_in_registers<2>(list, beg, count, s_mask);
-            else sort_bucket_in_registers<4>(list, beg, count, s_mask);
-            continue;
-        }
-        for (int w = threadIdx.x; w < kTileWords + kTileWords / 32; w += kBlock) s_mask[w] = 0u;
-        __syncthreads();
-        for (uint32_t base = beg; base < end; base += 4 * kBlock) {  // four loads in flight per thread
-            uint32_t v[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t i = base + j * kBlock + threadIdx.x;
-                v[j] = (i < end) ? list[i] : 0xffffffffu;
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if (v[j] != 0xffffffffu) {
-                    const uint32_t r = v[j] & ((1u << kTileShift) - 1u);
-                    const uint32_t word = r >> 5;
-                    atomicOr(&s_mask[word + (word >> 5)], 1u << (r & 31u));
-                }
-            }
-        }
-        __syncthreads();
-        // read-out in position order: thread t owns words t*32 .. t*32+31
-        const uint32_t* mine_words = s_mask + threadIdx.x * 33;
-        uint32_t mine = 0u;
-#pragma unroll 8
-        for (int j = 0; j < 32; ++j) mine += __popc(mine_words[j]);
-        uint32_t total;
-        uint32_t at = beg + block_exclusive_scan<uint32_t>(mine, s_scan, &total);
-        if (mine) {
-            const uint32_t first = (tile << kTileShift) + ((uint32_t)threadIdx.x << 10);
-            for (int j = 0; j < 32; ++j) {
-                uint32_t w = mine_words[j];
-                while (w) {
-                    const uint32_t idx = first + ((uint32_t)j << 5) + (__ffs(w) - 1);
-                    w &= w - 1u;
-                    if (at < end) list[at] = idx;
-                    ++at;
-                }
-            }
-        }
-        __syncthreads();  // s_mask is cleared again for the next tile
-    }
-}
-
-// ---------------------------------------------------------------- lengths, offsets, header
-
-__device__ __forceinline__ unsigned long long codeword_len(const Prob& P, uint32_t i, uint32_t* gap) {
-    const long long prev = i ? (long long)P.idx[i - 1] : -1ll;
-    const uint32_t g = (uint32_t)((long long)P.idx[i] - prev - 1);  // gap - 1 of Algorithm 3
-    *gap = g;
-    return (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
-}
+// ---------------------------------------------------------------- header
 
 __device__ __forceinline__ void store_u32(uint8_t* p, uint32_t v) { *reinterpret_cast<uint32_t*>(p) = v; }
 __device__ __forceinline__ void store_u64(uint8_t* p, unsigned long long v) {
@@ -236,109 +92,9 @@ __device__ __forceinline__ void write_header(const Prob& P, Ctl* ctl, bool ok, u
     store_u32(h + 40, (uint32_t)P.b);
     store_u32(h + 44, ok ? (P.mode == kModeValues ? SBC_SIDE_VALUES : __ldcg(&ctl->side)) : 0u);
     store_u32(h + 48, ok ? __float_as_uint(__ldcg(&ctl->mu32)) : 0u);
-    store_u32(h + 52, SBC_CHUNK_CODEWORDS);
+    store_u32(h + 52, P.chunk_cw);
     store_u32(h + 56, ok ? P.n_chunks : 0u);
     store_u32(h + 60, __ldcg(&ctl->status));
-}
-
-// Scan of the per-block bit counts (written by other blocks: read from L2) and the container
-// header, which is written always, so that a failed encode still leaves a header that says why.
-// One block.
-__device__ __forceinline__ void block_len_scan_header(const Prob& P, Ctl* ctl, unsigned long long* s_scan) {
-    const bool ok = __ldcg(&ctl->status) == 0u;  // uniform: nothing writes status while this kernel runs
-    unsigned long long total = 0ull;
-    if (ok) {
-        constexpr int kPer = 8;
-        for (uint32_t base = 0; base < P.n_len_blocks; base += kBlock * kPer) {
-            unsigned long long v[kPer];
-            unsigned long long sum = 0ull;
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) {
-                const uint32_t t = base + threadIdx.x * kPer + j;
-                v[j] = (t < P.n_len_blocks) ? __ldcg(P.blk_len + t) : 0ull;
-                sum += v[j];
-            }
-            unsigned long long part;
-            unsigned long long run = total + block_exclusive_scan<unsigned long long>(sum, s_scan, &part);
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) {
-                const uint32_t t = base + threadIdx.x * kPer + j;
-                if (t < P.n_len_blocks) P.blk_len[t] = run;
-                run += v[j];
-            }
-            total += part;
-        }
-    }
-    if (threadIdx.x == 0) write_header(P, ctl, ok, total);
-}
-
-// Bits of each block of kLenBlock codewords, and -- since this is the first
-// walk over the ordered position list -- the residual write-back
-// R_j = A_j - mu at the kept positions (Algorithm 1), in address order.  The block that finishes
-// last scans the block bit counts and writes the container header.
-__global__ void __launch_bounds__(kBlock) k_len_sum_residual(const Batch B) {
-    __shared__ Prob s_prob;
-    const Slot S = resolve(B, &s_prob);
-    const Prob& P = s_prob;
-    Ctl* ctl = P.ctl;
-    const bool failed = ctl->status != 0u;  // uniform over the grid: no kernel of this stage sets it
-    __shared__ unsigned long long s_scan[kBlock / 32 + 1];
-    constexpr int kPer = kLenBlock / kBlock;
-    const float mu = ctl->mu32;
-    const uint32_t k = (uint32_t)P.k;
-    // values mode: the kept values themselves are sent (they sit between the chunk table and the
-    // payload, in position order) and nothing of them stays in the residual
-    float* values = (P.mode == kModeValues)
-        ? reinterpret_cast<float*>(P.stream + SBC_HEADER_BYTES + (size_t)P.n_chunks * SBC_CHUNK_ENTRY_BYTES)
-        : nullptr;
-    // R_j - mu as a fire-and-forget atomic add of -mu (no load round trip): the same single fp32
-    // rounding as the subtraction.  The hardware's atomic adder treats subnormal operands and
-    // results as zero, which cannot change the result while |mu| >= 2^-100: a subnormal R_j is less
-    // than a quarter ulp of mu, and a non-zero difference of two values that close is a multiple of
-    // 2^-124.  Smaller |mu| (zero included) takes the load / subtract / store path.
-    const bool by_atomic = values == nullptr && fabsf(mu) >= 7.888609052e-31f;  // 2^-100
-    for (uint32_t blk = S.bx; blk < (failed ? 0u : P.n_len_blocks); blk += S.nb) {
-        const uint32_t i0 = blk * kLenBlock + threadIdx.x * kPer;
-        uint32_t pos[kPer];
-#pragma unroll
-        for (int j = 0; j < kPer; ++j) pos[j] = (i0 + j < k) ? P.idx[i0 + j] : 0u;
-        if (by_atomic) {
-            // lane-contiguous: one warp instruction covers 32 neighbouring positions of the list, so
-            // that updates of the same DRAM row reach the memory together (0.43 -> 0.39 ms for
-            // 10.7 M positions over 4 GiB against four consecutive positions per thread)
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) {
-                const uint32_t i = blk * kLenBlock + (uint32_t)j * kBlock + threadIdx.x;
-                if (i < k) atomicAdd(P.residual + P.idx[i], -mu);
-            }
-        } else {
-            float r[kPer];
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) r[j] = (i0 + j < k) ? P.residual[pos[j]] : 0.f;
-#pragma unroll
-            for (int j = 0; j < kPer; ++j) {
-                if (i0 + j < k) {
-                    if (values) values[i0 + j] = r[j];
-                    P.residual[pos[j]] = __fsub_rn(r[j], values ? r[j] : mu);
-                }
-            }
-        }
-        long long prev = (i0 && i0 < k) ? (long long)P.idx[i0 - 1] : -1ll;
-        unsigned long long sum = 0ull;
-#pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            if (i0 + j < k) {
-                const uint32_t g = (uint32_t)((long long)pos[j] - prev - 1);
-                sum += (unsigned long long)(g >> P.b) + 1ull + (unsigned long long)P.b;
-                prev = pos[j];
-            }
-        }
-        unsigned long long total;
-        block_exclusive_scan<unsigned long long>(sum, s_scan, &total);
-        if (threadIdx.x == 0) P.blk_len[blk] = total;
-    }
-    // by the block that finishes last: bit offset of every block, total bits, header
-    if (last_block_ticket(&ctl->done[ST_LEN], S.nb)) block_len_scan_header(P, ctl, s_scan);
 }
 
 // ---------------------------------------------------------------- bit packer
@@ -358,18 +114,15 @@ __device__ __forceinline__ void or_bits(uint32_t* words, unsigned long long off,
 
 // Codeword i (gap g, Golomb parameter b) at stream bit `off`: q = g >> b ones, a zero, then g's low
 // b bits MSB first (Algorithm 3), ORed into the zeroed payload; the first codeword of a chunk also
-// writes the chunk's table entry (bit offset, position of the codeword before it, taken from the
-// ascending position list).
-// `words` holds the payload from stream bit `bit_base` on (the payload itself: 0; a staging buffer
-// in shared memory: the bit at which the buffer starts, a multiple of 32).
-__device__ __forceinline__ void pack_codeword(uint32_t* words, unsigned long long bit_base, uint8_t* table, uint32_t i,
-                                              unsigned long long off, uint32_t g, int b, const uint32_t* positions) {
-    if (i % kChunkCodewords == 0) {
-        uint8_t* e = table + (size_t)(i / kChunkCodewords) * SBC_CHUNK_ENTRY_BYTES;
+// writes the chunk's table entry (bit offset, position of the codeword before it: prev_plus1 - 1).
+__device__ __forceinline__ void pack_codeword(uint32_t* words, uint8_t* table, uint32_t chunk_cw, uint32_t i,
+                                              unsigned long long off, uint32_t g, int b, uint32_t prev_plus1) {
+    if (i % chunk_cw == 0u) {
+        uint8_t* e = table + (size_t)(i / chunk_cw) * SBC_CHUNK_ENTRY_BYTES;
         store_u64(e, off);
-        store_u64(e + 8, (unsigned long long)(i ? (long long)positions[i - 1] : -1ll));
+        store_u64(e + 8, (unsigned long long)((long long)prev_plus1 - 1ll));
     }
-    unsigned long long pos = off - bit_base;
+    unsigned long long pos = off;
     uint32_t q = g >> b;
     // q ones: head up to a word boundary, whole words, then the rest
     if (q) {
@@ -382,41 +135,266 @@ __device__ __forceinline__ void pack_codeword(uint32_t* words, unsigned long lon
     or_bits(words, pos, 1 + b, g & ((1u << b) - 1u));
 }
 
-// Bit offset of every codeword (block scan over the lengths) and the payload bits themselves, every
-// codeword ORed into the zeroed payload on its own.  (Putting a block's bit range together in
-// shared memory first and storing whole words was measured slower: 79 instead of 62 us for 10.7 M
-// codewords; the atomics of many blocks on the L2-resident payload do not wait for one another.)
-__global__ void __launch_bounds__(kBlock) k_pack(const Batch B) {
+// ---------------------------------------------------------------- candidates in position order
+
+// Calls on_batch(composite, valid) for every 32 consecutive entries of the position-ordered
+// candidates of spans [span0, span1) of side `s`, in ascending order; lane j of a call holds entry
+// 32 * call + j.  All 32 lanes call and on_batch runs warp-uniformly.  The records of 32 spans are
+// read at once; a batch may straddle spans (lane j finds its span by a search over the scanned counts).
+template <typename F>
+__device__ __forceinline__ void walk_spans(const Prob& P, int s, uint32_t span0, uint32_t span1, F&& on_batch) {
+    const uint2* __restrict__ rec = P.span_rec[s];
+    const unsigned long long* __restrict__ list = P.list[s];
+    const uint32_t lane = lane_id();
+    const uint32_t list_cap = P.list_cap;
+    for (uint32_t sp = span0; sp < span1; sp += 32u) {
+        uint2 r = make_uint2(0u, 0u);
+        if (sp + lane < span1) r = rec[sp + lane];
+        if (r.x > list_cap || r.y > list_cap - r.x) r.y = 0u;  // a record that points outside the list holds nothing
+        const uint32_t incl = warp_inclusive_scan(r.y);
+        const uint32_t total = __shfl_sync(0xffffffffu, incl, 31);
+        const uint32_t excl = incl - r.y;
+        for (uint32_t t0 = 0u; t0 < total; t0 += 32u) {
+            const uint32_t t = t0 + lane;
+            const bool valid = t < total;
+            // the span of entry t: the last lane whose exclusive count is <= t
+            uint32_t at = 0u;
+#pragma unroll
+            for (uint32_t step = 16u; step > 0u; step >>= 1) {
+                const uint32_t e = __shfl_sync(0xffffffffu, excl, (int)((at + step) & 31u));
+                if (at + step < 32u && e <= t) at += step;
+            }
+            const uint32_t off = __shfl_sync(0xffffffffu, r.x, (int)at);
+            const uint32_t ex = __shfl_sync(0xffffffffu, excl, (int)at);
+            const unsigned long long c = valid ? list[off + (t - ex)] : 0ull;
+            on_batch(c, valid);
+        }
+    }
+}
+
+// Spans [first, last) of warp range `r` when n_spans spans are split evenly over n_ranges ranges.
+__device__ __forceinline__ void range_spans(uint32_t n_spans, uint32_t n_ranges, uint32_t r, uint32_t* first, uint32_t* last) {
+    const uint32_t per = (n_spans + n_ranges - 1u) / n_ranges;
+    *first = min(n_spans, r * per);
+    *last = min(n_spans, *first + per);
+}
+
+// `A` followed by `B` (ranges that lie one after the other): the code lengths of B's first entry,
+// whose gap reaches back to A's last, becomes an inner one.
+__device__ __forceinline__ RangeSum fold_ranges(RangeSum A, const RangeSum& B, int b) {
+    if (B.cnt == 0u) return A;
+    if (A.cnt == 0u) return B;
+    const uint32_t g = B.first - (A.last + 1u);
+    A.inner_bits += (unsigned long long)(g >> b) + 1ull + (unsigned long long)b + B.inner_bits;
+    A.cnt += B.cnt;
+    A.last = B.last;
+    return A;
+}
+__device__ __forceinline__ RangeSum load_range_sum(const RangeSum* p) {
+    RangeSum r;
+    r.cnt = __ldcg(&p->cnt); r.first = __ldcg(&p->first); r.last = __ldcg(&p->last); r.pad_ = 0u;
+    r.inner_bits = __ldcg(&p->inner_bits);
+    return r;
+}
+
+// Per warp range: number of kept entries, first and last kept position, and the code lengths of
+// all kept entries but the first (its gap reaches back into an earlier range); the same for the
+// block's eight ranges together.  The last block to finish combines the blocks in order: for every
+// block the rank of its first kept entry, the position kept just before it and the bit offset of
+// its first codeword; then the header.
+__global__ void __launch_bounds__(kBlock) k_span_count(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
-    if (P.ctl->status) return;
-    __shared__ unsigned long long s_scan[kBlock / 32 + 1];
-    constexpr int kPer = kLenBlock / kBlock;
-    uint32_t* words = reinterpret_cast<uint32_t*>(P.stream + P.payload_offset);
-    uint8_t* table = P.stream + SBC_HEADER_BYTES;
+    Ctl* ctl = P.ctl;
+    const bool failed = ctl->status != 0u;  // uniform over the grid: no kernel of this stage sets it before the ticket
+    const int s = (int)ctl->side;
+    const unsigned long long thr = ctl->thr[s];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    const unsigned lt = (1u << lane) - 1u;
+    constexpr uint32_t kWarps = kBlock / 32;
+    const uint32_t n_ranges = S.nb * kWarps;
+    const uint32_t range = S.bx * kWarps + warp;
     const int b = P.b;
-    for (uint32_t blk = S.bx; blk < P.n_len_blocks; blk += S.nb) {
-        unsigned long long len[kPer];
-        uint32_t gap[kPer];
-        unsigned long long sum = 0ull;
+    __shared__ RangeSum s_rs[kWarps];
+    if (!failed) {
+        uint32_t span0, span1;
+        range_spans(P.n_spans, n_ranges, range, &span0, &span1);
+        uint32_t cnt = 0u, first = 0u, prev_plus1 = 0u;  // prev_plus1: last kept position so far, plus one
+        unsigned long long bits = 0ull;                    // per lane; summed over the warp at the end
+        walk_spans(P, s, span0, span1, [&](unsigned long long c, bool valid) {
+            const bool kept = valid && c >= thr;
+            const unsigned m = __ballot_sync(0xffffffffu, kept);
+            if (m == 0u) return;  // warp-uniform
+            const uint32_t pos = composite_index(c);
+            const unsigned lower = m & lt;
+            const uint32_t before = __shfl_sync(0xffffffffu, pos, lower ? 31 - __clz((int)lower) : 0);
+            const bool range_first = cnt == 0u && lower == 0u;   // the first kept entry of the range
+            if (kept && !range_first) {
+                const uint32_t g = pos - (lower ? before + 1u : prev_plus1);
+                bits += (unsigned long long)(g >> b) + 1ull + (unsigned long long)b;
+            }
+            if (cnt == 0u) first = __shfl_sync(0xffffffffu, pos, __ffs((int)m) - 1);
+            prev_plus1 = __shfl_sync(0xffffffffu, pos, 31 - __clz((int)m)) + 1u;
+            cnt += (uint32_t)__popc(m);
+        });
 #pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            const uint32_t i = blk * kLenBlock + threadIdx.x * kPer + j;
-            len[j] = 0ull;
-            gap[j] = 0u;
-            if (i < (uint32_t)P.k) len[j] = codeword_len(P, i, &gap[j]);
-            sum += len[j];
+        for (int d = 16; d > 0; d >>= 1) bits += __shfl_down_sync(0xffffffffu, bits, d);
+        if (lane == 0u) {
+            RangeSum rs;
+            rs.cnt = cnt; rs.first = first; rs.last = prev_plus1 - 1u; rs.pad_ = 0u; rs.inner_bits = bits;
+            P.rng_sum[range] = rs;
+            s_rs[warp] = rs;
         }
-        unsigned long long off = P.blk_len[blk] + block_exclusive_scan<unsigned long long>(sum, s_scan, nullptr);
-#pragma unroll
-        for (int j = 0; j < kPer; ++j) {
-            const uint32_t i = blk * kLenBlock + threadIdx.x * kPer + j;
-            if (i >= (uint32_t)P.k) continue;
-            pack_codeword(words, 0ull, table, i, off, gap[j], b, P.idx);
-            off += len[j];
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            RangeSum all = s_rs[0];
+            for (uint32_t w = 1; w < kWarps; ++w) all = fold_ranges(all, s_rs[w], b);
+            P.blk_sum[S.bx] = all;
         }
     }
+    if (!last_block_ticket(&ctl->done[ST_ORDER], S.nb)) return;
+    // ---- the last block: blocks in order.  Thread t takes blocks [t * per, (t + 1) * per).
+    __shared__ uint32_t s_scan[kBlock / 32 + 1];
+    __shared__ unsigned long long s_scan64[kBlock / 32 + 1];
+    __shared__ uint32_t s_last[kBlock];   // per thread: last kept position + 1 within its blocks (0: none)
+    __shared__ RangeSum s_blk[kOrderBlocksMax];
+    if (failed || S.nb > kOrderBlocksMax) {
+        if (threadIdx.x == 0) {
+            if (!failed) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+            write_header(P, ctl, false, 0ull);
+        }
+        return;
+    }
+    for (uint32_t i = threadIdx.x; i < S.nb; i += kBlock) s_blk[i] = load_range_sum(P.blk_sum + i);
+    __syncthreads();
+    const uint32_t per = (S.nb + kBlock - 1u) / kBlock;
+    const uint32_t r0 = min(S.nb, threadIdx.x * per), r1 = min(S.nb, r0 + per);
+    RangeSum mine;
+    mine.cnt = 0u; mine.first = 0u; mine.last = 0u; mine.pad_ = 0u; mine.inner_bits = 0ull;
+    for (uint32_t r = r0; r < r1; ++r) mine = fold_ranges(mine, s_blk[r], b);
+    s_last[threadIdx.x] = mine.cnt ? mine.last + 1u : 0u;
+    uint32_t total_cnt;
+    uint32_t rank = block_exclusive_scan<uint32_t>(mine.cnt, s_scan, &total_cnt);
+    // last kept position before this thread's blocks: the nearest earlier thread that has one
+    uint32_t pp = 0u;
+    for (int t = (int)threadIdx.x - 1; t >= 0; --t)
+        if (s_last[t]) { pp = s_last[t]; break; }
+    // bits of this thread's blocks, now that the gap of its first entry is known
+    const unsigned long long my_bits =
+        mine.cnt ? (unsigned long long)((mine.first - pp) >> b) + 1ull + (unsigned long long)b + mine.inner_bits : 0ull;
+    unsigned long long total_bits;
+    unsigned long long bit = block_exclusive_scan<unsigned long long>(my_bits, s_scan64, &total_bits);
+    for (uint32_t r = r0; r < r1; ++r) {
+        RangeBase rb;
+        rb.rank = rank; rb.prev_plus1 = pp; rb.bit = bit;
+        P.blk_base[r] = rb;
+        const RangeSum& q = s_blk[r];
+        if (q.cnt == 0u) continue;
+        bit += (unsigned long long)((q.first - pp) >> b) + 1ull + (unsigned long long)b + q.inner_bits;
+        pp = q.last + 1u;
+        rank += q.cnt;
+    }
+    if (threadIdx.x == 0) {
+        ctl->kept_total = total_cnt;
+        const bool ok = total_cnt == (uint32_t)P.k;
+        if (!ok) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
+        write_header(P, ctl, ok, ok ? total_bits : 0ull);
+    }
+}
+
+// Second walk: every kept entry gets its rank and bit offset from the range's start values and
+// does its three jobs -- R_j -= mu (Algorithm 1), its codeword into the payload, and, if it
+// opens a chunk, the chunk's table entry (Algorithm 3).  A warp instruction covers 32 neighbouring
+// list entries, i.e. neighbouring positions of the tensor, so that updates of the same DRAM row
+// reach the memory together.
+__global__ void __launch_bounds__(kBlock) k_span_emit(const Batch B) {
+    __shared__ Prob s_prob;
+    const Slot S = resolve(B, &s_prob);
+    const Prob& P = s_prob;
+    Ctl* ctl = P.ctl;
+    if (ctl->status != 0u) return;
+    const int s = (int)ctl->side;
+    const unsigned long long thr = ctl->thr[s];
+    const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
+    const unsigned lt = (1u << lane) - 1u;
+    const uint32_t n_ranges = S.nb * (kBlock / 32);
+    const uint32_t range = S.bx * (kBlock / 32) + warp;
+    const int b = P.b;
+    const float mu = ctl->mu32;
+    const uint32_t k = (uint32_t)P.k, chunk_cw = P.chunk_cw;
+    uint32_t* words = reinterpret_cast<uint32_t*>(P.stream + P.payload_offset);
+    uint8_t* table = P.stream + SBC_HEADER_BYTES;
+    float* __restrict__ R = P.residual;
+    // values mode: the kept values themselves are sent (they sit between the chunk table and the
+    // payload, in position order) and nothing of them stays in the residual
+    float* values = (P.mode == kModeValues)
+        ? reinterpret_cast<float*>(P.stream + SBC_HEADER_BYTES + (size_t)P.n_chunks * SBC_CHUNK_ENTRY_BYTES)
+        : nullptr;
+    // R_j - mu as a fire-and-forget atomic add of -mu (no load round trip): the same single fp32
+    // rounding as the subtraction.  The hardware's atomic adder treats subnormal operands and
+    // results as zero, which cannot change the result while |mu| >= 2^-100: a subnormal R_j is less
+    // than a quarter ulp of mu, and a non-zero difference of two values that close is a multiple of
+    // 2^-124.  Smaller |mu| (zero included) takes the load / subtract / store path.
+    const bool by_atomic = values == nullptr && fabsf(mu) >= 7.888609052e-31f;  // 2^-100
+    uint32_t span0, span1;
+    range_spans(P.n_spans, n_ranges, range, &span0, &span1);
+    // where this warp's range starts: the block's start values, advanced over the block's earlier ranges
+    const RangeBase rb = P.blk_base[S.bx];
+    uint32_t rank = rb.rank, prev_plus1 = rb.prev_plus1;
+    unsigned long long bit = rb.bit;
+    {
+        RangeSum mine;
+        mine.cnt = 0u; mine.first = 0u; mine.last = 0u; mine.pad_ = 0u; mine.inner_bits = 0ull;
+        if (lane < kBlock / 32) mine = P.rng_sum[S.bx * (kBlock / 32) + lane];
+        for (uint32_t w = 0; w < warp; ++w) {  // warp-uniform bound
+            const uint32_t c = __shfl_sync(0xffffffffu, mine.cnt, (int)w);
+            const uint32_t f = __shfl_sync(0xffffffffu, mine.first, (int)w);
+            const uint32_t l = __shfl_sync(0xffffffffu, mine.last, (int)w);
+            const unsigned long long in = __shfl_sync(0xffffffffu, mine.inner_bits, (int)w);
+            if (c == 0u) continue;
+            bit += (unsigned long long)((f - prev_plus1) >> b) + 1ull + (unsigned long long)b + in;
+            prev_plus1 = l + 1u;
+            rank += c;
+        }
+    }
+    walk_spans(P, s, span0, span1, [&](unsigned long long c, bool valid) {
+        const bool kept = valid && c >= thr;
+        const unsigned m = __ballot_sync(0xffffffffu, kept);
+        if (m == 0u) return;  // warp-uniform
+        const uint32_t pos = composite_index(c);
+        const unsigned lower = m & lt;
+        const uint32_t before = __shfl_sync(0xffffffffu, pos, lower ? 31 - __clz((int)lower) : 0);
+        const uint32_t pp = lower ? before + 1u : prev_plus1;   // previous kept position, plus one
+        const uint32_t g = kept ? pos - pp : 0u;
+        const unsigned long long len = kept ? (unsigned long long)(g >> b) + 1ull + (unsigned long long)b : 0ull;
+        // bit offsets: 32-bit scan unless a long unary run is among the 32 (then 64-bit)
+        unsigned long long off;
+        if (__any_sync(0xffffffffu, len >= (1ull << 26))) {
+            const unsigned long long incl = warp_inclusive_scan(len);
+            off = bit + incl - len;
+            bit += __shfl_sync(0xffffffffu, incl, 31);
+        } else {
+            const uint32_t incl = warp_inclusive_scan((uint32_t)len);
+            off = bit + (incl - (uint32_t)len);
+            bit += __shfl_sync(0xffffffffu, incl, 31);
+        }
+        if (kept) {
+            const uint32_t i = rank + (uint32_t)__popc(lower);
+            if (i < k && pos < (uint32_t)P.n) {
+                if (by_atomic) {
+                    atomicAdd(R + pos, -mu);
+                } else {
+                    const float r = R[pos];
+                    if (values) values[i] = r;
+                    R[pos] = __fsub_rn(r, values ? r : mu);
+                }
+                pack_codeword(words, table, chunk_cw, i, off, g, b, pp);
+            }
+        }
+        prev_plus1 = __shfl_sync(0xffffffffu, pos, 31 - __clz((int)m)) + 1u;
+        rank += (uint32_t)__popc(m);
+    });
 }
 
 }  // namespace sbc

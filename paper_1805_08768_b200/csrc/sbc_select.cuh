@@ -1,9 +1,8 @@
-// Exact k-th largest composite of each candidate list (Algorithm 2: exactly k
+// Exact k-th largest composite of each side's candidates (Algorithm 2: exactly k
 // kept entries, equal values ordered by index), by MSB-first radix selection
 // with 11-bit digits over the 64-bit composites.  Each level keeps only the
 // entries that fall in the selected bucket, so the lists shrink quickly.
-// Then the exact sums, the two means, the side choice and mu (Algorithm 2),
-// and the residual write-back at the kept positions (Algorithm 1).
+// Then the exact sums, the two means, the side choice and mu (Algorithm 2).
 #pragma once
 #include "sbc_common.cuh"
 #include "../../include/sbc.h"
@@ -23,10 +22,9 @@ __device__ __forceinline__ uint32_t digit_of(unsigned long long c, int level, in
 }
 // Highest composite bit in which the entries of the selected part of the list can differ, and
 // (through *base) the bits above it, which they all share.
-__device__ __forceinline__ int select_top(const Prob& P, const Ctl* ctl, int s, const CandView& v,
-                                          unsigned long long* base) {
+__device__ __forceinline__ int select_top(const Prob& P, const Ctl* ctl, int s, unsigned long long* base) {
     *base = 0ull;
-    if (ctl->use_fallback || v.sure >= (uint32_t)P.k) return 63;  // exact route, or ranking the certain part
+    if (ctl->use_fallback) return 63;  // exact route: the whole key range
     const uint32_t lo = ctl->lo_key[s], hi = ctl->up_key[s] - 1u;  // band keys lie in [lo, hi]
     const uint32_t diff = lo ^ hi;
     const int top = 32 + (diff ? 31 - __clz(diff) : -1);
@@ -104,18 +102,17 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
     __shared__ Pick s_pick;
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
-    const CandView view = cand_view(P, ctl, s);
-    uint32_t begin, cnt, rank;
-    select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
+    const BandView view = band_view(P, ctl, s);
+    const uint32_t cnt = view.count, rank = view.rank;
     unsigned long long shared_bits;
-    const int top = select_top(P, ctl, s, view, &shared_bits);
+    const int top = select_top(P, ctl, s, &shared_bits);
     constexpr int kItems = 4;  // loads in flight per thread
     for (uint32_t base = S.bx * (kBlock * kItems); base < cnt; base += S.nb * (kBlock * kItems)) {
         unsigned long long c[kItems];
 #pragma unroll
         for (int j = 0; j < kItems; ++j) {
             const uint32_t i = base + j * kBlock + threadIdx.x;
-            c[j] = (i < cnt) ? view.at(begin + i) : 0ull;
+            c[j] = (i < cnt) ? view.src[i] : 0ull;
         }
 #pragma unroll
         for (int j = 0; j < kItems; ++j) {
@@ -138,7 +135,7 @@ __global__ void __launch_bounds__(kBlock) k_select_hist0(const Batch B) {
 #pragma unroll
             for (int j = 0; j < kFinishPer; ++j) {
                 const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
-                c[j] = (i < cnt) ? view.at(begin + i) : 0ull;
+                c[j] = (i < cnt) ? view.src[i] : 0ull;
             }
             const bool good = block_select_registers<kFinishPer>(c, cnt, rank, top, 0, shared_bits, s_hist, s_scan, &s_pick,
                                                                  &s_result, &thr);
@@ -177,11 +174,10 @@ __global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
     __shared__ uint32_t s_hist[kHistBins];
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     __shared__ Pick s_pick;
-    const CandView view = cand_view(P, ctl, s);
-    uint32_t begin, cnt, rank;
-    select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
+    const BandView view = band_view(P, ctl, s);
+    const uint32_t cnt = view.count, rank = view.rank;
     unsigned long long prefix;
-    const int top = select_top(P, ctl, s, view, &prefix);
+    const int top = select_top(P, ctl, s, &prefix);
     if (cnt > kSmallList) {  // cannot happen: cnt <= cap <= kSmallList is what the host checked
         if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
         return;
@@ -190,7 +186,7 @@ __global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
 #pragma unroll
     for (int j = 0; j < kPer; ++j) {
         const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
-        c[j] = (i < cnt) ? view.at(begin + i) : 0ull;
+        c[j] = (i < cnt) ? view.src[i] : 0ull;
     }
     __shared__ unsigned long long s_result;
     unsigned long long thr = 0ull;
@@ -220,12 +216,11 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
     __shared__ Pick s_pick;
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
-    const CandView view = cand_view(P, ctl, s);
+    const BandView view = band_view(P, ctl, s);
     unsigned long long shared_bits;
-    const int top = select_top(P, ctl, s, view, &shared_bits);
+    const int top = select_top(P, ctl, s, &shared_bits);
     if (LEVEL + 1 >= digit_levels(top)) return;  // the previous level was the last one
-    uint32_t begin = 0u, cnt = ctl->list_cnt[s][LEVEL], rank0;
-    if (LEVEL == 0) select_range(view, (uint32_t)P.k, &begin, &cnt, &rank0);  // the part of the list hist0 looked at
+    const uint32_t cnt = LEVEL == 0 ? view.count : ctl->list_cnt[s][LEVEL];
     const unsigned long long* __restrict__ src = P.buf[s][(LEVEL + 1) & 1];  // the previous level's output
     unsigned long long* __restrict__ dst = P.buf[s][LEVEL & 1];
     const uint32_t sel = digit_of(ctl->b_prefix[s], LEVEL, top);
@@ -235,7 +230,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter(const Batch B) {
 #pragma unroll
         for (int j = 0; j < kItems; ++j) {
             const uint32_t i = base + j * kBlock + threadIdx.x;
-            c[j] = (i < cnt) ? (LEVEL == 0 ? view.at(begin + i) : src[i]) : 0ull;
+            c[j] = (i < cnt) ? (LEVEL == 0 ? view.src[i] : src[i]) : 0ull;
             const bool m = (i < cnt) && digit_of(c[j], LEVEL, top) == sel;
             match |= m ? (1u << j) : 0u;
             warp_hist_add(s_hist, digit_of(c[j], LEVEL + 1, top), m);
@@ -357,11 +352,13 @@ __device__ double bins_to_double(const long long* bins, const uint32_t* nonzero)
     return neg ? -mag : mag;
 }
 
-// Sum the kept values of both lists exactly: a value is m * 2^(e-150) with an
+// Sum the kept values of both sides exactly: a value is m * 2^(e-150) with an
 // integer m of at most 24 bits, so one 64-bit integer per exponent holds the
 // sum of up to 2^39 of them and integer addition makes the result independent
-// of the order of the atomics.  grid.z = side.  The last block turns the bins
-// into mu+ and mu- and takes Algorithm 2's side decision.
+// of the order of the atomics.  On the fast route the entries above the sample's upper bound of the
+// threshold were summed while the streaming pass flushed them (pre_bins); only the band is read
+// here.  grid.z = side.  The last block turns the bins into mu+ and mu- and takes Algorithm 2's
+// side decision.
 __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
@@ -374,11 +371,8 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     __shared__ unsigned long long s_bins[2][256];
     s_bins[0][threadIdx.x] = 0ull;
     __syncthreads();
-    const CandView view = cand_view(P, ctl, s);
+    const BandView view = band_view(P, ctl, s);
     const unsigned long long thr = ctl->thr[s];
-    // Almost every kept value shares the exponent of the threshold value or the
-    // next one up: those two bins are summed in registers, the rest goes
-    // straight to the shared bins.
     const uint32_t thr_bits = ctl->sampled_ok ? __float_as_uint(s ? ctl->hi_f : ctl->lo_f)
                             : values_mode ? (uint32_t)(thr >> 32) : bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
     // Values within eight binades of the threshold's (nearly all of them) are summed in one
@@ -398,23 +392,13 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     if (!values_mode) {  // the means exist only for the binarised form
         constexpr int kItems = 8;  // loads in flight per thread
         const uint32_t stride = S.nb * kBlock * kItems;
-        for (uint32_t base = S.bx * kBlock * kItems + threadIdx.x; base < view.sure; base += stride) {  // front of the list
+        for (uint32_t base = S.bx * kBlock * kItems + threadIdx.x; base < view.count; base += stride) {
             unsigned long long c[kItems];
 #pragma unroll
-            for (int j = 0; j < kItems; ++j) c[j] = (base + j * kBlock < view.sure) ? view.src[base + j * kBlock] : 0ull;
+            for (int j = 0; j < kItems; ++j) c[j] = (base + j * kBlock < view.count) ? view.src[base + j * kBlock] : 0ull;
 #pragma unroll
             for (int j = 0; j < kItems; ++j)
-                if (base + j * kBlock < view.sure && c[j] >= thr) add(c[j]);
-        }
-        const unsigned long long* __restrict__ back = view.src + (view.cap - 1u);
-        const uint32_t n_back = view.total - view.sure;
-        for (uint32_t base = S.bx * kBlock * kItems + threadIdx.x; base < n_back; base += stride) {  // its back
-            unsigned long long c[kItems];
-#pragma unroll
-            for (int j = 0; j < kItems; ++j) c[j] = (base + j * kBlock < n_back) ? *(back - (base + j * kBlock)) : 0ull;
-#pragma unroll
-            for (int j = 0; j < kItems; ++j)
-                if (base + j * kBlock < n_back && c[j] >= thr) add(c[j]);
+                if (base + j * kBlock < view.count && c[j] >= thr) add(c[j]);
         }
     }
 #pragma unroll
@@ -427,7 +411,10 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
     }
     if (last_block_ticket(&ctl->done[ST_SUM], values_mode ? S.nb : S.nb * gridDim.z)) {
         __shared__ uint32_t s_nonzero[2][8];
-        const long long b0 = __ldcg(&ctl->bins[0][threadIdx.x]), b1 = __ldcg(&ctl->bins[1][threadIdx.x]);
+        // fast route: every entry above the upper bound is kept and was summed when it was flushed
+        const bool pre = !ctl->use_fallback && !values_mode;
+        const long long b0 = __ldcg(&ctl->bins[0][threadIdx.x]) + (pre ? __ldcg(&ctl->pre_bins[0][threadIdx.x]) : 0ll);
+        const long long b1 = __ldcg(&ctl->bins[1][threadIdx.x]) + (pre ? __ldcg(&ctl->pre_bins[1][threadIdx.x]) : 0ll);
         s_bins[0][threadIdx.x] = (unsigned long long)b0;
         s_bins[1][threadIdx.x] = (unsigned long long)b1;
         bins_nonzero_masks(b0, s_nonzero[0]);
@@ -436,7 +423,7 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
         if (threadIdx.x < 2) {  // one thread per side rounds its exact sum
             const double sum = bins_to_double(reinterpret_cast<const long long*>(s_bins[threadIdx.x]), s_nonzero[threadIdx.x]);
             // mean over the k selected entries, or over however many the sampled threshold let through
-            const double count = ctl->sampled_ok ? (double)min(__ldcg(&ctl->cand_cnt[threadIdx.x]), P.cap) : (double)P.k;
+            const double count = ctl->sampled_ok ? (double)__ldcg(&ctl->cand_cnt[threadIdx.x]) : (double)P.k;
             ctl->mu64[threadIdx.x] = threadIdx.x ? -sum / count : sum / count;
         }
         __syncthreads();
@@ -448,113 +435,14 @@ __global__ void __launch_bounds__(kBlock) k_sums_decide(const Batch B) {
             ctl->side = side;
             ctl->mu32 = mu;
             if (P.out_mu) *P.out_mu = mu;
-            const uint32_t k_final = ctl->sampled_ok ? min(__ldcg(&ctl->cand_cnt[side]), P.cap) : (uint32_t)P.k;
+            const uint32_t k_final = ctl->sampled_ok ? __ldcg(&ctl->cand_cnt[side]) : (uint32_t)P.k;
             ctl->k_final = k_final;
             if (P.sampled) {  // the kernels that follow size their work from the descriptor
+                const uint32_t cw = chunk_codewords_for(k_final);
                 S.G->k = k_final;
-                S.G->n_len_blocks = (k_final + kLenBlock - 1) / kLenBlock;
-                S.G->n_chunks = (k_final + kChunkCodewords - 1) / kChunkCodewords;
+                S.G->chunk_cw = cw;
+                S.G->n_chunks = (k_final + cw - 1u) / cw;
                 S.G->payload_offset = SBC_HEADER_BYTES + (unsigned long long)S.G->n_chunks * SBC_CHUNK_ENTRY_BYTES;
-            }
-        }
-    }
-}
-
-// Ordering of the kept positions, step 1: how many fall into each tile (2^kTileShift consecutive
-// positions).  Each block walks one contiguous span of the chosen side's list.  The list is nearly
-// in position order, so a span touches few tiles: their counts are kept in a shared-memory window
-// and each is added to the tile's global count with ONE atomic, whose return value is at the same
-// time the block's reserved range in the tile's bucket (kept for k_scatter).  Entries outside the
-// window are counted one warp group at a time in a second per-tile counter.
-__global__ void __launch_bounds__(kBlock) k_tile_count(const Batch B) {
-    __shared__ Prob s_prob;
-    const Slot S = resolve(B, &s_prob);
-    const Prob& P = s_prob;
-    Ctl* ctl = P.ctl;
-    if (ctl->status) return;
-    const int s = (int)ctl->side;
-    const CandView view = cand_view(P, ctl, s);
-    const unsigned long long thr = ctl->thr[s];
-    uint32_t* __restrict__ tile_out = P.tile_base;
-    __shared__ uint32_t s_win[kTileWindow];
-    for (int w = threadIdx.x; w < kTileWindow; w += kBlock) s_win[w] = 0u;
-    const uint32_t span = ((view.total + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
-    const uint32_t lo = min(view.total, S.bx * span), hi = min(view.total, lo + span);
-    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(view.at(lo)) >> kTileShift : 0u);
-    __syncthreads();
-    constexpr int kItems = 4;  // loads in flight per thread
-    for (uint32_t base = lo; base < hi; base += kBlock * kItems) {
-        unsigned long long cs[kItems];
-#pragma unroll
-        for (int j = 0; j < kItems; ++j) {
-            const uint32_t i = base + j * kBlock + threadIdx.x;
-            cs[j] = (i < hi) ? view.at(i) : 0ull;
-        }
-#pragma unroll
-        for (int j = 0; j < kItems; ++j) {
-            const bool kept = (base + j * kBlock + threadIdx.x < hi) && cs[j] >= thr;
-            const uint32_t tile = composite_index(cs[j]) >> kTileShift;
-            const uint32_t rel = tile - win0;
-            if (kept && rel < (uint32_t)kTileWindow) atomicAdd(&s_win[rel], 1u);
-            warp_group_add<false>(tile_out, tile, kept && rel >= (uint32_t)kTileWindow, nullptr);
-        }
-    }
-    __syncthreads();
-    for (int w = threadIdx.x; w < kTileWindow; w += kBlock) {
-        const uint32_t c = s_win[w];
-        P.blk_first[(size_t)S.bx * kTileWindow + w] = c ? atomicAdd(&P.tile_in[win0 + w], c) : 0u;
-    }
-}
-
-// Step 3 (after the scan of the tile counts): every kept position goes into its tile's bucket of
-// the position list.  A bucket holds first the ranges the counting blocks reserved, then the
-// entries that were outside their block's window.  Inside a bucket the order is arbitrary;
-// k_tile_sort puts each bucket in order afterwards.  Same spans and windows as k_tile_count.
-__global__ void __launch_bounds__(kBlock) k_scatter(const Batch B) {
-    __shared__ Prob s_prob;
-    const Slot S = resolve(B, &s_prob);
-    const Prob& P = s_prob;
-    Ctl* ctl = P.ctl;
-    if (ctl->status) return;
-    const int s = (int)ctl->side;
-    const CandView view = cand_view(P, ctl, s);
-    const unsigned long long thr = ctl->thr[s];
-    const uint32_t* __restrict__ tile_base = P.tile_base;
-    const uint32_t* __restrict__ tile_in = P.tile_in;
-    uint32_t* __restrict__ tile_fill = P.tile_fill;
-    uint32_t* __restrict__ out = P.idx;
-    const uint32_t k = (uint32_t)P.k;
-    __shared__ uint32_t s_win[kTileWindow];
-    __shared__ uint32_t s_first[kTileWindow];
-    for (int w = threadIdx.x; w < kTileWindow; w += kBlock) {
-        s_win[w] = 0u;
-        s_first[w] = P.blk_first[(size_t)S.bx * kTileWindow + w];
-    }
-    const uint32_t span = ((view.total + S.nb - 1) / S.nb + kBlock - 1) / kBlock * kBlock;
-    const uint32_t lo = min(view.total, S.bx * span), hi = min(view.total, lo + span);
-    const uint32_t win0 = tile_window_base(lo < hi ? composite_index(view.at(lo)) >> kTileShift : 0u);
-    __syncthreads();
-    constexpr int kItems = 4;  // loads in flight per thread
-    for (uint32_t base = lo; base < hi; base += kBlock * kItems) {
-        unsigned long long cs[kItems];
-#pragma unroll
-        for (int j = 0; j < kItems; ++j) {
-            const uint32_t i = base + j * kBlock + threadIdx.x;
-            cs[j] = (i < hi) ? view.at(i) : 0ull;
-        }
-#pragma unroll
-        for (int j = 0; j < kItems; ++j) {
-            const bool kept = (base + j * kBlock + threadIdx.x < hi) && cs[j] >= thr;
-            const uint32_t idx = composite_index(cs[j]);
-            const uint32_t tile = idx >> kTileShift;
-            const uint32_t rel = tile - win0;
-            const bool in_win = rel < (uint32_t)kTileWindow;
-            uint32_t first_g = 0u;
-            const uint32_t rank_g = warp_group_add<true>(tile_fill, tile, kept && !in_win, &first_g);
-            if (kept) {
-                const uint32_t slot = tile_base[tile] + (in_win ? s_first[rel] + atomicAdd(&s_win[rel], 1u)
-                                                                : tile_in[tile] + first_g + rank_g);
-                if (slot < k) out[slot] = idx;
             }
         }
     }

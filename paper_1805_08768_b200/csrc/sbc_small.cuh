@@ -39,17 +39,16 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
     if (threadIdx.x == 0) s_status = __ldcg(&ctl->status);
     __syncthreads();
     if (s_status == 0u) {
-        const CandView view = cand_view(P, ctl, s);
-        uint32_t begin, cnt, rank;
-        select_range(view, (uint32_t)P.k, &begin, &cnt, &rank);
+        const BandView view = band_view(P, ctl, s);   // short lists have no upper bound: every candidate is in the band
+        const uint32_t cnt = view.count, rank = view.rank;
         unsigned long long prefix, thr = 0ull;
-        const int top = select_top(P, ctl, s, view, &prefix);
-        bool good = cnt <= kSmallList && view.total <= kSmallList;  // what the host checked through the capacity
+        const int top = select_top(P, ctl, s, &prefix);
+        bool good = cnt <= kSmallList;  // what the host checked through the capacity
         unsigned long long c[kPer];
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
-            c[j] = (good && i < cnt) ? view.at(begin + i) : 0ull;
+            c[j] = (good && i < cnt) ? view.src[i] : 0ull;
         }
         good = good && block_select_registers<kPer>(c, cnt, rank, top, 0, prefix, s_hist, s_scan, &s_pick, &s_result, &thr);
         if (!good) {
@@ -65,13 +64,13 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
             const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
             long long acc_a = 0;
             constexpr int kLoads = 4;  // list entries in flight per thread
-            for (uint32_t base = threadIdx.x; base < view.total; base += kBlock * kLoads) {
+            for (uint32_t base = threadIdx.x; base < cnt; base += kBlock * kLoads) {
                 unsigned long long e[kLoads];
 #pragma unroll
-                for (int j = 0; j < kLoads; ++j) e[j] = (base + j * kBlock < view.total) ? view.at(base + j * kBlock) : 0ull;
+                for (int j = 0; j < kLoads; ++j) e[j] = (base + j * kBlock < cnt) ? view.src[base + j * kBlock] : 0ull;
 #pragma unroll
                 for (int j = 0; j < kLoads; ++j) {
-                    if (base + j * kBlock >= view.total || e[j] < thr) continue;
+                    if (base + j * kBlock >= cnt || e[j] < thr) continue;
                     const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(e[j] >> 32)));
                     const uint32_t ex = (bits >> 23) & 0xffu;
                     int m = (int)(bits & 0x7fffffu) | (ex ? 0x800000 : 0);
@@ -119,19 +118,20 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
     for (uint32_t i = threadIdx.x; i < kSmallKept; i += kBlock) s_pos[i] = 0xffffffffu;
     __syncthreads();
     {
-        const CandView view = cand_view(P, ctl, (int)side);
+        const BandView view = band_view(P, ctl, (int)side);
+        const uint32_t total = min(view.count, kSmallList);
         const unsigned long long thr = __ldcg(&ctl->thr[side]);
         constexpr int kLoads = 4;  // list entries in flight per thread
-        for (uint32_t base = 0; base < view.total; base += kBlock * kLoads) {
+        for (uint32_t base = 0; base < total; base += kBlock * kLoads) {
             unsigned long long e[kLoads];
 #pragma unroll
             for (int j = 0; j < kLoads; ++j) {
                 const uint32_t i = base + j * kBlock + threadIdx.x;
-                e[j] = (i < view.total) ? view.at(i) : 0ull;
+                e[j] = (i < total) ? view.src[i] : 0ull;
             }
 #pragma unroll
             for (int j = 0; j < kLoads; ++j) {  // one slot reservation per warp and step
-                const bool kept = base + j * kBlock + threadIdx.x < view.total && e[j] >= thr;
+                const bool kept = base + j * kBlock + threadIdx.x < total && e[j] >= thr;
                 const unsigned mask = __ballot_sync(0xffffffffu, kept);
                 uint32_t first = 0u;
                 if (lane_id() == 0 && mask) first = atomicAdd(&s_count, (uint32_t)__popc(mask));
@@ -173,7 +173,6 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
         gap[j] = 0u;
         if (i < k) {
             P.residual[pos[j]] = __fsub_rn(r[j], mu);
-            P.idx[i] = pos[j];
             gap[j] = (uint32_t)((long long)pos[j] - prev - 1);
             prev = (long long)pos[j];
             len_sum += (unsigned long long)(gap[j] >> b) + 1ull + (unsigned long long)b;
@@ -196,7 +195,7 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
     for (int j = 0; j < kCw; ++j) {
         const uint32_t i = i0 + j;
         if (i < k) {
-            pack_codeword(target, 0ull, table, i, off, gap[j], b, s_pos);
+            pack_codeword(target, table, P.chunk_cw, i, off, gap[j], b, i ? s_pos[i - 1] + 1u : 0u);
             off += (unsigned long long)(gap[j] >> b) + 1ull + (unsigned long long)b;
         }
     }

@@ -119,20 +119,26 @@ def test_short_list_form_and_its_limits(n, p, kind):
     check_against_oracle(upd, res, p)
 
 
-# The kept positions are ordered bucket by bucket (2^18 positions each): up to 256 per bucket by
-# comparison counting, up to 512 and up to 1024 by register sorting networks of two sizes, more
-# through a bitmask of the bucket.  One case per form, plus uneven buckets (all kept entries in the
-# first tenth of the tensor), where neighbouring buckets take different forms.
+# The kept positions come out in order because the candidates are gathered span by span (1, 2, 4 or
+# 8 steps of 512 elements, by tensor size) into per-warp regions and walked in span order.  Sizes
+# on both sides of every span length, sparse and dense spans, and uneven ones (all kept entries in
+# the first tenth of the tensor: ten times the expected candidates per span there, none elsewhere).
 @pytest.mark.parametrize("n,p,clustered", [
-    (1 << 23, 0.0005, False),   # ~131 per bucket (k = 4194: beyond the one-kernel form for short lists)
-    (1 << 22, 0.0015, False),   # ~393
-    (1 << 21, 0.003, False),    # ~786
-    (3_000_001, 0.0039, False), # ~1020: around the upper limit of the larger network
-    (1 << 21, 0.006, False),    # ~1573: bitmask
-    (1 << 24, 0.0004, True),    # 6710 kept entries in the first seven buckets
-    (1 << 24, 0.00025, True),   # 4194 kept entries in the first seven buckets
+    (1 << 23, 0.0005, False),   # k = 4194: just beyond the one-kernel form for short lists
+    (1 << 22, 0.0015, False),
+    (1 << 21, 0.003, False),
+    (3_000_001, 0.0039, False),
+    (1 << 21, 0.006, False),
+    (1 << 24, 0.0004, True),
+    (1 << 24, 0.00025, True),
+    (7_272_960 + 17, 0.004, False),   # 14206 steps: one short of two two-step spans per warp -> one-step spans
+    (7_273_472 + 17, 0.004, False),   # 14207 steps: two-step spans
+    (14_546_437, 0.002, False),       # 28412 steps: still two-step spans
+    (14_546_949, 0.002, False),       # 28413 steps: four-step spans
+    (29_093_381, 0.001, False),       # 56824 steps: still four-step spans
+    (29_093_893, 0.001, False),       # 56825 steps: eight-step spans
 ])
-def test_bucket_ordering_forms(n, p, clustered):
+def test_span_ordering_forms(n, p, clustered):
     rng = np.random.default_rng(zlib.crc32(f"buckets/{n}/{p}/{clustered}".encode()))
     upd = rng.standard_normal(n).astype(np.float32) * np.float32(1e-3)
     if clustered:
@@ -205,9 +211,10 @@ def test_selection_looks_only_at_the_band_between_the_two_bounds():
         assert np.array_equal(res.view(np.uint32), want_res.view(np.uint32))
 
 
-def test_upper_bound_below_the_threshold_selects_among_the_certain_entries():
-    # large entries only where the strided sample does not look: both bounds come out too low,
-    # more than k candidates pass the upper one, and the k-th largest is found among those
+def test_upper_bound_below_the_threshold_takes_the_exact_route():
+    # large entries only where the strided sample does not look: both bounds come out too low and k
+    # or more candidates pass the upper one, so it says nothing about what is kept; the thresholds
+    # are then searched over the whole tensor
     n, p = 1 << 23, 0.01
     k = oracle.kept_count(n, p)
     rng = np.random.default_rng(7)
@@ -219,10 +226,42 @@ def test_upper_bound_below_the_threshold_selects_among_the_certain_entries():
     want_res = np.zeros(n, dtype=np.float32)
     want_stream, want_mu = oracle.encode(upd, want_res, p)
     stream, mu, res, diag = encode_with_diag(upd, p)
-    assert diag.exact_route == 0
-    assert diag.certain[0] >= k and diag.certain[1] >= k
+    assert diag.exact_route == 1 and diag.regathered == 0
     assert np.array_equal(stream, want_stream) and mu.view(np.uint32) == want_mu.view(np.uint32)
     assert np.array_equal(res.view(np.uint32), want_res.view(np.uint32))
+
+
+@pytest.mark.parametrize("n,p,where", [
+    (1 << 23, 0.01, "front"),      # every kept entry inside the first 2 % of the tensor
+    (1 << 23, 0.01, "stripe"),     # inside one stripe in the middle, not aligned to anything
+    (1 << 22, 0.01, "front"),
+    (3_000_001, 0.02, "tail"),     # at the ragged end
+])
+def test_clustered_candidates_are_gathered_again_with_the_bounds_kept(n, p, where):
+    """The streaming pass gives each warp a fixed region for its candidates.  When nearly all
+    candidates sit in a few neighbouring spans, a region overflows; the sample's bounds are still
+    right, so only the gathering is redone (space reserved tile by tile), not the threshold search."""
+    rng = np.random.default_rng(zlib.crc32(f"cluster/{n}/{p}/{where}".encode()))
+    upd = (rng.standard_normal(n) * 1e-6).astype(np.float32)
+    # the strided sample must still see the large values' distribution: scale a contiguous part
+    width = n // 50
+    start = {"front": 0, "stripe": n // 2 + 12345, "tail": n - width}[where]
+    upd[start:start + width] *= np.float32(1e3)
+    want_res = np.zeros(n, dtype=np.float32)
+    want_stream, want_mu = oracle.encode(upd, want_res, p)
+    stream, mu, res, diag = encode_with_diag(upd, p)
+    assert diag.exact_route == 1 and diag.regathered == 1
+    assert np.array_equal(stream, want_stream) and mu.view(np.uint32) == want_mu.view(np.uint32)
+    assert np.array_equal(res.view(np.uint32), want_res.view(np.uint32))
+
+
+@pytest.mark.parametrize("n,p", [(1 << 22, 0.3), (1 << 21, 0.6), (1 << 20, 0.9), (700_001, 0.45)])
+def test_dense_selections(n, p):
+    # more candidates in one step of a warp than its stage holds: the stage is flushed between quarters of the step
+    rng = np.random.default_rng(zlib.crc32(f"dense/{n}/{p}".encode()))
+    upd = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    res = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    check_against_oracle(upd, res, p)
 
 
 def test_multi_round_residual_carry():

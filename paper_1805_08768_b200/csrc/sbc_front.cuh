@@ -216,11 +216,110 @@ constexpr int kPerThread = 4 * kUnroll;       // elements per thread per step
 static_assert(32 * kPerThread == kWarpChunk, "one warp step covers kWarpChunk elements");
 constexpr int kStage = 128;                   // staged candidates per warp per side
 constexpr int kBandStage = 64;                // staged band entries per warp per side (flushed from 32 on)
-constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 warps, 128 B in flight per thread)
+constexpr int kCollectBlocksPerSM = 2;        // persistent blocks per SM (16 warps, each with 128 B per thread in flight nearly all the time)
+
+// Shared-memory state of the candidate stages of one block of the streaming pass.
+struct StageState {
+    // the same for all warps of the block
+    uint32_t up_key[2];
+    int bin_a[2];                     // lowest of the eight binades the register accumulators cover
+    uint32_t cap_w, band_cap, use_runs, pad_;
+    unsigned long long* band[2];
+    uint32_t* band_cnt[2];
+    // per warp and side
+    unsigned long long* region[kBlock / 32][2];
+    uint32_t fill[kBlock / 32][2];    // candidates already in the region (or dropped, once it overflowed)
+    uint32_t bcnt[kBlock / 32][2];    // staged band entries
+    uint32_t n_sure[kBlock / 32][2];
+    uint32_t flags[kBlock / 32];      // bit 0: a non-finite candidate, bit 1: a region or band list overflowed
+    uint2 stage[kBlock / 32][2][kStage];   // staged candidates: x = bit pattern of A_i, y = i
+    unsigned long long bstage[kBlock / 32][2][kBandStage];
+    unsigned long long bins[2][256];  // exact sums of sure entries outside the accumulators' binades
+};
+
+// The `cnt` staged band entries of one side go to the band list (one atomic for all of them).
+// All lanes call, with the same `cnt`; the caller sets its count of staged entries back to zero.
+__device__ __forceinline__ void flush_band_stage(StageState& st, int warp, int s, uint32_t cnt) {
+    if (cnt == 0u) return;  // warp-uniform
+    const uint32_t lane = lane_id();
+    __syncwarp();
+    uint32_t first = 0u;
+    if (lane == 0u) first = atomicAdd(st.band_cnt[s], cnt);
+    first = __shfl_sync(0xffffffffu, first, 0);
+    unsigned long long* const dst = st.band[s];
+    if (first <= st.band_cap && cnt <= st.band_cap - first) {
+        for (uint32_t i = lane; i < cnt; i += 32u) dst[first + i] = st.bstage[warp][s][i];
+    } else if (lane == 0u) {
+        st.flags[warp] |= 2u;
+    }
+    __syncwarp();
+}
+
+// The `cnt` staged candidates of side `s` of this warp go to the warp's region, in the order they
+// were staged.  A staged candidate is the pair (bit pattern of A_i, i): the key, the composite,
+// the non-finite check, the exact sums of the entries at or above the sample's upper bound of the
+// threshold ("sure": known to be kept) and the copy of the others ("band") to the band list are
+// all done here, by 32 lanes at a time, and not where the candidate is found, by the one lane that
+// holds it.  Returns the lane's accumulator of the exact sums, advanced.  One copy of this code
+// serves every place that flushes (the streaming kernel is large enough as it is, and its
+// instruction fetch showed).  All lanes call.
+template <int MODE>
+__device__ __noinline__ long long flush_stage(StageState& st, int warp, int s, uint32_t cnt, long long acc) {
+    const uint32_t lane = lane_id();
+    const unsigned lt = (1u << lane) - 1u;
+    __syncwarp();
+    const uint32_t up_key = st.up_key[s], cap_w = st.cap_w;
+    const int bin_a = st.bin_a[s];
+    const bool use_runs = st.use_runs != 0u;
+    unsigned long long* const dst = st.region[warp][s];
+    const uint32_t fill = st.fill[warp][s];
+    const bool room = use_runs && fill <= cap_w && cnt <= cap_w - fill;
+    uint32_t bcnt = st.bcnt[warp][s], n_sure = 0u, flags = (use_runs && !room) ? 2u : 0u;
+    for (uint32_t i0 = 0u; i0 < cnt; i0 += 32u) {
+        const uint32_t i = i0 + lane;
+        const bool valid = i < cnt;
+        const uint2 e = valid ? st.stage[warp][s][i] : make_uint2(0u, 0u);
+        const uint32_t bits = e.x;
+        if ((bits & 0x7f800000u) == 0x7f800000u) flags |= 1u;   // padding lanes hold 0
+        const uint32_t skey = side_key(s, select_key(MODE, bits));
+        const unsigned long long c = make_composite(skey, e.y);
+        if (valid && room) dst[fill + i] = c;
+        const bool sure = valid && skey >= up_key;
+        const unsigned mb = __ballot_sync(0xffffffffu, valid && !sure);
+        n_sure += (uint32_t)__popc(__ballot_sync(0xffffffffu, sure));
+        if (MODE == kModeBinary && sure) {
+            const uint32_t ex = (bits >> 23) & 0xffu;
+            int m = (int)(bits & 0x7fffffu) | (ex ? 0x800000 : 0);
+            if (bits >> 31) m = -m;
+            const int bin = ex ? (int)ex - 1 : 0;
+            const uint32_t up = (uint32_t)(bin - bin_a);
+            if (up < 8u) acc += (long long)m << up;  // |m| < 2^24: at most 2^31 per entry, 2^62 over 2^31 entries
+            else atomicAdd(&st.bins[s][bin], (unsigned long long)(long long)m);
+        }
+        if (mb) {
+            if (valid && !sure) st.bstage[warp][s][bcnt + (uint32_t)__popc(mb & lt)] = c;
+            bcnt += (uint32_t)__popc(mb);
+            if (bcnt >= 32u) {   // room for another round of 32 is kept at all times
+                flush_band_stage(st, warp, s, bcnt);
+                bcnt = 0u;
+            }
+        }
+    }
+    flags = __reduce_or_sync(0xffffffffu, flags);
+    __syncwarp();
+    if (lane == 0u) {
+        st.fill[warp][s] = fill + cnt;
+        st.bcnt[warp][s] = bcnt;
+        st.n_sure[warp][s] += n_sure;
+        if (flags) st.flags[warp] |= flags;
+    }
+    __syncwarp();
+    return acc;
+}
 
 // The streaming pass: A = R + dW written over R (12 bytes per element), two float compares per
 // element, and a rare append of (key, index) composites.  Each thread has eight 16-byte loads in
-// flight before it touches any of them.
+// flight, and the loads of the next step are issued before the step at hand is looked through.
 //
 // A warp works through whole spans (span_steps consecutive steps of 512 elements), span after
 // span in ascending order, and appends each side's candidates, in position order, to a region of
@@ -228,9 +327,7 @@ constexpr int kCollectBlocksPerSM = 3;        // persistent blocks per SM (24 wa
 // span's entries start in the region and how many they are goes into the span's record, which is
 // all a later kernel needs to walk the candidates of the whole tensor in position order.
 // Candidates pass through a per-warp shared-memory stage so that the region is written in full
-// lines.  While a stage is flushed, entries at or above the sample's upper bound of the threshold
-// ("sure": known to be kept) are added to the exact sums right away; the others ("band") are also
-// copied to the unordered band list the exact selection works on (one atomic per 32 or more).
+// lines (see flush_stage).
 template <int MODE>
 __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(const Batch B) {
     __shared__ Prob s_prob;
@@ -238,12 +335,7 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
     const Prob& P = s_prob;
     Ctl* ctl = P.ctl;
     constexpr int kSides = (MODE == kModeValues) ? 1 : 2;
-    // A staged candidate is the pair (bit pattern of A_i, i): everything else (key, composite,
-    // checks, sums) is done when the stage is flushed, by 32 lanes at a time, and not when the
-    // candidate is found, by the one lane that holds it.
-    __shared__ uint2 s_stage[kBlock / 32][2][kStage];
-    __shared__ unsigned long long s_bstage[kBlock / 32][2][kBandStage];
-    __shared__ unsigned long long s_bins[2][256];
+    __shared__ StageState st;
     const int warp = threadIdx.x >> 5, lane = lane_id();
     const unsigned lt = (1u << lane) - 1u;
     const float lo = ctl->lo_f, hi = ctl->hi_f;
@@ -252,107 +344,78 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
     float* __restrict__ R = P.residual;
     const bool vec_ok = P.vec_ok != 0;
     const bool use_runs = P.use_runs != 0u;
-    const uint32_t cap_w = P.cap_w, band_cap = P.cap;
-    const uint32_t up_key0 = ctl->up_key[0], up_key1 = ctl->up_key[1];
-    // the exact sums of the sure entries: values within eight binades of the upper bound's are added
-    // in one register per side (units of the lowest of those binades), the rest in shared bins
-    int bin_a[2];
-#pragma unroll
-    for (int s = 0; s < 2; ++s) {
-        const uint32_t ub = bits_of_key(side_key(s, s ? up_key1 : up_key0));
-        bin_a[s] = max((int)((ub >> 23) & 0xffu) - 1, 0);
-    }
-    long long acc[2] = {0, 0};
-    s_bins[0][threadIdx.x] = 0ull;
-    s_bins[1][threadIdx.x] = 0ull;
-    __syncthreads();
-
+    const uint32_t cap_w = P.cap_w;
     const uint32_t total_warps = S.nb * (kBlock / 32);
     const uint32_t gw = S.bx * (kBlock / 32) + (uint32_t)warp;   // < P.main_warps: the grid is sized from the same plan
-    unsigned long long* const region0 = P.list[0] + (size_t)gw * cap_w;
-    unsigned long long* const region1 = P.list[1] + (size_t)gw * cap_w;
+    if (threadIdx.x < 2) {
+        const int s = threadIdx.x;
+        const uint32_t up_key = ctl->up_key[s];
+        st.up_key[s] = up_key;
+        // the exact sums of the sure entries: values within eight binades of the upper bound's are added
+        // in one register per lane and side (units of the lowest of those binades), the rest in shared bins
+        const uint32_t ub = bits_of_key(side_key(s, up_key));
+        st.bin_a[s] = max((int)((ub >> 23) & 0xffu) - 1, 0);
+        st.band[s] = P.band[s];
+        st.band_cnt[s] = &ctl->band_cnt[s];
+        if (s == 0) { st.cap_w = cap_w; st.band_cap = P.cap; st.use_runs = P.use_runs; }
+    }
+    if (lane < 2) {
+        st.region[warp][lane] = P.list[lane] + (size_t)gw * cap_w;
+        st.fill[warp][lane] = 0u;
+        st.bcnt[warp][lane] = 0u;
+        st.n_sure[warp][lane] = 0u;
+        if (lane == 0) st.flags[warp] = 0u;
+    }
+    st.bins[0][threadIdx.x] = 0ull;
+    st.bins[1][threadIdx.x] = 0ull;
+    __syncthreads();
+    long long acc[2] = {0, 0};
     uint32_t wcnt[2] = {0u, 0u};   // staged, not yet in the region
-    uint32_t fill[2] = {0u, 0u};   // already in the region (or dropped, once it overflowed)
-    uint32_t bcnt[2] = {0u, 0u};   // staged band entries
-    uint32_t n_cand[2] = {0u, 0u}, n_sure[2] = {0u, 0u};
-    bool bad = false, overflow = false;
-
-    // Staged band entries of one side go to the band list (one atomic for all of them).
-    auto flush_band = [&](int s) {
-        const uint32_t cnt = bcnt[s];
-        if (cnt == 0u) return;  // warp-uniform
-        __syncwarp();
-        uint32_t first = 0u;
-        if (lane == 0) first = atomicAdd(&ctl->band_cnt[s], cnt);
-        first = __shfl_sync(0xffffffffu, first, 0);
-        unsigned long long* const dst = P.band[s];
-        if (first <= band_cap && cnt <= band_cap - first) {
-            for (uint32_t i = lane; i < cnt; i += 32u) dst[first + i] = s_bstage[warp][s][i];
-        } else {
-            overflow = true;
-        }
-        __syncwarp();
-        bcnt[s] = 0u;
-    };
-    // Staged candidates of one side go to the warp's region, in the order they were staged.
     auto flush = [&](int s) {
-        const uint32_t cnt = wcnt[s];
-        if (cnt == 0u) return;  // warp-uniform
-        __syncwarp();
-        const uint32_t up_key = s ? up_key1 : up_key0;
-        unsigned long long* const dst = s ? region1 : region0;
-        const bool room = use_runs && fill[s] <= cap_w && cnt <= cap_w - fill[s];
-        if (use_runs && !room) overflow = true;
-        for (uint32_t i0 = 0u; i0 < cnt; i0 += 32u) {
-            const uint32_t i = i0 + lane;
-            const bool valid = i < cnt;
-            const uint2 e = valid ? s_stage[warp][s][i] : make_uint2(0u, 0u);
-            const uint32_t bits = e.x;
-            if ((bits & 0x7f800000u) == 0x7f800000u) bad = true;   // padding lanes hold 0
-            const uint32_t skey = side_key(s, select_key(MODE, bits));
-            const unsigned long long c = make_composite(skey, e.y);
-            if (valid && room) dst[fill[s] + i] = c;
-            const bool sure = valid && skey >= up_key;
-            const unsigned mb = __ballot_sync(0xffffffffu, valid && !sure);
-            n_sure[s] += (uint32_t)__popc(__ballot_sync(0xffffffffu, sure));
-            if (MODE == kModeBinary && sure) {
-                const uint32_t ex = (bits >> 23) & 0xffu;
-                int m = (int)(bits & 0x7fffffu) | (ex ? 0x800000 : 0);
-                if (bits >> 31) m = -m;
-                const int bin = ex ? (int)ex - 1 : 0;
-                const uint32_t up = (uint32_t)(bin - bin_a[s]);
-                if (up < 8u) acc[s] += (long long)m << up;  // |m| < 2^24: at most 2^31 per entry, 2^62 over 2^31 entries
-                else atomicAdd(&s_bins[s][bin], (unsigned long long)(long long)m);
-            }
-            if (mb) {
-                if (valid && !sure) s_bstage[warp][s][bcnt[s] + (uint32_t)__popc(mb & lt)] = c;
-                bcnt[s] += (uint32_t)__popc(mb);
-                if (bcnt[s] >= 32u) flush_band(s);   // room for another round of 32 is kept at all times
-            }
-        }
-        __syncwarp();
-        fill[s] += cnt;
+        if (wcnt[s]) acc[s] = flush_stage<MODE>(st, warp, s, wcnt[s], acc[s]);
         wcnt[s] = 0u;
     };
 
     const long long n_chunks = (n + kWarpChunk - 1) / kWarpChunk;
-    const uint32_t span_steps = P.span_steps, n_spans = P.n_spans;
-    for (uint32_t span = gw; span < n_spans; span += total_warps) {
-        const uint32_t span_first[2] = {fill[0] + wcnt[0], fill[1] + wcnt[1]};
-        for (uint32_t st = 0u; st < span_steps; ++st) {
-            const long long chunk = (long long)span * span_steps + st;
-            if (chunk >= n_chunks) break;
+    const uint32_t span_steps = P.span_steps, n_spans = P.n_spans;   // span_steps is a power of two
+    const uint32_t step_shift = 31u - (uint32_t)__clz((int)span_steps);
+    // This warp's spans are gw, gw + total_warps, ...; its steps are numbered through: step t is
+    // step t % span_steps of its (t / span_steps)-th span.
+    const uint32_t my_spans = gw < n_spans ? (n_spans - gw + total_warps - 1u) / total_warps : 0u;
+    const uint32_t my_steps = my_spans << step_shift;
+    auto chunk_at = [&](uint32_t t) -> long long {   // chunk of step t; -1 past the end of the tensor
+        if (t >= my_steps) return -1ll;
+        const long long c = ((long long)gw + (long long)(t >> step_shift) * total_warps) * span_steps + (t & (span_steps - 1u));
+        return c < n_chunks ? c : -1ll;
+    };
+    // The loads of a step are issued while the step before it is still being looked through for
+    // candidates (the registers they land in are free by then), so that a warp has loads in flight
+    // nearly all the time.  Only whole, aligned chunks are loaded ahead.
+    float4 x[kUnroll], r[kUnroll];
+    auto load_ahead = [&](long long chunk) -> bool {
+        if (chunk < 0 || !vec_ok || (chunk + 1) * kWarpChunk > n) return false;  // warp-uniform
+        const float4* __restrict__ u4 = reinterpret_cast<const float4*>(U + chunk * kWarpChunk) + lane;
+        const float4* __restrict__ r4 = reinterpret_cast<const float4*>(R + chunk * kWarpChunk) + lane;
+#pragma unroll
+        for (int u = 0; u < kUnroll; ++u) { x[u] = __ldcs(u4 + u * 32); r[u] = __ldcs(r4 + u * 32); }
+        return true;
+    };
+    bool vec_layout = load_ahead(chunk_at(0u));
+    uint32_t span_first[2] = {0u, 0u};
+    for (uint32_t t = 0u; t < my_steps; ++t) {
+        const uint32_t span = gw + (t >> step_shift) * total_warps;
+        if ((t & (span_steps - 1u)) == 0u) {
+            span_first[0] = st.fill[warp][0] + wcnt[0];
+            span_first[1] = st.fill[warp][1] + wcnt[1];
+        }
+        const long long chunk = chunk_at(t);
+        if (chunk >= 0) {
             const long long base = chunk * kWarpChunk;
             float a[kPerThread];
             unsigned inb = 0u;
-            const bool vec_layout = vec_ok && (base + kWarpChunk <= n);  // warp-uniform
             if (vec_layout) {
                 // thread owns elements base + (u*32 + lane)*4 + {0..3}, u = 0..kUnroll-1
-                const float4* __restrict__ u4 = reinterpret_cast<const float4*>(U + base) + lane;
                 float4* __restrict__ r4 = reinterpret_cast<float4*>(R + base) + lane;
-                float4 x[kUnroll], r[kUnroll];
-#pragma unroll
-                for (int u = 0; u < kUnroll; ++u) { x[u] = __ldcs(u4 + u * 32); r[u] = __ldcs(r4 + u * 32); }
 #pragma unroll
                 for (int u = 0; u < kUnroll; ++u) {
                     float4 y;
@@ -375,6 +438,8 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
                     }
                 }
             }
+            const bool this_vec = vec_layout;
+            vec_layout = load_ahead(chunk_at(t + 1u));
             unsigned mask[2] = {0u, 0u};
 #pragma unroll
             for (int j = 0; j < kPerThread; ++j) {
@@ -387,17 +452,22 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
             }
             mask[0] &= inb;
             mask[1] &= inb;
-            if (!__any_sync(0xffffffffu, (mask[0] | mask[1]) != 0u)) continue;
-            if (vec_layout) {
+            if (__any_sync(0xffffffffu, (mask[0] | mask[1]) != 0u)) {
+            if (this_vec) {
                 // Position order inside the step is (u, lane, element of the float4).  Per side and u,
                 // the number of candidates of every lane goes into one byte of a 64-bit word; one warp
                 // scan gives every (side, u, lane) its slot.
                 unsigned long long packed = 0ull;
 #pragma unroll
-                for (int s = 0; s < kSides; ++s)
-#pragma unroll
-                    for (int u = 0; u < kUnroll; ++u)
-                        packed |= (unsigned long long)__popc((mask[s] >> (4 * u)) & 0xfu) << (8 * (4 * s + u));
+                for (int s = 0; s < kSides; ++s) {
+                    // bits set per nibble of the 16-bit mask, each count then moved into a byte of its own
+                    uint32_t c = mask[s];
+                    c = c - ((c >> 1) & 0x5555u);
+                    c = (c & 0x3333u) + ((c >> 2) & 0x3333u);
+                    c = (c | (c << 8)) & 0x00ff00ffu;
+                    c = (c | (c << 4)) & 0x0f0f0f0fu;
+                    packed |= (unsigned long long)c << (32 * s);
+                }
                 const unsigned long long incl = warp_inclusive_scan(packed);   // at most 128 per byte: no carries
                 const unsigned long long tot = __shfl_sync(0xffffffffu, incl, 31);
                 const unsigned long long excl = incl - packed;
@@ -407,41 +477,37 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
                     const uint32_t tot4 = (uint32_t)(tot >> (32 * s)), excl4 = (uint32_t)(excl >> (32 * s));
                     const uint32_t tot_s = __dp4a(tot4, 0x01010101u, 0u);   // the four bytes added up
                     if (tot_s == 0u) continue;  // warp-uniform
-                    n_cand[s] += tot_s;
+                    uint2* const dst = &st.stage[warp][s][0];
                     if (tot_s > (uint32_t)kStage) {
                         // more candidates in one step than the stage holds (dense ties): row by row
                         // (a row is one u, at most 128 candidates), the stage flushed in between
 #pragma unroll
                         for (int u = 0; u < kUnroll; ++u) {
-                            const uint32_t t = (tot4 >> (8 * u)) & 0xffu;
-                            if (wcnt[s] + t > (uint32_t)kStage) flush(s);
+                            const uint32_t tu = (tot4 >> (8 * u)) & 0xffu;
+                            if (wcnt[s] + tu > (uint32_t)kStage) flush(s);
                             uint32_t slot = wcnt[s] + ((excl4 >> (8 * u)) & 0xffu);
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
-                                if ((mask[s] >> (4 * u + q)) & 1u) {
-                                    s_stage[warp][s][slot] = make_uint2(__float_as_uint(a[4 * u + q]), idx0 + (uint32_t)(u * 128 + q));
-                                    ++slot;
-                                }
+                                if ((mask[s] >> (4 * u + q)) & 1u) dst[slot] = make_uint2(__float_as_uint(a[4 * u + q]), idx0 + (uint32_t)(u * 128 + q));
+                                slot += (mask[s] >> (4 * u + q)) & 1u;
                             }
-                            wcnt[s] += t;
+                            wcnt[s] += tu;
                         }
                         continue;
                     }
                     if (wcnt[s] + tot_s > (uint32_t)kStage) flush(s);
-                    // element slots that hold a candidate in some lane: the others are skipped by the whole warp
+                    // rows (one u each) in which no lane holds a candidate are skipped by the whole warp
                     const unsigned any_lane = __reduce_or_sync(0xffffffffu, mask[s]);
                     uint32_t row = wcnt[s];
 #pragma unroll
                     for (int u = 0; u < kUnroll; ++u) {
                         if (((any_lane >> (4 * u)) & 0xfu) == 0u) continue;  // warp-uniform
+                        const uint32_t nib = (mask[s] >> (4 * u)) & 0xfu;
                         uint32_t slot = row + ((excl4 >> (8 * u)) & 0xffu);
 #pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            if (!((any_lane >> (4 * u + q)) & 1u)) continue;  // warp-uniform
-                            if ((mask[s] >> (4 * u + q)) & 1u) {
-                                s_stage[warp][s][slot] = make_uint2(__float_as_uint(a[4 * u + q]), idx0 + (uint32_t)(u * 128 + q));
-                                ++slot;
-                            }
+                        for (int q = 0; q < 4; ++q) {   // no branches: four predicated stores
+                            if ((nib >> q) & 1u) dst[slot] = make_uint2(__float_as_uint(a[4 * u + q]), idx0 + (uint32_t)(u * 128 + q));
+                            slot += (nib >> q) & 1u;
                         }
                         row += (tot4 >> (8 * u)) & 0xffu;
                     }
@@ -456,42 +522,41 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
                         const bool mine = (mask[s] >> j) & 1u;
                         const unsigned mm = __ballot_sync(0xffffffffu, mine);
                         if (mm == 0u) continue;
-                        const uint32_t t = (uint32_t)__popc(mm);
-                        if (wcnt[s] + t > (uint32_t)kStage) flush(s);
+                        const uint32_t tj = (uint32_t)__popc(mm);
+                        if (wcnt[s] + tj > (uint32_t)kStage) flush(s);
                         if (mine) {
                             float aj = a[0];  // a[j] without indexing the register array dynamically
 #pragma unroll
                             for (int jj = 1; jj < kPerThread; ++jj) aj = (jj == j) ? a[jj] : aj;
-                            s_stage[warp][s][wcnt[s] + (uint32_t)__popc(mm & lt)] =
+                            st.stage[warp][s][wcnt[s] + (uint32_t)__popc(mm & lt)] =
                                 make_uint2(__float_as_uint(aj), (uint32_t)(base + j * 32 + lane));
                         }
-                        wcnt[s] += t;
-                        n_cand[s] += t;
+                        wcnt[s] += tj;
                     }
                 }
             }
             __syncwarp();
+            }
         }
-        // where this span's candidates sit (staged entries keep their order and follow the flushed ones)
-        if (use_runs && lane < kSides) {
-            const int s = lane;
-            P.span_rec[s][span] = make_uint2(gw * cap_w + (s ? span_first[1] : span_first[0]),
-                                             (s ? fill[1] + wcnt[1] - span_first[1] : fill[0] + wcnt[0] - span_first[0]));
-        }
+        // end of a span: its record says where its candidates sit (staged entries keep their order
+        // and follow the flushed ones)
+        if ((t & (span_steps - 1u)) == span_steps - 1u && use_runs && lane < kSides)
+            P.span_rec[lane][span] = make_uint2(gw * cap_w + (lane ? span_first[1] : span_first[0]),
+                                                st.fill[warp][lane] + (lane ? wcnt[1] - span_first[1] : wcnt[0] - span_first[0]));
     }
 #pragma unroll
     for (int s = 0; s < kSides; ++s) {
         flush(s);
-        flush_band(s);
+        flush_band_stage(st, warp, s, st.bcnt[warp][s]);
     }
-    if (bad) atomicOr(&ctl->status, SBC_STATUS_NONFINITE);
     if (lane == 0) {
 #pragma unroll
         for (int s = 0; s < kSides; ++s) {
-            if (n_cand[s]) atomicAdd(&ctl->cand_cnt[s], n_cand[s]);
-            if (n_sure[s]) atomicAdd(&ctl->sure_cnt[s], n_sure[s]);
+            if (st.fill[warp][s]) atomicAdd(&ctl->cand_cnt[s], st.fill[warp][s]);
+            if (st.n_sure[warp][s]) atomicAdd(&ctl->sure_cnt[s], st.n_sure[warp][s]);
         }
-        if (overflow) atomicOr(&ctl->overflow, 1u);
+        if (st.flags[warp] & 1u) atomicOr(&ctl->status, SBC_STATUS_NONFINITE);
+        if (st.flags[warp] & 2u) atomicOr(&ctl->overflow, 1u);
     }
     if (MODE == kModeBinary) {
 #pragma unroll
@@ -499,12 +564,12 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
             long long v = acc[s];
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xffffffffu, v, d);
-            if (lane == 0 && v) atomicAdd(&s_bins[s][bin_a[s]], (unsigned long long)v);
+            if (lane == 0 && v) atomicAdd(&st.bins[s][st.bin_a[s]], (unsigned long long)v);
         }
         __syncthreads();
 #pragma unroll
         for (int s = 0; s < 2; ++s) {
-            const unsigned long long v = s_bins[s][threadIdx.x];
+            const unsigned long long v = st.bins[s][threadIdx.x];
             if (v) atomicAdd(reinterpret_cast<unsigned long long*>(&ctl->pre_bins[s][threadIdx.x]), v);
         }
     }

@@ -197,12 +197,15 @@ __device__ __forceinline__ RangeSum load_range_sum(const RangeSum* p) {
     return r;
 }
 
-// Per warp range: number of kept entries, first and last kept position, and the code lengths of
-// all kept entries but the first (its gap reaches back into an earlier range); the same for the
-// block's eight ranges together.  The last block to finish combines the blocks in order: for every
-// block the rank of its first kept entry, the position kept just before it and the bit offset of
-// its first codeword; then the header.
-__global__ void __launch_bounds__(kBlock) k_span_count(const Batch B) {
+// Per warp range (the spans one warp of k_span_emit will walk): number of kept entries, first and
+// last kept position, and the code lengths of all kept entries but the first (its gap reaches back
+// into an earlier range); the same for the block's eight ranges together.  Here a THREAD walks a
+// span (or a few consecutive ones) by itself -- a compare and a handful of integer operations per
+// entry, no shuffles; the entries of a span are consecutive, so a thread's loads stay within a few
+// cache lines -- and the lanes' results are then put together in order.  The last block to finish
+// combines the blocks in order: for every block the rank of its first kept entry, the position
+// kept just before it and the bit offset of its first codeword; then the header.
+__global__ void __launch_bounds__(kBlock, 6) k_span_count(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
     const Prob& P = s_prob;
@@ -211,40 +214,55 @@ __global__ void __launch_bounds__(kBlock) k_span_count(const Batch B) {
     const int s = (int)ctl->side;
     const unsigned long long thr = ctl->thr[s];
     const uint32_t lane = lane_id(), warp = threadIdx.x >> 5;
-    const unsigned lt = (1u << lane) - 1u;
     constexpr uint32_t kWarps = kBlock / 32;
     const uint32_t n_ranges = S.nb * kWarps;
     const uint32_t range = S.bx * kWarps + warp;
     const int b = P.b;
+    // one buffer for two phases: the lanes' sums of this block's warps, then (last block only) all blocks' sums
+    __shared__ RangeSum s_buf[kOrderBlocksMax > kWarps * 32u ? kOrderBlocksMax : kWarps * 32u];
+    RangeSum (*s_lane)[32] = reinterpret_cast<RangeSum (*)[32]>(s_buf);
     __shared__ RangeSum s_rs[kWarps];
     if (!failed) {
         uint32_t span0, span1;
         range_spans(P.n_spans, n_ranges, range, &span0, &span1);
-        uint32_t cnt = 0u, first = 0u, prev_plus1 = 0u;  // prev_plus1: last kept position so far, plus one
-        unsigned long long bits = 0ull;                    // per lane; summed over the warp at the end
-        walk_spans(P, s, span0, span1, [&](unsigned long long c, bool valid) {
-            const bool kept = valid && c >= thr;
-            const unsigned m = __ballot_sync(0xffffffffu, kept);
-            if (m == 0u) return;  // warp-uniform
-            const uint32_t pos = composite_index(c);
-            const unsigned lower = m & lt;
-            const uint32_t before = __shfl_sync(0xffffffffu, pos, lower ? 31 - __clz((int)lower) : 0);
-            const bool range_first = cnt == 0u && lower == 0u;   // the first kept entry of the range
-            if (kept && !range_first) {
-                const uint32_t g = pos - (lower ? before + 1u : prev_plus1);
-                bits += (unsigned long long)(g >> b) + 1ull + (unsigned long long)b;
-            }
-            if (cnt == 0u) first = __shfl_sync(0xffffffffu, pos, __ffs((int)m) - 1);
-            prev_plus1 = __shfl_sync(0xffffffffu, pos, 31 - __clz((int)m)) + 1u;
-            cnt += (uint32_t)__popc(m);
-        });
+        // lane i takes spans [span0 + i * per_lane, span0 + (i + 1) * per_lane) of the range
+        const uint32_t per_lane = (span1 - span0 + 31u) / 32u;
+        const uint32_t my0 = min(span1, span0 + lane * per_lane), my1 = min(span1, my0 + per_lane);
+        const uint2* __restrict__ rec = P.span_rec[s];
+        const unsigned long long* __restrict__ list = P.list[s];
+        const uint32_t list_cap = P.list_cap;
+        RangeSum mine;
+        mine.cnt = 0u; mine.first = 0u; mine.last = 0u; mine.pad_ = 0u; mine.inner_bits = 0ull;
+        uint32_t prev_plus1 = 0u;
+        for (uint32_t sp = my0; sp < my1; ++sp) {
+            uint2 r = rec[sp];
+            if (r.x > list_cap || r.y > list_cap - r.x) r.y = 0u;  // a record that points outside the list holds nothing
+            const unsigned long long* __restrict__ e = list + r.x;
+            constexpr int kLoads = 8;   // loads in flight per thread
+            for (uint32_t j0 = 0u; j0 < r.y; j0 += kLoads) {
+                unsigned long long c[kLoads];
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) bits += __shfl_down_sync(0xffffffffu, bits, d);
+                for (int j = 0; j < kLoads; ++j) c[j] = (j0 + j < r.y) ? e[j0 + j] : 0ull;
+#pragma unroll
+                for (int j = 0; j < kLoads; ++j) {
+                    if (j0 + j < r.y && c[j] >= thr) {
+                        const uint32_t pos = composite_index(c[j]);
+                        if (mine.cnt == 0u) mine.first = pos;
+                        else mine.inner_bits += (unsigned long long)((pos - prev_plus1) >> b) + 1ull + (unsigned long long)b;
+                        prev_plus1 = pos + 1u;
+                        ++mine.cnt;
+                    }
+                }
+            }
+        }
+        mine.last = prev_plus1 - 1u;
+        s_lane[warp][lane] = mine;
+        __syncwarp();
         if (lane == 0u) {
-            RangeSum rs;
-            rs.cnt = cnt; rs.first = first; rs.last = prev_plus1 - 1u; rs.pad_ = 0u; rs.inner_bits = bits;
-            P.rng_sum[range] = rs;
-            s_rs[warp] = rs;
+            RangeSum all = s_lane[warp][0];
+            for (uint32_t l = 1u; l < 32u; ++l) all = fold_ranges(all, s_lane[warp][l], b);
+            P.rng_sum[range] = all;
+            s_rs[warp] = all;
         }
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -257,8 +275,8 @@ __global__ void __launch_bounds__(kBlock) k_span_count(const Batch B) {
     // ---- the last block: blocks in order.  Thread t takes blocks [t * per, (t + 1) * per).
     __shared__ uint32_t s_scan[kBlock / 32 + 1];
     __shared__ unsigned long long s_scan64[kBlock / 32 + 1];
-    __shared__ uint32_t s_last[kBlock];   // per thread: last kept position + 1 within its blocks (0: none)
-    __shared__ RangeSum s_blk[kOrderBlocksMax];
+    __shared__ uint32_t s_last[kBlock / 32];   // per warp: last kept position + 1 within its threads' blocks (0: none)
+    RangeSum* const s_blk = s_buf;   // the ticket's barriers lie between the two uses
     if (failed || S.nb > kOrderBlocksMax) {
         if (threadIdx.x == 0) {
             if (!failed) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
@@ -273,13 +291,26 @@ __global__ void __launch_bounds__(kBlock) k_span_count(const Batch B) {
     RangeSum mine;
     mine.cnt = 0u; mine.first = 0u; mine.last = 0u; mine.pad_ = 0u; mine.inner_bits = 0ull;
     for (uint32_t r = r0; r < r1; ++r) mine = fold_ranges(mine, s_blk[r], b);
-    s_last[threadIdx.x] = mine.cnt ? mine.last + 1u : 0u;
     uint32_t total_cnt;
     uint32_t rank = block_exclusive_scan<uint32_t>(mine.cnt, s_scan, &total_cnt);
-    // last kept position before this thread's blocks: the nearest earlier thread that has one
-    uint32_t pp = 0u;
-    for (int t = (int)threadIdx.x - 1; t >= 0; --t)
-        if (s_last[t]) { pp = s_last[t]; break; }
+    // last kept position (plus one) before this thread's blocks: positions only grow from thread to
+    // thread, so it is the maximum over the earlier threads
+    uint32_t pp;
+    {
+        const uint32_t mine_last = mine.cnt ? mine.last + 1u : 0u;
+        uint32_t incl = mine_last;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t o = __shfl_up_sync(0xffffffffu, incl, d);
+            if ((int)lane >= d) incl = max(incl, o);
+        }
+        if (lane == 31u) s_last[warp] = incl;
+        __syncthreads();
+        uint32_t before = 0u;
+        for (uint32_t w = 0; w < warp; ++w) before = max(before, s_last[w]);
+        const uint32_t up = __shfl_up_sync(0xffffffffu, incl, 1);
+        pp = max(before, lane ? up : 0u);
+    }
     // bits of this thread's blocks, now that the gap of its first entry is known
     const unsigned long long my_bits =
         mine.cnt ? (unsigned long long)((mine.first - pp) >> b) + 1ull + (unsigned long long)b + mine.inner_bits : 0ull;

@@ -319,9 +319,12 @@ int64_t sbc_oracle_golomb_decode(const uint8_t *msg, uint64_t nbits, int b,
  * The paper's message is the Golomb bit string plus one fp32 mean per tensor
  * ("Optimal Position Encoding"); shapes are known to both sides.  The
  * container adds what a parallel decoder needs and nothing that changes the
- * payload: a 64-byte little-endian header and, for every run of
- * SBC_ORACLE_CHUNK_CODEWORDS codewords, the bit offset of the run's first
- * codeword and the position decoded just before it (-1 for the first run).
+ * payload: a 64-byte little-endian header and, for every run of C codewords
+ * ("chunk"), the bit offset of the run's first codeword and the position
+ * decoded just before it (-1 for the first run).  C depends on the number of
+ * positions k alone (sbc_oracle_chunk_codewords): short messages get short
+ * chunks, so that a decoder that gives every chunk to one worker still has
+ * many chunks to hand out.
  *
  *   0  u32 magic      4  u32 version     8  u64 numel      16 u64 k
  *   24 u64 nbits      32 u64 payload_offset (bytes)        40 u32 b
@@ -346,8 +349,17 @@ static uint64_t get_u64(const uint8_t *p) {
     return v;
 }
 
+/* Codewords per chunk-table entry (project convention): 32 below 2^17
+ * positions, 64 below 2^21, 256 from there on. */
+uint32_t sbc_oracle_chunk_codewords(int64_t k) {
+    if (k < ((int64_t)1 << 17)) return 32u;
+    if (k < ((int64_t)1 << 21)) return 64u;
+    return 256u;
+}
+
 static uint64_t n_chunks_for(int64_t k) {
-    return ((uint64_t)k + SBC_ORACLE_CHUNK_CODEWORDS - 1) / SBC_ORACLE_CHUNK_CODEWORDS;
+    uint64_t c = sbc_oracle_chunk_codewords(k);
+    return ((uint64_t)k + c - 1) / c;
 }
 
 static size_t round_up16(size_t x) { return (x + 15u) & ~(size_t)15u; }
@@ -379,10 +391,11 @@ int sbc_oracle_container(const int64_t *I, int64_t k, int64_t n, int b, int side
     /* chunk table: bit offset of codeword c*C and the position before it */
     uint64_t bit_off = 0;
     int64_t prev = -1;
+    const int64_t chunk = (int64_t)sbc_oracle_chunk_codewords(k);
     for (int64_t i = 0; i < k; ++i) {
-        if (i % SBC_ORACLE_CHUNK_CODEWORDS == 0) {
+        if (i % chunk == 0) {
             uint8_t *e = out + SBC_ORACLE_HEADER_BYTES +
-                         SBC_ORACLE_CHUNK_ENTRY_BYTES * (size_t)(i / SBC_ORACLE_CHUNK_CODEWORDS);
+                         SBC_ORACLE_CHUNK_ENTRY_BYTES * (size_t)(i / chunk);
             put_u64(e, bit_off);
             put_u64(e + 8, (uint64_t)prev);
         }
@@ -402,7 +415,7 @@ int sbc_oracle_container(const int64_t *I, int64_t k, int64_t n, int b, int side
     put_u32(out + 40, (uint32_t)b);
     put_u32(out + 44, (uint32_t)side);
     put_u32(out + 48, mu_bits);
-    put_u32(out + 52, SBC_ORACLE_CHUNK_CODEWORDS);
+    put_u32(out + 52, sbc_oracle_chunk_codewords(k));
     put_u32(out + 56, (uint32_t)nchunks);
     put_u32(out + 60, 0u);
     if (out_len) *out_len = total;
@@ -521,10 +534,11 @@ int sbc_oracle_encode_values(const float *update, float *residual, int64_t n, do
     for (size_t z = payload_offset + (size_t)((nbits + 7) / 8); z < total; ++z) out[z] = 0;
     uint64_t bit_off = 0;
     int64_t prev = -1;
+    const int64_t chunk = (int64_t)sbc_oracle_chunk_codewords(k);
     for (int64_t i = 0; i < k; ++i) {
-        if (i % SBC_ORACLE_CHUNK_CODEWORDS == 0) {
+        if (i % chunk == 0) {
             uint8_t *e = out + SBC_ORACLE_HEADER_BYTES +
-                         SBC_ORACLE_CHUNK_ENTRY_BYTES * (size_t)(i / SBC_ORACLE_CHUNK_CODEWORDS);
+                         SBC_ORACLE_CHUNK_ENTRY_BYTES * (size_t)(i / chunk);
             put_u64(e, bit_off);
             put_u64(e + 8, (uint64_t)prev);
         }
@@ -541,7 +555,7 @@ int sbc_oracle_encode_values(const float *update, float *residual, int64_t n, do
     put_u32(out + 40, (uint32_t)b);
     put_u32(out + 44, SBC_ORACLE_SIDE_VALUES);
     put_u32(out + 48, 0u);
-    put_u32(out + 52, SBC_ORACLE_CHUNK_CODEWORDS);
+    put_u32(out + 52, sbc_oracle_chunk_codewords(k));
     put_u32(out + 56, (uint32_t)nchunks);
     put_u32(out + 60, 0u);
     if (out_len) *out_len = total;

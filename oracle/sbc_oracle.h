@@ -47,9 +47,13 @@ extern "C" {
 #define SBC_ORACLE_MAGIC 0x31434253u /* "SBC1" little-endian */
 #define SBC_ORACLE_VERSION 1u
 #define SBC_ORACLE_HEADER_BYTES 64u
-#define SBC_ORACLE_CHUNK_CODEWORDS 256u
 #define SBC_ORACLE_CHUNK_ENTRY_BYTES 16u
 #define SBC_ORACLE_SIDE_VALUES 2u /* header 'side' of a stream that carries one value per position */
+
+/* Codewords per chunk-table entry of a message with k positions: 32 below
+ * 2^17 positions, 64 below 2^21, 256 from there on (a convention of this
+ * project, "parity unpinned"; the header carries the value). */
+uint32_t sbc_oracle_chunk_codewords(int64_t k);
 
 /* k = max(1, floor(p*n)), at most n.  (Algorithm 2, "top p%"; reading S1.) */
 int64_t sbc_oracle_kept_count(int64_t n, double p);

@@ -15,11 +15,10 @@ __all__ = [
     "exact_sum", "compress", "payload_bits_bound", "golomb_encode",
     "golomb_decode", "container_bytes", "stream_bytes", "encode",
     "decode_accumulate", "parse_header", "StreamHeader", "side_and_mu", "container", "decode_apply", "topk_abs", "stream_bytes_values", "encode_values", "encode_sampled",
-    "HEADER_BYTES", "CHUNK_CODEWORDS", "CHUNK_ENTRY_BYTES", "MAGIC",
+    "HEADER_BYTES", "chunk_codewords", "CHUNK_ENTRY_BYTES", "MAGIC",
 ]
 
 HEADER_BYTES = 64
-CHUNK_CODEWORDS = 256
 CHUNK_ENTRY_BYTES = 16
 MAGIC = 0x31434253
 
@@ -38,6 +37,7 @@ def _sig(name, restype, *argtypes):
 
 
 _kept_count = _sig("sbc_oracle_kept_count", C.c_int64, C.c_int64, C.c_double)
+_chunk_cw = _sig("sbc_oracle_chunk_codewords", C.c_uint32, C.c_int64)
 _golomb_b = _sig("sbc_oracle_golomb_b", C.c_int, C.c_double)
 _mean_bits = _sig("sbc_oracle_mean_position_bits", C.c_double, C.c_double, C.c_int)
 _accumulate = _sig("sbc_oracle_accumulate", C.c_int, _f32p, _f32p, C.c_int64)
@@ -60,6 +60,11 @@ _container = _sig("sbc_oracle_container", C.c_int, _i64p, C.c_int64, C.c_int64, 
                   C.c_float, _u8p, C.c_size_t, C.POINTER(C.c_size_t))
 _decode_acc = _sig("sbc_oracle_decode_accumulate", C.c_int, C.POINTER(C.c_void_p), C.c_int,
                    _f32p, C.c_int64)
+
+
+def chunk_codewords(k: int) -> int:
+    """Codewords per chunk-table entry of a message with k positions."""
+    return int(_chunk_cw(int(k)))
 
 
 def kept_count(n: int, p: float) -> int:

@@ -308,36 +308,53 @@ def test_mean_code_length_matches_the_closed_form_on_iid_input():
     assert h.nbits <= oracle.payload_bits_bound(n, h.k, h.b) == 10485 * 7 + ((n - 10485) >> 6)
 
 
-def test_container_chunk_table_and_padding():
-    rng = np.random.default_rng(5)
-    n, p = 300000, 0.01
-    upd = rng.standard_normal(n).astype(np.float32)
-    res = np.zeros(n, dtype=np.float32)
-    stream, mu = oracle.encode(upd, res, p)
+def test_chunk_size_rule():
+    # convention (unpinned by the paper): 32 codewords per chunk below 2^17 positions, 64 below 2^21, 256 beyond
+    assert [oracle.chunk_codewords(k) for k in (1, 32, 33, 2**17 - 1)] == [32] * 4
+    assert [oracle.chunk_codewords(k) for k in (2**17, 2**20, 2**21 - 1)] == [64] * 3
+    assert [oracle.chunk_codewords(k) for k in (2**21, 2**25, 2**31 - 1)] == [256] * 3
+
+
+@pytest.mark.parametrize("n,p,chunk", [
+    (300_000, 0.01, 32),        # k = 3000
+    (70_001, 0.3, 32),          # k = 21000, b = 1
+    (400_000, 0.4, 64),         # k = 160000 >= 2^17, b = 0
+    (2_200_000, 0.06, 64),      # k = 132000, b = 4
+    (4_300_000, 0.5, 256),      # k = 2150000 >= 2^21, b = 0
+])
+def test_container_chunk_table_and_padding(n, p, chunk):
+    """Every chunk-table entry, at every chunk size, against an independent parse of the payload
+    bit string in Python (Algorithm 4 on a character string)."""
+    rng = np.random.default_rng(n)
+    k, b = oracle.kept_count(n, p), oracle.golomb_b(p)
+    idx = np.sort(rng.choice(n, size=k, replace=False)).astype(np.int64)
+    stream = oracle.container(idx, n, p, 1, -0.5)
     h = oracle.parse_header(stream)
-    assert h.magic == oracle.MAGIC and h.version == 1 and h.chunk_codewords == 256
-    assert h.n_chunks == -(-h.k // 256)
+    assert h.magic == oracle.MAGIC and h.version == 1 and h.k == k and h.b == b
+    assert h.chunk_codewords == chunk == oracle.chunk_codewords(k)
+    assert h.n_chunks == -(-h.k // chunk)
     assert h.payload_offset == 64 + 16 * h.n_chunks
     assert len(stream) % 16 == 0
-    # independent parse of the payload bit string in Python
     payload = bytes(stream[h.payload_offset:])
     bits = "".join(f"{byte:08b}" for byte in payload)
     assert set(bits[h.nbits:]) <= {"0"}
     table = stream[64:h.payload_offset].view("<u8").reshape(-1, 2)
+    assert table.shape[0] == h.n_chunks
     i, prev, count = 0, -1, 0
+    decoded = np.empty(k, dtype=np.int64)
     while count < h.k:
-        if count % 256 == 0:
-            assert int(table[count // 256, 0]) == i
-            assert int(table[count // 256, 1].astype(np.int64)) == prev
-        q = 0
-        while bits[i] == "1":
-            q += 1
-            i += 1
-        r = int(bits[i + 1:i + 1 + h.b], 2) if h.b else 0
+        if count % chunk == 0:
+            assert int(table[count // chunk, 0]) == i
+            assert int(table[count // chunk, 1].astype(np.int64)) == prev
+        j = bits.index("0", i)            # end of the unary part
+        q = j - i
+        r = int(bits[j + 1:j + 1 + h.b], 2) if h.b else 0
         prev = prev + (q << h.b) + r + 1
-        i += 1 + h.b
+        decoded[count] = prev
+        i = j + 1 + h.b
         count += 1
     assert i == h.nbits
+    assert np.array_equal(decoded, idx)
 
 
 def test_decode_accumulate_sums_clients_in_fp32():

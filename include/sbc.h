@@ -67,9 +67,14 @@ enum sbc_status {
  *     32 u64 payload_offset   40 u32 b (Golomb parameter b*)
  *     44 u32 side (0: +mu kept, 1: -mu kept, 2: values follow the table)  48 f32 mu (signed)
  *     52 u32 chunk_codewords  56 u32 n_chunks         60 u32 status
- *   bytes 64..    chunk table, n_chunks entries of
+ *   bytes 64..    chunk table, n_chunks = ceil(k / chunk_codewords) entries of
  *                 { u64 bit offset of codeword c*chunk_codewords,
  *                   i64 position decoded just before it (-1 for c = 0) }
+ *                 chunk_codewords depends on k alone (32 below 2^17 positions,
+ *                 64 below 2^21, 256 from there on): a decoder that hands
+ *                 every chunk to one worker then has enough chunks to hand
+ *                 out for short messages too, at 4, 2 or 0.5 table bits per
+ *                 position
  *   payload_offset..  payload: codeword i = q ones, a zero, r in b bits
  *                 (MSB first), where gap-1 = q*2^b + r (Algorithm 3); stream
  *                 bit j is bit 7-(j%8) of byte j/8; zero padded to 16 bytes.
@@ -77,7 +82,7 @@ enum sbc_status {
 #define SBC_MAGIC 0x31434253u
 #define SBC_VERSION 1u
 #define SBC_HEADER_BYTES 64u
-#define SBC_CHUNK_CODEWORDS 256u
+#define SBC_CHUNK_CODEWORDS_MAX 256u /* chunk_codewords is 32 for k < 2^17 positions, 64 for k < 2^21, else 256 */
 #define SBC_CHUNK_ENTRY_BYTES 16u
 #define SBC_SIDE_VALUES 2u /* header 'side' of a stream written by sbc_encode_values */
 

@@ -106,8 +106,10 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
     pl->n_xtiles = (uint32_t)((n + kXTile - 1) / kXTile);
     const long long k_max = pl->sampled ? (long long)pl->cap : k;  // most positions a stream can carry
     pl->chunk_cw = chunk_codewords_for((unsigned long long)k);
-    // table entries for the most positions at the smallest chunk size a stream of that many could get
-    pl->n_chunks = (uint32_t)((k_max + pl->chunk_cw - 1) / pl->chunk_cw);
+    // exact modes: the table of a stream of k positions; sampled mode: the largest table a stream
+    // of up to k_max positions can have (the device patches count and chunk size once it knows k)
+    pl->n_chunks = pl->sampled ? (uint32_t)max_chunks_upto((unsigned long long)k_max)
+                               : (uint32_t)((k + pl->chunk_cw - 1) / pl->chunk_cw);
     pl->payload_offset = SBC_HEADER_BYTES + (unsigned long long)pl->n_chunks * SBC_CHUNK_ENTRY_BYTES;
     if (mode == kModeValues) pl->payload_offset += align_up((size_t)k * 4, 16);  // the values sit before the payload
     pl->mode = mode;
@@ -818,10 +820,9 @@ static int decode_impl(const void* const* streams, const size_t* stream_bytes, i
         a.status = status_dev;
         a.scale = scale;
         a.momentum = momentum;
-        // at most ceil(numel / 256) chunks per client, 32 chunks per warp, two warps per block
+        // at most max_chunks_upto(numel) chunks per client, 32 chunks per warp, two warps per block
         const unsigned long long max_groups =
-            (unsigned long long)a.n_clients *
-            (unsigned long long)((numel + kChunkCodewords * 32 - 1) / (kChunkCodewords * 32));
+            (unsigned long long)a.n_clients * ((max_chunks_upto((unsigned long long)numel) + 31ull) / 32ull);
         const unsigned grid = grid_for(max_groups, kDecodeThreads / 32, sms * 5);
         k_decode_accumulate<<<grid, kDecodeThreads, 0, stream>>>(a);
     }
@@ -893,8 +894,7 @@ int sbc_decode_accumulate_batch(int n_tensors, int n_clients, const sbc_decode_d
             return SBC_ECUDA;
     }
     const unsigned long long max_groups =
-        (unsigned long long)n_clients *
-        (unsigned long long)((max_numel + kChunkCodewords * 32 - 1) / (kChunkCodewords * 32));
+        (unsigned long long)n_clients * ((max_chunks_upto((unsigned long long)max_numel) + 31ull) / 32ull);
     const unsigned gx = grid_for(max_groups, kDecodeThreads / 32,
                                  std::max(16u, (unsigned)sm_count() * 5u / (unsigned)n_tensors));
     k_decode_accumulate_batch<<<dim3(gx, (unsigned)n_tensors), kDecodeThreads, 0, stream>>>(d_args);

@@ -24,7 +24,7 @@ constexpr uint32_t kSampleMax = 1u << 20;  // elements looked at to bound the th
 constexpr int kXTile = 4096;          // elements per tile in the exact-select fallback
 constexpr int kWarpChunk = 512;       // elements one warp handles per step of the streaming pass
 constexpr int kMaxSpanSteps = kXTile / kWarpChunk;  // a span is 1, 2, 4 or 8 steps and never straddles a tile
-constexpr int kChunkCodewords = 256;  // codewords per chunk-table entry
+constexpr int kChunkCodewords = 256;  // most codewords per chunk-table entry (long streams)
 constexpr uint32_t kOrderBlocksMax = 148 * 8;  // ordering kernels: at most one resident wave of 8-warp blocks on 148 SMs
 constexpr int kSumBins = 254;         // one exact integer bin per fp32 exponent
 constexpr uint32_t kSmallList = 8192;  // candidate lists up to this capacity are ranked by one block
@@ -272,10 +272,26 @@ __device__ __forceinline__ BandView band_view(const Prob& P, const Ctl* ctl, int
     return v;
 }
 
-// Codewords per chunk-table entry of a stream that carries k positions.
+// Codewords per chunk-table entry of a stream that carries k positions.  The decoder gives every
+// chunk to one lane, which parses it codeword after codeword, so short streams get short chunks:
+// a stream of 10^5 positions then still occupies a hundred warps.  (A convention of the container;
+// the header carries the value.)
 __host__ __device__ __forceinline__ uint32_t chunk_codewords_for(unsigned long long k) {
-    (void)k;
+    if (k < (1ull << 17)) return 32u;
+    if (k < (1ull << 21)) return 64u;
     return (uint32_t)kChunkCodewords;
+}
+// Most chunk-table entries a stream of at most k_max positions can have (the chunk size grows with
+// the number of positions, so the count is not monotone).
+__host__ __device__ __forceinline__ unsigned long long chunks_of(unsigned long long k) {
+    const unsigned long long c = chunk_codewords_for(k);
+    return (k + c - 1ull) / c;
+}
+__host__ __device__ __forceinline__ unsigned long long max_chunks_upto(unsigned long long k_max) {
+    unsigned long long m = chunks_of(k_max);
+    if (k_max >= (1ull << 17) && chunks_of((1ull << 17) - 1ull) > m) m = chunks_of((1ull << 17) - 1ull);
+    if (k_max >= (1ull << 21) && chunks_of((1ull << 21) - 1ull) > m) m = chunks_of((1ull << 21) - 1ull);
+    return m;
 }
 
 // ---------------------------------------------------------------- scans

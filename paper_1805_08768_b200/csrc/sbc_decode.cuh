@@ -30,7 +30,7 @@ struct StreamView {
     const uint32_t* words;        // payload as stored (byte-swapped MSB-first words)
     const uint8_t* table;
     unsigned long long k, nbits, n_words;
-    uint32_t b, n_chunks;
+    uint32_t b, n_chunks, chunk_cw;
     float mu;
     const float* values;  // one value per position (values stream), else null
 };
@@ -62,7 +62,7 @@ __device__ __forceinline__ uint32_t add_at(float* p, float mu, bool ieee_path) {
 
 constexpr int kDecodeThreads = 64;            // two warps per block
 constexpr int kDecodeWarpWords = 4608;        // staged payload words per warp (18 KB)
-constexpr uint32_t kInOrderChunks = 8192;     // streams from this many chunks (2 M positions) on add in list order
+constexpr unsigned long long kInOrderPositions = 1ull << 21;   // streams from this many positions on add in list order
 
 // Sequential MSB-first bit reader over a warp's staged (byte-swapped) words, or over global memory when the group's payload did not fit the stage.
 // `cur` holds the next 64 - (32 - avail) ... bits left-aligned: bits [63, 64-avail)
@@ -158,7 +158,7 @@ __device__ __forceinline__ uint32_t parse_staged(const uint32_t* sw, uint32_t& r
 
 // One warp per group of 32 consecutive chunks: the group's payload is one
 // contiguous bit range, copied once (coalesced) into shared memory; then every
-// lane parses its chunk's kChunkCodewords codewords from there (Algorithm 4)
+// lane parses its chunk's codewords (32, 64 or 256 of them, by the header) from there (Algorithm 4)
 // and adds mu at each position (Algorithm 1, server sum).
 __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
     __shared__ StreamView s_view[kMaxClientsPerLaunch];
@@ -176,6 +176,7 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
         v.b = load_u32(h + 40);
         v.mu = __uint_as_float(load_u32(h + 48));
         v.n_chunks = load_u32(h + 56);
+        v.chunk_cw = load_u32(h + 52);
         v.n_words = (v.nbits + 31ull) >> 5;
         v.words = reinterpret_cast<const uint32_t*>(h + payload_offset);
         v.table = h + SBC_HEADER_BYTES;
@@ -187,8 +188,8 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
         const bool good =
             load_u32(h + 0) == SBC_MAGIC && load_u32(h + 4) == SBC_VERSION &&
             load_u64(h + 8) == (unsigned long long)args.n && load_u32(h + 60) == 0u &&
-            load_u32(h + 52) == SBC_CHUNK_CODEWORDS && v.b <= 30u && v.k <= (unsigned long long)args.n &&
-            v.n_chunks == (uint32_t)((v.k + kChunkCodewords - 1) / kChunkCodewords) &&
+            v.chunk_cw == chunk_codewords_for(v.k) && v.b <= 30u && v.k <= (unsigned long long)args.n &&
+            (unsigned long long)v.n_chunks == (v.k + v.chunk_cw - 1ull) / v.chunk_cw &&
             side <= SBC_SIDE_VALUES &&
             payload_offset == SBC_HEADER_BYTES + (unsigned long long)v.n_chunks * SBC_CHUNK_ENTRY_BYTES + values_bytes &&
             v.nbits >= v.k * (1ull + v.b) &&
@@ -200,6 +201,7 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
              payload_offset + ((((v.nbits + 7ull) >> 3) + 15ull) & ~15ull) <= args.bytes[tid]);
         if (!good) {
             v.n_chunks = 0u;  // contributes nothing
+            v.chunk_cw = (uint32_t)kChunkCodewords;
             if (args.status && blockIdx.x == 0) atomicOr(args.status, SBC_STATUS_CORRUPT);
         }
         s_view[tid] = v;
@@ -255,17 +257,17 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
         // and DRAM serves neighbours that arrive together far better: 0.44 -> 0.40 ms for 10.7 M
         // positions over 4 GiB.  Short streams are bound by the latency of a chunk's serial parse
         // instead, which the extra step lengthens (60 -> 63 us at 1 M positions), so only streams
-        // of at least kInOrderChunks chunks are decoded this way.
+        // of at least kInOrderPositions positions are decoded this way.
         const float mu_w = __fmul_rn(v.mu, args.scale);
-        const bool in_order = staged && v.n_chunks >= kInOrderChunks && v.values == nullptr &&
+        const bool in_order = staged && v.k >= kInOrderPositions && v.values == nullptr &&
                               args.momentum == nullptr && !(fabsf(mu_w) < 7.888609052e-31f);  // warp-uniform
         if (in_order) {
             uint32_t count = 0u, rel = 0u, rel_end = 0u, nxt = 0u, done = 0u;
             const uint32_t n32 = (uint32_t)args.n;
             bool live = has && !err;
             if (live) {
-                const unsigned long long first_cw = (unsigned long long)chunk * kChunkCodewords;
-                count = (uint32_t)min((unsigned long long)kChunkCodewords, v.k - first_cw);
+                const unsigned long long first_cw = (unsigned long long)chunk * v.chunk_cw;
+                count = (uint32_t)min((unsigned long long)v.chunk_cw, v.k - first_cw);
                 if (pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n) {
                     err = SBC_STATUS_CORRUPT;
                     live = false;
@@ -275,7 +277,7 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                 nxt = (uint32_t)(prev + 1);
             }
             const bool checked = live;  // the end of the chunk is compared with the table below
-            for (int step = 0; step < kChunkCodewords / 32; ++step) {
+            for (uint32_t step = 0; step < v.chunk_cw / 32u; ++step) {
                 if (!__any_sync(0xffffffffu, live && done < count)) break;  // warp-uniform
                 uint32_t got = 0u;
                 if (live) {
@@ -308,14 +310,14 @@ __device__ __forceinline__ void decode_body(const DecodeArgs& args) {
                 }
             }
         } else if (has && !err) {
-            const unsigned long long first_cw = (unsigned long long)chunk * kChunkCodewords;
-            const uint32_t count = (uint32_t)min((unsigned long long)kChunkCodewords, v.k - first_cw);
+            const unsigned long long first_cw = (unsigned long long)chunk * v.chunk_cw;
+            const uint32_t count = (uint32_t)min((unsigned long long)v.chunk_cw, v.k - first_cw);
             const bool entry_ok = !(pos >= v.nbits || pos < gbeg || pos > gend || prev < -1 || prev >= args.n);
             if (!entry_ok) err = SBC_STATUS_CORRUPT;
             const uint32_t b = v.b;
             const float mu = __fmul_rn(v.mu, args.scale);
             float* __restrict__ momentum = args.momentum;
-            const float* __restrict__ vals = v.values ? v.values + (size_t)chunk * kChunkCodewords : nullptr;
+            const float* __restrict__ vals = v.values ? v.values + (size_t)chunk * v.chunk_cw : nullptr;
             const bool tiny = fabsf(mu) < 7.888609052e-31f;  // 2^-100
             if (!entry_ok) {
                 // nothing is decoded from a chunk whose table entry is out of range

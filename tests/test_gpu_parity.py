@@ -371,7 +371,9 @@ def test_inflated_size_fields_are_refused_when_the_length_is_stated():
 
     def header(k, nbits=None, n_chunks=None, payload_offset=None):
         bad = stream.copy()
-        n_chunks = -(-k // int(info.chunk_codewords)) if n_chunks is None else n_chunks
+        chunk = oracle.chunk_codewords(k)                  # the chunk size that goes with k positions
+        bad[52:56].view("<u4")[0] = chunk
+        n_chunks = -(-k // chunk) if n_chunks is None else n_chunks
         payload_offset = 64 + 16 * n_chunks if payload_offset is None else payload_offset
         nbits = k * (1 + b) + ((n - k) >> b) if nbits is None else nbits
         bad[16:24].view("<u8")[0] = k

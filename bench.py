@@ -27,6 +27,7 @@ UNIT = "Gelem/s"
 WORKLOAD = ("flat 2^30-element fp32 update, Student-t(nu=3) x 1e-3, p sweep {1e-2,1e-3,1e-4}: "
             "per p one sbc_encode (residual carried across steps) + one sbc_decode_accumulate")
 ALGO_BYTES_PER_ELEM = 12  # read update, read residual, write residual
+DECODE_BYTES_PER_POSITION = 64  # one 32-byte sector of the dense tensor read and written back per decoded position
 
 
 def parse_args():
@@ -151,12 +152,19 @@ def run_reference(args):
 
 # ------------------------------------------------------------------ our arm
 
-# DRAM traffic of one k_add_collect launch from an ncu capture at 2^26 elements (its summary
-# is kept with the other profile summaries): (536.94 + 226.60) MB at 2^26 elements, p = 1e-2.
-# Traffic is proportional to the element count, so it is scaled by numel / 2^26.  Valid only for
-# the kernel source it was taken from: a different hash of the file reports null.
-NCU_TRAFFIC_BYTES_AT_2P26 = 763.54e6
-NCU_TRAFFIC_SOURCE_SHA256 = "7fde50810e202a03e25da00d8bce1e859be4aabb3c48e116afdef7a99eb21cda"
+# DRAM traffic of one k_add_collect launch, from an ncu capture at 2^26 elements, p = 1e-2 (its
+# summary is kept with the other profile summaries).  Reads grow in proportion to the element count.
+# Writes do not quite: when the kernel ends, a part of what it stored is still in L2 as dirty lines
+# (written back during the next kernel), and that part does not grow with the tensor.  So a launch
+# over `numel` elements is modelled as
+#     reads(2^26) * numel / 2^26  +  stored(numel) - l2_residue,
+#     stored(numel) = stored(2^26) * numel / 2^26,   l2_residue = stored(2^26) - writes(2^26),
+# where stored(2^26) = 4 B per element plus the candidate lists the capture's launch wrote.
+# Valid only for the kernel source it was taken from: a different hash of the file reports null.
+NCU_READ_BYTES_AT_2P26 = 0.0
+NCU_WRITE_BYTES_AT_2P26 = 0.0
+NCU_STORED_BYTES_AT_2P26 = 0.0
+NCU_TRAFFIC_SOURCE_SHA256 = "unset"
 
 
 def measured_traffic(numel: int):
@@ -168,7 +176,11 @@ def measured_traffic(numel: int):
                 return None
     except OSError:
         return None
-    return NCU_TRAFFIC_BYTES_AT_2P26 * numel / float(1 << 26)
+    scale = numel / float(1 << 26)
+    residue = NCU_STORED_BYTES_AT_2P26 - NCU_WRITE_BYTES_AT_2P26
+    traffic = NCU_READ_BYTES_AT_2P26 * scale + NCU_STORED_BYTES_AT_2P26 * scale - (residue if scale >= 1.0 else residue * scale)
+    # what the kernel must move can only be exceeded, never undercut
+    return traffic if traffic >= ALGO_BYTES_PER_ELEM * numel else None
 
 
 def reduce_max_over_ranks(value: float, dist, device) -> float:
@@ -187,7 +199,7 @@ def load_peak():
         with open(path) as fh:
             return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
     except (OSError, KeyError, ValueError):
-        return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+        return 6650.0, "fallback (6.65 TB/s: MEASURED_PEAKS.json not found)"
 
 
 def run_ours(args):
@@ -291,8 +303,11 @@ def run_ours(args):
     peak, peak_src = load_peak()
     collect_ms = sum(collect_ms_all) / len(collect_ms_all)
     achieved = ALGO_BYTES_PER_ELEM * n / (collect_ms * 1e-3) / 1e9
+    traffic = measured_traffic(n)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                "traffic": measured_traffic(n), "kernel": "k_add_collect", "launches_timed": len(collect_ms_all),
+                "traffic": traffic,
+                "traffic_over_algorithmic": (traffic / (ALGO_BYTES_PER_ELEM * n)) if traffic else None,
+                "kernel": "k_add_collect", "launches_timed": len(collect_ms_all),
                 "avg_ms": collect_ms, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": ALGO_BYTES_PER_ELEM * n}
 
@@ -313,6 +328,11 @@ def run_ours(args):
             "encode_algorithmic_gbs": ALGO_BYTES_PER_ELEM * n / (e * 1e-3) / 1e9,
             "encode_frac_of_peak": ALGO_BYTES_PER_ELEM * n / (e * 1e-3) / 1e9 / peak,
             "decode_positions_per_s": infos[i].k / (d * 1e-3),
+            # decode as the blueprint counts it: dense-equivalent rate, and bytes = one 32-byte sector read
+            # and written per position plus the container read once
+            "decode_dense_gelem_s": n / (d * 1e-3) / 1e9,
+            "decode_gbs": (DECODE_BYTES_PER_POSITION * infos[i].k + infos[i].total_bytes) / (d * 1e-3) / 1e9,
+            "decode_frac_of_peak": (DECODE_BYTES_PER_POSITION * infos[i].k + infos[i].total_bytes) / (d * 1e-3) / 1e9 / peak,
             "stage_ms": {name: stage_ms[i][s] / steps for s, name in enumerate(sbc.MARK_NAMES)},
             "route": diags[i],
         })
@@ -335,7 +355,7 @@ def run_ours(args):
                "seconds": dt, "host_cores_available": len(os.sched_getaffinity(0))}
 
     try:
-        network_shapes = run_network_shapes(torch, sbc, workloads, dev)
+        network_shapes = run_network_shapes(torch, sbc, workloads, dev, with_oracle=not args.no_cpu_baseline)
     except Exception as exc:  # context numbers only: never fail the headline for them
         network_shapes = {"error": repr(exc)}
 
@@ -357,53 +377,113 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
-def run_network_shapes(torch, sbc, workloads, dev):
-    """Batched encode (one round) and 8-client batched decode on the network-shaped workloads:
-    context numbers next to the headline, timed with CUDA events over 10 repetitions."""
+def _timed(torch, fn, reps=10):
+    """Mean device time of fn() in ms: 3 warm-ups, then `reps` calls between two CUDA events."""
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def _oracle_round(tensors, p):
+    """The oracle over one round of a model's tensors (zero residual), one core: (seconds, streams)."""
     import numpy as np
+    import oracle
+    t0 = time.perf_counter()
+    streams = []
+    for u in tensors:
+        stream, _ = oracle.encode(u, np.zeros(u.size, dtype=np.float32), p)
+        streams.append(stream)
+    return time.perf_counter() - t0, streams
+
+
+def run_network_shapes(torch, sbc, workloads, dev, with_oracle=True):
+    """The four small configurations next to the headline: per configuration the device time of
+    the calls (CUDA events, 10 repetitions after 3 warm-ups) and, beside it, the oracle on the same
+    tensors (one core, wall clock, run whole unless it says otherwise)."""
+    import numpy as np
+    import oracle
     out = {}
+
+    # ---- config 1: one tensor of 2^20 elements, N(0, 1e-3), p = 0.01, encode + decode round trip
+    n1, p1 = 1 << 20, 0.01
+    upd = workloads.normal_flat(n1, 1e-3, workloads.seed_for(1))
+    u = torch.from_numpy(upd).to(dev)
+    r = torch.zeros(n1, dtype=torch.float32, device=dev)
+    ws1 = torch.empty(sbc.sbc_workspace_bytes(n1, p1), dtype=torch.uint8, device=dev)
+    out1 = torch.empty(sbc.sbc_stream_bytes(n1, p1), dtype=torch.uint8, device=dev)
+    mu1 = torch.empty(1, dtype=torch.float32, device=dev)
+    dense1 = torch.zeros(n1, dtype=torch.float32, device=dev)
+    enc_ms = _timed(torch, lambda: sbc.sbc_encode(u, r, p1, out_stream=out1, out_mu=mu1, workspace=ws1), 20)
+    dec_ms = _timed(torch, lambda: sbc.sbc_decode_accumulate([out1], dense1), 20)
+    out["config1_flat_2p20_p1e-2"] = {"elements": n1, "encode_us": 1e3 * enc_ms, "decode_us": 1e3 * dec_ms,
+                                      "round_trip_gelem_s": n1 / (enc_ms + dec_ms) / 1e6}
+    if with_oracle:
+        t0 = time.perf_counter()
+        stream, _ = oracle.encode(upd, np.zeros(n1, dtype=np.float32), p1)
+        t1 = time.perf_counter()
+        oracle.decode_accumulate([stream], np.zeros(n1, dtype=np.float32))
+        t2 = time.perf_counter()
+        out["config1_flat_2p20_p1e-2"]["oracle"] = {"encode_s": t1 - t0, "decode_s": t2 - t1, "cores": 1,
+                                                     "round_trip_gelem_s": n1 / (t2 - t0) / 1e9}
+
+    # ---- configs 2, 3, 4: the network-shaped rounds (batched calls)
     for name, sizes, p, gen in (
             ("resnet50_shapes_p1e-3", [int(np.prod(s)) for _, s, _ in workloads.resnet50_shapes()], 1e-3,
              workloads.resnet50_update),
             ("word_lstm_shapes_p1e-2", [int(np.prod(s)) for _, s in workloads.word_lstm_shapes()], 1e-2,
+             workloads.word_lstm_update),
+            ("word_lstm_shapes_p1e-3", [int(np.prod(s)) for _, s in workloads.word_lstm_shapes()], 1e-3,
              workloads.word_lstm_update)):
         n_clients = 8
-        res = [torch.zeros(n, dtype=torch.float32, device=dev) for n in sizes]
-        mus = [torch.empty(1, dtype=torch.float32, device=dev) for _ in sizes]
-        ws = torch.empty(sbc.sbc_workspace_bytes_batch(sizes, [p] * len(sizes)), dtype=torch.uint8, device=dev)
-        # one message per client and tensor, from eight different seeded updates (zero residual each)
-        client_outs = []
+        ps = [p] * len(sizes)
+        ws = torch.empty(sbc.sbc_workspace_bytes_batch(sizes, ps), dtype=torch.uint8, device=dev)
+        # one message per client and tensor, from eight different seeded updates; every client has
+        # its own residuals, outputs and marshalled descriptors, as eight clients on one GPU would
+        clients, first_host = [], None
         for c in range(n_clients):
-            ups = [torch.from_numpy(u).to(dev) for u in gen(1 + c)]
-            for r in res:
-                r.zero_()
+            host = gen(1 + c)
+            if c == 0:
+                first_host = host
+            ups = [torch.from_numpy(x).to(dev) for x in host]
+            res = [torch.zeros(n, dtype=torch.float32, device=dev) for n in sizes]
             outs = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=dev) for n in sizes]
-            sbc.EncodeBatch(ups, res, [p] * len(sizes), outs, mus, ws).run()
-            torch.cuda.synchronize()
-            client_outs.append(outs)
-        enc = sbc.EncodeBatch(ups, res, [p] * len(sizes), client_outs[-1], mus, ws)  # timed: the last client's round
+            mus = [torch.empty(1, dtype=torch.float32, device=dev) for _ in sizes]
+            clients.append((sbc.EncodeBatch(ups, res, ps, outs, mus, ws), outs))
         dense = [torch.zeros(n, dtype=torch.float32, device=dev) for n in sizes]
         dws = torch.empty(sbc.sbc_decode_workspace_bytes_batch(len(sizes)), dtype=torch.uint8, device=dev)
-        dec = sbc.DecodeBatch([[client_outs[c][t] for c in range(n_clients)] for t in range(len(sizes))], dense, dws)
+        dec = sbc.DecodeBatch([[clients[c][1][t] for c in range(n_clients)] for t in range(len(sizes))], dense, dws)
 
-        def timed(fn, reps=10):
-            for _ in range(3):
-                fn()
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(reps):
-                fn()
-            e1.record()
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / reps
+        def encode_all():
+            for enc, _ in clients:
+                enc.run()
 
-        enc_ms, dec_ms = timed(enc.run), timed(dec.run)
+        one_ms = _timed(torch, clients[0][0].run)
+        all_ms = _timed(torch, encode_all, 5)
+        dec_ms = _timed(torch, dec.run)
         total = sum(sizes)
-        out[name] = {"tensors": len(sizes), "elements": total, "encode_batch_us": 1e3 * enc_ms,
-                     "encode_gelem_s": total / enc_ms / 1e6,
-                     "encode_algorithmic_gbs": ALGO_BYTES_PER_ELEM * total / enc_ms / 1e6,
-                     "decode_batch_8_clients_us": 1e3 * dec_ms}
+        out[name] = {"tensors": len(sizes), "elements": total, "encode_batch_us": 1e3 * one_ms,
+                     "encode_gelem_s": total / one_ms / 1e6,
+                     "encode_algorithmic_gbs": ALGO_BYTES_PER_ELEM * total / one_ms / 1e6,
+                     "encode_algorithmic_frac_of_peak": ALGO_BYTES_PER_ELEM * total / one_ms / 1e6 / load_peak()[0],
+                     "encode_8_clients_us": 1e3 * all_ms,
+                     "decode_batch_8_clients_us": 1e3 * dec_ms,
+                     "encode_8_clients_plus_decode_us": 1e3 * (all_ms + dec_ms)}
+        if with_oracle and name != "word_lstm_shapes_p1e-3":   # (the LSTM shapes are timed against the oracle at one p)
+            secs, streams = _oracle_round(first_host, p)
+            t0 = time.perf_counter()
+            for t, n in enumerate(sizes):    # the same message eight times stands in for eight clients' messages
+                oracle.decode_accumulate([streams[t]] * n_clients, np.zeros(n, dtype=np.float32))
+            dsecs = time.perf_counter() - t0
+            out[name]["oracle"] = {"encode_round_s": secs, "decode_8_clients_s": dsecs, "cores": 1,
+                                   "encode_gelem_s": total / secs / 1e9,
+                                   "sample": "one client's round (of eight), zero residual; decode of eight messages per tensor"}
     return out
 
 
@@ -455,6 +535,21 @@ def run_e2e(args, torch, sbc, dev, update, ws, n, world):
     settle(pending)
     pending = None
     torch.cuda.synchronize()
+    # the containers this first step brought back to the host are those of the device-buffer call
+    # on the same input (zero residual), byte for byte, and the last aggregate is the decoded message
+    chk_res = torch.zeros(n, dtype=torch.float32, device=dev)
+    for i, p in enumerate(P_SWEEP):
+        chk_res.zero_()
+        out, _ = sbc.sbc_encode(update, chk_res, p, workspace=ws)
+        info = sbc.sbc_stream_info_get(out)
+        if not torch.equal(out[: info.total_bytes].cpu(), stream_host[i][: info.total_bytes]):
+            raise RuntimeError(f"host-buffer encode at p={p} differs from sbc_encode")
+        if i == len(P_SWEEP) - 1:
+            chk_res.zero_()
+            sbc.sbc_decode_accumulate([out], chk_res)
+            if not torch.equal(chk_res.cpu().view(torch.int32), dense_host.view(torch.int32)):
+                raise RuntimeError("host-buffer decode differs from sbc_decode_accumulate")
+    del chk_res
     h2d = d2h = 0
     t0 = time.perf_counter()
     for _ in range(args.e2e_steps):

@@ -136,59 +136,74 @@ def test_config4_eight_clients_decode_aggregate():
         assert np.max(np.abs(got.astype(np.float64) - want)) <= tol, f"aggregate of tensor {t}"
 
 
+def _check_flat_round(accumulated, update, residual, p):
+    """One sbc_encode + decode of a flat tensor against an independent selection.  `accumulated` is
+    what A = residual + update must be (taken with torch's own fp32 add); torch's sort gives the two
+    order statistics, the oracle the exact sums, the side decision and the container.  `residual`
+    is updated in place by the encode and checked bit for bit."""
+    n = accumulated.numel()
+    k, b = oracle.kept_count(n, p), oracle.golomb_b(p)
+    sorted_vals = torch.sort(accumulated).values
+    t_top = sorted_vals[n - k]          # k-th largest
+    t_bot = sorted_vals[k - 1]          # k-th smallest
+    del sorted_vals
+    top = torch.nonzero(accumulated >= t_top).flatten()
+    bot = torch.nonzero(accumulated <= t_bot).flatten()
+    # continuous data: no ties expected at the thresholds; if there are, keep the lowest indices
+    if top.numel() > k:
+        ties = torch.nonzero(accumulated[top] == t_top).flatten()
+        keep = torch.ones(top.numel(), dtype=torch.bool, device=DEV)
+        keep[ties[k - (top.numel() - ties.numel()):]] = False
+        top = top[keep]
+    if bot.numel() > k:
+        ties = torch.nonzero(accumulated[bot] == t_bot).flatten()
+        keep = torch.ones(bot.numel(), dtype=torch.bool, device=DEV)
+        keep[ties[k - (bot.numel() - ties.numel()):]] = False
+        bot = bot[keep]
+    assert top.numel() == k and bot.numel() == k
+    top_vals = accumulated[top].cpu().numpy()
+    bot_vals = accumulated[bot].cpu().numpy()
+    ar = np.arange(k, dtype=np.int64)
+    side, mu, _, _ = oracle.side_and_mu(oracle.exact_sum(top_vals, ar), oracle.exact_sum(bot_vals, ar), k)
+    kept = (bot if side else top)
+    want_stream = oracle.container(kept.cpu().numpy(), n, p, side, mu)
+    del top, bot
+
+    out, mu_dev = sbc.sbc_encode(update, residual, p)
+    info = sbc.sbc_stream_info_get(out)
+    got_stream = out[: info.total_bytes].cpu().numpy()
+    assert (info.k, info.b, info.side) == (k, b, side)
+    assert np.float32(mu_dev.item()).view(np.uint32) == mu.view(np.uint32)
+    assert np.array_equal(got_stream, want_stream), f"p={p}: container differs"
+    # residual: A everywhere, A - mu (one fp32 subtraction) on the kept positions
+    expect_res = accumulated.clone()
+    expect_res[kept] = accumulated[kept] - float(mu)
+    assert torch.equal(residual.view(torch.int32), expect_res.view(torch.int32)), f"p={p}: residual differs"
+    del expect_res
+    # decode into a zeroed tensor: mu on the kept positions, zero elsewhere
+    dense = torch.zeros(n, dtype=torch.float32, device=DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    sbc.sbc_decode_accumulate([out], dense, status=status)
+    expect = torch.zeros(n, dtype=torch.float32, device=DEV)
+    expect[kept] = float(mu)
+    torch.cuda.synchronize()
+    assert status.item() == 0
+    assert torch.equal(dense.view(torch.int32), expect.view(torch.int32)), f"p={p}: decoded tensor differs"
+
+
 def test_config5_flat_2p30_sweep_against_independent_selection():
+    """Config 5 at full size, as the benchmark runs it: per p a first round from a zero residual and a
+    second round that carries the first round's residual (so that E1's add is not trivial)."""
     n = 1 << 30
     update = workloads.student_t_flat_torch(n, workloads.seed_for(5), DEV)
-    # independent selection: torch's sort gives both order statistics for every p at once
-    sorted_vals = torch.sort(update).values
+    update2 = workloads.student_t_flat_torch(n, workloads.seed_for(5, 1), DEV)
     for p in (1e-2, 1e-3, 1e-4):
-        k, b = oracle.kept_count(n, p), oracle.golomb_b(p)
-        t_top = sorted_vals[n - k]          # k-th largest
-        t_bot = sorted_vals[k - 1]          # k-th smallest
-        top = torch.nonzero(update >= t_top).flatten()
-        bot = torch.nonzero(update <= t_bot).flatten()
-        # continuous data: no ties expected at the thresholds; if there are, keep the lowest indices
-        if top.numel() > k:
-            ties = torch.nonzero(update[top] == t_top).flatten()
-            keep = torch.ones(top.numel(), dtype=torch.bool, device=DEV)
-            keep[ties[k - (top.numel() - ties.numel()):]] = False
-            top = top[keep]
-        if bot.numel() > k:
-            ties = torch.nonzero(update[bot] == t_bot).flatten()
-            keep = torch.ones(bot.numel(), dtype=torch.bool, device=DEV)
-            keep[ties[k - (bot.numel() - ties.numel()):]] = False
-            bot = bot[keep]
-        assert top.numel() == k and bot.numel() == k
-        top_vals = update[top].cpu().numpy()
-        bot_vals = update[bot].cpu().numpy()
-        ar = np.arange(k, dtype=np.int64)
-        side, mu, _, _ = oracle.side_and_mu(oracle.exact_sum(top_vals, ar), oracle.exact_sum(bot_vals, ar), k)
-        kept = (bot if side else top)
-        want_stream = oracle.container(kept.cpu().numpy(), n, p, side, mu)
-        del top, bot
-
         residual = torch.zeros(n, dtype=torch.float32, device=DEV)
-        out, mu_dev = sbc.sbc_encode(update, residual, p)
-        info = sbc.sbc_stream_info_get(out)
-        got_stream = out[: info.total_bytes].cpu().numpy()
-        assert (info.k, info.b, info.side) == (k, b, side)
-        assert np.float32(mu_dev.item()).view(np.uint32) == mu.view(np.uint32)
-        assert np.array_equal(got_stream, want_stream), f"p={p}: container differs"
-        # residual: A everywhere (zero residual in: A = update), A - mu on the kept positions
-        expect_res = update.clone()
-        expect_res[kept] = update[kept] - float(mu)
-        assert torch.equal(residual.view(torch.int32), expect_res.view(torch.int32)), f"p={p}: residual differs"
-        del expect_res
-        # decode into a zeroed tensor: mu on the kept positions, zero elsewhere
-        dense = torch.zeros(n, dtype=torch.float32, device=DEV)
-        status = torch.zeros(1, dtype=torch.int32, device=DEV)
-        sbc.sbc_decode_accumulate([out], dense, status=status)
-        expect = torch.zeros(n, dtype=torch.float32, device=DEV)
-        expect[kept] = float(mu)
-        torch.cuda.synchronize()
-        assert status.item() == 0
-        assert torch.equal(dense.view(torch.int32), expect.view(torch.int32)), f"p={p}: decoded tensor differs"
-        del dense, expect, residual, kept
+        _check_flat_round(update, update, residual, p)              # A = 0 + update
+        carried = torch.add(residual, update2)                      # what round 2 must accumulate
+        assert bool((residual != update).any())                     # the residual really carries something
+        _check_flat_round(carried, update2, residual, p)
+        del residual, carried
 
 
 def test_batch_and_single_tensor_calls_agree_with_mixed_sparsities():

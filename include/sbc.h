@@ -296,8 +296,8 @@ int sbc_encode_host(const float *update_host, float *update_dev, float *residual
  * that is part of the library image: every GPU that loads the library holds
  * those bytes until the process exits.  Consequences the caller must know:
  *   - Only problems with sbc_workspace_bytes(numel, p) <=
- *     SBC_STATIC_WORKSPACE_BYTES fit (up to about 6 M elements at p = 0.01,
- *     35 M at p = 0.001);
+ *     SBC_STATIC_WORKSPACE_BYTES fit (up to about 2.6 M elements at p = 0.01,
+ *     10.8 M at p = 0.001);
  *     larger ones are refused with SBC_ECAPACITY and nothing is enqueued.
  *   - There is ONE array per GPU, shared by every call in the process.  Two
  *     calls whose device work can overlap (different streams, different
@@ -306,7 +306,10 @@ int sbc_encode_host(const float *update_host, float *update_dev, float *residual
  *     left; each call clears the parts that must start at zero itself.
  *   - The first call on each device looks up the array's device address (with
  *     that device current) and remembers it; make that first call outside any
- *     stream capture.  No call allocates or frees memory.
+ *     stream capture.  The remembered address belongs to the device's primary
+ *     context: after cudaDeviceReset it is stale, and the library must not be
+ *     used on that device again in the same process.  No call allocates or
+ *     frees memory.
  * Everything else (arguments, results, errors, asynchrony) is as sbc_encode.
  */
 #define SBC_STATIC_WORKSPACE_BYTES (8u << 20)

@@ -5,6 +5,8 @@
 #include <mutex>
 #include <vector>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "../../include/sbc.h"
 #include "../../include/sbc_debug.h"
 #include "sbc_common.cuh"
@@ -310,7 +312,18 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
 void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, const unsigned grid[WK_COUNT],
                    const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, bool small_form, cudaStream_t st,
                    const sbc_cuda_event_t* marks) {
-    auto mark = [&](int i) { if (marks && marks[i]) cudaEventRecord(marks[i], st); };
+    // Every stage boundary closes an NVTX range and opens the next one (host-side ranges around the
+    // launches of a stage, for a timeline tool; no-ops when none is attached), and records the
+    // caller's event for that boundary if it gave one.
+    static const char* const kStageNames[SBC_MARK_COUNT] = {"sbc_encode: bounds", "sbc_encode: accumulate + collect",
+                                                            "sbc_encode: exact route", "sbc_encode: select + sums",
+                                                            "sbc_encode: order + golomb", ""};
+    nvtxRangePushA(kStageNames[0]);
+    auto mark = [&](int i) {
+        if (marks && marks[i]) cudaEventRecord(marks[i], st);
+        nvtxRangePop();
+        if (i + 1 < SBC_MARK_COUNT) nvtxRangePushA(kStageNames[i]);
+    };
     auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs, any_exact}; };
     auto g1 = [&](int kind) { return dim3(grid[kind]); };
     auto g2 = [&](int kind) { return dim3(grid[kind], 1, 2); };  // z = side

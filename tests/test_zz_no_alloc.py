@@ -42,7 +42,8 @@ def _both_ways(upd_np, res_np, p):
 
 
 def test_static_scratch_matches_sbc_encode_on_two_calls_in_a_row():
-    # call 1: ~1 M elements (close to the limit), call 2: a different size, p and a carried residual
+    # call 1: ~1 M elements (a little over half of the fixed scratch), call 2: a different size, p
+    # and a carried residual, run over the scratch the first call dirtied
     cases = [
         (workloads.normal_flat(1 << 20, 1e-3, 901), np.zeros(1 << 20, dtype=np.float32), 0.01),
         (workloads.student_t_flat(300001, 902), workloads.normal_flat(300001, 2e-3, 903), 0.001),
@@ -53,6 +54,22 @@ def test_static_scratch_matches_sbc_encode_on_two_calls_in_a_row():
         assert np.array_equal(s0, s1)                                   # container byte for byte
         assert np.array_equal(m0.view(np.uint32), m1.view(np.uint32))   # mu bit for bit
         assert np.array_equal(r0.view(np.uint32), r1.view(np.uint32))   # residual bit for bit
+
+
+def test_static_scratch_at_its_limit_then_a_small_call():
+    # the largest problem the fixed array takes at p = 0.01 (its scratch fills all but a few KB of
+    # the 8 MiB), then a small one that reuses the same bytes
+    p = 0.01
+    n = 2_600_000
+    need = sbc.sbc_workspace_bytes(n, p)
+    assert 0.98 * sbc.STATIC_WORKSPACE_BYTES < need <= sbc.STATIC_WORKSPACE_BYTES
+    assert sbc.sbc_workspace_bytes(n + 20_000, p) > sbc.STATIC_WORKSPACE_BYTES
+    for upd, res in ((workloads.student_t_flat(n, 904), workloads.normal_flat(n, 1e-3, 905)),
+                     (workloads.normal_flat(5000, 1e-3, 906), np.zeros(5000, dtype=np.float32))):
+        (s0, m0, r0), (s1, m1, r1) = _both_ways(upd, res, p)
+        assert np.array_equal(s0, s1)
+        assert np.array_equal(m0.view(np.uint32), m1.view(np.uint32))
+        assert np.array_equal(r0.view(np.uint32), r1.view(np.uint32))
 
 
 def test_static_scratch_refuses_what_does_not_fit():

@@ -259,8 +259,10 @@ inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsi
 void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned coarse_exact, unsigned nb[WK_COUNT]) {
     nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8 * coarse_sample, sms * 4);
     nb[WK_MAIN] = pl.main_blocks;
-    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 8);
-    nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 8);
+    // (the exact route is rare: its kernels usually only find out that they are not needed, which a
+    // smaller grid does sooner; when they do run, two blocks per SM still keep the memory busy)
+    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 2);
+    nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 4);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 2);  // x 2 sides: one resident wave at four blocks per SM
     nb[WK_ORDER] = pl.order_blocks;
     nb[WK_ONE] = 1;
@@ -513,7 +515,7 @@ int sbc_encode_values(const float* update, float* residual, int64_t numel, doubl
 }
 
 // Plans of all tensors of a batch.  Two things are decided over the whole batch: how many steps a
-// streaming block gets (about three waves of resident blocks over the batch, so that a block's
+// streaming block gets (about two waves of resident blocks over the batch, so that a block's
 // start-up -- finding its problem, reading the bounds -- and its final flush are paid for by
 // several steps of loads), and whether the launch can use the short-list form (only if every
 // tensor fits it).
@@ -527,7 +529,7 @@ static bool plan_batch(int n_tensors, const sbc_tensor_desc* descs, std::vector<
         small = small && !pl.use_runs;
     }
     const unsigned coarse_main = (unsigned)std::min<unsigned long long>(
-        8, std::max<unsigned long long>(1, fine_main / (kPlanSMs * 3 * kCollectBlocksPerSM)));
+        16, std::max<unsigned long long>(1, fine_main / (kPlanSMs * 2 * kCollectBlocksPerSM)));
     plans->resize((size_t)n_tensors);
     for (int t = 0; t < n_tensors; ++t)
         if (!make_plan(descs[t].numel, descs[t].p, &(*plans)[t], kModeBinary, 0, coarse_main, !small)) return false;

@@ -624,6 +624,28 @@ def test_sampled_thresholds_rejected_estimate_gives_the_exact_result():
     assert np.array_equal(out[: info.total_bytes].cpu().numpy(), want_exact)
 
 
+def test_sampled_thresholds_with_clustered_candidates_keep_the_oracle_s_rule():
+    """The estimate is accepted when both sets hold between 1 and min(n, 2k + 1024) entries -- also
+    when nearly all of them sit in one stripe of the tensor, which overflows the streaming pass's
+    per-warp regions: the gathering is then redone with the same thresholds, not the selection."""
+    n, p, m = 1 << 22, 0.01, 200000
+    rng = np.random.default_rng(21)
+    upd = (rng.standard_normal(n) * 1e-6).astype(np.float32)
+    upd[n // 3: n // 3 + n // 50] *= np.float32(1e3)            # every large entry inside 2 % of the tensor
+    idx = rng.integers(0, n, m).astype(np.uint32)
+    out, info = check_sampled(upd, np.zeros(n, dtype=np.float32), p, idx)
+    k = oracle.kept_count(n, p)
+    assert info.k != k and 0.5 * k < info.k < 2 * k                # the sampled rule's count, not the exact one
+
+
+def test_values_mode_with_clustered_candidates():
+    n, p = 1 << 22, 0.01
+    rng = np.random.default_rng(22)
+    upd = (rng.standard_normal(n) * 1e-6).astype(np.float32)
+    upd[n - n // 40:] *= np.float32(1e3)
+    check_values_mode(upd, np.zeros(n, dtype=np.float32), p)
+
+
 def test_checkpoint_and_resume_reproduces_the_streams():
     # the residual is the only state: six rounds straight == three rounds, save/restore, three more
     n, p = 200000, 0.01

@@ -44,7 +44,7 @@ enum sbc_status {
     SBC_ECAPACITY = -2,  /* an output or workspace buffer is too small */
     SBC_ENONFINITE = -3, /* residual + update holds an Inf or NaN */
     SBC_ECORRUPT = -4,   /* a stream failed validation while decoding */
-    SBC_ETIMEOUT = -5,   /* a bounded device-side wait gave up (unused so far: no kernel waits) */
+    SBC_ETIMEOUT = -5,   /* a bounded device-side wait gave up (the exact route's grid barrier) */
     SBC_ECUDA = -6       /* a CUDA runtime call failed */
 };
 
@@ -53,6 +53,7 @@ enum sbc_status {
 #define SBC_STATUS_CORRUPT 0x2u
 #define SBC_STATUS_RANGE 0x4u /* a decoded position fell outside [0, numel) */
 #define SBC_STATUS_INTERNAL 0x8u
+#define SBC_STATUS_TIMEOUT 0x10u /* a bounded device-side wait gave up; the stream holds no payload */
 
 /*
  * Stream container (little-endian).  The paper's message is the Golomb bit
@@ -319,7 +320,8 @@ int sbc_encode_static(const float *update, float *residual, int64_t numel, doubl
 
 /* Copies the header of a device-resident stream to the host and fills
  * *host_out.  Synchronises `stream`.  Returns SBC_OK, SBC_ECORRUPT if the
- * magic/version are wrong, SBC_ENONFINITE if the status word says so. */
+ * magic/version are wrong, SBC_ENONFINITE or SBC_ETIMEOUT if the status word
+ * says so. */
 int sbc_stream_info_get(const void *stream_dev, sbc_stream_info *host_out,
                         sbc_cuda_stream_t stream);
 

@@ -38,6 +38,15 @@ typedef struct sbc_encode_diag {
 } sbc_encode_diag;
 int sbc_encode_diag_get(const void *workspace, sbc_encode_diag *host_out, sbc_cuda_stream_t stream);
 
+/* The one device-side wait of the library is the barrier between the steps of
+ * the exact route's kernel; it gives up after a bounded number of polls (about a
+ * quarter of a second) and the affected streams then carry SBC_STATUS_TIMEOUT.
+ * This call shows the bound at work without damaging anything: it enqueues a
+ * two-block kernel whose barrier waits for a third block that does not exist.
+ * scratch_dev: device, two uint32 (zeroed by the call); when the stream has run,
+ * scratch_dev[1] holds SBC_STATUS_TIMEOUT.  Asynchronous. */
+int sbc_debug_barrier_timeout(uint32_t *scratch_dev, sbc_cuda_stream_t stream);
+
 #ifdef __cplusplus
 }
 #endif

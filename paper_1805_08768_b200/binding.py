@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsbc_b200.so")
 
 SBC_OK, SBC_EINVAL, SBC_ECAPACITY, SBC_ENONFINITE, SBC_ECORRUPT, SBC_ETIMEOUT, SBC_ECUDA = 0, -1, -2, -3, -4, -5, -6
-STATUS_NONFINITE, STATUS_CORRUPT, STATUS_RANGE, STATUS_INTERNAL = 1, 2, 4, 8
+STATUS_NONFINITE, STATUS_CORRUPT, STATUS_RANGE, STATUS_INTERNAL, STATUS_TIMEOUT = 1, 2, 4, 8, 16
 _ERR = {SBC_EINVAL: "SBC_EINVAL", SBC_ECAPACITY: "SBC_ECAPACITY", SBC_ENONFINITE: "SBC_ENONFINITE",
         SBC_ECORRUPT: "SBC_ECORRUPT", SBC_ETIMEOUT: "SBC_ETIMEOUT", SBC_ECUDA: "SBC_ECUDA"}
 
@@ -28,6 +28,7 @@ EXPORTS = [
     "sbc_decode_accumulate_host", "sbc_encode_static", "sbc_workspace_bytes_batch", "sbc_encode_batch",
     "sbc_decode_workspace_bytes_batch", "sbc_decode_accumulate_batch", "sbc_decode_apply", "sbc_stream_bytes_values", "sbc_encode_values", "sbc_stream_bytes_sampled",
     "sbc_workspace_bytes_sampled", "sbc_encode_sampled", "sbc_decode_accumulate_sized", "sbc_decode_apply_sized",
+    "sbc_debug_barrier_timeout",
 ]
 SIDE_VALUES = 2
 STATIC_WORKSPACE_BYTES = 8 << 20
@@ -345,6 +346,16 @@ def sbc_encode_launches() -> int:
 
 def sbc_decode_launches(n_clients: int) -> int:
     return int(lib().sbc_decode_launches(n_clients))
+
+
+def sbc_debug_barrier_timeout(scratch: torch.Tensor, stream=None) -> None:
+    """Enqueue the kernel whose barrier cannot be passed; scratch[1] then holds STATUS_TIMEOUT."""
+    if not (scratch.is_cuda and scratch.dtype == torch.int32 and scratch.numel() >= 2):
+        raise TypeError("scratch must be an int32 CUDA tensor of at least two elements")
+    L = lib()
+    L.sbc_debug_barrier_timeout.restype = C.c_int
+    L.sbc_debug_barrier_timeout.argtypes = [C.c_void_p, C.c_void_p]
+    _check(L.sbc_debug_barrier_timeout(scratch.data_ptr(), _cuda_stream(stream)), "sbc_debug_barrier_timeout")
 
 
 def sbc_encode_diag_get(workspace: torch.Tensor, stream=None) -> EncodeDiag:

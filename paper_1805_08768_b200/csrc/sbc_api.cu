@@ -250,19 +250,14 @@ inline unsigned grid_for(unsigned long long work_items, unsigned per_block, unsi
     return (unsigned)g;
 }
 
-// Blocks one problem gets for each kind of work.  The two coarsening factors (1 for a single
-// problem) make the blocks of the sample kernels and of the exact-route kernels that many times
-// larger: every block of those kernels pays for clearing and flushing a shared-memory histogram
-// (or, for the exact route, usually just for finding out that it is not needed), and a batch of
-// hundreds of problems has parallelism to spare.  The streaming pass and the ordering kernels take
-// their grids from the plan (the layout of the ordered lists depends on them).
-void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned coarse_exact, unsigned nb[WK_COUNT]) {
+// Blocks one problem gets for each kind of work.  The coarsening factor (1 for a single problem)
+// makes the blocks of the sample kernels that many times larger: every block of those kernels
+// pays for clearing and flushing a shared-memory histogram, and a batch of hundreds of problems
+// has parallelism to spare.  The streaming pass and the ordering kernels take their grids from
+// the plan (the layout of the ordered lists depends on them).
+void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned nb[WK_COUNT]) {
     nb[WK_SAMPLE] = grid_for(pl.m, kBlock * 8 * coarse_sample, sms * 4);
     nb[WK_MAIN] = pl.main_blocks;
-    // (the exact route is rare: its kernels usually only find out that they are not needed, which a
-    // smaller grid does sooner; when they do run, two blocks per SM still keep the memory busy)
-    nb[WK_EXACT] = grid_for((unsigned long long)pl.n, kBlock * 16 * coarse_exact, sms * 2);
-    nb[WK_XTILE] = grid_for(pl.n_xtiles, coarse_exact, sms * 4);
     nb[WK_CAND] = grid_for(pl.cap, kBlock * 4, sms * 2);  // x 2 sides: one resident wave at four blocks per SM
     nb[WK_ORDER] = pl.order_blocks;
     nb[WK_ONE] = 1;
@@ -307,6 +302,23 @@ __global__ void __launch_bounds__(kBlock) k_zero_stream(const Batch B) {
     for (unsigned long long i = (unsigned long long)S.bx * kBlock + threadIdx.x; i < count;
          i += (unsigned long long)S.nb * kBlock)
         dst[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Grid of the exact route's cooperative kernel: two blocks per SM (fewer if fewer fit), all of which
+// must be resident at once.  Looked up once per device.
+unsigned exact_route_blocks() {
+    static std::mutex mu;
+    static unsigned cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148u;
+    std::lock_guard<std::mutex> lock(mu);
+    if (cached[dev] == 0u) {
+        int per_sm = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k_exact_route, kBlock, 0) != cudaSuccess || per_sm < 1)
+            per_sm = 1;
+        cached[dev] = (unsigned)sm_count() * (unsigned)std::min(per_sm, 2);
+    }
+    return cached[dev];
 }
 
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
@@ -357,13 +369,21 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
     else                     go(k_add_collect<kModeBinary>, g1(WK_MAIN), B(WK_MAIN), prefix != nullptr);
     mark(SBC_MARK_COLLECT);
 
-    // 2. exact route over A (returns immediately unless the bounds failed)
-    go(k_exact_hist<0>, g1(WK_EXACT), B(WK_EXACT));
-    go(k_exact_hist<1>, g1(WK_EXACT), B(WK_EXACT));
-    go(k_exact_hist<2>, g1(WK_EXACT), B(WK_EXACT));
-    go(k_exact_tiecount, g1(WK_XTILE), B(WK_XTILE));
-    go(k_exact_tiescan, g1(WK_ONE), B(WK_ONE));
-    go(k_exact_collect, g1(WK_XTILE), B(WK_XTILE));
+    // 2. exact route over A: one cooperative kernel (its steps meet at grid barriers), which returns
+    // at once unless the candidate pass failed for some problem of the launch
+    {
+        ExactLaunch xl = {d_probs, n_probs, any_exact, any_exact + 1};   // launch_exact and x_barrier are neighbours
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(exact_route_blocks());
+        cfg.blockDim = dim3(kBlock);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        cudaLaunchKernelEx(&cfg, k_exact_route, xl);
+    }
     mark(SBC_MARK_EXACT);
 
     // 3. exact k-th composite of each candidate list, sums, side
@@ -473,7 +493,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
     }
 
     unsigned grid[WK_COUNT];
-    block_counts(pl, (unsigned)sm_count(), 1u, 1u, grid);
+    block_counts(pl, (unsigned)sm_count(), 1u, grid);
     launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, !pl.use_runs, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
@@ -576,16 +596,15 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     uint8_t* rest = zero + zero_total;
 
     const unsigned sms = (unsigned)sm_count();
-    // aim at about six (sample) and two (exact route) blocks per SM over the whole batch
-    unsigned long long fine_sample = 0, fine_exact = 0;
+    // aim at about six sample blocks per SM over the whole batch
+    unsigned long long fine_sample = 0;
     for (int t = 0; t < n_tensors; ++t) {
         fine_sample += (plans[t].m + kBlock * 8 - 1) / (kBlock * 8);
-        fine_exact += (unsigned long long)(plans[t].n + kBlock * 16 - 1) / (kBlock * 16);
     }
     auto factor = [&](unsigned long long fine, unsigned per_sm) {
         return (unsigned)std::min<unsigned long long>(256, std::max<unsigned long long>(1, fine / (sms * per_sm)));
     };
-    const unsigned coarse_sample = factor(fine_sample, 6), coarse_exact = factor(fine_exact, 2);
+    const unsigned coarse_sample = factor(fine_sample, 6);
     const size_t row_len = (size_t)n_tensors + 1;
     std::vector<Prob> probs((size_t)n_tensors);
     std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
@@ -598,7 +617,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
             z += plans[t].zero_bytes;
             r += plans[t].rest_bytes;
             unsigned nb[WK_COUNT];
-            block_counts(plans[t], sms, coarse_sample, coarse_exact, nb);
+            block_counts(plans[t], sms, coarse_sample, nb);
             for (int kind = 0; kind < WK_COUNT; ++kind) {
                 uint32_t* row = prefix.data() + (size_t)kind * row_len;
                 const unsigned long long next = (unsigned long long)row[t] + nb[kind];
@@ -674,10 +693,17 @@ int sbc_encode_static(const float* update, float* residual, int64_t numel, doubl
                       (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
 }
 
-int sbc_encode_launches(void) { return 19; }  // set-up, 2 sample, 1 collect, 6 exact, 7 select, 2 ordering + Golomb
+int sbc_encode_launches(void) { return 14; }  // set-up, 2 sample, 1 collect, 1 exact route, 7 select, 2 ordering + Golomb
 
 int sbc_decode_launches(int n_clients) {
     return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;
+}
+
+int sbc_debug_barrier_timeout(uint32_t* scratch_dev, sbc_cuda_stream_t stream) {
+    if (!scratch_dev || ((uintptr_t)scratch_dev & 3)) return SBC_EINVAL;
+    if (cudaMemsetAsync(scratch_dev, 0, 8, stream) != cudaSuccess) return SBC_ECUDA;
+    k_debug_barrier_timeout<<<2, kBlock, 0, stream>>>(scratch_dev, scratch_dev + 1);
+    return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
 int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cuda_stream_t stream) {
@@ -805,6 +831,7 @@ int sbc_stream_info_get(const void* stream_dev, sbc_stream_info* host_out, sbc_c
     o.total_bytes = o.payload_offset + align_up((size_t)((o.nbits + 7) / 8), 16);
     if (o.magic != SBC_MAGIC || o.version != SBC_VERSION) return SBC_ECORRUPT;
     if (o.status & SBC_STATUS_NONFINITE) return SBC_ENONFINITE;
+    if (o.status & SBC_STATUS_TIMEOUT) return SBC_ETIMEOUT;
     if (o.status) return SBC_ECORRUPT;
     return SBC_OK;
 }

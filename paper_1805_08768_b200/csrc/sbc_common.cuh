@@ -43,6 +43,7 @@ struct Ctl {
     uint32_t status;            // SBC_STATUS_* bits
     uint32_t use_fallback;      // 1: the candidate pass did not bracket both thresholds
     uint32_t launch_exact;      // in the launch's first problem: some problem of the launch has use_fallback set
+    uint32_t x_barrier;         // in the launch's first problem: arrivals at the exact route's grid barriers
     uint32_t done[ST_COUNT];    // tickets for the last-block pattern
     // threshold bounds from the sample
     uint32_t s_bin0[2], s_rank[2];
@@ -199,17 +200,9 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
     return s;
 }
 
-// First lines of the exact-route kernels: false (for the whole grid) when no problem of the launch
-// needs them, which is the usual case, so that they end before looking for their problem.
-__device__ __forceinline__ bool launch_needs_exact_route(const Batch& B) {
-    cudaTriggerProgrammaticLaunchCompletion();
-    cudaGridDependencySynchronize();
-    return __ldcg(B.any_exact) != 0u;
-}
-
 // Kinds of work a kernel's grid is sized by (one prefix table per kind in a batch).
 enum WorkKind : int {
-    WK_SAMPLE = 0, WK_MAIN, WK_EXACT, WK_XTILE, WK_CAND, WK_ORDER, WK_ONE, WK_STREAM, WK_COUNT
+    WK_SAMPLE = 0, WK_MAIN, WK_CAND, WK_ORDER, WK_ONE, WK_STREAM, WK_COUNT
 };
 
 // What the kept entries of one warp range of the ordering kernels add up to (see k_span_count).

@@ -207,3 +207,22 @@ def test_long_stream_is_decoded_in_list_order_and_rejects_damage():
     assert run(bad)[0] != 0
     bad = stream.copy(); bad[table + 16 * 9000 + 8: table + 16 * 9000 + 16].view("<i8")[0] = 2**40  # absurd previous position
     assert run(bad)[0] & sbc.STATUS_CORRUPT
+
+
+def test_the_bounded_wait_of_the_exact_route_gives_up_and_reports_it():
+    """The exact route's steps meet at a barrier in global memory.  Its wait is bounded: a barrier
+    that cannot be passed (here: one that waits for a block that does not exist) ends by itself
+    after a fraction of a second and leaves a status word, and the device is as usable as before."""
+    scratch = torch.zeros(2, dtype=torch.int32, device=DEV)
+    sbc.sbc_debug_barrier_timeout(scratch)
+    torch.cuda.synchronize()
+    assert scratch[1].item() == sbc.STATUS_TIMEOUT
+    # the context is intact: an ordinary encode still matches the oracle afterwards
+    n, p = 100000, 0.01
+    upd = workloads.normal_flat(n, 1e-3, 77)
+    want_res = np.zeros(n, dtype=np.float32)
+    want_stream, _ = oracle.encode(upd, want_res, p)
+    r = torch.zeros(n, dtype=torch.float32, device=DEV)
+    out, _ = sbc.sbc_encode(torch.from_numpy(upd).to(DEV), r, p)
+    info = sbc.sbc_stream_info_get(out)
+    assert np.array_equal(out[: info.total_bytes].cpu().numpy(), want_stream)

@@ -102,7 +102,7 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
         target = (uint32_t)std::max<long long>(1, (long long)std::floor(p * (double)sampled_m));
         up = 0;  // every candidate is kept: nothing is selected afterwards
     }
-    if (k < 32768) up = 0;  // short lists: selecting over all of them costs less than the second bound
+    if (pl->cap <= kSmallList && !force_runs) up = 0;  // a list one block ranks in its registers has no use for the second bound
     pl->s_target = target;
     pl->s_up = up;
     pl->n_xtiles = (uint32_t)((n + kXTile - 1) / kXTile);
@@ -398,13 +398,8 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
         go(k_select_small, g2(WK_ONE), B(WK_ONE));
     } else {
         go(k_select_hist0, g2(WK_CAND), B(WK_CAND));
-        go(k_select_filter<0>, g2(WK_CAND), B(WK_CAND));
-        go(k_select_filter<1>, g2(WK_CAND), B(WK_CAND));
-        go(k_select_filter<2>, g2(WK_CAND), B(WK_CAND));
-        go(k_select_filter<3>, g2(WK_CAND), B(WK_CAND));
-        go(k_select_filter<4>, g2(WK_CAND), B(WK_CAND));
+        go(k_select_filter0, g2(WK_CAND), B(WK_CAND));
     }
-    go(k_sums_decide, g2(WK_CAND), B(WK_CAND));
     mark(SBC_MARK_SELECT);
 
     go(k_span_count, g1(WK_ORDER), B(WK_ORDER));
@@ -475,6 +470,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
     uint8_t* ws = static_cast<uint8_t*>(workspace);
     uint8_t* zero = ws + kProbSlotBytes;
     uint8_t* rest = zero + pl.zero_bytes;
+    const bool small_lists = pl.cap <= kSmallList, small_form = !pl.use_runs;
     Prob P = make_prob(a, pl, zero, rest);
     P.sample_idx = sample_idx;
     Prob* d_prob = reinterpret_cast<Prob*>(ws);
@@ -494,7 +490,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, grid);
-    launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, pl.cap <= kSmallList, !pl.use_runs, st, marks);
+    launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, small_lists, small_form, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -605,6 +601,8 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         return (unsigned)std::min<unsigned long long>(256, std::max<unsigned long long>(1, fine / (sms * per_sm)));
     };
     const unsigned coarse_sample = factor(fine_sample, 6);
+    bool small_lists = true;
+    for (int t = 0; t < n_tensors; ++t) small_lists = small_lists && plans[t].cap <= kSmallList;
     const size_t row_len = (size_t)n_tensors + 1;
     std::vector<Prob> probs((size_t)n_tensors);
     std::vector<uint32_t> prefix((size_t)WK_COUNT * row_len, 0u);
@@ -646,8 +644,6 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
     k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors, nullptr});
-    bool small_lists = true;
-    for (int t = 0; t < n_tensors; ++t) small_lists = small_lists && plans[t].cap <= kSmallList;
     launch_encode(d_probs, (uint32_t)n_tensors, &probs[0].ctl->launch_exact, grid, d_rows, kModeBinary, false, small_lists, all_small, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
@@ -693,7 +689,7 @@ int sbc_encode_static(const float* update, float* residual, int64_t numel, doubl
                       (size_t)SBC_STATIC_WORKSPACE_BYTES, stream);
 }
 
-int sbc_encode_launches(void) { return 14; }  // set-up, 2 sample, 1 collect, 1 exact route, 7 select, 2 ordering + Golomb
+int sbc_encode_launches(void) { return 9; }  // set-up, 2 sample, 1 collect, 1 exact route, 2 select + sums, 2 ordering + Golomb
 
 int sbc_decode_launches(int n_clients) {
     return n_clients <= 0 ? 0 : (n_clients + kMaxClientsPerLaunch - 1) / kMaxClientsPerLaunch;
@@ -718,7 +714,7 @@ int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cu
         cudaStreamSynchronize(stream) != cudaSuccess)
         return SBC_ECUDA;
     host_out->status = c.status;
-    host_out->exact_route = c.use_fallback;
+    host_out->exact_route = (c.use_fallback || c.regathered) ? 1u : 0u;
     host_out->candidates[0] = c.cand_cnt[0];
     host_out->candidates[1] = c.cand_cnt[1];
     host_out->capacity = P.cap;
@@ -727,7 +723,7 @@ int sbc_encode_diag_get(const void* workspace, sbc_encode_diag* host_out, sbc_cu
     host_out->mu_pos = c.mu64[0];
     host_out->mu_neg = c.mu64[1];
     for (int s = 0; s < 2; ++s) host_out->certain[s] = c.use_fallback ? 0u : c.sure_cnt[s];
-    host_out->regathered = (c.use_fallback && c.x_known) ? 1u : 0u;
+    host_out->regathered = c.regathered;
     return SBC_OK;
 }
 

@@ -15,6 +15,7 @@
 
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include "../../include/sbc.h"
 
 namespace sbc {
 
@@ -32,10 +33,7 @@ constexpr uint32_t kSmallList = 8192;  // candidate lists up to this capacity ar
 // Stages that use the "last block to finish does the serial step" pattern.
 enum Stage : int {
     ST_SAMPLE0 = 0, ST_SAMPLE1, ST_SAMPLE2, ST_COLLECT, ST_XH0, ST_XH1, ST_XH2,
-    ST_BH0_S0, ST_BH0_S1,
-    ST_BF0_S0, ST_BF0_S1, ST_BF1_S0, ST_BF1_S1, ST_BF2_S0, ST_BF2_S1,
-    ST_BF3_S0, ST_BF3_S1, ST_BF4_S0, ST_BF4_S1,
-    ST_SUM, ST_ORDER, ST_COUNT
+    ST_HIST_S0, ST_HIST_S1, ST_FILTER_S0, ST_FILTER_S1, ST_SUM, ST_ORDER, ST_COUNT
 };
 
 // Device-side control block of one encode call; zeroed before the first kernel.
@@ -60,13 +58,15 @@ struct Ctl {
     uint32_t band_cnt[2];
     uint32_t overflow;          // a warp's region of the ordered list, or a band list, did not hold its entries
     uint32_t x_known;           // exact route: the thresholds are already known (x_thr), only the gathering is redone
+    uint32_t regathered;        // the gathering was redone (what x_known asked for), and the fast route's kernels go on from there
     long long pre_bins[2][256]; // exact sums of the sure entries, gathered while they were flushed
     // exact select over A (fallback)
     uint32_t x_prefix[2], x_rank[2], x_thr[2], x_ties_take[2], x_ties_have[2];
+    unsigned long long x_min_inv[2];  // complement of the smallest composite the exact route gathered (zero: none yet)
     // select over the candidate lists
-    unsigned long long b_prefix[2];
+    unsigned long long b_prefix[2];   // digits of the k-th largest composite found so far (relative to SelectDigits::sub)
     uint32_t b_rank[2];
-    uint32_t list_cnt[2][6];
+    uint32_t list_cnt[2];             // entries that share the first digit with the k-th largest
     unsigned long long thr[2];  // kept <=> composite >= thr[side]
     uint32_t sel_done[2];       // thr[side] is final: the remaining selection kernels have nothing to do
     // sums and decision
@@ -86,7 +86,7 @@ struct Hists {
     uint32_t s1[2][2][kHistBins];  // [side][0: lower bound's bin, 1: upper bound's bin]
     uint32_t s2[2][1024];
     uint32_t x[3][2][kHistBins];
-    uint32_t b[6][2][kHistBins];
+    uint32_t b0[2][kHistBins];     // first digit of the entries the candidate select ranks
 };
 
 // Everything a kernel needs to know about one encode problem.  Lives in
@@ -265,6 +265,66 @@ __device__ __forceinline__ BandView band_view(const Prob& P, const Ctl* ctl, int
     return v;
 }
 
+// Digit schedule of the candidate select.  The entries it ranks lie in a known range of composites:
+// `sub` is the smallest composite the range can hold and `top` the highest bit in which an entry
+// can differ from it once `sub` is taken off.  Digits are 11 bits each, from bit `top` downwards
+// (the last one takes what is left).  Fast route: the band between the two sample bounds, a narrow
+// range of keys, so that already the first digit tells the entries apart; exact route: the whole
+// range of composites (six digits).
+struct SelectDigits {
+    int top;
+    unsigned long long sub;
+};
+__device__ __forceinline__ SelectDigits band_digits(const Ctl* ctl, int s) {
+    const uint32_t lo = ctl->lo_key[s], width = ctl->up_key[s] - 1u - lo;  // band keys lie in [lo, lo + width]
+    SelectDigits d;
+    d.top = 63 - __clz((int)width);   // 31 for width 0: only the index half differs
+    d.sub = (unsigned long long)lo << 32;
+    return d;
+}
+__device__ __forceinline__ SelectDigits select_digits(const Ctl* ctl, int s) {
+    if (ctl->use_fallback) { SelectDigits d; d.top = 63; d.sub = 0ull; return d; }
+    return band_digits(ctl, s);
+}
+__device__ __forceinline__ int digit_bits(int level, int top) { return max(0, min(11, top + 1 - 11 * level)); }
+__device__ __forceinline__ int digit_shift(int level, int top) { return max(0, top + 1 - 11 * (level + 1)); }
+__device__ __forceinline__ int digit_levels(int top) { return (top + 1 + 10) / 11; }
+// Digit `level` of a composite from which `sub` has already been taken off.
+__device__ __forceinline__ uint32_t digit_of(unsigned long long c, int level, int top) {
+    return (uint32_t)(c >> digit_shift(level, top)) & ((1u << digit_bits(level, top)) - 1u);
+}
+
+// Exact sum of fp32 values (Algorithm 2's means): a value is m * 2^(e-150) with an integer m of at
+// most 24 bits, so one 64-bit integer per exponent holds the sum of up to 2^39 of them and integer
+// addition makes the result independent of the order.  Values within eight binades above `bin_a`
+// (nearly all of them, when bin_a is the binade below the threshold's) are added in one register,
+// in units of the lowest of those binades; the rest goes to the 256 shared bins by atomics.
+struct ExactSum {
+    int bin_a;
+    long long acc;
+    __device__ __forceinline__ void start(uint32_t bits_near) {
+        bin_a = max((int)((bits_near >> 23) & 0xffu) - 1, 0);
+        acc = 0;
+    }
+    __device__ __forceinline__ void add(uint32_t bits, unsigned long long* s_bins) {
+        const uint32_t e = (bits >> 23) & 0xffu;
+        int m = (int)(bits & 0x7fffffu) | (e ? 0x800000 : 0);
+        if (bits >> 31) m = -m;
+        const int bin = e ? (int)e - 1 : 0;
+        const uint32_t up = (uint32_t)(bin - bin_a);
+        if (up < 8u) acc += (long long)m << up;   // |m| < 2^24: at most 2^31 per entry, 2^62 over 2^31 entries
+        else atomicAdd(&s_bins[bin], (unsigned long long)(long long)m);
+    }
+    // All lanes of every warp of the block call; the bins are complete after the next barrier.
+    __device__ __forceinline__ void finish(unsigned long long* s_bins) {
+        long long v = acc;
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xffffffffu, v, d);
+        if ((threadIdx.x & 31u) == 0u && v) atomicAdd(&s_bins[bin_a], (unsigned long long)v);
+        acc = 0;
+    }
+};
+
 // Codewords per chunk-table entry of a stream that carries k positions.  The decoder gives every
 // chunk to one lane, which parses it codeword after codeword, so short streams get short chunks:
 // a stream of 10^5 positions then still occupies a hundred warps.  (A convention of the container;
@@ -396,6 +456,19 @@ __device__ __forceinline__ void block_pick_desc(const uint32_t* hist, int nbins,
             }
             cum += h[j];
         }
+    }
+    __syncthreads();
+}
+
+// The bucket of the rank-th largest entry's first digit, from the finished histogram of the list
+// the candidate select ranks: the start of b_prefix / b_rank.  One block, all threads call.
+__device__ __forceinline__ void select_pick0(const Prob& P, Ctl* ctl, int s, uint32_t rank, int top, uint32_t* s_scan,
+                                             Pick* s_pick) {
+    block_pick_desc(P.hists->b0[s], 1 << digit_bits(0, top), false, rank, s_scan, s_pick);
+    if (threadIdx.x == 0) {
+        ctl->b_prefix[s] = (unsigned long long)s_pick->bin << digit_shift(0, top);
+        ctl->b_rank[s] = s_pick->rank;
+        if (!s_pick->found) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
     }
     __syncthreads();
 }

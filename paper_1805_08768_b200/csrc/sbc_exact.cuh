@@ -18,8 +18,9 @@
 
 namespace sbc {
 
-// Whether a problem takes the route.  Decided by the streaming pass and not changed afterwards, so
-// that every block of the route's kernel sees the same answer at any time.
+// Whether a problem takes the route.  Decided by the streaming pass and not changed before the
+// route's last step (one block per problem, which is then done with it), so that every block of
+// the route's kernel sees the same answer in every step that works on the problem.
 __device__ __forceinline__ bool exact_route_active(const Ctl* ctl) { return ctl->use_fallback != 0u; }
 
 // Shared memory of the exact route's kernel, used by one step at a time.
@@ -180,6 +181,7 @@ __device__ __forceinline__ void exact_collect_step(const Prob& P, uint32_t bx, u
     const bool one_sided = P.mode == kModeValues;  // magnitude selection has no second side
     const float* __restrict__ A = P.residual;
     const uint32_t span_steps = P.span_steps;
+    unsigned long long least[2] = {~0ull, ~0ull};  // smallest composite this thread gathered
     for (uint32_t tile = S.bx; tile < P.n_xtiles; tile += S.nb) {
         const long long wbase = (long long)tile * kXTile + (long long)warp * kWarpChunk;
         uint32_t key[kSteps];
@@ -255,8 +257,9 @@ __device__ __forceinline__ void exact_collect_step(const Prob& P, uint32_t bx, u
                 const unsigned mm = __ballot_sync(0xffffffffu, mine);
                 if (mine) {
                     const uint32_t slot = pos + (uint32_t)__popc(mm & lt);
-                    if (slot < P.list_cap)
-                        P.list[s][slot] = make_composite(side_key(s, key[j]), (uint32_t)(wbase + j * 32 + lane));
+                    const unsigned long long c = make_composite(side_key(s, key[j]), (uint32_t)(wbase + j * 32 + lane));
+                    if (slot < P.list_cap) P.list[s][slot] = c;
+                    least[s] = min(least[s], c);
                 }
                 pos += (uint32_t)__popc(mm);
             }
@@ -269,6 +272,34 @@ __device__ __forceinline__ void exact_collect_step(const Prob& P, uint32_t bx, u
             }
         }
         __syncthreads();  // the shared arrays are reused by the next tile
+    }
+    // the k-th largest composite of a side is the smallest one gathered (when exactly k were)
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+        unsigned long long v = ~least[s];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) v = max(v, __shfl_down_sync(0xffffffffu, v, d));
+        if (lane == 0 && v) atomicMax(&ctl->x_min_inv[s], v);
+    }
+}
+
+// What the kernels after the route go by.  Thresholds found here: the lists hold exactly the k
+// kept entries of each side, so the selection has nothing to do.  Gathering redone: the fast
+// route's lists are whole again, its kernels take over.  One thread of one block per problem.
+__device__ __forceinline__ void exact_final_step(const Prob& P) {
+    Ctl* ctl = P.ctl;
+    if (threadIdx.x != 0) return;
+    if (__ldcg(&ctl->x_known) != 0u) {
+        ctl->regathered = 1u;
+        ctl->use_fallback = 0u;
+        return;
+    }
+    const int sides = P.mode == kModeValues ? 1 : 2;
+    for (int s = 0; s < sides; ++s) {
+        const unsigned long long inv = __ldcg(&ctl->x_min_inv[s]);
+        ctl->thr[s] = ~inv;
+        ctl->sel_done[s] = 1u;
+        if (inv == 0ull || __ldcg(&ctl->cand_cnt[s]) != (uint32_t)P.k) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
     }
 }
 
@@ -315,7 +346,7 @@ __device__ __forceinline__ void load_problem(const ExactLaunch& L, uint32_t p, P
     __syncthreads();
 }
 
-enum ExactStepKind : int { XS_HIST0 = 0, XS_HIST1, XS_HIST2, XS_TIECOUNT, XS_TIESCAN, XS_COLLECT };
+enum ExactStepKind : int { XS_HIST0 = 0, XS_HIST1, XS_HIST2, XS_TIECOUNT, XS_TIESCAN, XS_COLLECT, XS_FINAL };
 
 // One step of the route for every problem of the launch that needs it.  Problems are looked at 256
 // at a time (every thread reads one problem's flags); all blocks see the same flags, so they all
@@ -331,14 +362,14 @@ __device__ __forceinline__ void exact_step_all(const ExactLaunch& L, Prob* s_pro
         if (p < L.n_probs) {
             const Ctl* ctl = L.probs[p].ctl;
             const bool active = exact_route_active(ctl);
-            const bool wanted = active && (STEP == XS_COLLECT || ctl->x_known == 0u);
+            const bool wanted = active && (STEP == XS_COLLECT || STEP == XS_FINAL || ctl->x_known == 0u);
             if (wanted) s_list[atomicAdd(s_count, 1u)] = p;   // any order: the problems are independent
         }
         __syncthreads();
         const uint32_t count = *s_count;
         for (uint32_t j = 0u; j < count; ++j) {
             const uint32_t q = s_list[j];
-            if (STEP == XS_TIESCAN && q % gridDim.x != blockIdx.x) continue;  // one block per problem (block-uniform)
+            if ((STEP == XS_TIESCAN || STEP == XS_FINAL) && q % gridDim.x != blockIdx.x) continue;  // one block per problem (block-uniform)
             load_problem(L, q, s_prob);
             if (STEP == XS_HIST0) exact_hist_step<0>(*s_prob, blockIdx.x, gridDim.x, sh);
             if (STEP == XS_HIST1) exact_hist_step<1>(*s_prob, blockIdx.x, gridDim.x, sh);
@@ -346,6 +377,7 @@ __device__ __forceinline__ void exact_step_all(const ExactLaunch& L, Prob* s_pro
             if (STEP == XS_TIECOUNT) exact_tiecount_step(*s_prob, blockIdx.x, gridDim.x, sh);
             if (STEP == XS_TIESCAN) exact_tiescan_step(*s_prob, sh);
             if (STEP == XS_COLLECT) exact_collect_step(*s_prob, blockIdx.x, gridDim.x, sh);
+            if (STEP == XS_FINAL) exact_final_step(*s_prob);
         }
     }
 }
@@ -384,7 +416,11 @@ __global__ void __launch_bounds__(kBlock) k_exact_route(const ExactLaunch L) {
     }
     if (ok) {
         exact_step_all<XS_COLLECT>(L, &s_prob, sh, s_list, &s_count);
-        return;
+        ok = grid_barrier(L.barrier, gridDim.x, epoch);
+        if (ok) {
+            exact_step_all<XS_FINAL>(L, &s_prob, sh, s_list, &s_count);
+            return;
+        }
     }
     // a barrier gave up: whatever needed the route has no lists to go on with
     for (uint32_t p = threadIdx.x; p < L.n_probs; p += kBlock) {

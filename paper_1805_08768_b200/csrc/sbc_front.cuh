@@ -591,17 +591,22 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
             if (!ok) {
                 atomicOr(B.any_exact, 1u);
                 // The exact route rebuilds the lists.  If only the placement failed (a warp's region
-                // or a band list too small for unevenly spread candidates) the bounds still hold:
-                // everything at or beyond them is gathered again, this time with space reserved tile by tile.
+                // too small for unevenly spread candidates) the bounds still hold, and so does everything
+                // that does not depend on where a candidate was put: the band list (it cannot overflow
+                // while the counts fit) and the counts and sums of the sure entries.  Only the ordered
+                // lists are gathered again, this time with space reserved tile by tile, and the fast
+                // route's kernels go on from there.
                 if (counts_ok && bounds_ok) {
                     ctl->x_known = 1u;
                     ctl->x_thr[0] = ctl->lo_key[0];
                     ctl->x_thr[1] = ctl->lo_key[1];
                 }
-                ctl->cand_cnt[0] = 0u;
+                else {
+                    ctl->sure_cnt[0] = 0u;
+                    ctl->sure_cnt[1] = 0u;
+                }
+                ctl->cand_cnt[0] = 0u;   // counted again as the lists are rebuilt
                 ctl->cand_cnt[1] = 0u;
-                ctl->sure_cnt[0] = 0u;
-                ctl->sure_cnt[1] = 0u;
             }
             ctl->sampled_ok = (counts_ok && P.sampled) ? 1u : 0u;
         }

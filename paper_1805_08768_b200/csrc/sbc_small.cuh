@@ -41,16 +41,17 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
     if (s_status == 0u) {
         const BandView view = band_view(P, ctl, s);   // short lists have no upper bound: every candidate is in the band
         const uint32_t cnt = view.count, rank = view.rank;
-        unsigned long long prefix, thr = 0ull;
-        const int top = select_top(P, ctl, s, &prefix);
+        unsigned long long thr = 0ull;
+        const SelectDigits dg = select_digits(ctl, s);
         bool good = cnt <= kSmallList;  // what the host checked through the capacity
         unsigned long long c[kPer];
 #pragma unroll
         for (int j = 0; j < kPer; ++j) {
             const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
-            c[j] = (good && i < cnt) ? view.src[i] : 0ull;
+            c[j] = (good && i < cnt) ? view.src[i] - dg.sub : 0ull;
         }
-        good = good && block_select_registers<kPer>(c, cnt, rank, top, 0, prefix, s_hist, s_scan, &s_pick, &s_result, &thr);
+        good = good && block_select_registers<kPer>(c, cnt, rank, dg.top, 0, 0ull, s_hist, s_scan, &s_pick, &s_result, &thr);
+        thr += dg.sub;
         if (!good) {
             if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);
         } else {

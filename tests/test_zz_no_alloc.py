@@ -60,7 +60,7 @@ def test_static_scratch_at_its_limit_then_a_small_call():
     # the largest problem the fixed array takes at p = 0.01 (its scratch fills all but a few KB of
     # the 8 MiB), then a small one that reuses the same bytes
     p = 0.01
-    n = 2_600_000
+    n = 2_670_000
     need = sbc.sbc_workspace_bytes(n, p)
     assert 0.98 * sbc.STATIC_WORKSPACE_BYTES < need <= sbc.STATIC_WORKSPACE_BYTES
     assert sbc.sbc_workspace_bytes(n + 20_000, p) > sbc.STATIC_WORKSPACE_BYTES

@@ -592,15 +592,16 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     uint8_t* rest = zero + zero_total;
 
     const unsigned sms = (unsigned)sm_count();
-    // aim at about six sample blocks per SM over the whole batch
-    unsigned long long fine_sample = 0;
-    for (int t = 0; t < n_tensors; ++t) {
-        fine_sample += (plans[t].m + kBlock * 8 - 1) / (kBlock * 8);
+    // Sample kernels: the smallest block size (in units of 2048 sampled elements) with which the
+    // blocks of the whole batch are resident at once (four per SM); a second, short wave would cost
+    // as much time again as the first.
+    unsigned coarse_sample = 1;
+    for (; coarse_sample < 256; ++coarse_sample) {
+        unsigned long long blocks = 0;
+        for (int t = 0; t < n_tensors; ++t)
+            blocks += (plans[t].m + (unsigned long long)kBlock * 8 * coarse_sample - 1) / ((unsigned long long)kBlock * 8 * coarse_sample);
+        if (blocks <= (unsigned long long)sms * 4) break;
     }
-    auto factor = [&](unsigned long long fine, unsigned per_sm) {
-        return (unsigned)std::min<unsigned long long>(256, std::max<unsigned long long>(1, fine / (sms * per_sm)));
-    };
-    const unsigned coarse_sample = factor(fine_sample, 6);
     bool small_lists = true;
     for (int t = 0; t < n_tensors; ++t) small_lists = small_lists && plans[t].cap <= kSmallList;
     const size_t row_len = (size_t)n_tensors + 1;

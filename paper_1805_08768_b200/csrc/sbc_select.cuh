@@ -69,6 +69,21 @@ __device__ __forceinline__ bool block_select_registers(const unsigned long long 
     return true;
 }
 
+// Highest bit set in any of a block's values (all threads call, result in all; s_tmp: one word per
+// warp).  A list that is ranked by one block starts its digits there: with no upper bound on its
+// keys the range the digits were laid out for is mostly empty at the top.
+__device__ __forceinline__ int block_top_bit(unsigned long long any_bits, unsigned long long* s_tmp) {
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) any_bits |= __shfl_xor_sync(0xffffffffu, any_bits, d);
+    __syncthreads();  // s_tmp may still be read from an earlier use
+    if (lane_id() == 0) s_tmp[threadIdx.x >> 5] = any_bits;
+    __syncthreads();
+    unsigned long long all = 0ull;
+#pragma unroll
+    for (int w = 0; w < kBlock / 32; ++w) all |= s_tmp[w];
+    return all ? 63 - __clzll((long long)all) : 0;
+}
+
 constexpr int kFinishPer = 8;  // entries per thread the short rest of a side is ranked from in registers
 constexpr uint32_t kFinishList = kFinishPer * kBlock;
 
@@ -420,6 +435,7 @@ __global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
     __shared__ unsigned long long s_result;
     __shared__ unsigned long long s_bins[2][256];
     __shared__ uint32_t s_nonzero[2][8];
+    __shared__ unsigned long long s_top[kBlock / 32];
     s_bins[0][threadIdx.x] = 0ull;
     const BandView view = band_view(P, ctl, s);
     const uint32_t cnt = view.count, rank = view.rank;
@@ -436,7 +452,11 @@ __global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
         unsigned long long thr_rel = 0ull;  // accepted sampled thresholds: every candidate is kept
         bool good = true;
         if (!ctl->sampled_ok) {
-            good = block_select_registers<kPer>(c, cnt, rank, dg.top, 0, 0ull, s_hist, s_scan, &s_pick, &s_result, &thr_rel);
+            unsigned long long bits = 0ull;
+#pragma unroll
+            for (int j = 0; j < kPer; ++j) bits |= c[j];
+            const int top = min(dg.top, block_top_bit(bits, s_top));
+            good = block_select_registers<kPer>(c, cnt, rank, top, 0, 0ull, s_hist, s_scan, &s_pick, &s_result, &thr_rel);
             if (threadIdx.x == 0) {
                 if (good) ctl->thr[s] = thr_rel + dg.sub;
                 else atomicOr(&ctl->status, SBC_STATUS_INTERNAL);

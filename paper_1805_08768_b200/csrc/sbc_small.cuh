@@ -50,7 +50,11 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
             const uint32_t i = (uint32_t)j * kBlock + threadIdx.x;
             c[j] = (good && i < cnt) ? view.src[i] - dg.sub : 0ull;
         }
-        good = good && block_select_registers<kPer>(c, cnt, rank, dg.top, 0, 0ull, s_hist, s_scan, &s_pick, &s_result, &thr);
+        unsigned long long bits = 0ull;
+#pragma unroll
+        for (int j = 0; j < kPer; ++j) bits |= c[j];
+        const int top = min(dg.top, block_top_bit(bits, s_scan64));
+        good = good && block_select_registers<kPer>(c, cnt, rank, top, 0, 0ull, s_hist, s_scan, &s_pick, &s_result, &thr);
         thr += dg.sub;
         if (!good) {
             if (threadIdx.x == 0) atomicOr(&ctl->status, SBC_STATUS_INTERNAL);

@@ -211,6 +211,34 @@ def test_selection_looks_only_at_the_band_between_the_two_bounds():
         assert np.array_equal(res.view(np.uint32), want_res.view(np.uint32))
 
 
+@pytest.mark.parametrize("ties", [5000, 40000])
+def test_many_equal_values_straddle_the_threshold_inside_the_band(ties):
+    # thousands of entries with exactly the value the k-th largest one has, half of them kept (the
+    # ones at the lowest positions): the bucket of the first select digit that holds the threshold
+    # then holds all of them, far more than one block ranks in its registers, and the selection has
+    # to work through the index half of the composites digit by digit
+    n, p = 1 << 23, 0.01
+    k = oracle.kept_count(n, p)
+    rng = np.random.default_rng(ties)
+    upd = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    order = np.argsort(upd)
+    v_pos, v_neg = upd[order[n - (k - ties // 2)]], upd[order[k - ties // 2 - 1]]
+    middle = order[n // 4: 3 * n // 4]                  # entries far from both thresholds
+    planted = rng.choice(middle, 2 * ties, replace=False)
+    upd[planted[:ties]] = v_pos
+    upd[planted[ties:]] = v_neg
+    assert np.count_nonzero(upd > v_pos) < k < np.count_nonzero(upd >= v_pos)
+    assert np.count_nonzero(upd < v_neg) < k < np.count_nonzero(upd <= v_neg)
+    want_res = np.zeros(n, dtype=np.float32)
+    want_stream, want_mu = oracle.encode(upd, want_res, p)
+    stream, mu, res, diag = encode_with_diag(upd, p)
+    assert diag.exact_route == 0                          # the sample's bounds still bracket both thresholds
+    assert np.array_equal(stream, want_stream) and mu.view(np.uint32) == want_mu.view(np.uint32)
+    assert np.array_equal(res.view(np.uint32), want_res.view(np.uint32))
+    # magnitude selection: with the negative side scaled down its k-th largest |value| is v_pos too
+    check_values_mode(np.where(upd > 0, upd, upd * np.float32(0.1)).astype(np.float32), np.zeros(n, dtype=np.float32), p)
+
+
 def test_upper_bound_below_the_threshold_takes_the_exact_route():
     # large entries only where the strided sample does not look: both bounds come out too low and k
     # or more candidates pass the upper one, so it says nothing about what is kept; the thresholds

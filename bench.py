@@ -290,6 +290,23 @@ def run_ours(args):
     if int(status.item()) != 0:
         raise RuntimeError(f"decoder reported status {int(status.item())}")
 
+    # The decode once more, per p, with the L2 cleaned between the caller's zero fill and the timed
+    # call (a read of 512 MB that nothing wrote): the timed decodes above start with the L2 full of
+    # the zero fill's dirty lines, which are written back while the decode's own lines come in.
+    # Reported beside decode_ms, not part of `value`.
+    dec_clean_ms = [0.0] * len(P_SWEEP)
+    clean_reps = 5
+    for i, p in enumerate(P_SWEEP):
+        for _ in range(clean_reps):
+            dense.zero_()
+            update[: 1 << 27].sum()
+            d0, d1 = new_events(2)
+            d0.record(cur)
+            sbc.sbc_decode_accumulate([streams[i]], dense, status=status)
+            d1.record(cur)
+            torch.cuda.synchronize()
+            dec_clean_ms[i] += d0.elapsed_time(d1) / clean_reps
+
     infos = [sbc.sbc_stream_info_get(s) for s in streams]
     diags = []
     for i, p in enumerate(P_SWEEP):  # one more untimed encode per p to read back which route it takes
@@ -335,6 +352,7 @@ def run_ours(args):
             "decode_dense_gelem_s": n / (d * 1e-3) / 1e9,
             "decode_gbs": (DECODE_BYTES_PER_POSITION * infos[i].k + infos[i].total_bytes) / (d * 1e-3) / 1e9,
             "decode_frac_of_peak": (DECODE_BYTES_PER_POSITION * infos[i].k + infos[i].total_bytes) / (d * 1e-3) / 1e9 / peak,
+            "decode_ms_clean_l2": dec_clean_ms[i],
             "stage_ms": {name: stage_ms[i][s] / steps for s, name in enumerate(sbc.MARK_NAMES)},
             "route": diags[i],
         })

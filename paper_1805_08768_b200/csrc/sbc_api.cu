@@ -324,8 +324,8 @@ unsigned exact_route_blocks() {
 // Enqueue every kernel of the encode path once; `grid[kind]` blocks and `prefix[kind]` (null for
 // a single problem) say how each kind of work is spread over the problems.
 void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, const unsigned grid[WK_COUNT],
-                   const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, bool small_form, cudaStream_t st,
-                   const sbc_cuda_event_t* marks) {
+                   const uint32_t* const* prefix, int mode, bool sampled, bool small_lists, bool small_form, bool dense_spans,
+                   cudaStream_t st, const sbc_cuda_event_t* marks) {
     // Every stage boundary closes an NVTX range and opens the next one (host-side ranges around the
     // launches of a stage, for a timeline tool; no-ops when none is attached), and records the
     // caller's event for that boundary if it gave one.
@@ -402,7 +402,8 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
     }
     mark(SBC_MARK_SELECT);
 
-    go(k_span_count, g1(WK_ORDER), B(WK_ORDER));
+    if (dense_spans) go(k_span_count<true>, g1(WK_ORDER), B(WK_ORDER));
+    else             go(k_span_count<false>, g1(WK_ORDER), B(WK_ORDER));
     go(k_span_emit, g1(WK_ORDER), B(WK_ORDER), false);
     mark(SBC_MARK_END);
 }
@@ -490,7 +491,8 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
 
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, grid);
-    launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, small_lists, small_form, st, marks);
+    launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, small_lists, small_form,
+                  (unsigned long long)pl.k >= 16ull * pl.n_spans, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 
@@ -645,7 +647,10 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
         grid[kind] = prefix[(size_t)kind * row_len + (size_t)n_tensors];
     }
     k_zero_stream<<<grid[WK_STREAM], kBlock, 0, st>>>(Batch{d_probs, d_rows[WK_STREAM], (uint32_t)n_tensors, nullptr});
-    launch_encode(d_probs, (uint32_t)n_tensors, &probs[0].ctl->launch_exact, grid, d_rows, kModeBinary, false, small_lists, all_small, st, nullptr);
+    unsigned long long k_total = 0, spans_total = 0;
+    for (int t = 0; t < n_tensors; ++t) { k_total += (unsigned long long)plans[t].k; spans_total += plans[t].n_spans; }
+    launch_encode(d_probs, (uint32_t)n_tensors, &probs[0].ctl->launch_exact, grid, d_rows, kModeBinary, false, small_lists, all_small,
+                  k_total >= 16ull * spans_total, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

@@ -199,12 +199,10 @@ __device__ __forceinline__ RangeSum load_range_sum(const RangeSum* p) {
 
 // Per warp range (the spans one warp of k_span_emit will walk): number of kept entries, first and
 // last kept position, and the code lengths of all kept entries but the first (its gap reaches back
-// into an earlier range); the same for the block's eight ranges together.  Here a THREAD walks a
-// span (or a few consecutive ones) by itself -- a compare and a handful of integer operations per
-// entry, no shuffles; the entries of a span are consecutive, so a thread's loads stay within a few
-// cache lines -- and the lanes' results are then put together in order.  The last block to finish
-// combines the blocks in order: for every block the rank of its first kept entry, the position
-// kept just before it and the bit offset of its first codeword; then the header.
+// into an earlier range); the same for the block's eight ranges together.  The last block to
+// finish combines the blocks in order: for every block the rank of its first kept entry, the
+// position kept just before it and the bit offset of its first codeword; then the header.
+template <bool DENSE_SPANS>
 __global__ void __launch_bounds__(kBlock, 6) k_span_count(const Batch B) {
     __shared__ Prob s_prob;
     const Slot S = resolve(B, &s_prob);
@@ -218,51 +216,87 @@ __global__ void __launch_bounds__(kBlock, 6) k_span_count(const Batch B) {
     const uint32_t n_ranges = S.nb * kWarps;
     const uint32_t range = S.bx * kWarps + warp;
     const int b = P.b;
-    // one buffer for two phases: the lanes' sums of this block's warps, then (last block only) all blocks' sums
+    // one buffer for two phases: the lanes' sums of this block's warps (long spans), then (last block only) all blocks' sums
     __shared__ RangeSum s_buf[kOrderBlocksMax > kWarps * 32u ? kOrderBlocksMax : kWarps * 32u];
     RangeSum (*s_lane)[32] = reinterpret_cast<RangeSum (*)[32]>(s_buf);
     __shared__ RangeSum s_rs[kWarps];
+    // DENSE_SPANS (the host's choice: sixteen kept entries or more per span on average): one THREAD
+    // walks a span by itself -- a compare and a handful of integer operations per entry, no
+    // shuffles; a thread's loads stay within a few cache lines.  Otherwise the warp walks its range
+    // 32 entries at a time, as k_span_emit does (with a thread per span nearly every load would be
+    // a sector of its own and the work of the lanes uneven).  Same result either way.
     if (!failed) {
         uint32_t span0, span1;
         range_spans(P.n_spans, n_ranges, range, &span0, &span1);
-        // lane i takes spans [span0 + i * per_lane, span0 + (i + 1) * per_lane) of the range
-        const uint32_t per_lane = (span1 - span0 + 31u) / 32u;
-        const uint32_t my0 = min(span1, span0 + lane * per_lane), my1 = min(span1, my0 + per_lane);
-        const uint2* __restrict__ rec = P.span_rec[s];
-        const unsigned long long* __restrict__ list = P.list[s];
-        const uint32_t list_cap = P.list_cap;
-        RangeSum mine;
-        mine.cnt = 0u; mine.first = 0u; mine.last = 0u; mine.pad_ = 0u; mine.inner_bits = 0ull;
-        uint32_t prev_plus1 = 0u;
-        for (uint32_t sp = my0; sp < my1; ++sp) {
-            uint2 r = rec[sp];
-            if (r.x > list_cap || r.y > list_cap - r.x) r.y = 0u;  // a record that points outside the list holds nothing
-            const unsigned long long* __restrict__ e = list + r.x;
-            constexpr int kLoads = 8;   // loads in flight per thread
-            for (uint32_t j0 = 0u; j0 < r.y; j0 += kLoads) {
-                unsigned long long c[kLoads];
+        if (DENSE_SPANS) {
+            // lane i takes spans [span0 + i * per_lane, span0 + (i + 1) * per_lane) of the range
+            const uint32_t per_lane = (span1 - span0 + 31u) / 32u;
+            const uint32_t my0 = min(span1, span0 + lane * per_lane), my1 = min(span1, my0 + per_lane);
+            const uint2* __restrict__ rec = P.span_rec[s];
+            const unsigned long long* __restrict__ list = P.list[s];
+            const uint32_t list_cap = P.list_cap;
+            RangeSum mine;
+            mine.cnt = 0u; mine.first = 0u; mine.last = 0u; mine.pad_ = 0u; mine.inner_bits = 0ull;
+            uint32_t pp1 = 0u;
+            for (uint32_t sp = my0; sp < my1; ++sp) {
+                uint2 r = rec[sp];
+                if (r.x > list_cap || r.y > list_cap - r.x) r.y = 0u;  // a record that points outside the list holds nothing
+                const unsigned long long* __restrict__ e = list + r.x;
+                constexpr int kLoads = 8;   // loads in flight per thread
+                for (uint32_t j0 = 0u; j0 < r.y; j0 += kLoads) {
+                    unsigned long long c[kLoads];
 #pragma unroll
-                for (int j = 0; j < kLoads; ++j) c[j] = (j0 + j < r.y) ? e[j0 + j] : 0ull;
+                    for (int j = 0; j < kLoads; ++j) c[j] = (j0 + j < r.y) ? e[j0 + j] : 0ull;
 #pragma unroll
-                for (int j = 0; j < kLoads; ++j) {
-                    if (j0 + j < r.y && c[j] >= thr) {
-                        const uint32_t pos = composite_index(c[j]);
-                        if (mine.cnt == 0u) mine.first = pos;
-                        else mine.inner_bits += (unsigned long long)((pos - prev_plus1) >> b) + 1ull + (unsigned long long)b;
-                        prev_plus1 = pos + 1u;
-                        ++mine.cnt;
+                    for (int j = 0; j < kLoads; ++j) {
+                        if (j0 + j < r.y && c[j] >= thr) {
+                            const uint32_t pos = composite_index(c[j]);
+                            if (mine.cnt == 0u) mine.first = pos;
+                            else mine.inner_bits += (unsigned long long)((pos - pp1) >> b) + 1ull + (unsigned long long)b;
+                            pp1 = pos + 1u;
+                            ++mine.cnt;
+                        }
                     }
                 }
             }
-        }
-        mine.last = prev_plus1 - 1u;
-        s_lane[warp][lane] = mine;
-        __syncwarp();
+            mine.last = pp1 - 1u;
+            // the lanes' sums in order, by lane 0
+            s_lane[warp][lane] = mine;
+            __syncwarp();
+            if (lane == 0u) {
+                RangeSum all = s_lane[warp][0];
+                for (uint32_t l = 1u; l < 32u; ++l) all = fold_ranges(all, s_lane[warp][l], b);
+                P.rng_sum[range] = all;
+                s_rs[warp] = all;
+            }
+        } else {
+        const unsigned lt = (1u << lane) - 1u;
+        uint32_t cnt = 0u, first = 0u, prev_plus1 = 0u;   // the same in all lanes
+        unsigned long long inner = 0ull;                   // each lane adds up the code lengths of the entries it sees
+        walk_spans(P, s, span0, span1, [&](unsigned long long c, bool valid) {
+            const bool kept = valid && c >= thr;
+            const unsigned m = __ballot_sync(0xffffffffu, kept);
+            if (m == 0u) return;  // warp-uniform
+            const uint32_t pos = composite_index(c);
+            const unsigned lower = m & lt;
+            const uint32_t before = __shfl_sync(0xffffffffu, pos, lower ? 31 - __clz((int)lower) : 0);
+            const bool opens = cnt == 0u && lower == 0u;   // the range's first kept entry: its gap reaches into an earlier range
+            if (kept && !opens) {
+                const uint32_t pp = lower ? before + 1u : prev_plus1;   // previous kept position, plus one
+                inner += (unsigned long long)((pos - pp) >> b) + 1ull + (unsigned long long)b;
+            }
+            if (cnt == 0u) first = __shfl_sync(0xffffffffu, pos, __ffs((int)m) - 1);
+            prev_plus1 = __shfl_sync(0xffffffffu, pos, 31 - __clz((int)m)) + 1u;
+            cnt += (uint32_t)__popc(m);
+        });
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) inner += __shfl_down_sync(0xffffffffu, inner, d);
         if (lane == 0u) {
-            RangeSum all = s_lane[warp][0];
-            for (uint32_t l = 1u; l < 32u; ++l) all = fold_ranges(all, s_lane[warp][l], b);
+            RangeSum all;
+            all.cnt = cnt; all.first = first; all.last = prev_plus1 - 1u; all.pad_ = 0u; all.inner_bits = inner;
             P.rng_sum[range] = all;
             s_rs[warp] = all;
+        }
         }
         __syncthreads();
         if (threadIdx.x == 0) {

@@ -1,5 +1,6 @@
 // Host side of the SBC C ABI: argument checks, workspace layout, kernel launches.
 // Declared and documented in include/sbc.h.
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -262,6 +263,7 @@ void block_counts(const Plan& pl, unsigned sms, unsigned coarse_sample, unsigned
     nb[WK_ORDER] = pl.order_blocks;
     nb[WK_ONE] = 1;
     nb[WK_STREAM] = grid_for(pl.stream_bytes, kBlock * 64, sms * 4);
+    nb[WK_PERM] = 0;
 }
 
 // Set-up of a single encode in one launch instead of two memsets and a descriptor kernel: the
@@ -338,7 +340,9 @@ void launch_encode(const Prob* d_probs, uint32_t n_probs, uint32_t* any_exact, c
         nvtxRangePop();
         if (i + 1 < SBC_MARK_COUNT) nvtxRangePushA(kStageNames[i]);
     };
-    auto B = [&](int kind) { return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs, any_exact}; };
+    auto B = [&](int kind) {
+        return Batch{d_probs, prefix ? prefix[kind] : nullptr, n_probs, any_exact, (prefix && kind == WK_ONE) ? prefix[WK_PERM] : nullptr};
+    };
     auto g1 = [&](int kind) { return dim3(grid[kind]); };
     auto g2 = [&](int kind) { return dim3(grid[kind], 1, 2); };  // z = side
     // Every kernel is launched with programmatic stream serialisation: its blocks may be placed
@@ -626,6 +630,13 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
                 row[t + 1] = (uint32_t)next;
             }
         }
+    }
+
+    {   // one-block kernels take the problems largest first
+        uint32_t* perm = prefix.data() + (size_t)WK_PERM * row_len;
+        for (int t = 0; t < n_tensors; ++t) perm[t] = (uint32_t)t;
+        std::stable_sort(perm, perm + n_tensors, [&](uint32_t a, uint32_t b) { return plans[a].n > plans[b].n; });
+        perm[n_tensors] = 0u;
     }
 
     cudaStream_t st = stream;

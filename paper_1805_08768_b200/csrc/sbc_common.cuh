@@ -146,6 +146,10 @@ struct Batch {
     const uint32_t* prefix;  // n_probs + 1 entries, or nullptr
     uint32_t n_probs;
     uint32_t* any_exact;     // one word per launch: non-zero once a problem needs the exact route
+    // One-block-per-problem kernels of a batch: slot i of the grid works on problem perm[i] (largest
+    // problems first: the grid can be larger than what is resident at once, and the blocks that
+    // have to wait for a free slot should be the short ones).  nullptr: slot i is problem i.
+    const uint32_t* perm;
 };
 struct Slot {
     const Prob* P;
@@ -186,7 +190,7 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
                 hi = min(hi, lo + step);
             }
             if (lane < 2u) s_slot[1 + lane] = B.prefix[lo + lane];
-            if (lane == 0u) s_slot[0] = lo;
+            if (lane == 0u) s_slot[0] = B.perm ? B.perm[lo] : lo;
         }
         __syncthreads();
         src = B.probs + s_slot[0]; s.bx = blockIdx.x - s_slot[1]; s.nb = s_slot[2] - s_slot[1];
@@ -202,7 +206,9 @@ __device__ __forceinline__ Slot resolve(const Batch& B, Prob* s_prob) {
 
 // Kinds of work a kernel's grid is sized by (one prefix table per kind in a batch).
 enum WorkKind : int {
-    WK_SAMPLE = 0, WK_MAIN, WK_CAND, WK_ORDER, WK_ONE, WK_STREAM, WK_COUNT
+    WK_SAMPLE = 0, WK_MAIN, WK_CAND, WK_ORDER, WK_ONE, WK_STREAM,
+    WK_PERM,   // not a kind of work: the row of the tables that holds the order in which one-block kernels take the problems
+    WK_COUNT
 };
 
 // What the kept entries of one warp range of the ordering kernels add up to (see k_span_count).

@@ -68,23 +68,18 @@ __global__ void __launch_bounds__(kBlock) k_small_finish(const Batch B) {
             const uint32_t thr_bits = bits_of_key(side_key(s, (uint32_t)(thr >> 32)));
             const int bin_a = max((int)((thr_bits >> 23) & 0xffu) - 1, 0);
             long long acc_a = 0;
-            constexpr int kLoads = 4;  // list entries in flight per thread
-            for (uint32_t base = threadIdx.x; base < cnt; base += kBlock * kLoads) {
-                unsigned long long e[kLoads];
+            const unsigned long long thr_rel = thr - dg.sub;   // the entries are still in the registers, with dg.sub taken off
 #pragma unroll
-                for (int j = 0; j < kLoads; ++j) e[j] = (base + j * kBlock < cnt) ? view.src[base + j * kBlock] : 0ull;
-#pragma unroll
-                for (int j = 0; j < kLoads; ++j) {
-                    if (base + j * kBlock >= cnt || e[j] < thr) continue;
-                    const uint32_t bits = bits_of_key(side_key(s, (uint32_t)(e[j] >> 32)));
-                    const uint32_t ex = (bits >> 23) & 0xffu;
-                    int m = (int)(bits & 0x7fffffu) | (ex ? 0x800000 : 0);
-                    if (bits >> 31) m = -m;
-                    const int bin = ex ? (int)ex - 1 : 0;
-                    const uint32_t up = (uint32_t)(bin - bin_a);
-                    if (up < 8u) acc_a += (long long)m << up;  // |m| < 2^24: at most 2^31 per entry
-                    else atomicAdd(reinterpret_cast<unsigned long long*>(&s_bins[bin]), (unsigned long long)(long long)m);
-                }
+            for (int j = 0; j < kPer; ++j) {
+                if ((uint32_t)j * kBlock + threadIdx.x >= cnt || c[j] < thr_rel) continue;
+                const uint32_t bits = bits_of_key(side_key(s, (uint32_t)((c[j] + dg.sub) >> 32)));
+                const uint32_t ex = (bits >> 23) & 0xffu;
+                int m = (int)(bits & 0x7fffffu) | (ex ? 0x800000 : 0);
+                if (bits >> 31) m = -m;
+                const int bin = ex ? (int)ex - 1 : 0;
+                const uint32_t up = (uint32_t)(bin - bin_a);
+                if (up < 8u) acc_a += (long long)m << up;  // |m| < 2^24: at most 2^31 per entry
+                else atomicAdd(reinterpret_cast<unsigned long long*>(&s_bins[bin]), (unsigned long long)(long long)m);
             }
 #pragma unroll
             for (int d = 16; d > 0; d >>= 1) acc_a += __shfl_down_sync(0xffffffffu, acc_a, d);

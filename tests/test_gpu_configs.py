@@ -233,6 +233,54 @@ def test_batch_and_single_tensor_calls_agree_with_mixed_sparsities():
         sbc.sbc_encode_batch(d_up, d_res, ps[:-1] + [1.5], outs, mus, ws)
 
 
+def test_batch_whose_problems_take_all_three_routes():
+    # one launch of the general chain in which a problem runs on the sample's bounds, one has its
+    # candidates gathered again (clustered), one has its thresholds searched over the whole tensor
+    # (the sample never sees its large values), one is all zeros and one is small: the exact
+    # route's kernel works on three of them at once and hands each back the right way
+    rng = np.random.default_rng(4711)
+    n_big = 1 << 21
+    plain = (rng.standard_t(3, n_big) * 1e-3).astype(np.float32)
+    clustered = (rng.standard_normal(n_big) * 1e-6).astype(np.float32)
+    clustered[n_big // 2 + 777: n_big // 2 + 777 + n_big // 50] *= np.float32(1e3)
+    hidden = (rng.standard_normal(n_big) * 1e-3).astype(np.float32)
+    k = oracle.kept_count(n_big, 0.01)
+    off_sample = np.flatnonzero((np.arange(n_big) // 32) % 16 != 0)
+    extra = rng.choice(off_sample, k, replace=False)
+    hidden[extra[: k // 2]] = (5e-3 + 1e-3 * rng.random(k // 2)).astype(np.float32)
+    hidden[extra[k // 2:]] = (-5e-3 - 1e-3 * rng.random(k - k // 2)).astype(np.float32)
+    zeros = np.zeros(300_000, dtype=np.float32)
+    small = (rng.standard_normal(5000) * 1e-3).astype(np.float32)
+    ups = [plain, clustered, hidden, zeros, small]
+    ps = [0.01, 0.01, 0.01, 0.01, 0.01]
+    sizes = [u.size for u in ups]
+    for rnd in range(2):                                  # second round: carried residuals
+        if rnd == 0:
+            res0 = [np.zeros(n, dtype=np.float32) for n in sizes]
+            d_res = [torch.from_numpy(r).to(DEV) for r in res0]
+            want_res = [r.copy() for r in res0]
+        want = [oracle.encode(u, r, p) for u, r, p in zip(ups, want_res, ps)]
+        d_up = [torch.from_numpy(u).to(DEV) for u in ups]
+        outs = [torch.empty(sbc.sbc_stream_bytes(n, p), dtype=torch.uint8, device=DEV) for n, p in zip(sizes, ps)]
+        mus = [torch.empty(1, dtype=torch.float32, device=DEV) for _ in sizes]
+        ws = torch.empty(sbc.sbc_workspace_bytes_batch(sizes, ps), dtype=torch.uint8, device=DEV)
+        sbc.sbc_encode_batch(d_up, d_res, ps, outs, mus, ws)
+        torch.cuda.synchronize()
+        for t, (ws_, wm) in enumerate(want):
+            info = sbc.sbc_stream_info_get(outs[t])
+            assert np.array_equal(outs[t][: info.total_bytes].cpu().numpy(), ws_), f"round {rnd}, tensor {t}"
+            assert np.float32(mus[t].item()).view(np.uint32) == wm.view(np.uint32), f"round {rnd}, tensor {t}"
+            assert np.array_equal(d_res[t].cpu().numpy().view(np.uint32), want_res[t].view(np.uint32)), f"round {rnd}, tensor {t}"
+    # the same three large tensors one by one: the routes are the ones this test is about
+    for u, want_route in ((plain, (0, 0)), (clustered, (1, 1)), (hidden, (1, 0))):
+        d_u = torch.from_numpy(u).to(DEV)
+        d_r = torch.zeros(u.size, dtype=torch.float32, device=DEV)
+        ws1 = torch.empty(sbc.sbc_workspace_bytes(u.size, 0.01), dtype=torch.uint8, device=DEV)
+        sbc.sbc_encode(d_u, d_r, 0.01, workspace=ws1)
+        diag = sbc.sbc_encode_diag_get(ws1)
+        assert (diag.exact_route, diag.regathered) == want_route
+
+
 @pytest.mark.parametrize("seed", [1, 2, 3])
 def test_batch_of_short_list_problems_with_ties_zeros_and_a_bad_tensor(seed):
     # every tensor keeps at most 3584 positions, so the whole batch takes the one-kernel back half;

@@ -242,22 +242,32 @@ __global__ void __launch_bounds__(kBlock, 6) k_span_count(const Batch B) {
                 uint2 r = rec[sp];
                 if (r.x > list_cap || r.y > list_cap - r.x) r.y = 0u;  // a record that points outside the list holds nothing
                 const unsigned long long* __restrict__ e = list + r.x;
-                constexpr int kLoads = 8;   // loads in flight per thread
-                for (uint32_t j0 = 0u; j0 < r.y; j0 += kLoads) {
-                    unsigned long long c[kLoads];
-#pragma unroll
-                    for (int j = 0; j < kLoads; ++j) c[j] = (j0 + j < r.y) ? e[j0 + j] : 0ull;
-#pragma unroll
-                    for (int j = 0; j < kLoads; ++j) {
-                        if (j0 + j < r.y && c[j] >= thr) {
-                            const uint32_t pos = composite_index(c[j]);
-                            if (mine.cnt == 0u) mine.first = pos;
-                            else mine.inner_bits += (unsigned long long)((pos - pp1) >> b) + 1ull + (unsigned long long)b;
-                            pp1 = pos + 1u;
-                            ++mine.cnt;
-                        }
+                auto take = [&](unsigned long long c) {
+                    if (c >= thr) {
+                        const uint32_t pos = composite_index(c);
+                        if (mine.cnt == 0u) mine.first = pos;
+                        else mine.inner_bits += (unsigned long long)((pos - pp1) >> b) + 1ull + (unsigned long long)b;
+                        pp1 = pos + 1u;
+                        ++mine.cnt;
                     }
+                };
+                // two entries per load (every lane's load is a sector of its own here, and the load
+                // unit takes such an instruction apart lane by lane: half as many instructions, half
+                // the time): an odd first entry and an odd last one by themselves
+                uint32_t j0 = 0u;
+                if ((r.x & 1u) && r.y) { take(e[0]); j0 = 1u; }
+                const ulonglong2* __restrict__ e2 = reinterpret_cast<const ulonglong2*>(e + j0);   // the lists start on 256-byte boundaries
+                const uint32_t pairs = (r.y - j0) >> 1;
+                constexpr int kLoads = 4;   // loads in flight per thread
+                for (uint32_t q0 = 0u; q0 < pairs; q0 += kLoads) {
+                    ulonglong2 v[kLoads];
+#pragma unroll
+                    for (int j = 0; j < kLoads; ++j) v[j] = (q0 + j < pairs) ? e2[q0 + j] : make_ulonglong2(0ull, 0ull);
+#pragma unroll
+                    for (int j = 0; j < kLoads; ++j)
+                        if (q0 + j < pairs) { take(v[j].x); take(v[j].y); }
                 }
+                if ((r.y - j0) & 1u) take(e[r.y - 1u]);
             }
             mine.last = pp1 - 1u;
             // the lanes' sums in order, by lane 0

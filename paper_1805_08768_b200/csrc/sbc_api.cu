@@ -36,6 +36,7 @@ struct Plan {
     uint32_t cap, m, n_xtiles, n_chunks, chunk_cw;
     uint32_t s_target, s_up;
     uint32_t main_blocks, main_warps, span_steps, n_spans, cap_w, list_cap, use_runs, order_blocks;
+    bool dense_spans;   // sixteen kept entries or more per span expected
     unsigned long long payload_offset;
     size_t stream_bytes;
     size_t zero_bytes, off_ctl, off_hists;                 // offsets inside the zero part
@@ -146,7 +147,10 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
         pl->list_cap = (uint32_t)std::min<unsigned long long>(std::max<unsigned long long>(regions, pl->cap), 0xfffffff0ull);
         if (regions > 0xfffffff0ull) return false;      // cannot happen below 2^31 elements
     }
-    pl->order_blocks = grid_for(pl->n_spans, (kBlock / 32) * 4, kOrderBlocksMax);   // four spans or more per warp
+    // four spans or more per warp; where spans are long (see k_span_count) as many blocks as it takes to
+    // give every lane of the counting walk one span, else one resident wave
+    pl->dense_spans = (unsigned long long)k >= 16ull * pl->n_spans;
+    pl->order_blocks = grid_for(pl->n_spans, (kBlock / 32) * 4, pl->dense_spans ? kOrderBlocksMax : kOrderBlocksWave);
 
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -496,7 +500,7 @@ static int encode_impl(int mode, const uint32_t* sample_idx, int64_t sample_m, c
     unsigned grid[WK_COUNT];
     block_counts(pl, (unsigned)sm_count(), 1u, grid);
     launch_encode(d_prob, 1u, &P.ctl->launch_exact, grid, nullptr, mode, pl.sampled != 0, small_lists, small_form,
-                  (unsigned long long)pl.k >= 16ull * pl.n_spans, st, marks);
+                  pl.dense_spans, st, marks);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

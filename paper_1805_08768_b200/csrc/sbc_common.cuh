@@ -26,7 +26,8 @@ constexpr int kXTile = 4096;          // elements per tile in the exact-select f
 constexpr int kWarpChunk = 512;       // elements one warp handles per step of the streaming pass
 constexpr int kMaxSpanSteps = kXTile / kWarpChunk;  // a span is 1, 2, 4 or 8 steps and never straddles a tile
 constexpr int kChunkCodewords = 256;  // most codewords per chunk-table entry (long streams)
-constexpr uint32_t kOrderBlocksMax = 148 * 8;  // ordering kernels: at most one resident wave of 8-warp blocks on 148 SMs
+constexpr uint32_t kOrderBlocksMax = 148 * 8;  // ordering kernels: most blocks a problem gets (long spans: one span per lane at 2^30 elements)
+constexpr uint32_t kOrderBlocksWave = 148 * 5; // ... and what is resident at once on 148 SMs (the walk that writes needs 48 registers): the grid for short spans
 constexpr int kSumBins = 254;         // one exact integer bin per fp32 exponent
 constexpr uint32_t kSmallList = 8192;  // candidate lists up to this capacity are ranked by one block
 

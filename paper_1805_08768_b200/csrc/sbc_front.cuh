@@ -453,7 +453,35 @@ __global__ void __launch_bounds__(kBlock, kCollectBlocksPerSM) k_add_collect(con
             mask[0] &= inb;
             mask[1] &= inb;
             if (__any_sync(0xffffffffu, (mask[0] | mask[1]) != 0u)) {
-            if (this_vec) {
+            if (this_vec && __all_sync(0xffffffffu, ((mask[0] & (mask[0] - 1u)) | (mask[1] & (mask[1] - 1u))) == 0u)) {
+                // No lane holds more than one candidate per side (nine steps in ten at p = 0.01):
+                // position order (row u, lane) comes from one ballot per row, no scan.
+                const uint32_t idx0 = (uint32_t)base + (uint32_t)lane * 4u;
+#pragma unroll
+                for (int s = 0; s < kSides; ++s) {
+                    const uint32_t m = mask[s];
+                    const unsigned b_any = __ballot_sync(0xffffffffu, m != 0u);
+                    if (b_any == 0u) continue;  // warp-uniform
+                    const unsigned b0 = __ballot_sync(0xffffffffu, (m & 0x000fu) != 0u);
+                    const unsigned b1 = __ballot_sync(0xffffffffu, (m & 0x00f0u) != 0u);
+                    const unsigned b2 = __ballot_sync(0xffffffffu, (m & 0x0f00u) != 0u);
+                    const unsigned b3 = b_any & ~(b0 | b1 | b2);
+                    const uint32_t tot_s = (uint32_t)__popc(b_any);
+                    if (wcnt[s] + tot_s > (uint32_t)kStage) flush(s);
+                    const uint32_t j = (uint32_t)__ffs((int)m) - 1u;   // the lane's candidate, if it has one
+                    const bool t0 = j & 1u, t1 = j & 2u, t2 = j & 4u, t3 = j & 8u;
+                    const float x0 = t0 ? a[1] : a[0], x1 = t0 ? a[3] : a[2], x2 = t0 ? a[5] : a[4], x3 = t0 ? a[7] : a[6];
+                    const float x4 = t0 ? a[9] : a[8], x5 = t0 ? a[11] : a[10], x6 = t0 ? a[13] : a[12], x7 = t0 ? a[15] : a[14];
+                    const float y0 = t1 ? x1 : x0, y1 = t1 ? x3 : x2, y2 = t1 ? x5 : x4, y3 = t1 ? x7 : x6;
+                    const float z0 = t2 ? y1 : y0, z1 = t2 ? y3 : y2;
+                    const float v = t3 ? z1 : z0;
+                    const unsigned row = t3 ? (t2 ? b3 : b2) : (t2 ? b1 : b0);
+                    const uint32_t before = (t3 || t2 ? (uint32_t)__popc(b0) : 0u) + (t3 ? (uint32_t)__popc(b1) : 0u) +
+                                            (t3 && t2 ? (uint32_t)__popc(b2) : 0u) + (uint32_t)__popc(row & lt);
+                    if (m) st.stage[warp][s][wcnt[s] + before] = make_uint2(__float_as_uint(v), idx0 + (j >> 2) * 128u + (j & 3u));
+                    wcnt[s] += tot_s;
+                }
+            } else if (this_vec) {
                 // Position order inside the step is (u, lane, element of the float4).  Per side and u,
                 // the number of candidates of every lane goes into one byte of a 64-bit word; one warp
                 // scan gives every (side, u, lane) its slot.

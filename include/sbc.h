@@ -251,8 +251,8 @@ enum sbc_mark {
     SBC_MARK_BOUNDS,    /* scratch cleared, threshold bounds estimated from the sample */
     SBC_MARK_COLLECT,   /* residual = A written, candidate lists gathered */
     SBC_MARK_EXACT,     /* exact-select route over A done (a no-op unless the bounds failed) */
-    SBC_MARK_SELECT,    /* k-th entries, means, side, mu, residual write-back done */
-    SBC_MARK_END,       /* positions compacted, Golomb payload, chunk table and header written */
+    SBC_MARK_SELECT,    /* k-th entries, means, side and mu found */
+    SBC_MARK_END,       /* kept positions walked in order: residual written back, Golomb payload, chunk table and header written */
     SBC_MARK_COUNT
 };
 int sbc_encode_ex(const float *update, float *residual, int64_t numel, double p,

@@ -417,7 +417,7 @@ __global__ void __launch_bounds__(kBlock) k_select_filter0(const Batch B) {
 // The whole selection and the sums of one side by ONE block, for lists of at most kSmallList
 // entries: the entries sit in registers, every level is a shared-memory histogram of the entries
 // that still match the prefix, and the walk stops as soon as the selected bucket holds a single
-// entry.  Same result as k_select_filter0 + k_select_tail; the host launches this kernel instead of
+// entry.  Same result as k_select_hist0 + k_select_filter0; the host launches this kernel instead of
 // those when every list of the launch is that small.  One block per problem, grid.z = side.
 __global__ void __launch_bounds__(kBlock) k_select_small(const Batch B) {
     __shared__ Prob s_prob;

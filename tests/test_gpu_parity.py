@@ -146,6 +146,19 @@ def test_span_ordering_forms(n, p, clustered):
     check_against_oracle(upd, np.zeros(n, dtype=np.float32), p)
 
 
+@pytest.mark.parametrize("n,p", [
+    ((1 << 25) + 4321, 0.0040),   # eight-step spans, 16.4 kept entries per span: a thread walks a span, 1184 blocks
+    ((1 << 25) + 4321, 0.0038),   # 15.6 per span: the warp walks its range, one resident wave of blocks
+    (1 << 22, 0.032),             # one-step spans on either side of the same limit
+    (1 << 22, 0.030),
+])
+def test_both_counting_walks_around_their_limit(n, p):
+    rng = np.random.default_rng(zlib.crc32(f"walks/{n}/{p}".encode()))
+    upd = (rng.standard_t(3, n) * 1e-3).astype(np.float32)
+    res = (rng.standard_normal(n) * 1e-4).astype(np.float32)
+    check_against_oracle(upd, res, p)
+
+
 @pytest.mark.parametrize("offset", [1, 2, 3])
 def test_encode_misaligned_pointers(offset):
     rng = np.random.default_rng(offset)

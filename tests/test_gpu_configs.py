@@ -200,7 +200,7 @@ def test_config5_flat_2p30_sweep_against_independent_selection():
     for p in (1e-2, 1e-3, 1e-4):
         residual = torch.zeros(n, dtype=torch.float32, device=DEV)
         _check_flat_round(update, update, residual, p)              # A = 0 + update
-        carried = torch.add(residual, update2)                      # what round 2 must accumulate
+        carried = torch.add(residual, update2)                      # what the second communication round must accumulate
         assert bool((residual != update).any())                     # the residual really carries something
         _check_flat_round(carried, update2, residual, p)
         del residual, carried

@@ -554,8 +554,16 @@ static bool plan_batch(int n_tensors, const sbc_tensor_desc* descs, std::vector<
         fine_main += (unsigned long long)(pl.n + kBlock * kPerThread - 1) / (kBlock * kPerThread);
         small = small && !pl.use_runs;
     }
-    const unsigned coarse_main = (unsigned)std::min<unsigned long long>(
+    unsigned coarse_main = (unsigned)std::min<unsigned long long>(
         16, std::max<unsigned long long>(1, fine_main / (kPlanSMs * 2 * kCollectBlocksPerSM)));
+    // a batch of a few large tensors: blocks of up to 32 x 4096 elements if all of them are then
+    // resident at once (a block's start-up and final flush cost as much as several steps)
+    for (unsigned c = coarse_main + 1; c <= 32; ++c) {
+        unsigned long long blocks = 0;
+        for (int t = 0; t < n_tensors; ++t)
+            blocks += ((unsigned long long)descs[t].numel + (unsigned long long)kBlock * kPerThread * c - 1) / ((unsigned long long)kBlock * kPerThread * c);
+        if (blocks <= (unsigned long long)kPlanSMs * kCollectBlocksPerSM) { coarse_main = c; break; }
+    }
     plans->resize((size_t)n_tensors);
     for (int t = 0; t < n_tensors; ++t)
         if (!make_plan(descs[t].numel, descs[t].p, &(*plans)[t], kModeBinary, 0, coarse_main, !small)) return false;

@@ -556,13 +556,21 @@ static bool plan_batch(int n_tensors, const sbc_tensor_desc* descs, std::vector<
     }
     unsigned coarse_main = (unsigned)std::min<unsigned long long>(
         16, std::max<unsigned long long>(1, fine_main / (kPlanSMs * 2 * kCollectBlocksPerSM)));
-    // a batch of a few large tensors: blocks of up to 32 x 4096 elements if all of them are then
-    // resident at once (a block's start-up and final flush cost as much as several steps)
-    for (unsigned c = coarse_main + 1; c <= 32; ++c) {
+    // Whole waves: with every tensor's block count rounded up, the rule above can leave a last wave
+    // that is half empty.  Blocks of up to 32 x 4096 elements if the batch then fits one resident
+    // wave (a few large tensors: a block's start-up and final flush cost as much as several
+    // steps), else the smallest blocks that fit two.
+    auto blocks_at = [&](unsigned c) {
         unsigned long long blocks = 0;
         for (int t = 0; t < n_tensors; ++t)
             blocks += ((unsigned long long)descs[t].numel + (unsigned long long)kBlock * kPerThread * c - 1) / ((unsigned long long)kBlock * kPerThread * c);
-        if (blocks <= (unsigned long long)kPlanSMs * kCollectBlocksPerSM) { coarse_main = c; break; }
+        return blocks;
+    };
+    const unsigned long long wave = (unsigned long long)kPlanSMs * kCollectBlocksPerSM;
+    if (blocks_at(32) <= wave) {
+        while (blocks_at(coarse_main) > wave) ++coarse_main;
+    } else if (blocks_at(32) <= 2 * wave) {
+        while (blocks_at(coarse_main) > 2 * wave) ++coarse_main;
     }
     plans->resize((size_t)n_tensors);
     for (int t = 0; t < n_tensors; ++t)

@@ -24,6 +24,9 @@ namespace {
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 constexpr size_t kProbSlotBytes = 512;  // one problem descriptor, padded
+// The counting walk with one thread per span pays only where there are spans enough to fill the
+// machine with threads (long spans of a small tensor leave most lanes without one).
+constexpr unsigned long long kDenseSpansMin = 65536;
 static_assert(sizeof(Prob) <= kProbSlotBytes, "descriptor must fit its slot");
 
 // Host-side plan of one encode problem: scalar parameters and the layout of its scratch, which
@@ -147,10 +150,10 @@ bool make_plan(long long n, double p, Plan* pl, int mode = kModeBinary, long lon
         pl->list_cap = (uint32_t)std::min<unsigned long long>(std::max<unsigned long long>(regions, pl->cap), 0xfffffff0ull);
         if (regions > 0xfffffff0ull) return false;      // cannot happen below 2^31 elements
     }
-    // four spans or more per warp; where spans are long (see k_span_count) as many blocks as it takes to
-    // give every lane of the counting walk one span, else one resident wave
-    pl->dense_spans = (unsigned long long)k >= 16ull * pl->n_spans;
-    pl->order_blocks = grid_for(pl->n_spans, (kBlock / 32) * 4, pl->dense_spans ? kOrderBlocksMax : kOrderBlocksWave);
+    // a span or more per warp; where spans are long and many (see k_span_count) as many blocks as it takes
+    // to give every lane of the counting walk one span, else one resident wave
+    pl->dense_spans = (unsigned long long)k >= 16ull * pl->n_spans && pl->n_spans >= kDenseSpansMin;
+    pl->order_blocks = grid_for(pl->n_spans, kBlock / 32, pl->dense_spans ? kOrderBlocksMax : kOrderBlocksWave);
 
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
@@ -681,7 +684,7 @@ int sbc_encode_batch(int n_tensors, const sbc_tensor_desc* descs, void* workspac
     unsigned long long k_total = 0, spans_total = 0;
     for (int t = 0; t < n_tensors; ++t) { k_total += (unsigned long long)plans[t].k; spans_total += plans[t].n_spans; }
     launch_encode(d_probs, (uint32_t)n_tensors, &probs[0].ctl->launch_exact, grid, d_rows, kModeBinary, false, small_lists, all_small,
-                  k_total >= 16ull * spans_total, st, nullptr);
+                  k_total >= 16ull * spans_total && spans_total >= kDenseSpansMin, st, nullptr);
     return cudaGetLastError() == cudaSuccess ? SBC_OK : SBC_ECUDA;
 }
 

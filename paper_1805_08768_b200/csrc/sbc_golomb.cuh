@@ -220,7 +220,8 @@ __global__ void __launch_bounds__(kBlock, 6) k_span_count(const Batch B) {
     __shared__ RangeSum s_buf[kOrderBlocksMax > kWarps * 32u ? kOrderBlocksMax : kWarps * 32u];
     RangeSum (*s_lane)[32] = reinterpret_cast<RangeSum (*)[32]>(s_buf);
     __shared__ RangeSum s_rs[kWarps];
-    // DENSE_SPANS (the host's choice: sixteen kept entries or more per span on average): one THREAD
+    // DENSE_SPANS (the host's choice: sixteen kept entries or more per span on average, and spans
+    // enough to give most threads of the machine one): one THREAD
     // walks a span by itself -- a compare and a handful of integer operations per entry, no
     // shuffles; a thread's loads stay within a few cache lines.  Otherwise the warp walks its range
     // 32 entries at a time, as k_span_emit does (with a thread per span nearly every load would be

@@ -297,8 +297,8 @@ int sbc_encode_host(const float *update_host, float *update_dev, float *residual
  * that is part of the library image: every GPU that loads the library holds
  * those bytes until the process exits.  Consequences the caller must know:
  *   - Only problems with sbc_workspace_bytes(numel, p) <=
- *     SBC_STATIC_WORKSPACE_BYTES fit (up to about 2.67 M elements at p = 0.01,
- *     11.0 M at p = 0.001);
+ *     SBC_STATIC_WORKSPACE_BYTES fit (up to about 2.6 M elements at p = 0.01,
+ *     10.7 M at p = 0.001);
  *     larger ones are refused with SBC_ECAPACITY and nothing is enqueued.
  *   - There is ONE array per GPU, shared by every call in the process.  Two
  *     calls whose device work can overlap (different streams, different

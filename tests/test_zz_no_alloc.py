@@ -60,7 +60,15 @@ def test_static_scratch_at_its_limit_then_a_small_call():
     # the largest problem the fixed array takes at p = 0.01 (its scratch fills all but a few KB of
     # the 8 MiB), then a small one that reuses the same bytes
     p = 0.01
-    n = 2_670_000
+    lo, hi = 1, 1 << 26                       # the largest n whose scratch fits, by bisection on the host
+    while hi - lo > 1:
+        mid = (lo + hi) // 2
+        if sbc.sbc_workspace_bytes(mid, p) <= sbc.STATIC_WORKSPACE_BYTES:
+            lo = mid
+        else:
+            hi = mid
+    n = lo - 1000
+    assert 2_000_000 < n < 4_000_000          # what the header says about the limit (about 2.6 M at p = 0.01)
     need = sbc.sbc_workspace_bytes(n, p)
     assert 0.98 * sbc.STATIC_WORKSPACE_BYTES < need <= sbc.STATIC_WORKSPACE_BYTES
     assert sbc.sbc_workspace_bytes(n + 20_000, p) > sbc.STATIC_WORKSPACE_BYTES

@@ -38,7 +38,43 @@ __global__ void __launch_bounds__(kBlock, 4) k_sample0(const Batch B) {
     for (int i = threadIdx.x; i < kHistBins; i += kBlock) s_hist[i] = 0u;
     __syncthreads();
     constexpr int kItems = 8;  // sampled elements per thread and step, all loads issued before any is used
+    const float* __restrict__ R = P.residual;
+    const float* __restrict__ U = P.update;
+    uint32_t* __restrict__ keys = P.sample_keys;
+    const uint32_t m = P.m;
+    const bool whole = (long long)m == P.n, by_arithmetic = P.sampled == 0;
+    const int mode = P.mode;
+    const unsigned long long step = P.sample_step;
     for (uint32_t base = S.bx * (kBlock * kItems); base < P.m; base += S.nb * (kBlock * kItems)) {
+        if (by_arithmetic && base + kBlock * kItems <= m) {
+            // Every slot of the step is a sample slot and its element follows from its number (in
+            // range by construction): 32-bit indices, the segment's line by adding up instead of
+            // multiplying (slot i + 256 j lies 8 j segments further on), no checks.  This kernel runs
+            // at the rate it issues instructions, not at the memory's.
+            uint32_t e[kItems];
+            const uint32_t i0 = base + threadIdx.x;
+            if (whole) {
+#pragma unroll
+                for (int j = 0; j < kItems; ++j) e[j] = i0 + (uint32_t)j * kBlock;
+            } else {
+                unsigned long long prod = (unsigned long long)(i0 >> 5) * step;
+#pragma unroll
+                for (int j = 0; j < kItems; ++j) {
+                    e[j] = (uint32_t)(prod >> 20) * 32u + (i0 & 31u);
+                    prod += (unsigned long long)(kBlock / 32) * step;
+                }
+            }
+            float r[kItems], u[kItems];
+#pragma unroll
+            for (int j = 0; j < kItems; ++j) { r[j] = R[e[j]]; u[j] = U[e[j]]; }
+#pragma unroll
+            for (int j = 0; j < kItems; ++j) {
+                const uint32_t key = select_key(mode, __float_as_uint(__fadd_rn(r[j], u[j])));
+                keys[i0 + (uint32_t)j * kBlock] = key;
+                atomicAdd(&s_hist[key >> 21], 1u);
+            }
+            continue;
+        }
         long long e[kItems];
         float r[kItems], u[kItems];
 #pragma unroll

@@ -161,12 +161,12 @@ def run_reference(args):
 #     stored(numel) = stored(2^26) * numel / 2^26,   l2_residue = stored(2^26) - writes(2^26),
 # where stored(2^26) = 4 B per element plus the candidate lists the capture's launch wrote.
 # Valid only for the kernel source it was taken from: a different hash of the file reports null.
-NCU_READ_BYTES_AT_2P26 = 537.12e6      # dram__bytes_read.sum
-NCU_WRITE_BYTES_AT_2P26 = 229.36e6     # dram__bytes_write.sum (during the kernel)
+NCU_READ_BYTES_AT_2P26 = 537.07e6      # dram__bytes_read.sum
+NCU_WRITE_BYTES_AT_2P26 = 229.18e6     # dram__bytes_write.sum (during the kernel)
 # 4 B x 2^26 of residual + 8 B x (717245 + 699450) ordered candidate entries + ~1.4 MB of band entries
 # + 0.26 MB of span records
 NCU_STORED_BYTES_AT_2P26 = 268.435456e6 + 11.33356e6 + 1.4e6 + 0.262144e6
-NCU_TRAFFIC_SOURCE_SHA256 = "f57535d1900fad3093898bc1bbf4e6d2145c29a0a8a4e6467caf4fc5b6dc991b"
+NCU_TRAFFIC_SOURCE_SHA256 = "623b599fadbfc6197856f6d23ed7ffa42ed7a04d2353a8c38a418ec21f92cb26"
 
 
 def measured_traffic(numel: int):
